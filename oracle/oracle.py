@@ -1,0 +1,171 @@
+"""ctypes front end of the float64 CPU oracle (test infrastructure only).
+
+Each function marshals numpy arrays to ``btard_oracle.c`` and returns numpy
+arrays; no arithmetic of the method is done in Python.
+"""
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+INIT_CALLER, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
+STOP_FIXED, STOP_EPS = 0, 1
+SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1
+STATUS_NOT_CONVERGED, STATUS_NONFINITE_ROW = 1, 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "btard_oracle.c")
+_LIB = os.path.join(_HERE, "libbtard_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with gcc (no fast-math, no fp contraction)."""
+    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC):
+        return _LIB
+    tmp = _LIB + ".tmp%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+           "-fno-fast-math", "-Wall", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            _lib = C.CDLL(build())
+            _lib.btard_oracle_max_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a, ty):
+    return a.ctypes.data_as(C.POINTER(ty)) if a is not None else None
+
+
+def max_threads():
+    return int(_load().btard_oracle_max_threads())
+
+
+def philox4x32_10(ctr, key):
+    """One Philox4x32-10 block: 4 counter words, 2 key words -> 4 output words."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    _load().btard_oracle_philox4x32_10(_p(c, C.c_uint32), _p(k, C.c_uint32), _p(out, C.c_uint32))
+    return out
+
+
+def random_vector(seed, p, k, part_len):
+    """Unnormalised fp32 coordinates of z_k for partition p."""
+    z = np.zeros(int(part_len), dtype=np.float32)
+    _load().btard_oracle_random_vector(C.c_uint64(int(seed)), C.c_int32(p), C.c_int32(k),
+                                       C.c_int64(int(part_len)), _p(z, C.c_float))
+    return z
+
+
+def partition_layout(d, P, mode=SPLIT_PAPER, align_elems=32):
+    off = np.zeros(P, dtype=np.int64)
+    ln = np.zeros(P, dtype=np.int64)
+    stride = C.c_int64(0)
+    rc = _load().btard_oracle_partition_layout(C.c_int64(int(d)), C.c_int32(P), C.c_int32(mode),
+                                               C.c_int32(align_elems), _p(off, C.c_int64),
+                                               _p(ln, C.c_int64), C.byref(stride))
+    if rc:
+        raise ValueError("partition_layout: invalid argument")
+    return off, ln, int(stride.value)
+
+
+def _as_g(g):
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    if g.ndim == 2:
+        g = g[None]
+    assert g.ndim == 3, "g must be [P][n][stride]"
+    return g
+
+
+def _per_part(x, P, dtype):
+    a = np.ascontiguousarray(np.broadcast_to(np.asarray(x, dtype=dtype), (P,)))
+    return a
+
+
+def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v0=None, stop_mode=STOP_FIXED,
+                  max_iters=1, eps=0.0):
+    """Batched CenteredClip.  g: [P][n][stride] fp32 (or [n][stride]).
+
+    Returns dict(v [P][stride] f64, resid_norm [P][n], iters [P], last_step_norm [P], status [P]).
+    """
+    g = _as_g(g)
+    P, n, stride = g.shape
+    ln = _per_part(stride if part_len is None else part_len, P, np.int64)
+    tau = _per_part(tau, P, np.float64)
+    if v0 is not None:
+        v0 = np.ascontiguousarray(v0, dtype=np.float32).reshape(P, stride)
+    v = np.zeros((P, stride), dtype=np.float64)
+    rn = np.zeros((P, n), dtype=np.float64)
+    it = np.zeros(P, dtype=np.int32)
+    ls = np.zeros(P, dtype=np.float64)
+    st = np.zeros(P, dtype=np.uint32)
+    rc = _load().btard_oracle_centered_clip(
+        _p(g, C.c_float), C.c_int32(n), C.c_int32(P), C.c_int64(stride), _p(ln, C.c_int64),
+        _p(tau, C.c_double), C.c_int32(init_mode), _p(v0, C.c_float), C.c_int32(stop_mode),
+        C.c_int32(max_iters), C.c_double(eps), _p(v, C.c_double), _p(rn, C.c_double),
+        _p(it, C.c_int32), _p(ls, C.c_double), _p(st, C.c_uint32))
+    if rc:
+        raise ValueError("centered_clip: invalid argument")
+    return dict(v=v, resid_norm=rn, iters=it, last_step_norm=ls, status=st)
+
+
+def verify(g, v, tau, seed, K=1, part_len=None, norm_in=None, want_resid_sum=False,
+           first_partition=0):
+    """Batched verification metadata.  v: [P][stride] fp32 (the vector a peer received).
+
+    ``first_partition`` shifts the partition index that keys the z stream, so that a
+    slab cut out of a larger tensor is verified with the z of its true position.
+    """
+    g = _as_g(g)
+    P, n, stride = g.shape
+    v = np.ascontiguousarray(v, dtype=np.float32).reshape(P, stride)
+    ln = _per_part(stride if part_len is None else part_len, P, np.int64)
+    tau = _per_part(tau, P, np.float64)
+    if norm_in is not None:
+        norm_in = np.ascontiguousarray(norm_in, dtype=np.float64).reshape(P, n)
+    out = dict(norm=np.zeros((P, n)), weight=np.zeros((P, n)), dot=np.zeros((P, n, K)),
+               s=np.zeros((P, n, K)), s_sum=np.zeros((P, K)), znorm2=np.zeros((P, K)),
+               resid_sum_norm=np.zeros(P), status=np.zeros(P, dtype=np.uint32))
+    rs = np.zeros((P, stride)) if want_resid_sum else None
+    lib = _load()
+    if first_partition == 0:
+        rc = lib.btard_oracle_verify(
+            _p(g, C.c_float), C.c_int32(n), C.c_int32(P), C.c_int64(stride), _p(ln, C.c_int64),
+            _p(v, C.c_float), _p(tau, C.c_double), C.c_uint64(int(seed)), C.c_int32(K),
+            _p(norm_in, C.c_double), _p(out["norm"], C.c_double), _p(out["weight"], C.c_double),
+            _p(out["dot"], C.c_double), _p(out["s"], C.c_double), _p(out["s_sum"], C.c_double),
+            _p(out["znorm2"], C.c_double), _p(out["resid_sum_norm"], C.c_double),
+            _p(rs, C.c_double), _p(out["status"], C.c_uint32))
+        if rc:
+            raise ValueError("verify: invalid argument")
+    else:
+        for p in range(P):
+            rsn = C.c_double(0.0)
+            stt = C.c_uint32(0)
+            rc = lib.btard_oracle_verify_one(
+                _p(g[p], C.c_float), C.c_int32(n), C.c_int64(stride), C.c_int64(int(ln[p])),
+                _p(v[p], C.c_float), C.c_double(float(tau[p])), C.c_uint64(int(seed)),
+                C.c_int32(first_partition + p), C.c_int32(K),
+                _p(norm_in[p], C.c_double) if norm_in is not None else None,
+                _p(out["norm"][p], C.c_double), _p(out["weight"][p], C.c_double),
+                _p(out["dot"][p], C.c_double), _p(out["s"][p], C.c_double),
+                _p(out["s_sum"][p], C.c_double), _p(out["znorm2"][p], C.c_double),
+                C.byref(rsn), _p(rs[p], C.c_double) if rs is not None else None, C.byref(stt))
+            if rc:
+                raise ValueError("verify: invalid argument")
+            out["resid_sum_norm"][p] = rsn.value
+            out["status"][p] = stt.value
+    if rs is not None:
+        out["resid_sum"] = rs
+    return out
