@@ -1,0 +1,214 @@
+/*
+ * btard.h — C ABI of the batched CenteredClip + verification library for one NVIDIA B200.
+ *
+ * The library implements the arithmetic core of Byzantine-Tolerant All-Reduce (BTARD,
+ * arXiv 2106.11257): the robust aggregation that replaces averaging in ButterflyClip
+ * (Alg. 2, line 5) and the metadata of Verifications 1-2 (Alg. 6).  The n peers are rows of
+ * one tensor in device memory; the P butterfly partitions are slabs of that tensor.
+ *
+ * Conventions
+ *   - Tensor layout: g is [P][n][row_stride] float32, v is [P][row_stride] float32, both in
+ *     device memory, 16-byte aligned, row_stride a multiple of 4.  Row i of slab p is peer i's
+ *     part p.  Only the first part_len[p] columns of slab p are data; what lies beyond is ignored
+ *     on input and written as 0 in v.
+ *   - Every pointer marked "device" is owned by the caller and must stay valid until the work
+ *     queued on `stream` has finished.  Pointers marked "host" are read before the call returns.
+ *   - Calls that take device buffers are asynchronous on `stream` (a cudaStream_t passed as
+ *     void*; NULL is the default stream), allocate nothing and never synchronise with the host.
+ *     Scratch memory comes from `workspace`, sized by the matching *_workspace() query.
+ *   - Return value: BTARD_OK, or a negative error; on error nothing was queued.  Conditions that
+ *     only the device can see are reported per partition in `status` (BTARD_STATUS_* bits).
+ */
+#ifndef BTARD_H_
+#define BTARD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BTARD_API __attribute__((visibility("default")))
+#else
+#define BTARD_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BTARD_OK 0
+#define BTARD_ERR_INVALID_ARG (-1)      /* NULL pointer, size out of range, tau < 0 or NaN ...   */
+#define BTARD_ERR_BAD_ALIGNMENT (-2)    /* pointer not 16-byte aligned / row_stride % 4 != 0      */
+#define BTARD_ERR_WORKSPACE_TOO_SMALL (-3)
+#define BTARD_ERR_CUDA (-4)             /* a CUDA call failed; see btard_last_cuda_error()        */
+#define BTARD_ERR_UNSUPPORTED (-5)      /* e.g. n_peers > BTARD_MAX_PEERS                          */
+
+#define BTARD_MAX_PEERS 256
+#define BTARD_MAX_Z 64
+
+#define BTARD_SPLIT_PAPER 0     /* first d mod P parts have ceil(d/P) entries, the rest floor(d/P)  */
+#define BTARD_SPLIT_CEIL_PAD 1  /* every part ceil(d/P) until d runs out; the tail part is short   */
+
+#define BTARD_INIT_CALLER_V0 0      /* v holds v^0 on entry                                         */
+#define BTARD_INIT_ZERO 1
+#define BTARD_INIT_MEAN 2
+#define BTARD_INIT_COORD_MEDIAN 3   /* coordinate-wise median of the n rows                         */
+
+#define BTARD_ALGO_DIRECT 0         /* one pass over g per iteration                                */
+#define BTARD_ALGO_GRAM 1           /* Gram matrix pass + iteration in coefficient space + combine  */
+
+#define BTARD_STOP_FIXED_ITERS 0    /* exactly max_iters updates                                    */
+#define BTARD_STOP_EPS 1            /* stop once ||v^{l+1} - v^l||_2 <= eps, at most max_iters       */
+
+#define BTARD_STATUS_NOT_CONVERGED 1u   /* EPS mode: max_iters reached with the last step > eps     */
+#define BTARD_STATUS_NONFINITE_ROW 2u   /* a row with non-finite residual norm got weight 0         */
+
+/*
+ * Split(v, n) of App. D.1 ("Basic building blocks"): offsets and lengths of the P parts of a
+ * vector of d coordinates, and the padded row length used to store one part.
+ * Host only, pure, no CUDA.  part_offset, part_len: host arrays of P entries (out).
+ * row_stride (out) = longest part rounded up to a multiple of align_elems (a multiple of 4).
+ * Errors: INVALID_ARG for d < 0, P < 1, unknown mode, align_elems < 4 or not a multiple of 4.
+ */
+BTARD_API int btard_partition_layout(int64_t d, int32_t P, int32_t mode, int32_t align_elems,
+                           int64_t* part_offset, int64_t* part_len, int64_t* row_stride);
+
+/*
+ * CenteredClip, App. D.2 eq. (CenteredClip), on all P partitions at once:
+ *     v^{l+1} = v^l + (1/n) sum_i (x_i - v^l) min{1, tau / ||x_i - v^l||_2},   x_i = g[p][i][:].
+ * A row whose residual norm is not finite takes weight 0 and is left out of the sum.
+ */
+typedef struct {
+    int32_t n_peers;             /* n, 1..BTARD_MAX_PEERS                                           */
+    int32_t n_partitions;        /* P >= 1                                                          */
+    int64_t row_stride;          /* elements, multiple of 4                                         */
+    const int64_t* part_len;     /* host [P], 0 <= part_len[p] <= row_stride                        */
+    const float* g;              /* device [P][n][row_stride], read only                            */
+    const double* tau;           /* host [P], clip radius per partition; >= 0, +inf allowed         */
+    int32_t init_mode;           /* BTARD_INIT_*                                                    */
+    int32_t algo;                /* BTARD_ALGO_*                                                    */
+    int32_t stop_mode;           /* BTARD_STOP_*                                                    */
+    int32_t max_iters;           /* >= 1                                                            */
+    double eps;                  /* used in EPS mode, >= 0                                          */
+    float* v;                    /* device [P][row_stride]; in: v^0 if CALLER_V0; out: result       */
+    int32_t* iters;              /* device [P] out: updates applied                                 */
+    double* last_step_norm;      /* device [P] out: ||v^{I} - v^{I-1}||_2                           */
+    double* resid_norm;          /* device [P][n] out: ||x_i - v||_2 at the returned v              */
+    uint32_t* status;            /* device [P] out: BTARD_STATUS_* bits                             */
+    void* workspace;             /* device, 256-byte aligned                                        */
+    size_t workspace_bytes;
+    void* stream;                /* cudaStream_t                                                    */
+} btard_cclip_args;
+
+/* Bytes of workspace btard_centered_clip needs for these arguments (0 on invalid arguments).
+   Reads only the sizes and modes, no pointer. */
+BTARD_API size_t btard_centered_clip_workspace(const btard_cclip_args* args);
+BTARD_API int btard_centered_clip(const btard_cclip_args* args);
+
+/*
+ * Verification metadata, Sec. 3.1 eq. (2) and Alg. 6 lines 6-14, for all partitions:
+ *     norm_i = ||g_i - v||_2,  w_i = min{1, tau/norm_i},
+ *     dot_ik = <g_i - v, z_k>  with z_k = GetRandomVector(seed) restricted to partition p, unnormalised,
+ *     s_ik   = w_i dot_ik / ||z_k||_2   (the paper's s_i^j = <z[j], Delta_i^j>),
+ *     s_sum_k = sum_i s_ik,  resid_sum = sum_i w_i (g_i - v)   (both ~ 0 at the fixed point, eq. (1)).
+ * z_k for partition p is keyed by (seed, partition_base + p, k); see btard_random_vector.
+ */
+typedef struct {
+    int32_t n_peers;
+    int32_t n_partitions;
+    int64_t row_stride;
+    const int64_t* part_len;     /* host [P]                                                        */
+    const float* g;              /* device [P][n][row_stride]                                       */
+    const float* v;              /* device [P][row_stride]: the aggregate as a peer received it     */
+    const double* tau;           /* host [P]                                                        */
+    uint64_t seed;               /* shared seed r (output of the multi-party generator)             */
+    int32_t n_z;                 /* K, 1..BTARD_MAX_Z random vectors per partition                  */
+    int32_t partition_base;      /* global index of slab 0 (0 unless the tensor is a shard)         */
+    const double* resid_norm_in; /* device [P][n] norms at v (e.g. from btard_centered_clip) or NULL:
+                                    NULL costs one more pass over g                                 */
+    double* norm;                /* device [P][n] out                                               */
+    double* weight;              /* device [P][n] out                                               */
+    double* dot;                 /* device [P][n][K] out                                            */
+    double* s;                   /* device [P][n][K] out                                            */
+    double* s_sum;               /* device [P][K] out                                               */
+    double* znorm2;              /* device [P][K] out: ||z_k||_2^2 over the part_len[p] coordinates */
+    double* resid_sum_norm;      /* device [P] out: ||sum_i w_i (g_i - v)||_2                       */
+    float* resid_sum;            /* device [P][row_stride] out, or NULL                             */
+    uint32_t* status;            /* device [P] out                                                  */
+    void* workspace;
+    size_t workspace_bytes;
+    void* stream;
+} btard_verify_args;
+
+BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* args);
+BTARD_API int btard_verify_projections(const btard_verify_args* args);
+
+/*
+ * GetRandomVector (Alg. 6 line 5) made visible: writes the unnormalised float32 coordinates
+ * z_k[0 .. part_len) of partition p to device memory (z_out, 16-byte aligned, room for
+ * part_len rounded up to a multiple of 4).  Coordinates 4q..4q+3 are the Box-Muller images of the
+ * four words of Philox4x32-10 with counter (q, p, k, 0x42544152) and key (seed low, seed high).
+ * Bit-exact against the CPU oracle.  Asynchronous on `stream`.
+ */
+BTARD_API int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t part_len, float* z_out,
+                        void* stream);
+
+/*
+ * The same aggregation + verification with HOST buffers: copies g to the device, runs
+ * btard_centered_clip (DIRECT) and btard_verify_projections, copies the results back and waits for
+ * `stream`.  All device memory comes from device_scratch (sized by btard_aggregate_host_scratch).
+ * Host output pointers may be NULL to skip that copy, except v.  Pinned host memory makes the
+ * copies asynchronous and fast; pageable memory works too.
+ */
+typedef struct {
+    int32_t n_peers;
+    int32_t n_partitions;
+    int64_t row_stride;
+    const int64_t* part_len;     /* host [P] */
+    const double* tau;           /* host [P] */
+    const float* g;              /* HOST [P][n][row_stride] */
+    int32_t init_mode;           /* CALLER_V0: v holds v^0 on entry */
+    int32_t stop_mode;
+    int32_t max_iters;
+    double eps;
+    uint64_t seed;
+    int32_t n_z;
+    float* v;                    /* HOST [P][row_stride] out (in for CALLER_V0) */
+    int32_t* iters;              /* HOST [P] out */
+    double* last_step_norm;      /* HOST [P] out */
+    double* norm;                /* HOST [P][n] out */
+    double* weight;              /* HOST [P][n] out */
+    double* dot;                 /* HOST [P][n][K] out */
+    double* s;                   /* HOST [P][n][K] out */
+    double* s_sum;               /* HOST [P][K] out */
+    double* znorm2;              /* HOST [P][K] out */
+    double* resid_sum_norm;      /* HOST [P] out */
+    uint32_t* status;            /* HOST [P] out: OR of the two calls' status words */
+    void* device_scratch;        /* device, 256-byte aligned */
+    size_t device_scratch_bytes;
+    void* stream;
+} btard_host_args;
+
+BTARD_API size_t btard_aggregate_host_scratch(const btard_host_args* args);
+BTARD_API int btard_aggregate_host(const btard_host_args* args);
+
+/* The cudaError_t (as int) of the last failed CUDA call made by this thread inside the library. */
+BTARD_API int btard_last_cuda_error(void);
+
+/*
+ * Optional per-kernel timing for benchmarks (no counterpart in the paper).  While enabled, every
+ * streaming kernel the library launches is bracketed by CUDA events on the caller's stream.
+ * btard_profile_collect waits for the recorded events, adds up elapsed milliseconds and launch counts
+ * per kernel kind into total_ms[kind] / launches[kind] (host arrays of n_kinds >= 5 entries:
+ * 0 median start, 1 init pass, 2 CenteredClip iteration pass, 3 verification pass, 4 other) and
+ * forgets them.  Process-wide state; not meant for concurrent use from several threads.
+ */
+BTARD_API void btard_profile_enable(int on);
+BTARD_API int btard_profile_collect(double* total_ms, int64_t* launches, int32_t n_kinds);
+
+/* Number of kernels the library has launched from this process so far (for accounting). */
+BTARD_API int64_t btard_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BTARD_H_ */

@@ -1,0 +1,317 @@
+"""ctypes binding of libbtard.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch tensors (device memory and streams are torch's); every step of the computation
+runs in the library's kernels.  Missing library => ImportError-like failure at first use, never a
+fallback.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
+ALGO_DIRECT, ALGO_GRAM = 0, 1
+STOP_FIXED_ITERS, STOP_EPS = 0, 1
+SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1
+STATUS_NOT_CONVERGED, STATUS_NONFINITE_ROW = 1, 2
+
+EXPORTS = [
+    "btard_partition_layout", "btard_centered_clip_workspace", "btard_centered_clip",
+    "btard_verify_projections_workspace", "btard_verify_projections", "btard_random_vector",
+    "btard_aggregate_host_scratch", "btard_aggregate_host", "btard_last_cuda_error",
+    "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
+]
+
+_ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
+           -4: "CUDA error", -5: "unsupported"}
+
+
+class BtardError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        extra = ""
+        if code == -4:
+            extra = " (cudaError %d)" % lib().btard_last_cuda_error()
+        super().__init__("%s: %s%s" % (where, _ERRORS.get(code, "error %d" % code), extra))
+
+
+class CclipArgs(C.Structure):
+    _fields_ = [("n_peers", C.c_int32), ("n_partitions", C.c_int32), ("row_stride", C.c_int64),
+                ("part_len", C.c_void_p), ("g", C.c_void_p), ("tau", C.c_void_p),
+                ("init_mode", C.c_int32), ("algo", C.c_int32), ("stop_mode", C.c_int32),
+                ("max_iters", C.c_int32), ("eps", C.c_double), ("v", C.c_void_p),
+                ("iters", C.c_void_p), ("last_step_norm", C.c_void_p), ("resid_norm", C.c_void_p),
+                ("status", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("stream", C.c_void_p)]
+
+
+class VerifyArgs(C.Structure):
+    _fields_ = [("n_peers", C.c_int32), ("n_partitions", C.c_int32), ("row_stride", C.c_int64),
+                ("part_len", C.c_void_p), ("g", C.c_void_p), ("v", C.c_void_p), ("tau", C.c_void_p),
+                ("seed", C.c_uint64), ("n_z", C.c_int32), ("partition_base", C.c_int32),
+                ("resid_norm_in", C.c_void_p), ("norm", C.c_void_p), ("weight", C.c_void_p),
+                ("dot", C.c_void_p), ("s", C.c_void_p), ("s_sum", C.c_void_p),
+                ("znorm2", C.c_void_p), ("resid_sum_norm", C.c_void_p), ("resid_sum", C.c_void_p),
+                ("status", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("stream", C.c_void_p)]
+
+
+class HostArgs(C.Structure):
+    _fields_ = [("n_peers", C.c_int32), ("n_partitions", C.c_int32), ("row_stride", C.c_int64),
+                ("part_len", C.c_void_p), ("tau", C.c_void_p), ("g", C.c_void_p),
+                ("init_mode", C.c_int32), ("stop_mode", C.c_int32), ("max_iters", C.c_int32),
+                ("eps", C.c_double), ("seed", C.c_uint64), ("n_z", C.c_int32), ("v", C.c_void_p),
+                ("iters", C.c_void_p), ("last_step_norm", C.c_void_p), ("norm", C.c_void_p),
+                ("weight", C.c_void_p), ("dot", C.c_void_p), ("s", C.c_void_p),
+                ("s_sum", C.c_void_p), ("znorm2", C.c_void_p), ("resid_sum_norm", C.c_void_p),
+                ("status", C.c_void_p), ("device_scratch", C.c_void_p),
+                ("device_scratch_bytes", C.c_size_t), ("stream", C.c_void_p)]
+
+
+_lib = None
+
+
+def library_path():
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbtard.so")
+
+
+def lib():
+    """Loads libbtard.so (built by paper_2106_11257_b200/build.py); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise OSError("libbtard.so is not built: run `python -m paper_2106_11257_b200.build` "
+                          "(there is no CPU fallback)")
+        L = C.CDLL(path)
+        L.btard_partition_layout.restype = C.c_int
+        L.btard_partition_layout.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                             C.c_void_p, C.c_void_p, C.POINTER(C.c_int64)]
+        L.btard_centered_clip_workspace.restype = C.c_size_t
+        L.btard_centered_clip_workspace.argtypes = [C.POINTER(CclipArgs)]
+        L.btard_centered_clip.restype = C.c_int
+        L.btard_centered_clip.argtypes = [C.POINTER(CclipArgs)]
+        L.btard_verify_projections_workspace.restype = C.c_size_t
+        L.btard_verify_projections_workspace.argtypes = [C.POINTER(VerifyArgs)]
+        L.btard_verify_projections.restype = C.c_int
+        L.btard_verify_projections.argtypes = [C.POINTER(VerifyArgs)]
+        L.btard_random_vector.restype = C.c_int
+        L.btard_random_vector.argtypes = [C.c_uint64, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                          C.c_void_p]
+        L.btard_aggregate_host_scratch.restype = C.c_size_t
+        L.btard_aggregate_host_scratch.argtypes = [C.POINTER(HostArgs)]
+        L.btard_aggregate_host.restype = C.c_int
+        L.btard_aggregate_host.argtypes = [C.POINTER(HostArgs)]
+        L.btard_last_cuda_error.restype = C.c_int
+        L.btard_kernel_launch_count.restype = C.c_int64
+        L.btard_profile_enable.restype = None
+        L.btard_profile_enable.argtypes = [C.c_int]
+        L.btard_profile_collect.restype = C.c_int
+        L.btard_profile_collect.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+        _lib = L
+    return _lib
+
+
+def kernel_launch_count():
+    return int(lib().btard_kernel_launch_count())
+
+
+KERNEL_KINDS = ("median", "init", "iter", "verify", "other")
+
+
+def profile_enable(on):
+    lib().btard_profile_enable(1 if on else 0)
+
+
+def profile_collect():
+    """Returns {kind: (total_ms, launches)} for the kernels timed since the last call."""
+    ms = np.zeros(len(KERNEL_KINDS), dtype=np.float64)
+    cnt = np.zeros(len(KERNEL_KINDS), dtype=np.int64)
+    _check(lib().btard_profile_collect(ms.ctypes.data, cnt.ctypes.data, len(KERNEL_KINDS)),
+           "btard_profile_collect")
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def last_cuda_error():
+    return int(lib().btard_last_cuda_error())
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise BtardError(rc, where)
+
+
+def partition_layout(d, P, mode=SPLIT_PAPER, align_elems=32):
+    """Host-only.  Returns (part_offset[P], part_len[P], row_stride)."""
+    off = np.zeros(P, dtype=np.int64)
+    ln = np.zeros(P, dtype=np.int64)
+    stride = C.c_int64(0)
+    _check(lib().btard_partition_layout(int(d), int(P), int(mode), int(align_elems),
+                                        off.ctypes.data, ln.ctypes.data, C.byref(stride)),
+           "btard_partition_layout")
+    return off, ln, int(stride.value)
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _stream_ptr(stream):
+    torch = _torch()
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _host_arr(x, P, dtype):
+    return np.ascontiguousarray(np.broadcast_to(np.asarray(x, dtype=dtype), (P,)))
+
+
+def centered_clip_workspace(n, P, row_stride, stop_mode=STOP_EPS):
+    a = CclipArgs(n_peers=n, n_partitions=P, row_stride=row_stride, stop_mode=stop_mode)
+    return int(lib().btard_centered_clip_workspace(C.byref(a)))
+
+
+def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v=None, stop_mode=STOP_FIXED_ITERS,
+                  max_iters=1, eps=0.0, algo=ALGO_DIRECT, workspace=None, out=None, stream=None):
+    """g: CUDA float32 [P][n][row_stride].  Returns dict of CUDA tensors
+    (v, iters, last_step_norm, resid_norm, status).  Asynchronous on the current stream."""
+    torch = _torch()
+    assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
+    P, n, stride = g.shape
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    tau_h = _host_arr(tau, P, np.float64)
+    dev = g.device
+    if v is None:
+        assert init_mode != INIT_CALLER_V0, "CALLER_V0 needs v"
+        v = torch.empty((P, stride), dtype=torch.float32, device=dev)
+    assert v.is_cuda and v.dtype == torch.float32 and v.is_contiguous() and v.numel() == P * stride
+    o = out if out is not None else dict(
+        iters=torch.empty(P, dtype=torch.int32, device=dev),
+        last_step_norm=torch.empty(P, dtype=torch.float64, device=dev),
+        resid_norm=torch.empty((P, n), dtype=torch.float64, device=dev),
+        status=torch.empty(P, dtype=torch.int32, device=dev))
+    need = centered_clip_workspace(n, P, stride, stop_mode)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    a = CclipArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
+                  g=g.data_ptr(), tau=tau_h.ctypes.data, init_mode=init_mode, algo=algo,
+                  stop_mode=stop_mode, max_iters=max_iters, eps=eps, v=v.data_ptr(),
+                  iters=o["iters"].data_ptr(), last_step_norm=o["last_step_norm"].data_ptr(),
+                  resid_norm=o["resid_norm"].data_ptr(), status=o["status"].data_ptr(),
+                  workspace=workspace.data_ptr(), workspace_bytes=workspace.numel(),
+                  stream=_stream_ptr(stream))
+    with torch.cuda.device(dev):
+        _check(lib().btard_centered_clip(C.byref(a)), "btard_centered_clip")
+    res = dict(o)
+    res["v"] = v
+    res["workspace"] = workspace
+    return res
+
+
+def verify_projections_workspace(n, P, row_stride, K):
+    a = VerifyArgs(n_peers=n, n_partitions=P, row_stride=row_stride, n_z=K)
+    return int(lib().btard_verify_projections_workspace(C.byref(a)))
+
+
+def verify_projections(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None, partition_base=0,
+                       want_resid_sum=False, workspace=None, out=None, stream=None):
+    """Returns dict of CUDA tensors: norm, weight [P][n]; dot, s [P][n][K]; s_sum, znorm2 [P][K];
+    resid_sum_norm [P]; status [P]; resid_sum [P][row_stride] if asked."""
+    torch = _torch()
+    assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
+    P, n, stride = g.shape
+    assert v.is_cuda and v.dtype == torch.float32 and v.is_contiguous() and v.numel() == P * stride
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    tau_h = _host_arr(tau, P, np.float64)
+    dev = g.device
+    f64 = dict(dtype=torch.float64, device=dev)
+    o = out if out is not None else dict(
+        norm=torch.empty((P, n), **f64), weight=torch.empty((P, n), **f64),
+        dot=torch.empty((P, n, K), **f64), s=torch.empty((P, n, K), **f64),
+        s_sum=torch.empty((P, K), **f64), znorm2=torch.empty((P, K), **f64),
+        resid_sum_norm=torch.empty(P, **f64), status=torch.empty(P, dtype=torch.int32, device=dev))
+    rs = None
+    if want_resid_sum:
+        rs = o.get("resid_sum")
+        if rs is None:
+            rs = torch.zeros((P, stride), dtype=torch.float32, device=dev)
+    need = verify_projections_workspace(n, P, stride, K)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if resid_norm_in is not None:
+        assert resid_norm_in.is_cuda and resid_norm_in.dtype == torch.float64 and resid_norm_in.is_contiguous()
+    a = VerifyArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
+                   g=g.data_ptr(), v=v.data_ptr(), tau=tau_h.ctypes.data, seed=int(seed), n_z=K,
+                   partition_base=partition_base,
+                   resid_norm_in=resid_norm_in.data_ptr() if resid_norm_in is not None else None,
+                   norm=o["norm"].data_ptr(), weight=o["weight"].data_ptr(), dot=o["dot"].data_ptr(),
+                   s=o["s"].data_ptr(), s_sum=o["s_sum"].data_ptr(), znorm2=o["znorm2"].data_ptr(),
+                   resid_sum_norm=o["resid_sum_norm"].data_ptr(),
+                   resid_sum=rs.data_ptr() if rs is not None else None, status=o["status"].data_ptr(),
+                   workspace=workspace.data_ptr(), workspace_bytes=workspace.numel(),
+                   stream=_stream_ptr(stream))
+    with torch.cuda.device(dev):
+        _check(lib().btard_verify_projections(C.byref(a)), "btard_verify_projections")
+    res = dict(o)
+    if rs is not None:
+        res["resid_sum"] = rs
+    res["workspace"] = workspace
+    return res
+
+
+def random_vector(seed, p, k, part_len, device="cuda", stream=None):
+    """Unnormalised fp32 z_k of partition p as a CUDA tensor of part_len entries."""
+    torch = _torch()
+    padded = (int(part_len) + 3) // 4 * 4
+    z = torch.zeros(max(padded, 4), dtype=torch.float32, device=device)
+    with torch.cuda.device(z.device):
+        _check(lib().btard_random_vector(int(seed), int(p), int(k), int(part_len), z.data_ptr(),
+                                         _stream_ptr(stream)), "btard_random_vector")
+    return z[:int(part_len)]
+
+
+def aggregate_host_scratch(n, P, row_stride, K):
+    a = HostArgs(n_peers=n, n_partitions=P, row_stride=row_stride, n_z=K)
+    return int(lib().btard_aggregate_host_scratch(C.byref(a)))
+
+
+def aggregate_host(g_host, tau, seed, K=1, part_len=None, init_mode=INIT_COORD_MEDIAN, v_host=None,
+                   stop_mode=STOP_FIXED_ITERS, max_iters=1, eps=0.0, scratch=None, out=None,
+                   device="cuda", stream=None):
+    """Whole aggregation + verification from HOST tensors (ideally pinned); blocks until done.
+    Returns dict of host tensors."""
+    torch = _torch()
+    assert not g_host.is_cuda and g_host.dtype == torch.float32 and g_host.dim() == 3 and g_host.is_contiguous()
+    P, n, stride = g_host.shape
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    tau_h = _host_arr(tau, P, np.float64)
+    pin = g_host.is_pinned()
+
+    def host(shape, dtype):
+        return torch.empty(shape, dtype=dtype, pin_memory=pin)
+    o = out if out is not None else dict(
+        v=v_host if v_host is not None else host((P, stride), torch.float32),
+        iters=host(P, torch.int32), last_step_norm=host(P, torch.float64),
+        norm=host((P, n), torch.float64), weight=host((P, n), torch.float64),
+        dot=host((P, n, K), torch.float64), s=host((P, n, K), torch.float64),
+        s_sum=host((P, K), torch.float64), znorm2=host((P, K), torch.float64),
+        resid_sum_norm=host(P, torch.float64), status=host(P, torch.int32))
+    need = aggregate_host_scratch(n, P, stride, K)
+    if scratch is None:
+        scratch = torch.empty(need, dtype=torch.uint8, device=device)
+    a = HostArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
+                 tau=tau_h.ctypes.data, g=g_host.data_ptr(), init_mode=init_mode,
+                 stop_mode=stop_mode, max_iters=max_iters, eps=eps, seed=int(seed), n_z=K,
+                 v=o["v"].data_ptr(), iters=o["iters"].data_ptr(),
+                 last_step_norm=o["last_step_norm"].data_ptr(), norm=o["norm"].data_ptr(),
+                 weight=o["weight"].data_ptr(), dot=o["dot"].data_ptr(), s=o["s"].data_ptr(),
+                 s_sum=o["s_sum"].data_ptr(), znorm2=o["znorm2"].data_ptr(),
+                 resid_sum_norm=o["resid_sum_norm"].data_ptr(), status=o["status"].data_ptr(),
+                 device_scratch=scratch.data_ptr(), device_scratch_bytes=scratch.numel(),
+                 stream=_stream_ptr(stream))
+    with torch.cuda.device(scratch.device):
+        _check(lib().btard_aggregate_host(C.byref(a)), "btard_aggregate_host")
+    res = dict(o)
+    res["scratch"] = scratch
+    return res

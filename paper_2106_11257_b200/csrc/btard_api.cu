@@ -1,0 +1,451 @@
+// C ABI entry points: argument validation, workspace carving and the sequence of launches.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "btard_common.h"
+
+namespace btard {
+
+static thread_local int g_last_cuda_error = 0;
+static std::atomic<long long> g_launches{0};
+
+void set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// ---- optional kernel timing ---------------------------------------------------------------------
+namespace {
+struct ProfRecord { int kind; cudaEvent_t a, b; };
+std::mutex g_prof_mu;
+bool g_prof_on = false;
+std::vector<ProfRecord> g_prof_records;
+std::vector<cudaEvent_t> g_prof_pool;
+cudaEvent_t g_prof_open = nullptr;
+
+cudaEvent_t prof_event()
+{
+    if (!g_prof_pool.empty()) { cudaEvent_t e = g_prof_pool.back(); g_prof_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return e;
+}
+}  // namespace
+
+void prof_begin(int kind, cudaStream_t st)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    if (!g_prof_on) return;
+    g_prof_open = prof_event();
+    if (g_prof_open) cudaEventRecord(g_prof_open, st);
+}
+
+void prof_end(int kind, cudaStream_t st)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    if (!g_prof_on || !g_prof_open) return;
+    cudaEvent_t b = prof_event();
+    if (!b) { g_prof_pool.push_back(g_prof_open); g_prof_open = nullptr; return; }
+    cudaEventRecord(b, st);
+    g_prof_records.push_back(ProfRecord{kind, g_prof_open, b});
+    g_prof_open = nullptr;
+}
+
+int sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+        (void)cudaGetLastError();
+        return 148;   // B200
+    }
+    return sms;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_common(int n, int P, long long stride, const int64_t* part_len, const double* tau)
+{
+    if (n < 1 || P < 1 || P > 65535 || stride < 4 || !part_len || !tau) return BTARD_ERR_INVALID_ARG;
+    if (n > BTARD_MAX_PEERS) return BTARD_ERR_UNSUPPORTED;
+    if (stride % 4 != 0) return BTARD_ERR_BAD_ALIGNMENT;
+    if (stride > (1LL << 33)) return BTARD_ERR_UNSUPPORTED;   // 32-bit Philox block index
+    for (int p = 0; p < P; ++p) {
+        if (part_len[p] < 0 || part_len[p] > stride) return BTARD_ERR_INVALID_ARG;
+        if (!(tau[p] >= 0.0)) return BTARD_ERR_INVALID_ARG;   // rejects NaN too
+    }
+    return BTARD_OK;
+}
+
+struct CclipWorkspace {
+    size_t table, part[2], done, v_lo, v_lo_bytes, total;
+};
+
+// EPS mode carries v as fp32 + a bf16 correction so that the stop test sees steps far below the
+// rounding of v; FIXED mode needs no such thing.
+CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, const Geometry& geo)
+{
+    CclipWorkspace w;
+    size_t off = 0;
+    w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
+    const size_t part_bytes = sizeof(double) * (size_t)P * geo.cpp * (n + 1);
+    w.part[0] = off; off = align_up(off + part_bytes, 256);
+    w.part[1] = off; off = align_up(off + part_bytes, 256);
+    w.done = off; off = align_up(off + sizeof(int) * P, 256);
+    w.v_lo_bytes = (stop_mode == BTARD_STOP_EPS) ? sizeof(unsigned short) * (size_t)P * stride : 0;
+    w.v_lo = off; off = align_up(off + w.v_lo_bytes, 256);
+    w.total = off;
+    return w;
+}
+
+struct VerifyWorkspace {
+    size_t table, part, norms, cpart, total;
+};
+
+VerifyWorkspace verify_ws_layout(int n, int P, const VerifyGeometry& vg, const Geometry& cg)
+{
+    VerifyWorkspace w;
+    size_t off = 0;
+    w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
+    w.part = off; off = align_up(off + sizeof(double) * (size_t)P * vg.g.cpp * vg.slots, 256);
+    w.norms = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
+    w.cpart = off; off = align_up(off + sizeof(double) * (size_t)P * cg.cpp * (n + 1), 256);
+    w.total = off;
+    return w;
+}
+
+int upload_table(PartEntry* dev, int P, const int64_t* part_len, const double* tau, cudaStream_t st)
+{
+    std::vector<PartEntry> host((size_t)P);
+    for (int p = 0; p < P; ++p) { host[p].len = part_len[p]; host[p].tau = tau[p]; }
+    // The source is pageable: the runtime stages it before returning, so `host` may go away.
+    BTARD_CUDA_TRY(cudaMemcpyAsync(dev, host.data(), sizeof(PartEntry) * P, cudaMemcpyHostToDevice, st));
+    return BTARD_OK;
+}
+
+}  // namespace
+}  // namespace btard
+
+using namespace btard;
+
+extern "C" {
+
+int btard_last_cuda_error(void) { return g_last_cuda_error; }
+int64_t btard_kernel_launch_count(void) { return (int64_t)g_launches.load(); }
+
+void btard_profile_enable(int on)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = (on != 0);
+}
+
+int btard_profile_collect(double* total_ms, int64_t* launches, int32_t n_kinds)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    if (!total_ms || !launches || n_kinds < KIND_COUNT) return BTARD_ERR_INVALID_ARG;
+    for (int i = 0; i < n_kinds; ++i) { total_ms[i] = 0.0; launches[i] = 0; }
+    int rc = BTARD_OK;
+    for (const ProfRecord& r : g_prof_records) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(r.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.a, r.b);
+        if (e != cudaSuccess) { set_cuda_error(e); rc = BTARD_ERR_CUDA; }
+        else { total_ms[r.kind] += ms; launches[r.kind] += 1; }
+        g_prof_pool.push_back(r.a);
+        g_prof_pool.push_back(r.b);
+    }
+    g_prof_records.clear();
+    return rc;
+}
+
+int btard_partition_layout(int64_t d, int32_t P, int32_t mode, int32_t align_elems,
+                           int64_t* part_offset, int64_t* part_len, int64_t* row_stride)
+{
+    if (d < 0 || P < 1 || align_elems < 4 || align_elems % 4 != 0) return BTARD_ERR_INVALID_ARG;
+    if (!part_offset || !part_len || !row_stride) return BTARD_ERR_INVALID_ARG;
+    if (mode != BTARD_SPLIT_PAPER && mode != BTARD_SPLIT_CEIL_PAD) return BTARD_ERR_INVALID_ARG;
+    const int64_t base = d / P, extra = d % P, big = base + (extra != 0);
+    int64_t at = 0, longest = 0;
+    for (int32_t j = 0; j < P; ++j) {
+        int64_t len;
+        if (mode == BTARD_SPLIT_PAPER) len = base + (j < extra ? 1 : 0);
+        else len = (d - at < big) ? d - at : big;
+        part_offset[j] = at;
+        part_len[j] = len;
+        at += len;
+        if (len > longest) longest = len;
+    }
+    if (longest == 0) longest = 1;
+    *row_stride = (longest + align_elems - 1) / align_elems * align_elems;
+    return BTARD_OK;
+}
+
+size_t btard_centered_clip_workspace(const btard_cclip_args* a)
+{
+    if (!a || a->n_peers < 1 || a->n_peers > BTARD_MAX_PEERS || a->n_partitions < 1 ||
+        a->row_stride < 4)
+        return 0;
+    const Geometry geo = cclip_geometry(a->n_peers, a->n_partitions, a->row_stride);
+    return cclip_ws_layout(a->n_peers, a->n_partitions, a->row_stride, a->stop_mode, geo).total;
+}
+
+int btard_centered_clip(const btard_cclip_args* a)
+{
+    if (!a) return BTARD_ERR_INVALID_ARG;
+    int rc = check_common(a->n_peers, a->n_partitions, a->row_stride, a->part_len, a->tau);
+    if (rc != BTARD_OK) return rc;
+    if (!a->g || !a->v || !a->iters || !a->last_step_norm || !a->resid_norm || !a->status ||
+        !a->workspace)
+        return BTARD_ERR_INVALID_ARG;
+    if (a->max_iters < 1 || !(a->eps >= 0.0)) return BTARD_ERR_INVALID_ARG;
+    if (a->init_mode < BTARD_INIT_CALLER_V0 || a->init_mode > BTARD_INIT_COORD_MEDIAN)
+        return BTARD_ERR_INVALID_ARG;
+    if (a->stop_mode != BTARD_STOP_FIXED_ITERS && a->stop_mode != BTARD_STOP_EPS)
+        return BTARD_ERR_INVALID_ARG;
+    if (a->algo != BTARD_ALGO_DIRECT) return BTARD_ERR_UNSUPPORTED;
+    if (!aligned16(a->g) || !aligned16(a->v) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
+        return BTARD_ERR_BAD_ALIGNMENT;
+
+    const int n = a->n_peers, P = a->n_partitions;
+    const Geometry geo = cclip_geometry(n, P, a->row_stride);
+    const CclipWorkspace ws = cclip_ws_layout(n, P, a->row_stride, a->stop_mode, geo);
+    if (a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)a->stream;
+    char* base = (char*)a->workspace;
+
+    CclipLaunch L{};
+    L.g = a->g; L.v = a->v;
+    L.table = (const PartEntry*)(base + ws.table);
+    L.done = (int*)(base + ws.done);
+    L.iters = a->iters; L.last_step = a->last_step_norm; L.resid_norm = a->resid_norm;
+    L.status = a->status;
+    L.stride = a->row_stride; L.n = n; L.P = P;
+    L.stop_mode = a->stop_mode; L.max_iters = a->max_iters; L.eps2 = a->eps * a->eps;
+    double* part[2] = {(double*)(base + ws.part[0]), (double*)(base + ws.part[1])};
+
+    rc = upload_table((PartEntry*)(base + ws.table), P, a->part_len, a->tau, st);
+    if (rc != BTARD_OK) return rc;
+    if (ws.v_lo_bytes) {
+        L.v_lo = (unsigned short*)(base + ws.v_lo);
+        BTARD_CUDA_TRY(cudaMemsetAsync(L.v_lo, 0, ws.v_lo_bytes, st));
+    }
+
+    // Init pass: v^0 and the residual norms at v^0 (slot buffer 0).
+    L.init_mode = a->init_mode;
+    if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
+        rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
+        if (rc != BTARD_OK) return rc;
+        L.init_mode = BTARD_INIT_CALLER_V0;
+    }
+    L.part_in = nullptr; L.part_out = part[0]; L.l = 0;
+    rc = launch_cclip_pass(L, geo, PASS_INIT, st);
+    if (rc != BTARD_OK) return rc;
+
+    // Update l reads the slots of buffer l % 2 and writes buffer (l + 1) % 2.
+    for (int l = 0; l < a->max_iters; ++l) {
+        L.l = l; L.part_in = part[l & 1]; L.part_out = part[(l + 1) & 1];
+        rc = launch_cclip_pass(L, geo, PASS_ITER, st);
+        if (rc != BTARD_OK) return rc;
+    }
+    L.part_in = part[a->max_iters & 1];
+    return launch_cclip_finalize(L, geo, st);
+}
+
+size_t btard_verify_projections_workspace(const btard_verify_args* a)
+{
+    if (!a || a->n_peers < 1 || a->n_peers > BTARD_MAX_PEERS || a->n_partitions < 1 ||
+        a->row_stride < 4 || a->n_z < 1)
+        return 0;
+    const VerifyGeometry vg = verify_geometry(a->n_peers, a->n_partitions, a->row_stride, a->n_z);
+    const Geometry cg = cclip_geometry(a->n_peers, a->n_partitions, a->row_stride);
+    return verify_ws_layout(a->n_peers, a->n_partitions, vg, cg).total;
+}
+
+int btard_verify_projections(const btard_verify_args* a)
+{
+    if (!a) return BTARD_ERR_INVALID_ARG;
+    int rc = check_common(a->n_peers, a->n_partitions, a->row_stride, a->part_len, a->tau);
+    if (rc != BTARD_OK) return rc;
+    if (!a->g || !a->v || !a->norm || !a->weight || !a->dot || !a->s || !a->s_sum || !a->znorm2 ||
+        !a->resid_sum_norm || !a->status || !a->workspace)
+        return BTARD_ERR_INVALID_ARG;
+    if (a->n_z < 1 || a->n_z > BTARD_MAX_Z || a->partition_base < 0) return BTARD_ERR_INVALID_ARG;
+    if (!aligned16(a->g) || !aligned16(a->v) || (a->resid_sum && !aligned16(a->resid_sum)) ||
+        (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
+        return BTARD_ERR_BAD_ALIGNMENT;
+
+    const int n = a->n_peers, P = a->n_partitions, K = a->n_z;
+    const VerifyGeometry vg = verify_geometry(n, P, a->row_stride, K);
+    const Geometry cg = cclip_geometry(n, P, a->row_stride);
+    const VerifyWorkspace ws = verify_ws_layout(n, P, vg, cg);
+    if (a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)a->stream;
+    char* base = (char*)a->workspace;
+    PartEntry* table = (PartEntry*)(base + ws.table);
+    rc = upload_table(table, P, a->part_len, a->tau, st);
+    if (rc != BTARD_OK) return rc;
+
+    const double* norms = a->resid_norm_in;
+    if (!norms) {   // one more pass: residual norms at v
+        CclipLaunch L{};
+        L.g = a->g; L.v = const_cast<float*>(a->v); L.table = table;
+        L.part_out = (double*)(base + ws.cpart);
+        L.stride = a->row_stride; L.n = n; L.P = P;
+        rc = launch_cclip_pass(L, cg, PASS_NORMS, st);
+        if (rc != BTARD_OK) return rc;
+        rc = launch_partials_to_norms(L.part_out, (double*)(base + ws.norms), n, P, cg.cpp, st);
+        if (rc != BTARD_OK) return rc;
+        norms = (const double*)(base + ws.norms);
+    }
+
+    VerifyLaunch V{};
+    V.g = a->g; V.v = a->v; V.table = table; V.norm_in = norms;
+    V.part_out = (double*)(base + ws.part);
+    V.resid_sum = a->resid_sum;
+    V.norm = a->norm; V.weight = a->weight; V.dot = a->dot; V.s = a->s; V.s_sum = a->s_sum;
+    V.znorm2 = a->znorm2; V.resid_sum_norm = a->resid_sum_norm; V.status = a->status;
+    V.stride = a->row_stride; V.n = n; V.P = P; V.K = K; V.p_base = a->partition_base;
+    V.seed_lo = (uint32_t)a->seed; V.seed_hi = (uint32_t)(a->seed >> 32);
+    for (int k0 = 0; k0 < K; k0 += vg.KT) {
+        V.k0 = k0;
+        V.kc = (K - k0 < vg.KT) ? K - k0 : vg.KT;
+        rc = launch_verify(V, vg, st);
+        if (rc != BTARD_OK) return rc;
+    }
+    return BTARD_OK;
+}
+
+int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t part_len, float* z_out,
+                        void* stream)
+{
+    if (p < 0 || k < 0 || part_len < 0 || (part_len > 0 && !z_out)) return BTARD_ERR_INVALID_ARG;
+    if (part_len > (1LL << 33)) return BTARD_ERR_UNSUPPORTED;
+    if (!aligned16(z_out)) return BTARD_ERR_BAD_ALIGNMENT;
+    return launch_random_vector(seed, p, k, part_len, z_out, (cudaStream_t)stream);
+}
+
+// ---- host-buffer path ---------------------------------------------------------------------------
+namespace {
+struct HostScratch {
+    size_t g, v, iters, last_step, resid_norm, status_c, status_v, norm, weight, dot, s, s_sum,
+        znorm2, rsn, ws_c, ws_v, total;
+    size_t ws_c_bytes, ws_v_bytes;
+};
+
+HostScratch host_layout(const btard_host_args* a)
+{
+    HostScratch h{};
+    const size_t n = a->n_peers, P = a->n_partitions, S = (size_t)a->row_stride, K = a->n_z;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes, 256); return at; };
+    h.g = take(sizeof(float) * P * n * S);
+    h.v = take(sizeof(float) * P * S);
+    h.iters = take(sizeof(int32_t) * P);
+    h.last_step = take(sizeof(double) * P);
+    h.resid_norm = take(sizeof(double) * P * n);
+    h.status_c = take(sizeof(uint32_t) * P);
+    h.status_v = take(sizeof(uint32_t) * P);
+    h.norm = take(sizeof(double) * P * n);
+    h.weight = take(sizeof(double) * P * n);
+    h.dot = take(sizeof(double) * P * n * K);
+    h.s = take(sizeof(double) * P * n * K);
+    h.s_sum = take(sizeof(double) * P * K);
+    h.znorm2 = take(sizeof(double) * P * K);
+    h.rsn = take(sizeof(double) * P);
+    btard_cclip_args ca{};
+    ca.n_peers = a->n_peers; ca.n_partitions = a->n_partitions; ca.row_stride = a->row_stride;
+    ca.stop_mode = BTARD_STOP_EPS;   // the larger of the two layouts
+    h.ws_c_bytes = btard_centered_clip_workspace(&ca);
+    btard_verify_args va{};
+    va.n_peers = a->n_peers; va.n_partitions = a->n_partitions; va.row_stride = a->row_stride;
+    va.n_z = a->n_z;
+    h.ws_v_bytes = btard_verify_projections_workspace(&va);
+    h.ws_c = take(h.ws_c_bytes);
+    h.ws_v = take(h.ws_v_bytes);
+    h.total = off;
+    return h;
+}
+
+bool host_sizes_ok(const btard_host_args* a)
+{
+    return a && a->n_peers >= 1 && a->n_peers <= BTARD_MAX_PEERS && a->n_partitions >= 1 &&
+           a->row_stride >= 4 && a->n_z >= 1 && a->n_z <= BTARD_MAX_Z;
+}
+}  // namespace
+
+size_t btard_aggregate_host_scratch(const btard_host_args* a)
+{
+    if (!host_sizes_ok(a)) return 0;
+    return host_layout(a).total;
+}
+
+int btard_aggregate_host(const btard_host_args* a)
+{
+    if (!host_sizes_ok(a) || !a->g || !a->v || !a->device_scratch) return BTARD_ERR_INVALID_ARG;
+    int rc = check_common(a->n_peers, a->n_partitions, a->row_stride, a->part_len, a->tau);
+    if (rc != BTARD_OK) return rc;
+    if (reinterpret_cast<uintptr_t>(a->device_scratch) & 255u) return BTARD_ERR_BAD_ALIGNMENT;
+    const HostScratch h = host_layout(a);
+    if (a->device_scratch_bytes < h.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)a->stream;
+    char* base = (char*)a->device_scratch;
+    const size_t n = a->n_peers, P = a->n_partitions, S = (size_t)a->row_stride, K = a->n_z;
+
+    BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.g, a->g, sizeof(float) * P * n * S, cudaMemcpyHostToDevice, st));
+    if (a->init_mode == BTARD_INIT_CALLER_V0)
+        BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.v, a->v, sizeof(float) * P * S, cudaMemcpyHostToDevice, st));
+
+    btard_cclip_args ca{};
+    ca.n_peers = a->n_peers; ca.n_partitions = a->n_partitions; ca.row_stride = a->row_stride;
+    ca.part_len = a->part_len; ca.g = (const float*)(base + h.g); ca.tau = a->tau;
+    ca.init_mode = a->init_mode; ca.algo = BTARD_ALGO_DIRECT; ca.stop_mode = a->stop_mode;
+    ca.max_iters = a->max_iters; ca.eps = a->eps; ca.v = (float*)(base + h.v);
+    ca.iters = (int32_t*)(base + h.iters); ca.last_step_norm = (double*)(base + h.last_step);
+    ca.resid_norm = (double*)(base + h.resid_norm); ca.status = (uint32_t*)(base + h.status_c);
+    ca.workspace = base + h.ws_c; ca.workspace_bytes = h.ws_c_bytes; ca.stream = a->stream;
+    rc = btard_centered_clip(&ca);
+    if (rc != BTARD_OK) return rc;
+
+    btard_verify_args va{};
+    va.n_peers = a->n_peers; va.n_partitions = a->n_partitions; va.row_stride = a->row_stride;
+    va.part_len = a->part_len; va.g = ca.g; va.v = ca.v; va.tau = a->tau; va.seed = a->seed;
+    va.n_z = a->n_z; va.partition_base = 0; va.resid_norm_in = ca.resid_norm;
+    va.norm = (double*)(base + h.norm); va.weight = (double*)(base + h.weight);
+    va.dot = (double*)(base + h.dot); va.s = (double*)(base + h.s);
+    va.s_sum = (double*)(base + h.s_sum); va.znorm2 = (double*)(base + h.znorm2);
+    va.resid_sum_norm = (double*)(base + h.rsn); va.resid_sum = nullptr;
+    va.status = (uint32_t*)(base + h.status_v);
+    va.workspace = base + h.ws_v; va.workspace_bytes = h.ws_v_bytes; va.stream = a->stream;
+    rc = btard_verify_projections(&va);
+    if (rc != BTARD_OK) return rc;
+
+    auto back = [&](void* dst, size_t off, size_t bytes) -> cudaError_t {
+        if (!dst) return cudaSuccess;
+        return cudaMemcpyAsync(dst, base + off, bytes, cudaMemcpyDeviceToHost, st);
+    };
+    BTARD_CUDA_TRY(back(a->v, h.v, sizeof(float) * P * S));
+    BTARD_CUDA_TRY(back(a->iters, h.iters, sizeof(int32_t) * P));
+    BTARD_CUDA_TRY(back(a->last_step_norm, h.last_step, sizeof(double) * P));
+    BTARD_CUDA_TRY(back(a->norm, h.norm, sizeof(double) * P * n));
+    BTARD_CUDA_TRY(back(a->weight, h.weight, sizeof(double) * P * n));
+    BTARD_CUDA_TRY(back(a->dot, h.dot, sizeof(double) * P * n * K));
+    BTARD_CUDA_TRY(back(a->s, h.s, sizeof(double) * P * n * K));
+    BTARD_CUDA_TRY(back(a->s_sum, h.s_sum, sizeof(double) * P * K));
+    BTARD_CUDA_TRY(back(a->znorm2, h.znorm2, sizeof(double) * P * K));
+    BTARD_CUDA_TRY(back(a->resid_sum_norm, h.rsn, sizeof(double) * P));
+    std::vector<uint32_t> sc, sv;
+    if (a->status) {
+        sc.resize(P); sv.resize(P);
+        BTARD_CUDA_TRY(cudaMemcpyAsync(sc.data(), base + h.status_c, sizeof(uint32_t) * P, cudaMemcpyDeviceToHost, st));
+        BTARD_CUDA_TRY(cudaMemcpyAsync(sv.data(), base + h.status_v, sizeof(uint32_t) * P, cudaMemcpyDeviceToHost, st));
+    }
+    BTARD_CUDA_TRY(cudaStreamSynchronize(st));
+    if (a->status)
+        for (size_t p = 0; p < P; ++p) a->status[p] = sc[p] | sv[p];
+    return BTARD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,481 @@
+// CenteredClip streaming passes (App. D.2, eq. (CenteredClip)) for sm_100a.
+//
+// One pass reads the [P][n][row_stride] tensor exactly once.  A CTA owns a contiguous range of
+// column tiles of one partition; a thread keeps R rows x 4 columns of the current tile in
+// registers (R independent 128-bit loads in flight), so that the update of v and the residual
+// norms at the *updated* v come out of the same registers:
+//
+//   weights w_i from the norms the previous pass left behind      (prologue, per CTA)
+//   u[c]  = (1/n) sum_i w_i (x_i[c] - v[c]);  v'[c] = v[c] + u[c]  (eq. (CenteredClip))
+//   norm2_i += (x_i[c] - v'[c])^2;  step2 += u[c]^2               (feeds the next pass)
+//
+// Cross-CTA sums are not atomics: every CTA writes its partial sums to its own slot and the next
+// pass adds the slots of its partition in a fixed order, so results are reproducible run to run.
+// The stop rule is evaluated the same way by every CTA of a partition at the top of each pass.
+#include "btard_common.h"
+
+namespace btard {
+namespace {
+
+__device__ __forceinline__ float4 ld_stream(const float* p)
+{
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+
+__device__ __forceinline__ double warp_sum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Clip weight min{1, tau/rho} from the squared norm; non-finite norms give 0.
+__device__ __forceinline__ float clip_weight(double norm2, double tau, bool& nonfinite)
+{
+    const double rho = sqrt(norm2);
+    if (!isfinite(rho)) { nonfinite = true; return 0.0f; }
+    if (rho <= tau) return 1.0f;
+    return (float)(tau / rho);
+}
+
+struct KernelArgs {
+    CclipLaunch a;
+    int RG, CL, tiles, cpp;
+};
+
+// Records the end state of a partition (called by one CTA of it).
+__device__ void finish_partition(const KernelArgs& k, int p, const double* sums, int iters_done,
+                                 bool eps_mode)
+{
+    const int n = k.a.n;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) k.a.resid_norm[(size_t)p * n + i] = sqrt(sums[i]);
+    if (threadIdx.x == 0) {
+        const double step2 = sums[n];
+        k.a.iters[p] = iters_done;
+        k.a.last_step[p] = sqrt(step2);
+        unsigned st = 0;
+        for (int i = 0; i < n; ++i)
+            if (!isfinite(sums[i])) st |= BTARD_STATUS_NONFINITE_ROW;
+        if (eps_mode && !(step2 <= k.a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
+        atomicOr(&k.a.status[p], st);
+        k.a.done[p] = 1;
+    }
+}
+
+// bf16 <-> fp32 for the low-order part of v (round to nearest even; inputs are finite and tiny).
+__device__ __forceinline__ uint32_t bf16_bits(float f)
+{
+    const uint32_t u = __float_as_uint(f);
+    return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+__device__ __forceinline__ float bf16_value(uint32_t b) { return __uint_as_float(b << 16); }
+
+// v + s as an unevaluated sum hi + lo (Knuth's TwoSum), lo then rounded to bf16.
+__device__ __forceinline__ void two_sum_bf16(float v, float s, float& hi, float& lo, uint32_t& lo_bits)
+{
+    hi = __fadd_rn(v, s);
+    const float bb = __fadd_rn(hi, -v);
+    const float err = __fadd_rn(__fadd_rn(v, -__fadd_rn(hi, -bb)), __fadd_rn(s, -bb));
+    lo_bits = bf16_bits(err);
+    lo = bf16_value(lo_bits);
+}
+
+// COMP (PASS_ITER only): v is carried as hi + lo, hi the fp32 output vector and lo a bf16 correction
+// in the workspace, so that the update and the stop test do not drown in the rounding of v.
+template <int R, int MODE, bool COMP>
+__global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
+{
+    extern __shared__ float4 sh_x[];                  // [2][RG][CL] exchange of partial column sums
+    __shared__ double sh_sum[BTARD_MAX_PEERS + 1];
+    __shared__ float sh_w[BTARD_MAX_PEERS];
+    __shared__ double sh_red[16][17];
+    __shared__ int sh_flag;
+
+    const CclipLaunch& a = k.a;
+    const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
+    const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const long long stride = a.stride;
+    const long long len = a.table[p].len;
+    const double tau = a.table[p].tau;
+
+    float Wsum = 0.0f;
+    if (MODE == PASS_ITER) {
+        if (a.done[p]) return;
+        // Sum the previous pass's slots in a fixed order: norms at the current v, and its step.
+        const double* src = a.part_in + (size_t)p * cpp * (n + 1);
+        for (int i = tid; i <= n; i += blockDim.x) {
+            double s = 0.0;
+            for (int c = 0; c < cpp; ++c) s += src[(size_t)c * (n + 1) + i];
+            sh_sum[i] = s;
+        }
+        __syncthreads();
+        const bool converged = (a.stop_mode == BTARD_STOP_EPS) && a.l >= 1 && (sh_sum[n] <= a.eps2);
+        if (converged) {                              // same decision in every CTA of the partition
+            if (j == 0) finish_partition(k, p, sh_sum, a.l, true);
+            return;
+        }
+        if (tid == 0) sh_flag = 0;
+        __syncthreads();
+        for (int i = tid; i < n; i += blockDim.x) {
+            bool bad = false;
+            sh_w[i] = clip_weight(sh_sum[i], tau, bad);
+            if (bad) sh_flag = 1;
+        }
+        __syncthreads();
+        if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+        for (int i = 0; i < n; ++i) Wsum += sh_w[i];
+    } else if (MODE == PASS_INIT) {
+        if (j == 0 && tid == 0) { a.done[p] = 0; a.status[p] = 0; }
+    }
+    (void)Wsum;
+
+    float w[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int i = rg * R + r;
+        w[r] = (MODE == PASS_ITER && i < n) ? sh_w[i] : 0.0f;
+    }
+
+    float acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.0f;
+    float step_acc = 0.0f;
+
+    const long long t0 = (long long)k.tiles * j / cpp, t1 = (long long)k.tiles * (j + 1) / cpp;
+    const float* gp = a.g + (size_t)p * n * stride;
+    float* vp = a.v + (size_t)p * stride;
+    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
+    const float nf = (float)n;
+
+    for (long long t = t0; t < t1; ++t) {
+        const long long col = (t * CL + cl) * 4;
+        const bool valid = col < stride;
+        float4 x[R];
+        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f);      // low-order part of v (COMP)
+        if (valid) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int i = rg * R + r;
+                x[r] = (i < n) ? ld_stream(gp + (size_t)i * stride + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (MODE != PASS_INIT || a.init_mode == BTARD_INIT_CALLER_V0)
+                v4 = *reinterpret_cast<const float4*>(vp + col);
+            if (COMP) {
+                const uint2 lb = *reinterpret_cast<const uint2*>(lop + col);
+                lo4 = make_float4(bf16_value(lb.x & 0xFFFFu), bf16_value(lb.x >> 16),
+                                  bf16_value(lb.y & 0xFFFFu), bf16_value(lb.y >> 16));
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len, m3 = col + 3 < len;
+
+        float4 vn = v4;                                // v after this pass
+        if (MODE == PASS_ITER || (MODE == PASS_INIT && a.init_mode == BTARD_INIT_MEAN)) {
+            float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                if (MODE == PASS_ITER) {
+                    if (w[r] != 0.0f) {                // weight 0: the row is left out, not multiplied
+                        s4.x = fmaf(w[r], (x[r].x - v4.x) - lo4.x, s4.x);
+                        s4.y = fmaf(w[r], (x[r].y - v4.y) - lo4.y, s4.y);
+                        s4.z = fmaf(w[r], (x[r].z - v4.z) - lo4.z, s4.z);
+                        s4.w = fmaf(w[r], (x[r].w - v4.w) - lo4.w, s4.w);
+                    }
+                } else {
+                    s4.x += x[r].x; s4.y += x[r].y; s4.z += x[r].z; s4.w += x[r].w;
+                }
+            }
+            if (RG > 1) {                              // add the row groups' partial column sums
+                float4* buf = sh_x + (size_t)(t & 1) * RG * CL;
+                buf[rg * CL + cl] = s4;
+                __syncthreads();
+                s4 = buf[cl];
+                for (int q = 1; q < RG; ++q) {
+                    const float4 o = buf[q * CL + cl];
+                    s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
+                }
+            }
+            const float4 u = make_float4(s4.x / nf, s4.y / nf, s4.z / nf,
+                                         s4.w / nf);
+            if (MODE == PASS_ITER) {
+                if (COMP) {
+                    uint32_t b0, b1, b2, b3;
+                    two_sum_bf16(v4.x, lo4.x + u.x, vn.x, lo4.x, b0);
+                    two_sum_bf16(v4.y, lo4.y + u.y, vn.y, lo4.y, b1);
+                    two_sum_bf16(v4.z, lo4.z + u.z, vn.z, lo4.z, b2);
+                    two_sum_bf16(v4.w, lo4.w + u.w, vn.w, lo4.w, b3);
+                    if (!m0) { b0 = 0; lo4.x = 0.f; }
+                    if (!m1) { b1 = 0; lo4.y = 0.f; }
+                    if (!m2) { b2 = 0; lo4.z = 0.f; }
+                    if (!m3) { b3 = 0; lo4.w = 0.f; }
+                    if (rg == 0 && valid)
+                        *reinterpret_cast<uint2*>(lop + col) = make_uint2(b0 | (b1 << 16), b2 | (b3 << 16));
+                } else {
+                    vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+                }
+                if (rg == 0)
+                    step_acc += (m0 ? u.x * u.x : 0.f) + (m1 ? u.y * u.y : 0.f) +
+                                (m2 ? u.z * u.z : 0.f) + (m3 ? u.w * u.w : 0.f);
+            } else {
+                vn = u;
+            }
+        } else if (MODE == PASS_INIT && a.init_mode == BTARD_INIT_ZERO) {
+            vn = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (!m0) vn.x = 0.f;
+        if (!m1) vn.y = 0.f;
+        if (!m2) vn.z = 0.f;
+        if (!m3) vn.w = 0.f;
+        if (MODE != PASS_NORMS && rg == 0 && valid) *reinterpret_cast<float4*>(vp + col) = vn;
+
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float dx = m0 ? (x[r].x - vn.x) - lo4.x : 0.f, dy = m1 ? (x[r].y - vn.y) - lo4.y : 0.f;
+            const float dz = m2 ? (x[r].z - vn.z) - lo4.z : 0.f, dw = m3 ? (x[r].w - vn.w) - lo4.w : 0.f;
+            acc[r] += fmaf(dx, dx, fmaf(dy, dy, fmaf(dz, dz, dw * dw)));
+        }
+    }
+
+    // CTA reduction: lanes of a warp share a row group, so a warp reduces R rows at once.
+    const int warp = tid >> 5, lane = tid & 31, wpg = CL >> 5;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const double s = warp_sum((double)acc[r]);
+        if (lane == 0) sh_red[warp][r] = s;
+    }
+    {
+        const double s = warp_sum((double)step_acc);
+        if (lane == 0) sh_red[warp][16] = s;
+    }
+    __syncthreads();
+    double* dst = a.part_out + ((size_t)p * cpp + j) * (n + 1);
+    for (int i = tid; i <= n; i += blockDim.x) {
+        double s = 0.0;
+        if (i < n) {
+            const int g0 = (i / R) * wpg;
+            for (int q = 0; q < wpg; ++q) s += sh_red[g0 + q][i % R];
+        } else {
+            for (int q = 0; q < wpg; ++q) s += sh_red[q][16];
+        }
+        dst[i] = s;
+    }
+}
+
+// After the last pass: partitions still running take iters = max_iters.
+__global__ void cclip_finalize_kernel(const KernelArgs k)
+{
+    __shared__ double sh_sum[BTARD_MAX_PEERS + 1];
+    const CclipLaunch& a = k.a;
+    const int p = blockIdx.x, n = a.n;
+    if (a.done[p]) return;
+    const double* src = a.part_in + (size_t)p * k.cpp * (n + 1);
+    for (int i = threadIdx.x; i <= n; i += blockDim.x) {
+        double s = 0.0;
+        for (int c = 0; c < k.cpp; ++c) s += src[(size_t)c * (n + 1) + i];
+        sh_sum[i] = s;
+    }
+    __syncthreads();
+    finish_partition(k, p, sh_sum, a.max_iters, a.stop_mode == BTARD_STOP_EPS);
+}
+
+__global__ void partials_to_norms_kernel(const double* part, double* norm, int n, int cpp)
+{
+    const int p = blockIdx.x;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        double s = 0.0;
+        for (int c = 0; c < cpp; ++c) s += part[((size_t)p * cpp + c) * (n + 1) + i];
+        norm[(size_t)p * n + i] = sqrt(s);
+    }
+}
+
+// ---- coordinate-wise median start ---------------------------------------------------------------
+// Order-preserving map of float bit patterns to unsigned integers (IEEE total order).
+__device__ __forceinline__ uint32_t order_key(float f)
+{
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(uint32_t key)
+{
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7FFFFFFFu) : ~key);
+}
+
+// One thread sorts the n values of one column in registers with a bitonic network of N2 >= n
+// inputs (missing inputs are the largest key).
+template <int N2>
+__global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float* v,
+                                                          const PartEntry* table, long long stride,
+                                                          int n)
+{
+    const int p = blockIdx.y;
+    const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= stride) return;
+    const long long len = table[p].len;
+    float out = 0.0f;
+    if (c < len) {
+        const float* gp = g + (size_t)p * n * stride + c;
+        uint32_t key[N2];
+#pragma unroll
+        for (int i = 0; i < N2; ++i) key[i] = (i < n) ? order_key(__ldcs(gp + (size_t)i * stride)) : 0xFFFFFFFFu;
+#pragma unroll
+        for (int kk = 2; kk <= N2; kk <<= 1) {
+#pragma unroll
+            for (int jj = kk >> 1; jj > 0; jj >>= 1) {
+#pragma unroll
+                for (int i = 0; i < N2; ++i) {
+                    const int l = i ^ jj;
+                    if (l > i) {
+                        const uint32_t lo = min(key[i], key[l]), hi = max(key[i], key[l]);
+                        const bool up = (i & kk) == 0;
+                        key[i] = up ? lo : hi;
+                        key[l] = up ? hi : lo;
+                    }
+                }
+            }
+        }
+        // n is a run-time value: pick the two middle keys without dynamic register indexing.
+        uint32_t ka = 0, kb = 0;
+        const int ia = (n - 1) >> 1, ib = n >> 1;
+#pragma unroll
+        for (int i = 0; i < N2; ++i) {
+            if (i == ia) ka = key[i];
+            if (i == ib) kb = key[i];
+        }
+        out = (float)(((double)key_value(ka) + (double)key_value(kb)) * 0.5);
+    }
+    v[(size_t)p * stride + c] = out;
+}
+
+// Any n: rank every value by counting (O(n^2) compares per column), pick the two middle ranks.
+__global__ void median_rank_kernel(const float* g, float* v, const PartEntry* table,
+                                   long long stride, int n)
+{
+    const int p = blockIdx.y;
+    const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= stride) return;
+    const long long len = table[p].len;
+    float out = 0.0f;
+    if (c < len) {
+        const float* gp = g + (size_t)p * n * stride + c;
+        const int ia = (n - 1) >> 1, ib = n >> 1;
+        uint32_t ka = 0, kb = 0;
+        for (int i = 0; i < n; ++i) {
+            const uint32_t ki = order_key(gp[(size_t)i * stride]);
+            int rank = 0;
+            for (int q = 0; q < n; ++q) {
+                const uint32_t kq = order_key(gp[(size_t)q * stride]);
+                rank += (kq < ki) || (kq == ki && q < i);
+            }
+            if (rank == ia) ka = ki;
+            if (rank == ib) kb = ki;
+        }
+        out = (float)(((double)key_value(ka) + (double)key_value(kb)) * 0.5);
+    }
+    v[(size_t)p * stride + c] = out;
+}
+
+template <int R>
+int launch_pass_r(const KernelArgs& ka, int mode, int threads, size_t smem, int grid, cudaStream_t st)
+{
+    const int kind = (mode == PASS_ITER) ? KIND_ITER : (mode == PASS_INIT) ? KIND_INIT : KIND_OTHER;
+    prof_begin(kind, st);
+    switch (mode) {
+        case PASS_INIT: cclip_pass_kernel<R, PASS_INIT, false><<<grid, threads, smem, st>>>(ka); break;
+        case PASS_ITER:
+            if (ka.a.v_lo) cclip_pass_kernel<R, PASS_ITER, true><<<grid, threads, smem, st>>>(ka);
+            else cclip_pass_kernel<R, PASS_ITER, false><<<grid, threads, smem, st>>>(ka);
+            break;
+        default: cclip_pass_kernel<R, PASS_NORMS, false><<<grid, threads, smem, st>>>(ka); break;
+    }
+    prof_end(kind, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+}  // namespace
+
+Geometry cclip_geometry(int n, int P, long long stride)
+{
+    Geometry g;
+    g.R = (n <= 4) ? 4 : (n <= 8) ? 8 : 16;
+    g.RG = (n + g.R - 1) / g.R;
+    g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 8) ? 64 : 32;
+    g.threads = g.RG * g.CL;
+    const long long cols = 4LL * g.CL;
+    g.tiles = (int)((stride + cols - 1) / cols);
+    // Enough CTAs to fill every SM twice over, few enough tiles per CTA to bound the fp32 running
+    // sums, and a total close to a whole number of waves.
+    const int ctas_per_sm = (g.threads <= 256) ? 2 : 1;
+    const int slots = sm_count() * ctas_per_sm;
+    int cmin = (g.tiles + kMaxTilesPerCta - 1) / kMaxTilesPerCta;
+    if (cmin < 1) cmin = 1;
+    int want = (slots + P - 1) / P;
+    if (want < cmin) want = cmin;
+    if (want > g.tiles) want = g.tiles;
+    if (want < 1) want = 1;
+    int best = want;
+    double best_eff = -1.0;
+    for (int c = want; c <= want + 8 && c <= (g.tiles > 0 ? g.tiles : 1); ++c) {
+        const long long total = (long long)c * P;
+        const long long waves = (total + slots - 1) / slots;
+        const double eff = (double)total / (double)(waves * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = c; }
+    }
+    g.cpp = best;
+    return g;
+}
+
+int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st)
+{
+    KernelArgs ka{a, geo.RG, geo.CL, geo.tiles, geo.cpp};
+    const size_t smem = (geo.RG > 1) ? sizeof(float4) * 2 * geo.RG * geo.CL : 0;
+    const int grid = a.P * geo.cpp;
+    switch (geo.R) {
+        case 4: return launch_pass_r<4>(ka, mode, geo.threads, smem, grid, st);
+        case 8: return launch_pass_r<8>(ka, mode, geo.threads, smem, grid, st);
+        default: return launch_pass_r<16>(ka, mode, geo.threads, smem, grid, st);
+    }
+}
+
+int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st)
+{
+    KernelArgs ka{a, geo.RG, geo.CL, geo.tiles, geo.cpp};
+    cclip_finalize_kernel<<<a.P, 128, 0, st>>>(ka);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_partials_to_norms(const double* part, double* norm, int n, int P, int cpp, cudaStream_t st)
+{
+    partials_to_norms_kernel<<<P, 128, 0, st>>>(part, norm, n, cpp);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
+                       int P, cudaStream_t st)
+{
+    const int threads = 128;
+    dim3 grid((unsigned)((stride + threads - 1) / threads), (unsigned)P);
+    prof_begin(KIND_MEDIAN, st);
+    if (n <= 2) median_sort_kernel<2><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n <= 4) median_sort_kernel<4><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n <= 8) median_sort_kernel<8><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n <= 16) median_sort_kernel<16><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n <= 32) median_sort_kernel<32><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n <= 64) median_sort_kernel<64><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else median_rank_kernel<<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    prof_end(KIND_MEDIAN, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+}  // namespace btard

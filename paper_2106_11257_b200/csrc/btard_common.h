@@ -1,0 +1,111 @@
+// Shared declarations of the library's translation units (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/btard.h"
+
+namespace btard {
+
+// Per-partition constants the kernels read from the workspace.
+struct PartEntry {
+    long long len;   // number of real columns
+    double tau;      // clip radius
+};
+
+// How one streaming pass is cut into CTAs.  A CTA is RG row groups x CL column lanes; a thread
+// owns R consecutive rows of its group and 4 consecutive columns of every tile it visits.
+struct Geometry {
+    int R;        // rows per thread (compile-time choice, one of the instantiated values)
+    int RG;       // row groups = ceil(n / R)
+    int CL;       // column lanes (multiple of 32)
+    int threads;  // RG * CL
+    int tiles;    // tiles per partition = ceil(row_stride / (4 CL))
+    int cpp;      // CTAs per partition
+};
+
+constexpr int kMaxTilesPerCta = 64;   // bounds the length of every fp32 running sum (256 terms)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Error bookkeeping (thread local).
+void set_cuda_error(cudaError_t e);
+void count_launch(int n = 1);
+
+// Optional per-kernel timing (off by default): CUDA events around every launch of a kind.
+enum KernelKind { KIND_MEDIAN = 0, KIND_INIT = 1, KIND_ITER = 2, KIND_VERIFY = 3, KIND_OTHER = 4,
+                  KIND_COUNT = 5 };
+void prof_begin(int kind, cudaStream_t st);
+void prof_end(int kind, cudaStream_t st);
+int sm_count();
+
+#define BTARD_CUDA_TRY(expr)                         \
+    do {                                             \
+        cudaError_t e__ = (expr);                    \
+        if (e__ != cudaSuccess) {                    \
+            ::btard::set_cuda_error(e__);            \
+            return BTARD_ERR_CUDA;                   \
+        }                                            \
+    } while (0)
+
+// ---- CenteredClip passes (btard_cclip.cu) -------------------------------------------------------
+enum PassMode { PASS_INIT = 0, PASS_ITER = 1, PASS_NORMS = 2 };
+
+struct CclipLaunch {
+    const float* g;
+    float* v;                 // PASS_NORMS never writes it
+    unsigned short* v_lo;     // device [P][stride] bf16 low-order part of v, or nullptr (plain fp32 v)
+    const PartEntry* table;   // device [P]
+    const double* part_in;    // device [P][cpp][n+1] partial sums of the previous pass
+    double* part_out;         // device [P][cpp][n+1]
+    int* done;                // device [P]
+    int32_t* iters;
+    double* last_step;
+    double* resid_norm;
+    uint32_t* status;
+    long long stride;
+    int n, P;
+    int l;                    // index of the update this pass applies (PASS_ITER)
+    int stop_mode, max_iters;
+    double eps2;
+    int init_mode;            // PASS_INIT
+};
+
+Geometry cclip_geometry(int n, int P, long long stride);
+int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
+int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
+int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
+                       int P, cudaStream_t st);
+// norm2 partial sums -> norms (sqrt of the per-partition sums), used when verification is asked to
+// compute the norms itself.
+int launch_partials_to_norms(const double* part, double* norm, int n, int P, int cpp,
+                             cudaStream_t st);
+
+// ---- verification (btard_verify.cu) -------------------------------------------------------------
+struct VerifyLaunch {
+    const float* g;
+    const float* v;
+    const PartEntry* table;
+    const double* norm_in;    // device [P][n]
+    double* part_out;         // device [P][cpp][slots]
+    float* resid_sum;         // device [P][stride] or nullptr
+    double *norm, *weight, *dot, *s, *s_sum, *znorm2, *resid_sum_norm;
+    uint32_t* status;
+    long long stride;
+    int n, P, K, k0, kc;      // this launch covers z indices k0 .. k0+kc-1
+    int p_base;
+    uint32_t seed_lo, seed_hi;
+};
+
+struct VerifyGeometry {
+    Geometry g;
+    int KT;      // z vectors per launch (compile-time choice)
+    int slots;   // doubles per CTA in part_out
+};
+
+VerifyGeometry verify_geometry(int n, int P, long long stride, int K);
+int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t st);
+int launch_random_vector(uint64_t seed, int p, int k, long long len, float* z, cudaStream_t st);
+
+}  // namespace btard

@@ -1,0 +1,353 @@
+// Verification pass (Sec. 3.1 eq. (2); Alg. 6 lines 5-14) for sm_100a: one read of the
+// [P][n][row_stride] tensor produces, per partition, the projections <g_i - v, z_k> on K random
+// directions, ||z_k||^2, and the clipped-residual sum sum_i w_i (g_i - v) with its norm.
+//
+// z is generated on the fly: the CTA's threads share the Philox/Box-Muller work of a
+// [K][tile columns] block of z, stage it in shared memory (double buffered), and every thread then
+// multiplies its R rows x 4 columns of residuals against it.  Per-thread accumulators are fp32 over
+// at most kMaxTilesPerCta tiles; everything that crosses threads is fp64, written to per-CTA slots
+// and summed in a fixed order by the finalize kernel.
+#include "btard_common.h"
+#include "btard_philox.cuh"
+
+namespace btard {
+namespace {
+
+__device__ __forceinline__ double warp_sum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
+    return x;
+}
+
+struct VArgs {
+    VerifyLaunch a;
+    int RG, CL, tiles, cpp, slots;
+};
+
+// slot layout per CTA: [n*KT] dots (row-major i, k), [KT] znorm2, [1] squared norm of resid_sum
+template <int R, int KT>
+__global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
+{
+    extern __shared__ float4 sh_dyn[];   // z: [2][KT][CL], then column sums: [2][RG][CL]
+    __shared__ float sh_w[BTARD_MAX_PEERS];
+    __shared__ double sh_red[16][R * KT + KT + 1];
+
+    const VerifyLaunch& a = k.a;
+    const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
+    const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL, nthr = blockDim.x;
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const long long stride = a.stride, len = a.table[p].len;
+    const double tau = a.table[p].tau;
+    float4* sh_z = sh_dyn;
+    float4* sh_s = sh_dyn + 2 * KT * CL;
+
+    for (int i = tid; i < n; i += nthr) {
+        const double rho = a.norm_in[(size_t)p * n + i];
+        float w = 0.0f;
+        if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+        sh_w[i] = w;
+    }
+    __syncthreads();
+    float w[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int i = rg * R + r;
+        w[r] = (i < n) ? sh_w[i] : 0.0f;
+    }
+
+    float acc[R][KT];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int q = 0; q < KT; ++q) acc[r][q] = 0.0f;
+    float zz[KT];
+#pragma unroll
+    for (int q = 0; q < KT; ++q) zz[q] = 0.0f;
+    float rs2 = 0.0f;
+
+    const long long t0 = (long long)k.tiles * j / cpp, t1 = (long long)k.tiles * (j + 1) / cpp;
+    const float* gp = a.g + (size_t)p * n * stride;
+    const float* vp = a.v + (size_t)p * stride;
+    float* rsp = a.resid_sum ? a.resid_sum + (size_t)p * stride : nullptr;
+    const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
+    const uint32_t pg = (uint32_t)(a.p_base + p);
+
+    // Adds up the row groups' column sums of tile tt (written one tile earlier).
+    auto consume_sums = [&](long long tt) {
+        if (rg != 0) return;
+        const long long col = (tt * CL + cl) * 4;
+        if (col >= stride) return;
+        const float4* buf = sh_s + (size_t)(tt & 1) * RG * CL;
+        float4 s4 = buf[cl];
+        for (int q = 1; q < RG; ++q) {
+            const float4 o = buf[q * CL + cl];
+            s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
+        }
+        rs2 += fmaf(s4.x, s4.x, fmaf(s4.y, s4.y, fmaf(s4.z, s4.z, s4.w * s4.w)));
+        if (rsp) *reinterpret_cast<float4*>(rsp + col) = s4;
+    };
+
+    for (long long t = t0; t < t1; ++t) {
+        // 1. this tile's block of z
+        float4* zb = sh_z + (size_t)(t & 1) * KT * CL;
+        for (int idx = tid; idx < KT * CL; idx += nthr) {
+            const int kq = idx / CL, cq = idx % CL;
+            const long long col = (t * CL + cq) * 4;
+            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (kq < a.kc && col < len) {
+                z = z_quad((uint32_t)(col >> 2), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
+                if (col + 1 >= len) z.y = 0.f;
+                if (col + 2 >= len) z.z = 0.f;
+                if (col + 3 >= len) z.w = 0.f;
+            }
+            zb[kq * CL + cq] = z;
+        }
+        __syncthreads();
+        if (first_chunk && t > t0) consume_sums(t - 1);
+
+        // 2. residuals of this thread's rows and columns
+        const long long col = (t * CL + cl) * 4;
+        const bool valid = col < stride;
+        const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len, m3 = col + 3 < len;
+        float4 x[R];
+        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int i = rg * R + r;
+                x[r] = (i < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)i * stride + col))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            v4 = *reinterpret_cast<const float4*>(vp + col);
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            x[r].x = m0 ? x[r].x - v4.x : 0.f;
+            x[r].y = m1 ? x[r].y - v4.y : 0.f;
+            x[r].z = m2 ? x[r].z - v4.z : 0.f;
+            x[r].w = m3 ? x[r].w - v4.w : 0.f;
+        }
+        // 3. projections
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            const float4 z = zb[q * CL + cl];
+            if (rg == 0) zz[q] += fmaf(z.x, z.x, fmaf(z.y, z.y, fmaf(z.z, z.z, z.w * z.w)));
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                acc[r][q] += fmaf(x[r].x, z.x, fmaf(x[r].y, z.y, fmaf(x[r].z, z.z, x[r].w * z.w)));
+        }
+        // 4. clipped-residual column sums of this row group
+        if (first_chunk) {
+            float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                if (w[r] != 0.0f) {
+                    s4.x = fmaf(w[r], x[r].x, s4.x);
+                    s4.y = fmaf(w[r], x[r].y, s4.y);
+                    s4.z = fmaf(w[r], x[r].z, s4.z);
+                    s4.w = fmaf(w[r], x[r].w, s4.w);
+                }
+            }
+            sh_s[(size_t)(t & 1) * RG * CL + rg * CL + cl] = s4;
+        }
+    }
+    __syncthreads();
+    if (first_chunk && t1 > t0) consume_sums(t1 - 1);
+
+    // CTA reduction
+    const int warp = tid >> 5, lane = tid & 31, wpg = CL >> 5;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            const double s = warp_sum((double)acc[r][q]);
+            if (lane == 0) sh_red[warp][r * KT + q] = s;
+        }
+#pragma unroll
+    for (int q = 0; q < KT; ++q) {
+        const double s = warp_sum((double)zz[q]);
+        if (lane == 0) sh_red[warp][R * KT + q] = s;
+    }
+    {
+        const double s = warp_sum((double)rs2);
+        if (lane == 0) sh_red[warp][R * KT + KT] = s;
+    }
+    __syncthreads();
+    double* dst = a.part_out + ((size_t)p * cpp + j) * k.slots;
+    const int total = n * KT + KT + 1;
+    for (int e = tid; e < total; e += nthr) {
+        double s = 0.0;
+        if (e < n * KT) {
+            const int i = e / KT, q = e % KT;
+            const int g0 = (i / R) * wpg;
+            for (int u = 0; u < wpg; ++u) s += sh_red[g0 + u][(i % R) * KT + q];
+        } else {
+            const int q = e - n * KT;                  // znorm2 slots, then the resid-sum slot
+            for (int u = 0; u < wpg; ++u) s += sh_red[u][R * KT + q];
+        }
+        dst[e] = s;
+    }
+}
+
+// Sums the CTA slots of a partition in a fixed order and writes the outputs of z indices
+// k0 .. k0+kc-1 (and, with the first chunk, the per-row and per-partition values).
+__global__ void verify_finalize_kernel(const VArgs k, int KT)
+{
+    extern __shared__ double sh_v[];     // [slots]
+    __shared__ float sh_wf[BTARD_MAX_PEERS];
+    const VerifyLaunch& a = k.a;
+    const int p = blockIdx.x, n = a.n, K = a.K;
+    const int total = n * KT + KT + 1;
+    const double* src = a.part_out + (size_t)p * k.cpp * k.slots;
+    for (int e = threadIdx.x; e < total; e += blockDim.x) {
+        double s = 0.0;
+        for (int c = 0; c < k.cpp; ++c) s += src[(size_t)c * k.slots + e];
+        sh_v[e] = s;
+    }
+    const double tau = a.table[p].tau;
+    bool bad = false;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const double rho = a.norm_in[(size_t)p * n + i];
+        float w = 0.0f;
+        if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+        else bad = true;
+        sh_wf[i] = w;
+        if (a.k0 == 0) {
+            a.norm[(size_t)p * n + i] = rho;
+            a.weight[(size_t)p * n + i] = (double)w;
+        }
+    }
+    if (a.k0 == 0 && threadIdx.x == 0) a.status[p] = 0;
+    __syncthreads();
+    if (bad) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+    for (int e = threadIdx.x; e < n * a.kc; e += blockDim.x) {
+        const int i = e / a.kc, q = e % a.kc;
+        const double d = sh_v[i * KT + q];
+        const double zn = sqrt(sh_v[n * KT + q]);
+        a.dot[((size_t)p * n + i) * K + a.k0 + q] = d;
+        a.s[((size_t)p * n + i) * K + a.k0 + q] = (sh_wf[i] == 0.0f) ? 0.0 : (double)sh_wf[i] * d / zn;
+    }
+    for (int q = threadIdx.x; q < a.kc; q += blockDim.x) {
+        const double zn = sqrt(sh_v[n * KT + q]);
+        double ss = 0.0;
+        for (int i = 0; i < n; ++i)
+            if (sh_wf[i] != 0.0f) ss += (double)sh_wf[i] * sh_v[i * KT + q] / zn;
+        a.s_sum[(size_t)p * K + a.k0 + q] = ss;
+        a.znorm2[(size_t)p * K + a.k0 + q] = sh_v[n * KT + q];
+    }
+    if (a.k0 == 0 && threadIdx.x == 0) a.resid_sum_norm[p] = sqrt(sh_v[n * KT + KT]);
+}
+
+__global__ void random_vector_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t p, uint32_t kz,
+                                     long long len, float* z)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (4 * q >= len) return;
+    float4 v = z_quad((uint32_t)q, p, kz, seed_lo, seed_hi);
+    if (4 * q + 1 >= len) v.y = 0.f;
+    if (4 * q + 2 >= len) v.z = 0.f;
+    if (4 * q + 3 >= len) v.w = 0.f;
+    *reinterpret_cast<float4*>(z + 4 * q) = v;
+}
+
+template <int R, int KT>
+int launch_rk(const VArgs& va, int threads, size_t smem, int grid, cudaStream_t st)
+{
+    prof_begin(KIND_VERIFY, st);
+    verify_kernel<R, KT><<<grid, threads, smem, st>>>(va);
+    prof_end(KIND_VERIFY, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+template <int R>
+int launch_r(const VArgs& va, int KT, int threads, size_t smem, int grid, cudaStream_t st)
+{
+    if (KT == 1) return launch_rk<R, 1>(va, threads, smem, grid, st);
+    if (KT == 2) return launch_rk<R, 2>(va, threads, smem, grid, st);
+    if constexpr (R <= 8) {                 // 16 rows per thread never run more than 2 vectors
+        if (KT == 4) return launch_rk<R, 4>(va, threads, smem, grid, st);
+        if (KT == 8) return launch_rk<R, 8>(va, threads, smem, grid, st);
+    }
+    return BTARD_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
+{
+    VerifyGeometry vg;
+    Geometry& g = vg.g;
+    g.R = (n <= 16) ? 4 : 8;
+    g.RG = (n + g.R - 1) / g.R;
+    g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 4) ? 64 : 32;
+    g.threads = g.RG * g.CL;      // n <= 256 with R = 8 gives at most 32 x 32 = 1024
+    if (g.threads > 512) {        // keep CTAs at 512 threads: more rows per thread would be needed
+        g.R = 16;
+        g.RG = (n + 15) / 16;
+        g.CL = 32;
+        g.threads = g.RG * g.CL;
+    }
+    int kt = 1;
+    while (kt < K && kt < 8) kt <<= 1;
+    if (g.R == 16 && kt > 2) kt = 2;          // 16 rows per thread: keep the accumulators in registers
+    vg.KT = kt;
+    const long long cols = 4LL * g.CL;
+    g.tiles = (int)((stride + cols - 1) / cols);
+    const int ctas_per_sm = (g.threads <= 256) ? 2 : 1;
+    const int slots = sm_count() * ctas_per_sm;
+    int cmin = (g.tiles + kMaxTilesPerCta - 1) / kMaxTilesPerCta;
+    int want = (slots + P - 1) / P;
+    if (want < cmin) want = cmin;
+    if (want > g.tiles) want = g.tiles;
+    if (want < 1) want = 1;
+    int best = want;
+    double best_eff = -1.0;
+    for (int c = want; c <= want + 8 && c <= (g.tiles > 0 ? g.tiles : 1); ++c) {
+        const long long total = (long long)c * P;
+        const long long waves = (total + slots - 1) / slots;
+        const double eff = (double)total / (double)(waves * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = c; }
+    }
+    g.cpp = best;
+    vg.slots = n * kt + kt + 1;
+    return vg;
+}
+
+int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t st)
+{
+    const Geometry& g = vg.g;
+    VArgs va{a, g.RG, g.CL, g.tiles, g.cpp, vg.slots};
+    const size_t smem = sizeof(float4) * (2 * (size_t)vg.KT * g.CL + 2 * (size_t)g.RG * g.CL);
+    const int grid = a.P * g.cpp;
+    int rc;
+    switch (g.R) {
+        case 4: rc = launch_r<4>(va, vg.KT, g.threads, smem, grid, st); break;
+        case 8: rc = launch_r<8>(va, vg.KT, g.threads, smem, grid, st); break;
+        default: rc = launch_r<16>(va, vg.KT, g.threads, smem, grid, st); break;
+    }
+    if (rc != BTARD_OK) return rc;
+    verify_finalize_kernel<<<a.P, 128, sizeof(double) * vg.slots, st>>>(va, vg.KT);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_random_vector(uint64_t seed, int p, int k, long long len, float* z, cudaStream_t st)
+{
+    const long long quads = (len + 3) / 4;
+    if (quads == 0) return BTARD_OK;
+    const int threads = 256;
+    random_vector_kernel<<<(unsigned)((quads + threads - 1) / threads), threads, 0, st>>>(
+        (uint32_t)seed, (uint32_t)(seed >> 32), (uint32_t)p, (uint32_t)k, len, z);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+}  // namespace btard

@@ -1,0 +1,330 @@
+"""GPU-vs-oracle parity through the C ABI (run on a B200: `pytest -m gpu`).
+
+Tolerances: bit-exact for z, layout and indices; relative L2 <= 1e-5 per partition for v, norms,
+weights, dots and s in fixed-iteration mode; near-zero sums compared absolutely against the scale of
+their terms; iteration counts equal or +-1 in eps mode.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+import paper_2106_11257_b200 as btard
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-5
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    den = np.linalg.norm(b)
+    return np.linalg.norm(a - b) / den if den > 0 else np.linalg.norm(a)
+
+
+def cpu(t):
+    return t.detach().cpu().numpy()
+
+
+def run_gpu_cclip(g_np, tau, lens, **kw):
+    g = torch.from_numpy(np.ascontiguousarray(g_np)).cuda()
+    v0 = kw.pop("v0", None)
+    v = torch.from_numpy(np.ascontiguousarray(v0)).cuda().clone() if v0 is not None else None
+    r = btard.centered_clip(g, tau, part_len=lens, v=v, **kw)
+    torch.cuda.synchronize()
+    return g, r
+
+
+def check_cclip(r, ref, lens, eps_mode=False):
+    P = ref["v"].shape[0]
+    v = cpu(r["v"])
+    it = cpu(r["iters"])
+    for p in range(P):
+        L = int(lens[p])
+        if eps_mode:
+            assert abs(int(it[p]) - int(ref["iters"][p])) <= 1, (p, it[p], ref["iters"][p])
+            if it[p] != ref["iters"][p]:
+                continue
+        else:
+            assert it[p] == ref["iters"][p]
+        assert rel_l2(v[p, :L], ref["v"][p, :L]) <= RTOL, ("v", p)
+        assert np.all(v[p, L:] == 0)
+        assert rel_l2(cpu(r["resid_norm"])[p], ref["resid_norm"][p]) <= RTOL
+        ls, lr = cpu(r["last_step_norm"])[p], ref["last_step_norm"][p]
+        # the last step is a difference of nearly equal vectors: absolute floor from fp32 v
+        assert abs(ls - lr) <= 1e-4 * lr + 3e-7 * (1 + np.linalg.norm(ref["v"][p, :L])), (p, ls, lr)
+
+
+# ----------------------------------------------------------------------------- z and layout
+@pytest.mark.parametrize("seed,p,k,length", [(0, 0, 0, 1024), (0x1234567890ABCDEF, 3, 2, 4099),
+                                             (7, 15, 7, 698373), (2 ** 64 - 1, 63, 63, 1),
+                                             (5, 1, 0, 2), (5, 1, 0, 3), (5, 1, 0, 0), (9, 0, 1, 1 << 22)])
+def test_random_vector_is_bit_exact(seed, p, k, length):
+    z = cpu(btard.random_vector(seed, p, k, length))
+    ref = oracle.random_vector(seed, p, k, length)
+    assert np.array_equal(z.view(np.uint32), ref.view(np.uint32))
+
+
+def test_random_vector_rare_words():
+    """Exhaustive over the polynomial's inputs is too much; sweep many blocks so that every exponent
+    bucket of u and both sign bits occur, still bit for bit."""
+    z = cpu(btard.random_vector(123456789, 5, 3, 1 << 24))
+    ref = oracle.random_vector(123456789, 5, 3, 1 << 24)
+    assert np.array_equal(z.view(np.uint32), ref.view(np.uint32))
+
+
+# ----------------------------------------------------------------------------- CenteredClip
+def make_case(rng, P, n, stride, lens, far_rows=0, scale=0.02):
+    g = (rng.standard_normal((P, n, stride)) * scale).astype(np.float32)
+    g += rng.standard_normal((P, 1, stride)).astype(np.float32)          # common mean
+    if far_rows:
+        g[:, :far_rows] = (rng.standard_normal((P, far_rows, stride)) * 5).astype(np.float32)
+    for p in range(P):
+        g[p, :, lens[p]:] = 77.0                                           # garbage in the pad
+    return g
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 7, 8, 16, 23, 64, 100, 256])
+@pytest.mark.parametrize("init", [btard.INIT_ZERO, btard.INIT_MEAN, btard.INIT_COORD_MEDIAN,
+                                  btard.INIT_CALLER_V0])
+def test_fixed_iterations_match_oracle(n, init):
+    rng = np.random.default_rng(100 + n)
+    P, stride = 3, 5024
+    lens = np.array([5024, 4097, 0 if n % 2 else 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.5, 1.0, 2.0])
+    v0 = None
+    if init == btard.INIT_CALLER_V0:
+        v0 = rng.standard_normal((P, stride)).astype(np.float32)
+    ref = oracle.centered_clip(g, tau, lens, init_mode=init, v0=v0, max_iters=6)
+    _, r = run_gpu_cclip(g, tau, lens, init_mode=init, v0=v0, max_iters=6)
+    check_cclip(r, ref, lens)
+
+
+def test_many_tiles_per_cta_and_many_ctas():
+    """One long partition: several CTAs, each with many tiles, plus a ragged last tile."""
+    rng = np.random.default_rng(5)
+    P, n, stride = 2, 16, 1_000_032
+    lens = np.array([1_000_001, 999_999])
+    g = make_case(rng, P, n, stride, lens, far_rows=5, scale=0.001)
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=4)
+    check_cclip(r, ref, lens)
+
+
+def test_config1_fixed_and_eps():
+    w = workloads.make_workload(1)
+    g = w.g.numpy()
+    ref = oracle.centered_clip(g, w.tau, w.part_len, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=50)
+    _, r = run_gpu_cclip(g, w.tau, w.part_len, init_mode=btard.INIT_COORD_MEDIAN, max_iters=50)
+    check_cclip(r, ref, w.part_len)
+    ref = oracle.centered_clip(g, w.tau, w.part_len, init_mode=oracle.INIT_COORD_MEDIAN,
+                               stop_mode=oracle.STOP_EPS, max_iters=100, eps=1e-6)
+    _, r = run_gpu_cclip(g, w.tau, w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
+                         stop_mode=btard.STOP_EPS, max_iters=100, eps=1e-6)
+    check_cclip(r, ref, w.part_len, eps_mode=True)
+    assert cpu(r["status"])[0] == ref["status"][0] == 0
+
+
+def test_eps_mode_counts_and_cap_flag():
+    rng = np.random.default_rng(6)
+    P, n, stride = 4, 8, 2048
+    lens = np.array([2048, 2000, 1, 1027])
+    g = make_case(rng, P, n, stride, lens, far_rows=2)
+    for eps, cap in [(1e-3, 200), (1e-5, 200), (1e-5, 3)]:
+        ref = oracle.centered_clip(g, 0.7, lens, init_mode=oracle.INIT_MEAN, stop_mode=oracle.STOP_EPS,
+                                   max_iters=cap, eps=eps)
+        _, r = run_gpu_cclip(g, 0.7, lens, init_mode=btard.INIT_MEAN, stop_mode=btard.STOP_EPS,
+                             max_iters=cap, eps=eps)
+        check_cclip(r, ref, lens, eps_mode=True)
+        same = cpu(r["iters"]) == ref["iters"]
+        assert np.array_equal(cpu(r["status"])[same] & 1, ref["status"][same] & 1)
+    assert len(set(ref["iters"])) >= 1
+
+
+def test_special_radii():
+    rng = np.random.default_rng(7)
+    P, n, stride = 3, 5, 1024
+    lens = np.array([1024, 1000, 999])
+    g = make_case(rng, P, n, stride, lens)
+    tau = np.array([np.inf, 0.0, 1e-3])
+    ref = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_ZERO, max_iters=3)
+    _, r = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_ZERO, max_iters=3)
+    check_cclip(r, ref, lens)
+    v = cpu(r["v"])
+    assert rel_l2(v[0, :1024], g[0].astype(np.float64).mean(0)) < 1e-6     # tau = inf: the mean
+    assert np.all(v[1] == 0)                                               # tau = 0: never moves
+
+
+def test_non_finite_rows_take_weight_zero():
+    rng = np.random.default_rng(8)
+    P, n, stride = 2, 6, 1024
+    lens = np.array([1024, 1024])
+    g = make_case(rng, P, n, stride, lens)
+    g[0, 2, 17] = np.nan
+    g[1, 4, 900] = np.inf
+    g[1, 0, 3] = -np.inf
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_ZERO, max_iters=4)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_ZERO, max_iters=4)
+    v = cpu(r["v"])
+    assert np.all(np.isfinite(v))
+    for p in range(P):
+        assert rel_l2(v[p], ref["v"][p]) <= RTOL
+        assert cpu(r["status"])[p] & btard.STATUS_NONFINITE_ROW
+        assert ref["status"][p] & oracle.STATUS_NONFINITE_ROW
+    rn = cpu(r["resid_norm"])
+    assert np.array_equal(np.isfinite(rn), np.isfinite(ref["resid_norm"]))
+
+
+def test_peer_and_partition_indexing():
+    """Row i / slab p of every output belongs to peer i / partition p: distinct magnitudes."""
+    P, n, stride = 4, 5, 256
+    g = np.zeros((P, n, stride), dtype=np.float32)
+    for p in range(P):
+        for i in range(n):
+            g[p, i, :] = (p + 1) * 10 + i
+    lens = np.full(P, stride)
+    ref = oracle.centered_clip(g, np.inf, lens, init_mode=oracle.INIT_ZERO, max_iters=1)
+    _, r = run_gpu_cclip(g, np.inf, lens, init_mode=btard.INIT_ZERO, max_iters=1)
+    assert np.allclose(cpu(r["resid_norm"]), ref["resid_norm"], rtol=1e-6)
+    assert np.allclose(cpu(r["v"]), ref["v"], rtol=1e-6)
+
+
+# ----------------------------------------------------------------------------- verification
+def check_verify(out, ref, K):
+    P, n = ref["norm"].shape
+    for p in range(P):
+        for key in ("norm", "weight", "dot", "s"):
+            assert rel_l2(cpu(out[key])[p], ref[key][p]) <= RTOL, (key, p)
+        assert np.allclose(cpu(out["znorm2"])[p], ref["znorm2"][p], rtol=1e-6)
+        scale = np.abs(ref["s"][p]).sum(0) + 1e-300
+        assert np.all(np.abs(cpu(out["s_sum"])[p] - ref["s_sum"][p]) <= RTOL * scale), ("s_sum", p)
+        rscale = (ref["weight"][p] * ref["norm"][p]).sum() + 1e-300
+        assert abs(cpu(out["resid_sum_norm"])[p] - ref["resid_sum_norm"][p]) <= RTOL * rscale
+
+
+@pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (5, 3), (16, 8), (16, 1), (23, 4), (64, 4), (64, 8),
+                                 (64, 11), (100, 2), (200, 5)])
+def test_verify_matches_oracle(n, K):
+    rng = np.random.default_rng(200 + n + K)
+    P, stride = 3, 5024
+    lens = np.array([5024, 4097, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.5, 1.0, 2.0])
+    refc = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=8)
+    v32 = refc["v"].astype(np.float32)
+    seed = 0xABCDEF0123 + n
+    gd = torch.from_numpy(g).cuda()
+    vd = torch.from_numpy(v32).cuda()
+    # norms computed by the library itself
+    ref = oracle.verify(g, v32, tau, seed, K=K, part_len=lens, want_resid_sum=True)
+    out = btard.verify_projections(gd, vd, tau, seed, K=K, part_len=lens, want_resid_sum=True)
+    torch.cuda.synchronize()
+    check_verify(out, ref, K)
+    for p in range(P):
+        L = lens[p]
+        rs = cpu(out["resid_sum"])[p]
+        scale = (ref["weight"][p] * ref["norm"][p]).sum()
+        assert np.linalg.norm(rs[:L] - ref["resid_sum"][p, :L]) <= RTOL * scale
+    # norms handed over from the aggregation
+    nin = refc["resid_norm"]
+    ref2 = oracle.verify(g, v32, tau, seed, K=K, part_len=lens, norm_in=nin)
+    out2 = btard.verify_projections(gd, vd, tau, seed, K=K, part_len=lens,
+                                    resid_norm_in=torch.from_numpy(nin).cuda())
+    torch.cuda.synchronize()
+    check_verify(out2, ref2, K)
+
+
+def test_verify_partition_base_keys_z():
+    rng = np.random.default_rng(9)
+    P, n, stride, K = 2, 4, 1024, 2
+    lens = np.array([1024, 1001])
+    g = make_case(rng, P, n, stride, lens)
+    v = np.zeros((P, stride), dtype=np.float32)
+    ref = oracle.verify(g, v, 1.0, 11, K=K, part_len=lens, first_partition=5)
+    out = btard.verify_projections(torch.from_numpy(g).cuda(), torch.from_numpy(v).cuda(), 1.0, 11, K=K,
+                                   part_len=lens, partition_base=5)
+    torch.cuda.synchronize()
+    check_verify(out, ref, K)
+
+
+def test_wrong_aggregate_is_exposed_on_the_gpu_too():
+    """Aggregation attack (App. C): a modified v makes sum_i s_i visibly non-zero."""
+    w = workloads.make_workload(1)
+    g = w.g.cuda()
+    r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
+                            stop_mode=btard.STOP_EPS, max_iters=500, eps=1e-7)
+    good = btard.verify_projections(g, r["v"], w.tau, 0, K=4, part_len=w.part_len,
+                                    resid_norm_in=r["resid_norm"])
+    bad_v = r["v"] + 0.01 * torch.randn_like(r["v"])
+    bad = btard.verify_projections(g, bad_v, w.tau, 0, K=4, part_len=w.part_len)
+    torch.cuda.synchronize()
+    sg, sb = cpu(good["s_sum"])[0], cpu(bad["s_sum"])[0]
+    scale = np.abs(cpu(good["s"])[0]).sum(0)
+    assert np.all(np.abs(sg) < 1e-4 * scale)
+    assert np.all(np.abs(sb) > 10 * np.abs(sg))
+
+
+# ----------------------------------------------------------------------------- host-buffer path
+def test_aggregate_host_matches_device_path():
+    rng = np.random.default_rng(10)
+    P, n, stride, K = 3, 16, 4128, 2
+    lens = np.array([4128, 4100, 4001])
+    g = make_case(rng, P, n, stride, lens, far_rows=4)
+    gh = torch.from_numpy(g).pin_memory()
+    h = btard.aggregate_host(gh, 1.0, 77, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                             max_iters=7)
+    gd = torch.from_numpy(g).cuda()
+    r = btard.centered_clip(gd, 1.0, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=7)
+    o = btard.verify_projections(gd, r["v"], 1.0, 77, K=K, part_len=lens, resid_norm_in=r["resid_norm"])
+    torch.cuda.synchronize()
+    assert torch.equal(h["v"], r["v"].cpu())
+    for key in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm"):
+        assert torch.equal(h[key], o[key].cpu()), key
+    assert torch.equal(h["iters"], r["iters"].cpu())
+
+
+# ----------------------------------------------------------------------------- full-size configs
+def _full_config(cfg, sample, max_iters=None, stop=None):
+    """Runs configuration `cfg` at full size on the GPU in the benchmark's launch configuration and
+    compares the sampled partitions with the oracle."""
+    w = workloads.make_workload(cfg, device="cuda")
+    stop_mode = w.stop_mode if stop is None else stop
+    iters = w.max_iters if max_iters is None else max_iters
+    r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
+                            stop_mode=stop_mode, max_iters=iters, eps=w.eps)
+    o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                 resid_norm_in=r["resid_norm"])
+    torch.cuda.synchronize()
+    for p in sample:
+        gp = cpu(w.g[p:p + 1])
+        lens = w.part_len[p:p + 1]
+        ref = oracle.centered_clip(gp, w.tau[p], lens, init_mode=oracle.INIT_COORD_MEDIAN,
+                                   stop_mode=stop_mode, max_iters=iters, eps=w.eps)
+        sub = {k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}
+        check_cclip(sub, ref, lens, eps_mode=(stop_mode == btard.STOP_EPS))
+        vp = cpu(r["v"][p:p + 1])
+        nin = cpu(r["resid_norm"][p:p + 1])
+        refv = oracle.verify(gp, vp, w.tau[p], w.zseed, K=w.K, part_len=lens, norm_in=nin,
+                             first_partition=p)
+        subo = {k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2",
+                                          "resid_sum_norm")}
+        check_verify(subo, refv, w.K)
+    return w, r, o
+
+
+def test_config2_full_size_sampled():
+    w, r, o = _full_config(2, sample=[0, 15])
+    # fixed-iteration parity at full size as well (eps mode may differ by one update)
+    _full_config(2, sample=[7], max_iters=10, stop=btard.STOP_FIXED_ITERS)
+
+
+def test_config3_full_size_sampled():
+    _full_config(3, sample=[3, 15], max_iters=10, stop=btard.STOP_FIXED_ITERS)
+    _full_config(3, sample=[9])
+
+
+def test_config4_full_size_sampled():
+    _full_config(4, sample=[0, 63])
+    _full_config(4, sample=[31], max_iters=5, stop=btard.STOP_FIXED_ITERS)
