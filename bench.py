@@ -119,6 +119,8 @@ def run_ours(args):
     btard.lib()
 
     w = workloads.make_workload(args.config, device="cuda")
+    if args.max_iters:
+        w.max_iters = args.max_iters
     g = w.g
     P, n, stride = g.shape
     dev = g.device
@@ -289,6 +291,8 @@ def run_reference(args):
     P = wmeta.P
     sample = list(range(0, P, max(1, P // max(1, min(cores, P)))))[:cores]
     w = workloads.make_workload(args.config, device="cpu", partitions=sample)
+    if args.max_iters:
+        w.max_iters = args.max_iters
     g = w.g.numpy()
     iters = None
 
@@ -328,6 +332,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

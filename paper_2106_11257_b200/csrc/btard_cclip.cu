@@ -12,6 +12,8 @@
 // Cross-CTA sums are not atomics: every CTA writes its partial sums to its own slot and the next
 // pass adds the slots of its partition in a fixed order, so results are reproducible run to run.
 // The stop rule is evaluated the same way by every CTA of a partition at the top of each pass.
+#include <type_traits>
+
 #include "btard_common.h"
 
 namespace btard {
@@ -87,7 +89,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 {
     extern __shared__ float4 sh_x[];                  // [2][RG][CL] exchange of partial column sums
     __shared__ double sh_sum[BTARD_MAX_PEERS + 1];
-    __shared__ float sh_w[BTARD_MAX_PEERS];
+    __shared__ float sh_w[BTARD_MAX_PEERS + 16];      // zero beyond row n - 1
     __shared__ double sh_red[16][17];
     __shared__ int sh_flag;
 
@@ -99,7 +101,6 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const long long len = a.table[p].len;
     const double tau = a.table[p].tau;
 
-    float Wsum = 0.0f;
     if (MODE == PASS_ITER) {
         if (a.done[p]) return;
         // Sum the previous pass's slots in a fixed order: norms at the current v, and its step.
@@ -117,40 +118,43 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
         if (tid == 0) sh_flag = 0;
         __syncthreads();
-        for (int i = tid; i < n; i += blockDim.x) {
+        for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) {
             bool bad = false;
-            sh_w[i] = clip_weight(sh_sum[i], tau, bad);
+            sh_w[i] = (i < n) ? clip_weight(sh_sum[i], tau, bad) : 0.0f;
             if (bad) sh_flag = 1;
         }
         __syncthreads();
         if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
-        for (int i = 0; i < n; ++i) Wsum += sh_w[i];
     } else if (MODE == PASS_INIT) {
         if (j == 0 && tid == 0) { a.done[p] = 0; a.status[p] = 0; }
     }
-    (void)Wsum;
-
-    float w[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const int i = rg * R + r;
-        w[r] = (MODE == PASS_ITER && i < n) ? sh_w[i] : 0.0f;
-    }
+    const float* wrow = sh_w + rg * R;                // this thread's R clip weights
 
     float acc[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[r] = 0.0f;
     float step_acc = 0.0f;
 
-    const long long t0 = (long long)k.tiles * j / cpp, t1 = (long long)k.tiles * (j + 1) / cpp;
     const float* gp = a.g + (size_t)p * n * stride;
     float* vp = a.v + (size_t)p * stride;
     unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
     const float nf = (float)n;
 
-    for (long long t = t0; t < t1; ++t) {
-        const long long col = (t * CL + cl) * 4;
-        const bool valid = col < stride;
+    // This CTA's share of the partition, in groups of 4 columns ("quads"), cut on 128-byte lines.
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cpp) q1 &= ~7LL;
+    const long long full_quads = len >> 2;             // quads that lie entirely inside the data
+
+    // One tile: CL quads starting at quad qb.  MASKED = false when every lane's quad is inside both
+    // the CTA's range and the data, so no predicate is needed.
+    auto tile = [&](auto masked_tag, long long qb, int parity) {
+        constexpr bool MASKED = decltype(masked_tag)::value;
+        const long long col = (qb + cl) * 4;
+        const bool valid = !MASKED || (qb + cl < q1);
+        const bool m0 = !MASKED || (valid && col < len), m1 = !MASKED || (valid && col + 1 < len);
+        const bool m2 = !MASKED || (valid && col + 2 < len), m3 = !MASKED || (valid && col + 3 < len);
         float4 x[R];
         float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f);      // low-order part of v (COMP)
@@ -171,26 +175,32 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 #pragma unroll
             for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len, m3 = col + 3 < len;
+        if (MODE != PASS_INIT) {                       // residuals at the current v
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = (x[r].x - v4.x) - lo4.x; x[r].y = (x[r].y - v4.y) - lo4.y;
+                x[r].z = (x[r].z - v4.z) - lo4.z; x[r].w = (x[r].w - v4.w) - lo4.w;
+            }
+        }
 
         float4 vn = v4;                                // v after this pass
+        float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);   // what the represented v moved by
         if (MODE == PASS_ITER || (MODE == PASS_INIT && a.init_mode == BTARD_INIT_MEAN)) {
             float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 if (MODE == PASS_ITER) {
-                    if (w[r] != 0.0f) {                // weight 0: the row is left out, not multiplied
-                        s4.x = fmaf(w[r], (x[r].x - v4.x) - lo4.x, s4.x);
-                        s4.y = fmaf(w[r], (x[r].y - v4.y) - lo4.y, s4.y);
-                        s4.z = fmaf(w[r], (x[r].z - v4.z) - lo4.z, s4.z);
-                        s4.w = fmaf(w[r], (x[r].w - v4.w) - lo4.w, s4.w);
+                    const float wr = wrow[r];
+                    if (wr != 0.0f) {                  // weight 0: the row is left out, not multiplied
+                        s4.x = fmaf(wr, x[r].x, s4.x); s4.y = fmaf(wr, x[r].y, s4.y);
+                        s4.z = fmaf(wr, x[r].z, s4.z); s4.w = fmaf(wr, x[r].w, s4.w);
                     }
                 } else {
                     s4.x += x[r].x; s4.y += x[r].y; s4.z += x[r].z; s4.w += x[r].w;
                 }
             }
             if (RG > 1) {                              // add the row groups' partial column sums
-                float4* buf = sh_x + (size_t)(t & 1) * RG * CL;
+                float4* buf = sh_x + (size_t)parity * RG * CL;
                 buf[rg * CL + cl] = s4;
                 __syncthreads();
                 s4 = buf[cl];
@@ -199,23 +209,26 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
                     s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
                 }
             }
-            const float4 u = make_float4(s4.x / nf, s4.y / nf, s4.z / nf,
-                                         s4.w / nf);
+            const float4 u = make_float4(s4.x / nf, s4.y / nf, s4.z / nf, s4.w / nf);
             if (MODE == PASS_ITER) {
                 if (COMP) {
                     uint32_t b0, b1, b2, b3;
-                    two_sum_bf16(v4.x, lo4.x + u.x, vn.x, lo4.x, b0);
-                    two_sum_bf16(v4.y, lo4.y + u.y, vn.y, lo4.y, b1);
-                    two_sum_bf16(v4.z, lo4.z + u.z, vn.z, lo4.z, b2);
-                    two_sum_bf16(v4.w, lo4.w + u.w, vn.w, lo4.w, b3);
-                    if (!m0) { b0 = 0; lo4.x = 0.f; }
-                    if (!m1) { b1 = 0; lo4.y = 0.f; }
-                    if (!m2) { b2 = 0; lo4.z = 0.f; }
-                    if (!m3) { b3 = 0; lo4.w = 0.f; }
+                    float4 ln;
+                    two_sum_bf16(v4.x, lo4.x + u.x, vn.x, ln.x, b0);
+                    two_sum_bf16(v4.y, lo4.y + u.y, vn.y, ln.y, b1);
+                    two_sum_bf16(v4.z, lo4.z + u.z, vn.z, ln.z, b2);
+                    two_sum_bf16(v4.w, lo4.w + u.w, vn.w, ln.w, b3);
+                    if (!m0) b0 = 0;
+                    if (!m1) b1 = 0;
+                    if (!m2) b2 = 0;
+                    if (!m3) b3 = 0;
+                    dv = make_float4((vn.x - v4.x) + (ln.x - lo4.x), (vn.y - v4.y) + (ln.y - lo4.y),
+                                     (vn.z - v4.z) + (ln.z - lo4.z), (vn.w - v4.w) + (ln.w - lo4.w));
                     if (rg == 0 && valid)
                         *reinterpret_cast<uint2*>(lop + col) = make_uint2(b0 | (b1 << 16), b2 | (b3 << 16));
                 } else {
                     vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+                    dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
                 }
                 if (rg == 0)
                     step_acc += (m0 ? u.x * u.x : 0.f) + (m1 ? u.y * u.y : 0.f) +
@@ -231,13 +244,20 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         if (!m2) vn.z = 0.f;
         if (!m3) vn.w = 0.f;
         if (MODE != PASS_NORMS && rg == 0 && valid) *reinterpret_cast<float4*>(vp + col) = vn;
+        if (MODE == PASS_INIT) dv = vn;                // x still holds the rows themselves
 
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const float dx = m0 ? (x[r].x - vn.x) - lo4.x : 0.f, dy = m1 ? (x[r].y - vn.y) - lo4.y : 0.f;
-            const float dz = m2 ? (x[r].z - vn.z) - lo4.z : 0.f, dw = m3 ? (x[r].w - vn.w) - lo4.w : 0.f;
+        for (int r = 0; r < R; ++r) {                  // residuals at the new v
+            const float dx = m0 ? x[r].x - dv.x : 0.f, dy = m1 ? x[r].y - dv.y : 0.f;
+            const float dz = m2 ? x[r].z - dv.z : 0.f, dw = m3 ? x[r].w - dv.w : 0.f;
             acc[r] += fmaf(dx, dx, fmaf(dy, dy, fmaf(dz, dz, dw * dw)));
         }
+    };
+
+    int parity = 0;
+    for (long long qb = q0; qb < q1; qb += CL, parity ^= 1) {
+        if (qb + CL <= q1 && qb + CL <= full_quads) tile(std::false_type{}, qb, parity);
+        else tile(std::true_type{}, qb, parity);
     }
 
     // CTA reduction: lanes of a warp share a row group, so a warp reduces R rows at once.
@@ -399,6 +419,41 @@ int launch_pass_r(const KernelArgs& ka, int mode, int threads, size_t smem, int 
 
 }  // namespace
 
+// Resident CTAs per SM of the iteration kernel for this shape (2 when no device can be asked).
+static int iter_ctas_per_sm(int R, int threads, size_t smem)
+{
+    int nb = 0;
+    cudaError_t e;
+    if (R == 4) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_pass_kernel<4, PASS_ITER, true>, threads, smem);
+    else if (R == 8) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_pass_kernel<8, PASS_ITER, true>, threads, smem);
+    else e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_pass_kernel<16, PASS_ITER, true>, threads, smem);
+    if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 2; }
+    return nb;
+}
+
+// CTAs per partition: the smallest count that respects the bound on tiles per CTA, then the count
+// within reach that fills whole waves of resident CTAs best.
+int choose_ctas_per_partition(int P, long long quads, int CL, int slots)
+{
+    long long cmin = (quads + (long long)(kMaxTilesPerCta - 1) * CL - 1) / ((long long)(kMaxTilesPerCta - 1) * CL);
+    if (cmin < 1) cmin = 1;
+    long long cmax_work = (quads + 7) / 8;             // never less than one 128-byte line per CTA
+    if (cmax_work < 1) cmax_work = 1;
+    long long lo = cmin, hi = cmin + (4LL * slots + P - 1) / P;
+    if (lo > cmax_work) lo = cmax_work;
+    if (hi > cmax_work) hi = cmax_work;
+    long long best = lo;
+    double best_score = -1.0;
+    for (long long c = lo; c <= hi; ++c) {
+        const long long total = c * P;
+        const long long waves = (total + slots - 1) / slots;
+        double score = (double)total / (double)(waves * slots);     // fraction of the last wave used
+        if (total < slots) score *= 0.5;                            // under one wave: SMs idle
+        if (score > best_score + 1e-9) { best_score = score; best = c; }
+    }
+    return (int)best;
+}
+
 Geometry cclip_geometry(int n, int P, long long stride)
 {
     Geometry g;
@@ -406,27 +461,10 @@ Geometry cclip_geometry(int n, int P, long long stride)
     g.RG = (n + g.R - 1) / g.R;
     g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 8) ? 64 : 32;
     g.threads = g.RG * g.CL;
-    const long long cols = 4LL * g.CL;
-    g.tiles = (int)((stride + cols - 1) / cols);
-    // Enough CTAs to fill every SM twice over, few enough tiles per CTA to bound the fp32 running
-    // sums, and a total close to a whole number of waves.
-    const int ctas_per_sm = (g.threads <= 256) ? 2 : 1;
-    const int slots = sm_count() * ctas_per_sm;
-    int cmin = (g.tiles + kMaxTilesPerCta - 1) / kMaxTilesPerCta;
-    if (cmin < 1) cmin = 1;
-    int want = (slots + P - 1) / P;
-    if (want < cmin) want = cmin;
-    if (want > g.tiles) want = g.tiles;
-    if (want < 1) want = 1;
-    int best = want;
-    double best_eff = -1.0;
-    for (int c = want; c <= want + 8 && c <= (g.tiles > 0 ? g.tiles : 1); ++c) {
-        const long long total = (long long)c * P;
-        const long long waves = (total + slots - 1) / slots;
-        const double eff = (double)total / (double)(waves * slots);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = c; }
-    }
-    g.cpp = best;
+    g.tiles = 0;
+    const size_t smem = (g.RG > 1) ? sizeof(float4) * 2 * g.RG * g.CL : 0;
+    const int slots = sm_count() * iter_ctas_per_sm(g.R, g.threads, smem);
+    g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, slots);
     return g;
 }
 

@@ -21,7 +21,7 @@ struct Geometry {
     int RG;       // row groups = ceil(n / R)
     int CL;       // column lanes (multiple of 32)
     int threads;  // RG * CL
-    int tiles;    // tiles per partition = ceil(row_stride / (4 CL))
+    int tiles;    // unused
     int cpp;      // CTAs per partition
 };
 
@@ -73,6 +73,7 @@ struct CclipLaunch {
 };
 
 Geometry cclip_geometry(int n, int P, long long stride);
+int choose_ctas_per_partition(int P, long long quads, int CL, int slots);
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
 int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,

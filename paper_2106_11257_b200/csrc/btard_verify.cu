@@ -66,19 +66,23 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     for (int q = 0; q < KT; ++q) zz[q] = 0.0f;
     float rs2 = 0.0f;
 
-    const long long t0 = (long long)k.tiles * j / cpp, t1 = (long long)k.tiles * (j + 1) / cpp;
+    // This CTA's share of the partition in groups of 4 columns, cut on 128-byte lines.
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cpp) q1 &= ~7LL;
     const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v + (size_t)p * stride;
     float* rsp = a.resid_sum ? a.resid_sum + (size_t)p * stride : nullptr;
     const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
     const uint32_t pg = (uint32_t)(a.p_base + p);
 
-    // Adds up the row groups' column sums of tile tt (written one tile earlier).
-    auto consume_sums = [&](long long tt) {
+    // Adds up the row groups' column sums of the tile at quad qb (written one tile earlier).
+    auto consume_sums = [&](long long qb, int par) {
         if (rg != 0) return;
-        const long long col = (tt * CL + cl) * 4;
-        if (col >= stride) return;
-        const float4* buf = sh_s + (size_t)(tt & 1) * RG * CL;
+        if (qb + cl >= q1) return;
+        const long long col = (qb + cl) * 4;
+        const float4* buf = sh_s + (size_t)par * RG * CL;
         float4 s4 = buf[cl];
         for (int q = 1; q < RG; ++q) {
             const float4 o = buf[q * CL + cl];
@@ -88,14 +92,15 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
         if (rsp) *reinterpret_cast<float4*>(rsp + col) = s4;
     };
 
-    for (long long t = t0; t < t1; ++t) {
+    int par = 0;
+    for (long long qb = q0; qb < q1; qb += CL, par ^= 1) {
         // 1. this tile's block of z
-        float4* zb = sh_z + (size_t)(t & 1) * KT * CL;
+        float4* zb = sh_z + (size_t)par * KT * CL;
         for (int idx = tid; idx < KT * CL; idx += nthr) {
             const int kq = idx / CL, cq = idx % CL;
-            const long long col = (t * CL + cq) * 4;
+            const long long col = (qb + cq) * 4;
             float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kq < a.kc && col < len) {
+            if (kq < a.kc && qb + cq < q1 && col < len) {
                 z = z_quad((uint32_t)(col >> 2), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
                 if (col + 1 >= len) z.y = 0.f;
                 if (col + 2 >= len) z.z = 0.f;
@@ -104,12 +109,13 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
             zb[kq * CL + cq] = z;
         }
         __syncthreads();
-        if (first_chunk && t > t0) consume_sums(t - 1);
+        if (first_chunk && qb > q0) consume_sums(qb - CL, par ^ 1);
 
         // 2. residuals of this thread's rows and columns
-        const long long col = (t * CL + cl) * 4;
-        const bool valid = col < stride;
-        const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len, m3 = col + 3 < len;
+        const long long col = (qb + cl) * 4;
+        const bool valid = qb + cl < q1;
+        const bool m0 = valid && col < len, m1 = valid && col + 1 < len;
+        const bool m2 = valid && col + 2 < len, m3 = valid && col + 3 < len;
         float4 x[R];
         float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
         if (valid) {
@@ -152,11 +158,11 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
                     s4.w = fmaf(w[r], x[r].w, s4.w);
                 }
             }
-            sh_s[(size_t)(t & 1) * RG * CL + rg * CL + cl] = s4;
+            sh_s[(size_t)par * RG * CL + rg * CL + cl] = s4;
         }
     }
     __syncthreads();
-    if (first_chunk && t1 > t0) consume_sums(t1 - 1);
+    if (first_chunk && q1 > q0) consume_sums(q0 + (q1 - q0 - 1) / CL * CL, par ^ 1);
 
     // CTA reduction
     const int warp = tid >> 5, lane = tid & 31, wpg = CL >> 5;
@@ -277,6 +283,29 @@ int launch_r(const VArgs& va, int KT, int threads, size_t smem, int grid, cudaSt
     return BTARD_ERR_UNSUPPORTED;
 }
 
+template <int R>
+int occ_r(int KT, int threads, size_t smem, int* nb)
+{
+    cudaError_t e = cudaErrorInvalidValue;
+    if (KT == 1) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 1>, threads, smem);
+    else if (KT == 2) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 2>, threads, smem);
+    if constexpr (R <= 8) {
+        if (KT == 4) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 4>, threads, smem);
+        else if (KT == 8) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 8>, threads, smem);
+    }
+    return (int)e;
+}
+
+int verify_ctas_per_sm(int R, int KT, int threads, size_t smem)
+{
+    int nb = 0, e;
+    if (R == 4) e = occ_r<4>(KT, threads, smem, &nb);
+    else if (R == 8) e = occ_r<8>(KT, threads, smem, &nb);
+    else e = occ_r<16>(KT, threads, smem, &nb);
+    if (e != 0 || nb < 1) { (void)cudaGetLastError(); return 2; }
+    return nb;
+}
+
 }  // namespace
 
 VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
@@ -297,24 +326,10 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     while (kt < K && kt < 8) kt <<= 1;
     if (g.R == 16 && kt > 2) kt = 2;          // 16 rows per thread: keep the accumulators in registers
     vg.KT = kt;
-    const long long cols = 4LL * g.CL;
-    g.tiles = (int)((stride + cols - 1) / cols);
-    const int ctas_per_sm = (g.threads <= 256) ? 2 : 1;
-    const int slots = sm_count() * ctas_per_sm;
-    int cmin = (g.tiles + kMaxTilesPerCta - 1) / kMaxTilesPerCta;
-    int want = (slots + P - 1) / P;
-    if (want < cmin) want = cmin;
-    if (want > g.tiles) want = g.tiles;
-    if (want < 1) want = 1;
-    int best = want;
-    double best_eff = -1.0;
-    for (int c = want; c <= want + 8 && c <= (g.tiles > 0 ? g.tiles : 1); ++c) {
-        const long long total = (long long)c * P;
-        const long long waves = (total + slots - 1) / slots;
-        const double eff = (double)total / (double)(waves * slots);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = c; }
-    }
-    g.cpp = best;
+    g.tiles = 0;
+    const size_t smem = sizeof(float4) * (2 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
+    const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, g.threads, smem);
+    g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, slots);
     vg.slots = n * kt + kt + 1;
     return vg;
 }
