@@ -81,7 +81,7 @@ int check_common(int n, int P, long long stride, const int64_t* part_len, const 
 }
 
 struct CclipWorkspace {
-    size_t table, part[2], done, v_lo, v_lo_bytes, total;
+    size_t table, slots, tot[2], flags, flags_bytes, v_lo, v_lo_bytes, total;
 };
 
 // EPS mode carries v as fp32 + a bf16 correction so that the stop test sees steps far below the
@@ -91,10 +91,11 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, co
     CclipWorkspace w;
     size_t off = 0;
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
-    const size_t part_bytes = sizeof(double) * (size_t)P * geo.cpp * (n + 1);
-    w.part[0] = off; off = align_up(off + part_bytes, 256);
-    w.part[1] = off; off = align_up(off + part_bytes, 256);
-    w.done = off; off = align_up(off + sizeof(int) * P, 256);
+    w.slots = off; off = align_up(off + sizeof(double) * (size_t)P * geo.cpp * (n + 1), 256);
+    w.tot[0] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
+    w.tot[1] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
+    w.flags_bytes = sizeof(int) * 2 * (size_t)P;              // done[P], ticket[P]
+    w.flags = off; off = align_up(off + w.flags_bytes, 256);
     w.v_lo_bytes = (stop_mode == BTARD_STOP_EPS) ? sizeof(unsigned short) * (size_t)P * stride : 0;
     w.v_lo = off; off = align_up(off + w.v_lo_bytes, 256);
     w.total = off;
@@ -102,7 +103,7 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, co
 }
 
 struct VerifyWorkspace {
-    size_t table, part, norms, cpart, total;
+    size_t table, part, norms, cslots, ctot, cticket, total;
 };
 
 VerifyWorkspace verify_ws_layout(int n, int P, const VerifyGeometry& vg, const Geometry& cg)
@@ -112,7 +113,9 @@ VerifyWorkspace verify_ws_layout(int n, int P, const VerifyGeometry& vg, const G
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
     w.part = off; off = align_up(off + sizeof(double) * (size_t)P * vg.g.cpp * vg.slots, 256);
     w.norms = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
-    w.cpart = off; off = align_up(off + sizeof(double) * (size_t)P * cg.cpp * (n + 1), 256);
+    w.cslots = off; off = align_up(off + sizeof(double) * (size_t)P * cg.cpp * (n + 1), 256);
+    w.ctot = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
+    w.cticket = off; off = align_up(off + sizeof(unsigned int) * (size_t)P, 256);
     w.total = off;
     return w;
 }
@@ -219,15 +222,18 @@ int btard_centered_clip(const btard_cclip_args* a)
     CclipLaunch L{};
     L.g = a->g; L.v = a->v;
     L.table = (const PartEntry*)(base + ws.table);
-    L.done = (int*)(base + ws.done);
+    L.done = (int*)(base + ws.flags);
+    L.ticket = (unsigned int*)(base + ws.flags) + P;
+    L.slots = (double*)(base + ws.slots);
     L.iters = a->iters; L.last_step = a->last_step_norm; L.resid_norm = a->resid_norm;
     L.status = a->status;
     L.stride = a->row_stride; L.n = n; L.P = P;
     L.stop_mode = a->stop_mode; L.max_iters = a->max_iters; L.eps2 = a->eps * a->eps;
-    double* part[2] = {(double*)(base + ws.part[0]), (double*)(base + ws.part[1])};
+    double* tot[2] = {(double*)(base + ws.tot[0]), (double*)(base + ws.tot[1])};
 
     rc = upload_table((PartEntry*)(base + ws.table), P, a->part_len, a->tau, st);
     if (rc != BTARD_OK) return rc;
+    BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.flags, 0, ws.flags_bytes, st));
     if (ws.v_lo_bytes) {
         L.v_lo = (unsigned short*)(base + ws.v_lo);
         BTARD_CUDA_TRY(cudaMemsetAsync(L.v_lo, 0, ws.v_lo_bytes, st));
@@ -240,17 +246,17 @@ int btard_centered_clip(const btard_cclip_args* a)
         if (rc != BTARD_OK) return rc;
         L.init_mode = BTARD_INIT_CALLER_V0;
     }
-    L.part_in = nullptr; L.part_out = part[0]; L.l = 0;
+    L.tot_in = nullptr; L.tot_out = tot[0]; L.l = 0;
     rc = launch_cclip_pass(L, geo, PASS_INIT, st);
     if (rc != BTARD_OK) return rc;
 
-    // Update l reads the slots of buffer l % 2 and writes buffer (l + 1) % 2.
+    // Update l reads the totals in buffer l % 2 and writes buffer (l + 1) % 2.
     for (int l = 0; l < a->max_iters; ++l) {
-        L.l = l; L.part_in = part[l & 1]; L.part_out = part[(l + 1) & 1];
+        L.l = l; L.tot_in = tot[l & 1]; L.tot_out = tot[(l + 1) & 1];
         rc = launch_cclip_pass(L, geo, PASS_ITER, st);
         if (rc != BTARD_OK) return rc;
     }
-    L.part_in = part[a->max_iters & 1];
+    L.tot_in = tot[a->max_iters & 1];
     return launch_cclip_finalize(L, geo, st);
 }
 
@@ -292,11 +298,14 @@ int btard_verify_projections(const btard_verify_args* a)
     if (!norms) {   // one more pass: residual norms at v
         CclipLaunch L{};
         L.g = a->g; L.v = const_cast<float*>(a->v); L.table = table;
-        L.part_out = (double*)(base + ws.cpart);
+        L.slots = (double*)(base + ws.cslots);
+        L.tot_out = (double*)(base + ws.ctot);
+        L.ticket = (unsigned int*)(base + ws.cticket);
+        BTARD_CUDA_TRY(cudaMemsetAsync(L.ticket, 0, sizeof(unsigned int) * (size_t)P, st));
         L.stride = a->row_stride; L.n = n; L.P = P;
         rc = launch_cclip_pass(L, cg, PASS_NORMS, st);
         if (rc != BTARD_OK) return rc;
-        rc = launch_partials_to_norms(L.part_out, (double*)(base + ws.norms), n, P, cg.cpp, st);
+        rc = launch_totals_to_norms(L.tot_out, (double*)(base + ws.norms), n, P, st);
         if (rc != BTARD_OK) return rc;
         norms = (const double*)(base + ws.norms);
     }

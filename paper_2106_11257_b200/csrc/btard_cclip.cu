@@ -9,9 +9,10 @@
 //   u[c]  = (1/n) sum_i w_i (x_i[c] - v[c]);  v'[c] = v[c] + u[c]  (eq. (CenteredClip))
 //   norm2_i += (x_i[c] - v'[c])^2;  step2 += u[c]^2               (feeds the next pass)
 //
-// Cross-CTA sums are not atomics: every CTA writes its partial sums to its own slot and the next
-// pass adds the slots of its partition in a fixed order, so results are reproducible run to run.
-// The stop rule is evaluated the same way by every CTA of a partition at the top of each pass.
+// Cross-CTA sums are not floating-point atomics: every CTA writes its partial sums to its own slot,
+// and the CTA of a partition that finishes last (an integer ticket, nobody waits) adds the slots in
+// a fixed order, so results are reproducible run to run.  The stop rule is evaluated the same way
+// by every CTA of a partition at the top of the next pass, from those totals.
 #include <type_traits>
 
 #include "btard_common.h"
@@ -91,6 +92,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     __shared__ double sh_sum[BTARD_MAX_PEERS + 1];
     __shared__ float sh_w[BTARD_MAX_PEERS + 16];      // zero beyond row n - 1
     __shared__ double sh_red[16][17];
+    __shared__ double sh_part[512 + BTARD_MAX_PEERS + 1];
     __shared__ int sh_flag;
 
     const CclipLaunch& a = k.a;
@@ -103,13 +105,9 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 
     if (MODE == PASS_ITER) {
         if (a.done[p]) return;
-        // Sum the previous pass's slots in a fixed order: norms at the current v, and its step.
-        const double* src = a.part_in + (size_t)p * cpp * (n + 1);
-        for (int i = tid; i <= n; i += blockDim.x) {
-            double s = 0.0;
-            for (int c = 0; c < cpp; ++c) s += src[(size_t)c * (n + 1) + i];
-            sh_sum[i] = s;
-        }
+        // Totals the previous pass left behind: squared norms at the current v, and its squared step.
+        const double* src = a.tot_in + (size_t)p * (n + 1);
+        for (int i = tid; i <= n; i += blockDim.x) sh_sum[i] = __ldcg(src + i);
         __syncthreads();
         const bool converged = (a.stop_mode == BTARD_STOP_EPS) && a.l >= 1 && (sh_sum[n] <= a.eps2);
         if (converged) {                              // same decision in every CTA of the partition
@@ -128,6 +126,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     } else if (MODE == PASS_INIT) {
         if (j == 0 && tid == 0) { a.done[p] = 0; a.status[p] = 0; }
     }
+    (void)tau;
     const float* wrow = sh_w + rg * R;                // this thread's R clip weights
 
     float acc[R];
@@ -138,7 +137,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const float* gp = a.g + (size_t)p * n * stride;
     float* vp = a.v + (size_t)p * stride;
     unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
-    const float nf = (float)n;
+    const float inv_n = 1.0f / (float)n;
 
     // This CTA's share of the partition, in groups of 4 columns ("quads"), cut on 128-byte lines.
     const long long Q = stride >> 2;
@@ -209,7 +208,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
                     s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
                 }
             }
-            const float4 u = make_float4(s4.x / nf, s4.y / nf, s4.z / nf, s4.w / nf);
+            const float4 u = make_float4(s4.x * inv_n, s4.y * inv_n, s4.z * inv_n, s4.w * inv_n);
             if (MODE == PASS_ITER) {
                 if (COMP) {
                     uint32_t b0, b1, b2, b3;
@@ -272,7 +271,8 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         if (lane == 0) sh_red[warp][16] = s;
     }
     __syncthreads();
-    double* dst = a.part_out + ((size_t)p * cpp + j) * (n + 1);
+    double* slots = a.slots + (size_t)p * cpp * (n + 1);
+    double* dst = slots + (size_t)j * (n + 1);
     for (int i = tid; i <= n; i += blockDim.x) {
         double s = 0.0;
         if (i < n) {
@@ -283,6 +283,33 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
         dst[i] = s;
     }
+
+    // The CTA that finishes last adds up the partition's slots (fixed grouping, fixed order) and
+    // leaves the totals for the next pass.  No CTA waits for another.
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sh_flag = (atomicAdd(&a.ticket[p], 1u) == (unsigned)(cpp - 1));
+    __syncthreads();
+    if (!sh_flag) return;
+    __threadfence();
+    const int per = n + 1;
+    int groups = blockDim.x / per;
+    if (groups < 1) groups = 1;
+    if (groups > cpp) groups = cpp;
+    for (int e = tid; e < groups * per; e += blockDim.x) {
+        const int cg = e / per, i = e - cg * per;
+        double s = 0.0;
+        for (int c = cg; c < cpp; c += groups) s += __ldcg(slots + (size_t)c * per + i);
+        sh_part[e] = s;
+    }
+    __syncthreads();
+    double* tot = a.tot_out + (size_t)p * per;
+    for (int i = tid; i < per; i += blockDim.x) {
+        double s = 0.0;
+        for (int cg = 0; cg < groups; ++cg) s += sh_part[cg * per + i];
+        tot[i] = s;
+    }
+    if (tid == 0) a.ticket[p] = 0;
 }
 
 // After the last pass: partitions still running take iters = max_iters.
@@ -292,24 +319,17 @@ __global__ void cclip_finalize_kernel(const KernelArgs k)
     const CclipLaunch& a = k.a;
     const int p = blockIdx.x, n = a.n;
     if (a.done[p]) return;
-    const double* src = a.part_in + (size_t)p * k.cpp * (n + 1);
-    for (int i = threadIdx.x; i <= n; i += blockDim.x) {
-        double s = 0.0;
-        for (int c = 0; c < k.cpp; ++c) s += src[(size_t)c * (n + 1) + i];
-        sh_sum[i] = s;
-    }
+    const double* src = a.tot_in + (size_t)p * (n + 1);
+    for (int i = threadIdx.x; i <= n; i += blockDim.x) sh_sum[i] = src[i];
     __syncthreads();
     finish_partition(k, p, sh_sum, a.max_iters, a.stop_mode == BTARD_STOP_EPS);
 }
 
-__global__ void partials_to_norms_kernel(const double* part, double* norm, int n, int cpp)
+__global__ void totals_to_norms_kernel(const double* tot, double* norm, int n)
 {
     const int p = blockIdx.x;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        double s = 0.0;
-        for (int c = 0; c < cpp; ++c) s += part[((size_t)p * cpp + c) * (n + 1) + i];
-        norm[(size_t)p * n + i] = sqrt(s);
-    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        norm[(size_t)p * n + i] = sqrt(tot[(size_t)p * (n + 1) + i]);
 }
 
 // ---- coordinate-wise median start ---------------------------------------------------------------
@@ -489,9 +509,9 @@ int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_
     return BTARD_OK;
 }
 
-int launch_partials_to_norms(const double* part, double* norm, int n, int P, int cpp, cudaStream_t st)
+int launch_totals_to_norms(const double* tot, double* norm, int n, int P, cudaStream_t st)
 {
-    partials_to_norms_kernel<<<P, 128, 0, st>>>(part, norm, n, cpp);
+    totals_to_norms_kernel<<<P, 128, 0, st>>>(tot, norm, n);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
     return BTARD_OK;

@@ -57,8 +57,10 @@ struct CclipLaunch {
     float* v;                 // PASS_NORMS never writes it
     unsigned short* v_lo;     // device [P][stride] bf16 low-order part of v, or nullptr (plain fp32 v)
     const PartEntry* table;   // device [P]
-    const double* part_in;    // device [P][cpp][n+1] partial sums of the previous pass
-    double* part_out;         // device [P][cpp][n+1]
+    double* slots;            // device [P][cpp][n+1] per-CTA partial sums of the running pass
+    const double* tot_in;     // device [P][n+1] totals of the previous pass
+    double* tot_out;          // device [P][n+1] totals of this pass
+    unsigned int* ticket;     // device [P] CTAs of the partition that have finished (0 between passes)
     int* done;                // device [P]
     int32_t* iters;
     double* last_step;
@@ -78,10 +80,8 @@ int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaS
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
 int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
                        int P, cudaStream_t st);
-// norm2 partial sums -> norms (sqrt of the per-partition sums), used when verification is asked to
-// compute the norms itself.
-int launch_partials_to_norms(const double* part, double* norm, int n, int P, int cpp,
-                             cudaStream_t st);
+// squared-norm totals -> norms, used when verification is asked to compute the norms itself.
+int launch_totals_to_norms(const double* tot, double* norm, int n, int P, cudaStream_t st);
 
 // ---- verification (btard_verify.cu) -------------------------------------------------------------
 struct VerifyLaunch {
