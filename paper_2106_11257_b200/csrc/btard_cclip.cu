@@ -22,7 +22,7 @@ namespace {
 
 __device__ __forceinline__ float4 ld_stream(const float* p)
 {
-    return __ldcs(reinterpret_cast<const float4*>(p));
+    return __ldg(reinterpret_cast<const float4*>(p));
 }
 
 __device__ __forceinline__ double warp_sum(double x)
@@ -98,7 +98,11 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const CclipLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
-    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    // Consecutive passes sweep the tensor in opposite directions, so that a pass starts on the
+    // lines the previous one touched last and finds part of them still in L2.
+    const bool rev = (MODE == PASS_ITER) && ((a.l & 1) == 0);
+    const int bid = rev ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+    const int p = bid / cpp, j = bid % cpp;
     const long long stride = a.stride;
     const long long len = a.table[p].len;
     const double tau = a.table[p].tau;
@@ -253,10 +257,11 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
     };
 
-    int parity = 0;
-    for (long long qb = q0; qb < q1; qb += CL, parity ^= 1) {
-        if (qb + CL <= q1 && qb + CL <= full_quads) tile(std::false_type{}, qb, parity);
-        else tile(std::true_type{}, qb, parity);
+    const long long ntiles = (q1 - q0 + CL - 1) / CL;
+    for (long long t = 0; t < ntiles; ++t) {
+        const long long qb = q0 + (rev ? ntiles - 1 - t : t) * CL;
+        if (qb + CL <= q1 && qb + CL <= full_quads) tile(std::false_type{}, qb, (int)(t & 1));
+        else tile(std::true_type{}, qb, (int)(t & 1));
     }
 
     // CTA reduction: lanes of a warp share a row group, so a warp reduces R rows at once.
