@@ -23,6 +23,7 @@ struct Geometry {
     int threads;  // RG * CL
     int tiles;    // unused
     int cpp;      // CTAs per partition
+    int slots;    // CTAs resident on the whole GPU at once
 };
 
 constexpr int kMaxTilesPerCta = 64;   // bounds the length of every fp32 running sum (256 terms)

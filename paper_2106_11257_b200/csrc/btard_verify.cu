@@ -329,6 +329,7 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     g.tiles = 0;
     const size_t smem = sizeof(float4) * (2 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
     const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, g.threads, smem);
+    g.slots = slots;
     g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, slots);
     vg.slots = n * kt + kt + 1;
     return vg;
