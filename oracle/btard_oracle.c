@@ -318,7 +318,8 @@ int btard_oracle_verify_one(const float *g, int32_t n, int64_t stride, int64_t l
             double acc = 0.0;
             for (int64_t c = 0; c < len; ++c) acc += ((double)x[c] - vd[c]) * (double)z[c];
             dot[(int64_t)i * K + k] = acc;
-            double sik = (weight[i] == 0.0) ? 0.0 : weight[i] * acc / sqrt(zz);
+            /* an empty partition has no coordinates: the inner product is the empty sum, 0 */
+            double sik = (weight[i] == 0.0 || zz == 0.0) ? 0.0 : weight[i] * acc / sqrt(zz);
             s[(int64_t)i * K + k] = sik;
             s_sum[k] += sik;
         }

@@ -235,13 +235,14 @@ __global__ void verify_finalize_kernel(const VArgs k, int KT)
         const double d = sh_v[i * KT + q];
         const double zn = sqrt(sh_v[n * KT + q]);
         a.dot[((size_t)p * n + i) * K + a.k0 + q] = d;
-        a.s[((size_t)p * n + i) * K + a.k0 + q] = (sh_wf[i] == 0.0f) ? 0.0 : (double)sh_wf[i] * d / zn;
+        a.s[((size_t)p * n + i) * K + a.k0 + q] =
+            (sh_wf[i] == 0.0f || zn == 0.0) ? 0.0 : (double)sh_wf[i] * d / zn;
     }
     for (int q = threadIdx.x; q < a.kc; q += blockDim.x) {
         const double zn = sqrt(sh_v[n * KT + q]);
         double ss = 0.0;
         for (int i = 0; i < n; ++i)
-            if (sh_wf[i] != 0.0f) ss += (double)sh_wf[i] * sh_v[i * KT + q] / zn;
+            if (sh_wf[i] != 0.0f && zn != 0.0) ss += (double)sh_wf[i] * sh_v[i * KT + q] / zn;
         a.s_sum[(size_t)p * K + a.k0 + q] = ss;
         a.znorm2[(size_t)p * K + a.k0 + q] = sh_v[n * KT + q];
     }

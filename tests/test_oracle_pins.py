@@ -422,3 +422,12 @@ def test_partition_index_keys_z():
         assert np.array_equal(full[key][1:], sub[key])
     z = oracle.random_vector(8, 2, 1, 7).astype(np.float64)
     assert np.allclose(full["dot"][2, :, 1], g[2][:, :7].astype(np.float64) @ z, rtol=1e-12)
+
+
+def test_empty_partition_projects_to_zero():
+    """No coordinates: the inner product <z, Delta> is the empty sum."""
+    g = np.ones((2, 3, 8), dtype=np.float32)
+    v = np.zeros((2, 8), dtype=np.float32)
+    out = oracle.verify(g, v, 1.0, seed=1, K=2, part_len=np.array([0, 8]))
+    assert np.all(out["s"][0] == 0) and np.all(out["s_sum"][0] == 0) and np.all(out["znorm2"][0] == 0)
+    assert np.all(np.isfinite(out["s"]))
