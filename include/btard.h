@@ -143,6 +143,31 @@ BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* arg
 BTARD_API int btard_verify_projections(const btard_verify_args* args);
 
 /*
+ * btard_verify_projections without caller-supplied scratch.  The paper has no counterpart: this is
+ * a packaging variant of the call above, same arguments, same kernels, same outputs.
+ *
+ * It is for callers that cannot give the library a workspace because they cannot allocate device
+ * memory: a plug-in running inside a process whose framework has already claimed the whole GPU for
+ * its own memory pool (cudaMalloc would fail), or a latency-critical loop that must never call
+ * cudaMalloc / cudaFree because those may synchronise the device.  The caller still passes inputs
+ * and outputs; `workspace` and `workspace_bytes` in the arguments are ignored.
+ *
+ * The scratch is a fixed array of BTARD_STATIC_SCRATCH_BYTES inside the library's device image; every
+ * GPU that loads the library holds it until the process exits.  Problems whose scratch need exceeds
+ * it (many partitions, very long rows, many z vectors) are refused with
+ * BTARD_ERR_WORKSPACE_TOO_SMALL and nothing is queued; use btard_verify_projections for those.
+ * The call allocates nothing, on the device or on the host heap.
+ *
+ * The first call on each device looks up the array's device address (one driver query, with that
+ * device current); make that first call outside any stream capture.  All calls on one GPU share the
+ * array: calls that may overlap on the GPU (other streams or threads) race on it and must be
+ * serialised by the caller.  Nothing needs to persist in it between calls; what must start at zero
+ * is cleared on `stream` by each call.
+ */
+#define BTARD_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
+BTARD_API int btard_verify_projections_static(const btard_verify_args* args);
+
+/*
  * GetRandomVector (Alg. 6 line 5) made visible: writes the unnormalised float32 coordinates
  * z_k[0 .. part_len) of partition p to device memory (z_out, 16-byte aligned, room for
  * part_len rounded up to a multiple of 4).  Coordinates 4q..4q+3 are the Box-Muller images of the

@@ -20,6 +20,7 @@ EXPORTS = [
     "btard_verify_projections_workspace", "btard_verify_projections", "btard_random_vector",
     "btard_aggregate_host_scratch", "btard_aggregate_host", "btard_last_cuda_error",
     "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
+    "btard_verify_projections_static",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -95,6 +96,8 @@ def lib():
         L.btard_verify_projections_workspace.argtypes = [C.POINTER(VerifyArgs)]
         L.btard_verify_projections.restype = C.c_int
         L.btard_verify_projections.argtypes = [C.POINTER(VerifyArgs)]
+        L.btard_verify_projections_static.restype = C.c_int
+        L.btard_verify_projections_static.argtypes = [C.POINTER(VerifyArgs)]
         L.btard_random_vector.restype = C.c_int
         L.btard_random_vector.argtypes = [C.c_uint64, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
                                           C.c_void_p]
@@ -257,6 +260,45 @@ def verify_projections(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None, 
     if rs is not None:
         res["resid_sum"] = rs
     res["workspace"] = workspace
+    return res
+
+
+def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None,
+                              partition_base=0, want_resid_sum=False, out=None, stream=None):
+    """verify_projections for callers that cannot allocate device memory: the library's built-in
+    scratch array is used instead of a workspace.  Pass `out` (pre-made output tensors, same keys as
+    verify_projections returns) to keep this wrapper from allocating too; calls on one GPU must not
+    overlap.  Raises BtardError("workspace too small") when the problem exceeds the built-in array."""
+    torch = _torch()
+    assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
+    P, n, stride = g.shape
+    assert v.is_cuda and v.dtype == torch.float32 and v.is_contiguous() and v.numel() == P * stride
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    tau_h = _host_arr(tau, P, np.float64)
+    dev = g.device
+    f64 = dict(dtype=torch.float64, device=dev)
+    o = out if out is not None else dict(
+        norm=torch.empty((P, n), **f64), weight=torch.empty((P, n), **f64),
+        dot=torch.empty((P, n, K), **f64), s=torch.empty((P, n, K), **f64),
+        s_sum=torch.empty((P, K), **f64), znorm2=torch.empty((P, K), **f64),
+        resid_sum_norm=torch.empty(P, **f64), status=torch.empty(P, dtype=torch.int32, device=dev))
+    rs = o.get("resid_sum") if want_resid_sum else None
+    if want_resid_sum and rs is None:
+        rs = torch.zeros((P, stride), dtype=torch.float32, device=dev)
+    a = VerifyArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
+                   g=g.data_ptr(), v=v.data_ptr(), tau=tau_h.ctypes.data, seed=int(seed), n_z=K,
+                   partition_base=partition_base,
+                   resid_norm_in=resid_norm_in.data_ptr() if resid_norm_in is not None else None,
+                   norm=o["norm"].data_ptr(), weight=o["weight"].data_ptr(), dot=o["dot"].data_ptr(),
+                   s=o["s"].data_ptr(), s_sum=o["s_sum"].data_ptr(), znorm2=o["znorm2"].data_ptr(),
+                   resid_sum_norm=o["resid_sum_norm"].data_ptr(),
+                   resid_sum=rs.data_ptr() if rs is not None else None, status=o["status"].data_ptr(),
+                   workspace=None, workspace_bytes=0, stream=_stream_ptr(stream))
+    with torch.cuda.device(dev):
+        _check(lib().btard_verify_projections_static(C.byref(a)), "btard_verify_projections_static")
+    res = dict(o)
+    if rs is not None:
+        res["resid_sum"] = rs
     return res
 
 
