@@ -170,8 +170,8 @@ def _host_arr(x, P, dtype):
     return np.ascontiguousarray(np.broadcast_to(np.asarray(x, dtype=dtype), (P,)))
 
 
-def centered_clip_workspace(n, P, row_stride, stop_mode=STOP_EPS):
-    a = CclipArgs(n_peers=n, n_partitions=P, row_stride=row_stride, stop_mode=stop_mode)
+def centered_clip_workspace(n, P, row_stride, stop_mode=STOP_EPS, algo=ALGO_DIRECT):
+    a = CclipArgs(n_peers=n, n_partitions=P, row_stride=row_stride, stop_mode=stop_mode, algo=algo)
     return int(lib().btard_centered_clip_workspace(C.byref(a)))
 
 
@@ -194,7 +194,7 @@ def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v=None, stop_mode=
         last_step_norm=torch.empty(P, dtype=torch.float64, device=dev),
         resid_norm=torch.empty((P, n), dtype=torch.float64, device=dev),
         status=torch.empty(P, dtype=torch.int32, device=dev))
-    need = centered_clip_workspace(n, P, stride, stop_mode)
+    need = centered_clip_workspace(n, P, stride, stop_mode, algo)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
     a = CclipArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,

@@ -82,22 +82,33 @@ int check_common(int n, int P, long long stride, const int64_t* part_len, const 
 
 struct CclipWorkspace {
     size_t table, slots, tot[2], flags, flags_bytes, v_lo, v_lo_bytes, total;
+    size_t gslots, gram, coef;      // Gram variant only
 };
+
+constexpr int kMaxGramPeers = 128;
 
 // EPS mode carries v as fp32 + a bf16 correction so that the stop test sees steps far below the
 // rounding of v; FIXED mode needs no such thing.
-CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, const Geometry& geo)
+CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, int algo,
+                               const Geometry& geo)
 {
-    CclipWorkspace w;
+    CclipWorkspace w{};
     size_t off = 0;
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
     w.slots = off; off = align_up(off + sizeof(double) * (size_t)P * geo.cpp * (n + 1), 256);
     w.tot[0] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
     w.tot[1] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
-    w.flags_bytes = sizeof(int) * 2 * (size_t)P;              // done[P], ticket[P]
+    w.flags_bytes = sizeof(int) * 3 * (size_t)P;              // done[P], ticket[P], Gram ticket[P]
     w.flags = off; off = align_up(off + w.flags_bytes, 256);
-    w.v_lo_bytes = (stop_mode == BTARD_STOP_EPS) ? sizeof(unsigned short) * (size_t)P * stride : 0;
+    const bool gram = (algo == BTARD_ALGO_GRAM);
+    w.v_lo_bytes = (stop_mode == BTARD_STOP_EPS && !gram) ? sizeof(unsigned short) * (size_t)P * stride : 0;
     w.v_lo = off; off = align_up(off + w.v_lo_bytes, 256);
+    if (gram && n <= kMaxGramPeers) {
+        const GramGeometry gg = gram_geometry(n, P, stride);
+        w.gslots = off; off = align_up(off + sizeof(double) * (size_t)P * gg.cpp * gg.entries, 256);
+        w.gram = off; off = align_up(off + sizeof(double) * (size_t)P * gg.entries, 256);
+        w.coef = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
+    }
     w.total = off;
     return w;
 }
@@ -192,7 +203,7 @@ size_t btard_centered_clip_workspace(const btard_cclip_args* a)
         a->row_stride < 4)
         return 0;
     const Geometry geo = cclip_geometry(a->n_peers, a->n_partitions, a->row_stride);
-    return cclip_ws_layout(a->n_peers, a->n_partitions, a->row_stride, a->stop_mode, geo).total;
+    return cclip_ws_layout(a->n_peers, a->n_partitions, a->row_stride, a->stop_mode, a->algo, geo).total;
 }
 
 int btard_centered_clip(const btard_cclip_args* a)
@@ -208,13 +219,14 @@ int btard_centered_clip(const btard_cclip_args* a)
         return BTARD_ERR_INVALID_ARG;
     if (a->stop_mode != BTARD_STOP_FIXED_ITERS && a->stop_mode != BTARD_STOP_EPS)
         return BTARD_ERR_INVALID_ARG;
-    if (a->algo != BTARD_ALGO_DIRECT) return BTARD_ERR_UNSUPPORTED;
+    if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM) return BTARD_ERR_INVALID_ARG;
+    if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (!aligned16(a->g) || !aligned16(a->v) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
         return BTARD_ERR_BAD_ALIGNMENT;
 
     const int n = a->n_peers, P = a->n_partitions;
     const Geometry geo = cclip_geometry(n, P, a->row_stride);
-    const CclipWorkspace ws = cclip_ws_layout(n, P, a->row_stride, a->stop_mode, geo);
+    const CclipWorkspace ws = cclip_ws_layout(n, P, a->row_stride, a->stop_mode, a->algo, geo);
     if (a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)a->stream;
     char* base = (char*)a->workspace;
@@ -247,6 +259,31 @@ int btard_centered_clip(const btard_cclip_args* a)
         L.init_mode = BTARD_INIT_CALLER_V0;
     }
     L.tot_in = nullptr; L.tot_out = tot[0]; L.l = 0;
+    if (a->algo == BTARD_ALGO_GRAM) {
+        // v <- v0 (a median start is already in v), G = (g - v0)(g - v0)^T, iterate on coefficients,
+        // then one pass forms v and the residual norms at v.
+        if (a->init_mode != BTARD_INIT_COORD_MEDIAN && a->init_mode != BTARD_INIT_CALLER_V0) {
+            rc = launch_cclip_pass(L, geo, PASS_INIT, st);
+            if (rc != BTARD_OK) return rc;
+        }
+        const GramGeometry gg = gram_geometry(n, P, a->row_stride);
+        GramLaunch G{};
+        G.g = a->g; G.v0 = a->v; G.table = L.table;
+        G.slots = (double*)(base + ws.gslots); G.gram = (double*)(base + ws.gram);
+        G.ticket = (unsigned int*)(base + ws.flags) + 2 * P;
+        G.coef = (double*)(base + ws.coef);
+        G.iters = a->iters; G.last_step = a->last_step_norm; G.status = a->status;
+        G.stride = a->row_stride; G.n = n; G.P = P;
+        G.stop_mode = a->stop_mode; G.max_iters = a->max_iters; G.eps2 = a->eps * a->eps;
+        rc = launch_gram(G, gg, st);
+        if (rc != BTARD_OK) return rc;
+        rc = launch_gram_iterate(G, gg, st);
+        if (rc != BTARD_OK) return rc;
+        L.coef = G.coef;
+        rc = launch_cclip_pass(L, geo, PASS_COMBINE, st);
+        if (rc != BTARD_OK) return rc;
+        return launch_gram_finalize(L.tot_out, a->resid_norm, a->status, n, P, st);
+    }
     rc = launch_cclip_pass(L, geo, PASS_INIT, st);
     if (rc != BTARD_OK) return rc;
 

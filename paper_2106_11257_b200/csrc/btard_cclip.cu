@@ -111,6 +111,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
     // Consecutive passes sweep the tensor in opposite directions, so that a pass starts on the
     // lines the previous one touched last and finds part of them still in L2.
+    constexpr bool UPDATE = (MODE == PASS_ITER || MODE == PASS_COMBINE);   // v moves in this pass
     const bool rev = (MODE == PASS_ITER) && ((a.l & 1) == 0);
     const int bid = rev ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
     const int p = bid / cpp, j = bid % cpp;
@@ -138,6 +139,11 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
         __syncthreads();
         if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+    } else if (MODE == PASS_COMBINE) {
+        // v = v0 + sum_i a_i (x_i - v0): the update formula with weights n a_i.
+        for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x)
+            sh_w[i] = (i < n) ? (float)((double)n * a.coef[(size_t)p * n + i]) : 0.0f;
+        __syncthreads();
     } else if (MODE == PASS_INIT) {
         if (j == 0 && tid == 0) { a.done[p] = 0; a.status[p] = 0; }
     }
@@ -199,11 +205,11 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 
         float4 vn = v4;                                // v after this pass
         float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);   // what the represented v moved by
-        if (MODE == PASS_ITER || (MODE == PASS_INIT && a.init_mode == BTARD_INIT_MEAN)) {
+        if (UPDATE || (MODE == PASS_INIT && a.init_mode == BTARD_INIT_MEAN)) {
             float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                if (MODE == PASS_ITER) {
+                if (UPDATE) {
                     const float wr = wrow[r];
                     if (wr != 0.0f) {                  // weight 0: the row is left out, not multiplied
                         s4.x = fmaf(wr, x[r].x, s4.x); s4.y = fmaf(wr, x[r].y, s4.y);
@@ -224,7 +230,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
                 }
             }
             const float4 u = make_float4(s4.x * inv_n, s4.y * inv_n, s4.z * inv_n, s4.w * inv_n);
-            if (MODE == PASS_ITER) {
+            if (UPDATE) {
                 if (COMP) {
                     uint32_t b0, b1, b2, b3;
                     float4 ln;
@@ -441,7 +447,8 @@ __global__ void median_rank_kernel(const float* g, float* v, const PartEntry* ta
 template <int R>
 int launch_pass_r(const KernelArgs& ka, int mode, int threads, size_t smem, int grid, cudaStream_t st)
 {
-    const int kind = (mode == PASS_ITER) ? KIND_ITER : (mode == PASS_INIT) ? KIND_INIT : KIND_OTHER;
+    const int kind = (mode == PASS_ITER) ? KIND_ITER : (mode == PASS_INIT) ? KIND_INIT
+                                              : (mode == PASS_COMBINE) ? KIND_COMBINE : KIND_OTHER;
     prof_begin(kind, st);
     switch (mode) {
         case PASS_INIT: cclip_pass_kernel<R, PASS_INIT, false><<<grid, threads, smem, st>>>(ka); break;
@@ -449,6 +456,7 @@ int launch_pass_r(const KernelArgs& ka, int mode, int threads, size_t smem, int 
             if (ka.a.v_lo) cclip_pass_kernel<R, PASS_ITER, true><<<grid, threads, smem, st>>>(ka);
             else cclip_pass_kernel<R, PASS_ITER, false><<<grid, threads, smem, st>>>(ka);
             break;
+        case PASS_COMBINE: cclip_pass_kernel<R, PASS_COMBINE, false><<<grid, threads, smem, st>>>(ka); break;
         default: cclip_pass_kernel<R, PASS_NORMS, false><<<grid, threads, smem, st>>>(ka); break;
     }
     prof_end(kind, st);

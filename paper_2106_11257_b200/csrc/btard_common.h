@@ -36,7 +36,7 @@ void count_launch(int n = 1);
 
 // Optional per-kernel timing (off by default): CUDA events around every launch of a kind.
 enum KernelKind { KIND_MEDIAN = 0, KIND_INIT = 1, KIND_ITER = 2, KIND_VERIFY = 3, KIND_OTHER = 4,
-                  KIND_COUNT = 5 };
+                  KIND_GRAM = 5, KIND_COEF = 6, KIND_COMBINE = 7, KIND_COUNT = 8 };
 void prof_begin(int kind, cudaStream_t st);
 void prof_end(int kind, cudaStream_t st);
 int sm_count();
@@ -51,7 +51,7 @@ int sm_count();
     } while (0)
 
 // ---- CenteredClip passes (btard_cclip.cu) -------------------------------------------------------
-enum PassMode { PASS_INIT = 0, PASS_ITER = 1, PASS_NORMS = 2 };
+enum PassMode { PASS_INIT = 0, PASS_ITER = 1, PASS_NORMS = 2, PASS_COMBINE = 3 };
 
 struct CclipLaunch {
     const float* g;
@@ -62,6 +62,7 @@ struct CclipLaunch {
     const double* tot_in;     // device [P][n+1] totals of the previous pass
     double* tot_out;          // device [P][n+1] totals of this pass
     unsigned int* ticket;     // device [P] CTAs of the partition that have finished (0 between passes)
+    const double* coef;       // device [P][n] combination coefficients (PASS_COMBINE)
     int* done;                // device [P]
     int32_t* iters;
     double* last_step;
@@ -83,6 +84,40 @@ int launch_median_init(const float* g, float* v, const PartEntry* table, long lo
                        int P, cudaStream_t st);
 // squared-norm totals -> norms, used when verification is asked to compute the norms itself.
 int launch_totals_to_norms(const double* tot, double* norm, int n, int P, cudaStream_t st);
+
+// ---- Gram-matrix variant (btard_gram.cu) --------------------------------------------------------
+struct GramGeometry {
+    int NB;        // 8-row blocks = ceil(n / 8)
+    int nblk;      // upper-triangular 8x8 blocks = NB (NB + 1) / 2
+    int KG;        // column groups per CTA = 256 / nblk
+    int NP;        // padded row count in shared memory (8 NB + 4)
+    int TK;        // columns per tile
+    int cpp;       // CTAs per partition
+    int entries;   // doubles per Gram slot = 64 nblk
+    size_t smem;   // dynamic shared memory of the Gram kernel
+};
+struct GramLaunch {
+    const float* g;
+    const float* v0;            // device [P][stride] centre of the Gram matrix
+    const PartEntry* table;
+    double* slots;              // device [P][cpp][entries]
+    double* gram;               // device [P][entries] summed blocks
+    unsigned int* ticket;       // device [P]
+    double* coef;               // device [P][n] out of the coefficient iteration
+    int32_t* iters;
+    double* last_step;
+    uint32_t* status;
+    long long stride;
+    int n, P;
+    int stop_mode, max_iters;
+    double eps2;
+};
+GramGeometry gram_geometry(int n, int P, long long stride);
+int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st);
+int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st);
+// resid_norm from the totals of the combine pass
+int launch_gram_finalize(const double* tot, double* resid_norm, uint32_t* status, int n, int P,
+                         cudaStream_t st);
 
 // ---- verification (btard_verify.cu) -------------------------------------------------------------
 struct VerifyLaunch {

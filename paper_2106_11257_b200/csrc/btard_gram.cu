@@ -1,0 +1,338 @@
+// Gram-matrix variant of CenteredClip (same fixed-point iteration, App. D.2 eq. (CenteredClip),
+// carried out in the n-dimensional space of combination coefficients).
+//
+// With R_i = x_i - v0 and G = R R^T (n x n), every iterate is v^l = v0 + sum_j a_j R_j and
+//     ||x_i - v^l||^2 = G_ii - 2 (G a)_i + a^T G a,
+//     a^{l+1} = a^l + (w - W a^l) / n,   w_i = min{1, tau / ||x_i - v^l||},  W = sum_i w_i,
+//     ||v^{l+1} - v^l||^2 = da^T G da.
+// So the tensor is read once to build G (this file), the iteration runs on n x n numbers in fp64,
+// and one more pass forms v = v0 + sum_j a_j R_j (the combine mode of the streaming kernel).
+//
+// G is a dense contraction over the columns.  It is computed here on the fp32 FMA pipes: the
+// products of residuals that differ by orders of magnitude (attacked rows) must stay accurate to
+// about 1e-6 relative for the subtraction above, which rules out single-pass TF32.
+#include "btard_common.h"
+
+namespace btard {
+namespace {
+
+struct GArgs {
+    GramLaunch a;
+    GramGeometry g;
+};
+
+constexpr int kGramThreads = 256;
+constexpr int kPre = 6;   // float4 registers per thread for the tile in flight
+
+// Upper-triangular block index -> (bi, bj), bi <= bj.
+__device__ __forceinline__ void block_coords(int blk, int NB, int& bi, int& bj)
+{
+    bi = 0;
+    int rem = blk;
+    while (rem >= NB - bi) { rem -= NB - bi; ++bi; }
+    bj = bi + rem;
+}
+
+__global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
+{
+    extern __shared__ __align__(16) float sh[];
+    __shared__ int sh_last;
+    const GramLaunch& a = k.a;
+    const int n = a.n, NB = k.g.NB, nblk = k.g.nblk, KG = k.g.KG, NP = k.g.NP, TK = k.g.TK;
+    const int CH = NP >> 2, cpp = k.g.cpp, tid = threadIdx.x;
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const long long stride = a.stride, len = a.table[p].len;
+    const float* gp = a.g + (size_t)p * n * stride;
+    const float* vp = a.v0 + (size_t)p * stride;
+
+    // columns of this CTA, cut on 128-byte lines
+    long long c0 = stride * j / cpp, c1 = stride * (j + 1) / cpp;
+    if (j > 0) c0 &= ~31LL;
+    if (j + 1 < cpp) c1 &= ~31LL;
+    const int ntiles = (int)((c1 - c0 + TK - 1) / TK);
+
+    const bool active = tid < nblk * KG;
+    const int kg = tid / nblk, blk = tid % nblk;
+    int bi = 0, bj = 0;
+    if (active) block_coords(blk, NB, bi, bj);
+
+    float* As0 = sh;
+    float* As1 = sh + (size_t)TK * NP;
+    for (int e = tid; e < 2 * TK * NP; e += kGramThreads) sh[e] = 0.0f;   // pad rows stay zero
+    __syncthreads();
+
+    const int q4 = TK >> 2;                 // float4 per row of a tile
+    const int nload = n * q4;
+    float4 pre[kPre];
+
+    auto load_tile = [&](long long cb) {
+#pragma unroll
+        for (int m = 0; m < kPre; ++m) {
+            const int e = tid + kGramThreads * m;
+            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (e < nload) {
+                const int row = e / q4, c4 = e - row * q4;
+                const long long col = cb + 4 * c4;
+                if (col < c1) {
+                    const float4 x = __ldcs(reinterpret_cast<const float4*>(gp + (size_t)row * stride + col));
+                    const float4 v = *reinterpret_cast<const float4*>(vp + col);
+                    r.x = (col < len) ? x.x - v.x : 0.f;
+                    r.y = (col + 1 < len) ? x.y - v.y : 0.f;
+                    r.z = (col + 2 < len) ? x.z - v.z : 0.f;
+                    r.w = (col + 3 < len) ? x.w - v.w : 0.f;
+                }
+            }
+            pre[m] = r;
+        }
+    };
+    // Transposed store: As[kk][row], with the 16-byte chunks of a k-row rotated by kk/4 so that the
+    // 32 lanes (consecutive kk, same row) do not all hit one bank.
+    auto store_tile = [&](float* As) {
+#pragma unroll
+        for (int m = 0; m < kPre; ++m) {
+            const int e = tid + kGramThreads * m;
+            if (e < nload) {
+                const int row = e / q4, c4 = e - row * q4;
+                const int ch = row >> 2, sub = row & 3;
+                const int phys = ((ch + c4) % CH) * 4 + sub;      // kk >> 2 == c4 for kk = 4 c4 + q
+                float* dst = As + (size_t)(4 * c4) * NP + phys;
+                dst[0] = pre[m].x;
+                dst[NP] = pre[m].y;
+                dst[2 * NP] = pre[m].z;
+                dst[3 * NP] = pre[m].w;
+            }
+        }
+    };
+
+    float acc[8][8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[r][c] = 0.0f;
+
+    if (ntiles > 0) {
+        load_tile(c0);
+        store_tile(As0);
+    }
+    __syncthreads();
+    for (int t = 0; t < ntiles; ++t) {
+        const float* As = (t & 1) ? As1 : As0;
+        if (t + 1 < ntiles) load_tile(c0 + (long long)(t + 1) * TK);
+        if (active) {
+            for (int kk = kg; kk < TK; kk += KG) {
+                const float* row = As + (size_t)kk * NP;
+                const int s = kk >> 2;
+                const float4 i0 = *reinterpret_cast<const float4*>(row + ((2 * bi + s) % CH) * 4);
+                const float4 i1 = *reinterpret_cast<const float4*>(row + ((2 * bi + 1 + s) % CH) * 4);
+                const float4 j0 = *reinterpret_cast<const float4*>(row + ((2 * bj + s) % CH) * 4);
+                const float4 j1 = *reinterpret_cast<const float4*>(row + ((2 * bj + 1 + s) % CH) * 4);
+                const float ai[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
+                const float aj[8] = {j0.x, j0.y, j0.z, j0.w, j1.x, j1.y, j1.z, j1.w};
+#pragma unroll
+                for (int r = 0; r < 8; ++r)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) acc[r][c] = fmaf(ai[r], aj[c], acc[r][c]);
+            }
+        }
+        if (t + 1 < ntiles) store_tile((t & 1) ? As0 : As1);
+        __syncthreads();
+    }
+
+    // Add the column groups' partial blocks in fp64, fixed order, through shared memory.
+    float* scratch = sh;                                  // [64][256]
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) scratch[(r * 8 + c) * kGramThreads + tid] = active ? acc[r][c] : 0.0f;
+    __syncthreads();
+    const int entries = k.g.entries;
+    double* slots = a.slots + (size_t)p * cpp * entries;
+    double* dst = slots + (size_t)j * entries;
+    for (int idx = tid; idx < entries; idx += kGramThreads) {
+        const int b = idx >> 6, e = idx & 63;
+        double s = 0.0;
+        for (int q = 0; q < KG; ++q) s += (double)scratch[e * kGramThreads + q * nblk + b];
+        dst[idx] = s;
+    }
+
+    // The CTA that finishes last adds the partition's slots (nobody waits).
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sh_last = (atomicAdd(&a.ticket[p], 1u) == (unsigned)(cpp - 1));
+    __syncthreads();
+    if (!sh_last) return;
+    __threadfence();
+    double* out = a.gram + (size_t)p * entries;
+    for (int idx = tid; idx < entries; idx += kGramThreads) {
+        double s = 0.0;
+#pragma unroll 8
+        for (int c = 0; c < cpp; ++c) s += __ldcg(slots + (size_t)c * entries + idx);
+        out[idx] = s;
+    }
+    if (tid == 0) a.ticket[p] = 0;
+}
+
+// Sum over the threads of the CTA (fixed order).
+__device__ double block_sum(double x, double* red)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
+    __syncthreads();
+    if (lane == 0) red[warp] = x;
+    __syncthreads();
+    double s = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
+    return s;
+}
+
+// The fixed-point iteration on coefficients, one CTA per partition, fp64.
+__global__ void __launch_bounds__(kGramThreads) gram_iterate_kernel(const GArgs k)
+{
+    extern __shared__ __align__(16) double G[];          // [n][n], then delta[n]
+    __shared__ double red[8];
+    const GramLaunch& a = k.a;
+    const int n = a.n, NB = k.g.NB, nblk = k.g.nblk, tid = threadIdx.x;
+    const int p = blockIdx.x;
+    double* delta = G + (size_t)n * n;
+    const double* src = a.gram + (size_t)p * k.g.entries;
+    for (int idx = tid; idx < nblk * 64; idx += blockDim.x) {
+        const int b = idx >> 6, e = idx & 63;
+        int bi, bj;
+        block_coords(b, NB, bi, bj);
+        const int i = 8 * bi + (e >> 3), jj = 8 * bj + (e & 7);
+        if (i < n && jj < n) {
+            const double val = src[idx];
+            G[(size_t)i * n + jj] = val;
+            if (bi != bj) G[(size_t)jj * n + i] = val;
+        }
+    }
+    __syncthreads();
+
+    const double tau = a.table[p].tau;
+    const int i = tid;
+    const bool row = i < n;
+    const double gii = row ? G[(size_t)i * n + i] : 0.0;
+    const bool bad = row && !isfinite(gii);
+    double ai = 0.0, Gai = 0.0, step2 = 0.0;
+    int iters = 0;
+    for (int l = 0; l < a.max_iters; ++l) {
+        const double aGa = block_sum((row && !bad) ? ai * Gai : 0.0, red);
+        double w = 0.0;
+        if (row && !bad) {
+            double rho2 = gii - 2.0 * Gai + aGa;
+            if (rho2 < 0.0) rho2 = 0.0;
+            const double rho = sqrt(rho2);
+            if (isfinite(rho)) w = (rho <= tau) ? 1.0 : tau / rho;
+        }
+        const double W = block_sum(w, red);
+        const double d = (row && !bad) ? (w - W * ai) / (double)n : 0.0;
+        if (row) delta[i] = d;
+        __syncthreads();
+        double Gd = 0.0;
+        if (row && !bad) {
+            for (int q = 0; q < n; ++q) {
+                const double dq = delta[q];
+                if (dq != 0.0) Gd += G[(size_t)q * n + i] * dq;     // G is symmetric: column read
+            }
+        }
+        step2 = block_sum((row && !bad) ? d * Gd : 0.0, red);
+        ai += d;
+        Gai += Gd;
+        iters = l + 1;
+        if (a.stop_mode == BTARD_STOP_EPS && step2 <= a.eps2) break;
+    }
+    if (step2 < 0.0) step2 = 0.0;
+    if (row) a.coef[(size_t)p * n + i] = ai;
+    const double anybad = block_sum(bad ? 1.0 : 0.0, red);
+    if (tid == 0) {
+        a.iters[p] = iters;
+        a.last_step[p] = sqrt(step2);
+        unsigned st = 0;
+        if (anybad > 0.0) st |= BTARD_STATUS_NONFINITE_ROW;
+        if (a.stop_mode == BTARD_STOP_EPS && !(step2 <= a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
+        a.status[p] = st;
+    }
+}
+
+__global__ void gram_finalize_kernel(const double* tot, double* resid_norm, uint32_t* status, int n)
+{
+    const int p = blockIdx.x;
+    bool bad = false;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const double v = tot[(size_t)p * (n + 1) + i];
+        resid_norm[(size_t)p * n + i] = sqrt(v);
+        if (!isfinite(v)) bad = true;
+    }
+    if (bad) atomicOr(&status[p], BTARD_STATUS_NONFINITE_ROW);
+}
+
+}  // namespace
+
+GramGeometry gram_geometry(int n, int P, long long stride)
+{
+    GramGeometry g;
+    g.NB = (n + 7) / 8;
+    g.nblk = g.NB * (g.NB + 1) / 2;
+    g.KG = kGramThreads / g.nblk;
+    if (g.KG < 1) g.KG = 1;
+    g.NP = 8 * g.NB;
+    int tk = ((4096 / (g.NP + 4) + 16) / 32) * 32;
+    if (tk < 32) tk = 32;
+    if (tk > 256) tk = 256;
+    while ((long long)n * (tk / 4) > (long long)kPre * kGramThreads && tk > 32) tk -= 32;
+    g.TK = tk;
+    g.entries = g.nblk * 64;
+    size_t tiles = sizeof(float) * 2 * (size_t)g.TK * g.NP;
+    size_t scratch = sizeof(float) * 64 * kGramThreads;
+    g.smem = tiles > scratch ? tiles : scratch;
+    // every fp32 accumulator sums at most 4096 products before it enters fp64
+    const long long max_cols = 4096LL * g.KG;
+    long long cmin = (stride + max_cols - 1) / max_cols;
+    const int slots = sm_count() * 2;
+    long long c = (slots + P - 1) / P;
+    if (c < cmin) c = cmin;
+    const long long most = (stride + 127) / 128;
+    if (c > most) c = most;
+    if (c < 1) c = 1;
+    g.cpp = (int)c;
+    return g;
+}
+
+int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
+{
+    GArgs ga{a, geo};
+    if (geo.smem > 48 * 1024)
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
+    prof_begin(KIND_GRAM, st);
+    gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
+    prof_end(KIND_GRAM, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
+{
+    GArgs ga{a, geo};
+    const size_t smem = sizeof(double) * ((size_t)a.n * a.n + a.n);
+    if (smem > 48 * 1024)
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_iterate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    prof_begin(KIND_COEF, st);
+    gram_iterate_kernel<<<a.P, kGramThreads, smem, st>>>(ga);
+    prof_end(KIND_COEF, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_gram_finalize(const double* tot, double* resid_norm, uint32_t* status, int n, int P,
+                         cudaStream_t st)
+{
+    gram_finalize_kernel<<<P, 128, 0, st>>>(tot, resid_norm, status, n);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+}  // namespace btard

@@ -191,6 +191,45 @@ def test_peer_and_partition_indexing():
     assert np.allclose(cpu(r["v"]), ref["v"], rtol=1e-6)
 
 
+# ----------------------------------------------------------------------------- Gram variant
+@pytest.mark.parametrize("n", [1, 3, 8, 16, 23, 64, 100, 128])
+@pytest.mark.parametrize("init", [btard.INIT_MEAN, btard.INIT_COORD_MEDIAN, btard.INIT_CALLER_V0])
+def test_gram_mode_matches_oracle(n, init):
+    """Same iteration in coefficient space: must equal the direct oracle, cancellation included
+    (a third of the rows are 100x farther than the rest)."""
+    rng = np.random.default_rng(300 + n)
+    P, stride = 3, 5024
+    lens = np.array([5024, 4097, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.5, 1.0, 2.0])
+    v0 = None
+    if init == btard.INIT_CALLER_V0:
+        v0 = (g[:, n // 3:].mean(axis=1) + 0.01).astype(np.float32)
+    ref = oracle.centered_clip(g, tau, lens, init_mode=init, v0=v0, max_iters=12)
+    _, r = run_gpu_cclip(g, tau, lens, init_mode=init, v0=v0, max_iters=12, algo=btard.ALGO_GRAM)
+    check_cclip(r, ref, lens)
+
+
+def test_gram_mode_eps_and_long_rows():
+    rng = np.random.default_rng(11)
+    P, n, stride = 2, 16, 1_000_032
+    lens = np.array([1_000_001, 999_999])
+    g = make_case(rng, P, n, stride, lens, far_rows=5, scale=0.001)
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN,
+                               stop_mode=oracle.STOP_EPS, max_iters=300, eps=1e-6)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, stop_mode=btard.STOP_EPS,
+                         max_iters=300, eps=1e-6, algo=btard.ALGO_GRAM)
+    check_cclip(r, ref, lens, eps_mode=True)
+    assert np.array_equal(cpu(r["status"]) & 1, ref["status"] & 1)
+
+
+def test_gram_mode_rejects_too_many_peers():
+    g = torch.zeros((1, 129, 64), device="cuda")
+    with pytest.raises(btard.BtardError) as e:
+        btard.centered_clip(g, 1.0, init_mode=btard.INIT_ZERO, max_iters=1, algo=btard.ALGO_GRAM)
+    assert e.value.code == -5
+
+
 # ----------------------------------------------------------------------------- verification
 def check_verify(out, ref, K):
     P, n = ref["norm"].shape
@@ -286,14 +325,15 @@ def test_aggregate_host_matches_device_path():
 
 
 # ----------------------------------------------------------------------------- full-size configs
-def _full_config(cfg, sample, max_iters=None, stop=None):
+def _full_config(cfg, sample, max_iters=None, stop=None, algo=None):
     """Runs configuration `cfg` at full size on the GPU in the benchmark's launch configuration and
     compares the sampled partitions with the oracle."""
     w = workloads.make_workload(cfg, device="cuda")
     stop_mode = w.stop_mode if stop is None else stop
     iters = w.max_iters if max_iters is None else max_iters
     r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
-                            stop_mode=stop_mode, max_iters=iters, eps=w.eps)
+                            stop_mode=stop_mode, max_iters=iters, eps=w.eps,
+                            algo=btard.ALGO_DIRECT if algo is None else algo)
     o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
                                  resid_norm_in=r["resid_norm"])
     torch.cuda.synchronize()
@@ -328,3 +368,24 @@ def test_config3_full_size_sampled():
 def test_config4_full_size_sampled():
     _full_config(4, sample=[0, 63])
     _full_config(4, sample=[31], max_iters=5, stop=btard.STOP_FIXED_ITERS)
+
+
+def test_config2_and_4_gram_mode_full_size_sampled():
+    _full_config(2, sample=[5], max_iters=20, stop=btard.STOP_FIXED_ITERS, algo=btard.ALGO_GRAM)
+    _full_config(4, sample=[17], algo=btard.ALGO_GRAM)
+
+
+def test_config5_shape_sampled():
+    """Config 5 at a quarter of its length (16 GiB of rows): fixed 20 iterations and the Gram variant
+    side by side, one partition checked against the oracle."""
+    w = workloads.make_workload(5, device="cuda", d=1 << 26)
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
+        r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
+                                stop_mode=btard.STOP_FIXED_ITERS, max_iters=20, algo=algo)
+        torch.cuda.synchronize()
+        p = 41
+        gp = cpu(w.g[p:p + 1])
+        ref = oracle.centered_clip(gp, w.tau[p], w.part_len[p:p + 1], init_mode=oracle.INIT_COORD_MEDIAN,
+                                   max_iters=20)
+        sub = {k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}
+        check_cclip(sub, ref, w.part_len[p:p + 1])
