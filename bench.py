@@ -85,13 +85,15 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def algorithmic_bytes(w, iters):
+def algorithmic_bytes(w, iters, gram=False):
     """Bytes the method must move for one aggregation: one init pass, one pass per update and one
-    verification pass over each partition's [n][row_stride] rows, each with v read and written."""
+    verification pass over each partition's [n][row_stride] rows, each with v read and written.
+    The Gram variant needs a Gram pass, a combine pass and the verification pass, whatever the
+    number of updates."""
     n, stride = w.n, w.row_stride
     per_pass = n * stride * 4 * (1.0 + 2.0 / n)
     input_only = n * stride * 4
-    passes = [2 + int(i) for i in iters]
+    passes = [3 for _ in iters] if gram else [2 + int(i) for i in iters]
     return sum(passes) * input_only, sum(passes) * per_pass, passes
 
 
@@ -124,14 +126,15 @@ def run_ours(args):
     g = w.g
     P, n, stride = g.shape
     dev = g.device
-    ws_c = torch.empty(btard.centered_clip_workspace(n, P, stride, w.stop_mode), dtype=torch.uint8, device=dev)
+    algo = btard.ALGO_GRAM if args.algo == "gram" else btard.ALGO_DIRECT
+    ws_c = torch.empty(btard.centered_clip_workspace(n, P, stride, w.stop_mode, algo), dtype=torch.uint8, device=dev)
     ws_v = torch.empty(btard.verify_projections_workspace(n, P, stride, w.K), dtype=torch.uint8, device=dev)
     v = torch.empty((P, stride), dtype=torch.float32, device=dev)
     state = {}
 
     def step():
         r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=w.init_mode, v=v,
-                                stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps,
+                                stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps, algo=algo,
                                 workspace=ws_c, out=state.get("c"))
         state["c"] = {k: r[k] for k in ("iters", "last_step_norm", "resid_norm", "status")}
         o = btard.verify_projections(g, v, w.tau, w.zseed, K=w.K, part_len=w.part_len,
@@ -168,7 +171,7 @@ def run_ours(args):
 
     iters = state["c"]["iters"].cpu().numpy()
     status = state["c"]["status"].cpu().numpy()
-    in_bytes, alg_bytes, passes = algorithmic_bytes(w, iters)
+    in_bytes, alg_bytes, passes = algorithmic_bytes(w, iters, gram=(args.algo == "gram"))
     ms_step = ms_total / args.steps
     if dist:
         t = torch.tensor([ms_step], dtype=torch.float64, device=dev)
@@ -178,7 +181,7 @@ def run_ours(args):
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----------
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.algo == "direct":
         gh = torch.empty(g.shape, dtype=torch.float32, pin_memory=True)
         gh.copy_(g)
         scratch = torch.empty(btard.aggregate_host_scratch(n, P, stride, w.K), dtype=torch.uint8, device=dev)
@@ -251,11 +254,12 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "config %d: n=%d peers, d=%d, P=%d partitions, row_stride=%d" %
                                (args.config, w.n, w.d, w.P, w.row_stride),
-                   "init": "coordinate median", "stop": "eps" if w.stop_mode else "fixed",
+                   "algo": args.algo, "init": "coordinate median", "stop": "eps" if w.stop_mode else "fixed",
                    "max_iters": w.max_iters, "eps": w.eps, "K": w.K,
                    "iters_per_partition": [int(i) for i in iters],
                    "not_converged_partitions": int((status & 1).sum()),
-                   "passes_counted": "1 init + iters + 1 verify per partition",
+                   "passes_counted": ("1 Gram + 1 combine + 1 verify per partition" if args.algo == "gram"
+                                      else "1 init + iters + 1 verify per partition"),
                    "l2": "input (%.0f MB) larger than L2 (126 MB), no flush" % (g.numel() * 4 / 1e6),
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
         "fraction_of_hbm_peak": value / world / peak, "hbm_peak_gbs": peak, "hbm_peak_kind": peak_kind,
@@ -332,6 +336,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--algo", default="direct", choices=["direct", "gram"])
     ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

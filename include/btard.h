@@ -223,8 +223,9 @@ BTARD_API int btard_last_cuda_error(void);
  * Optional per-kernel timing for benchmarks (no counterpart in the paper).  While enabled, every
  * streaming kernel the library launches is bracketed by CUDA events on the caller's stream.
  * btard_profile_collect waits for the recorded events, adds up elapsed milliseconds and launch counts
- * per kernel kind into total_ms[kind] / launches[kind] (host arrays of n_kinds >= 5 entries:
- * 0 median start, 1 init pass, 2 CenteredClip iteration pass, 3 verification pass, 4 other) and
+ * per kernel kind into total_ms[kind] / launches[kind] (host arrays of n_kinds >= 8 entries:
+ * 0 median start, 1 init pass, 2 CenteredClip iteration pass, 3 verification pass, 4 other,
+ * 5 Gram pass, 6 coefficient iteration, 7 combine pass) and
  * forgets them.  Process-wide state; not meant for concurrent use from several threads.
  */
 BTARD_API void btard_profile_enable(int on);

@@ -119,7 +119,7 @@ def kernel_launch_count():
     return int(lib().btard_kernel_launch_count())
 
 
-KERNEL_KINDS = ("median", "init", "iter", "verify", "other")
+KERNEL_KINDS = ("median", "init", "iter", "verify", "other", "gram", "coef", "combine")
 
 
 def profile_enable(on):

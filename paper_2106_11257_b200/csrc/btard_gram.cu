@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
     __shared__ int sh_last;
     const GramLaunch& a = k.a;
     const int n = a.n, NB = k.g.NB, nblk = k.g.nblk, KG = k.g.KG, NP = k.g.NP, TK = k.g.TK;
-    const int CH = NP >> 2, cpp = k.g.cpp, tid = threadIdx.x;
+    const int CHM = (NP >> 2) - 1, cpp = k.g.cpp, tid = threadIdx.x;   // NP/4 is a power of two
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
     const long long stride = a.stride, len = a.table[p].len;
     const float* gp = a.g + (size_t)p * n * stride;
@@ -85,8 +85,8 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
             pre[m] = r;
         }
     };
-    // Transposed store: As[kk][row], with the 16-byte chunks of a k-row rotated by kk/4 so that the
-    // 32 lanes (consecutive kk, same row) do not all hit one bank.
+    // Transposed store: As[kk][row], with the 16-byte chunks of a k-row permuted (XOR with kk/4) so
+    // that the 32 lanes (consecutive kk, same row) do not all hit one bank.
     auto store_tile = [&](float* As) {
 #pragma unroll
         for (int m = 0; m < kPre; ++m) {
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
             if (e < nload) {
                 const int row = e / q4, c4 = e - row * q4;
                 const int ch = row >> 2, sub = row & 3;
-                const int phys = ((ch + c4) % CH) * 4 + sub;      // kk >> 2 == c4 for kk = 4 c4 + q
+                const int phys = ((ch ^ c4) & CHM) * 4 + sub;     // kk >> 2 == c4 for kk = 4 c4 + q
                 float* dst = As + (size_t)(4 * c4) * NP + phys;
                 dst[0] = pre[m].x;
                 dst[NP] = pre[m].y;
@@ -122,10 +122,10 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
             for (int kk = kg; kk < TK; kk += KG) {
                 const float* row = As + (size_t)kk * NP;
                 const int s = kk >> 2;
-                const float4 i0 = *reinterpret_cast<const float4*>(row + ((2 * bi + s) % CH) * 4);
-                const float4 i1 = *reinterpret_cast<const float4*>(row + ((2 * bi + 1 + s) % CH) * 4);
-                const float4 j0 = *reinterpret_cast<const float4*>(row + ((2 * bj + s) % CH) * 4);
-                const float4 j1 = *reinterpret_cast<const float4*>(row + ((2 * bj + 1 + s) % CH) * 4);
+                const float4 i0 = *reinterpret_cast<const float4*>(row + (((2 * bi) ^ s) & CHM) * 4);
+                const float4 i1 = *reinterpret_cast<const float4*>(row + (((2 * bi + 1) ^ s) & CHM) * 4);
+                const float4 j0 = *reinterpret_cast<const float4*>(row + (((2 * bj) ^ s) & CHM) * 4);
+                const float4 j1 = *reinterpret_cast<const float4*>(row + (((2 * bj + 1) ^ s) & CHM) * 4);
                 const float ai[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
                 const float aj[8] = {j0.x, j0.y, j0.z, j0.w, j1.x, j1.y, j1.z, j1.w};
 #pragma unroll
@@ -276,11 +276,17 @@ GramGeometry gram_geometry(int n, int P, long long stride)
     g.nblk = g.NB * (g.NB + 1) / 2;
     g.KG = kGramThreads / g.nblk;
     if (g.KG < 1) g.KG = 1;
-    g.NP = 8 * g.NB;
-    int tk = ((4096 / (g.NP + 4) + 16) / 32) * 32;
-    if (tk < 32) tk = 32;
-    if (tk > 256) tk = 256;
-    while ((long long)n * (tk / 4) > (long long)kPre * kGramThreads && tk > 32) tk -= 32;
+    if (g.KG > 64) g.KG = 64;
+    int chunks = 2;                                    // 16-byte chunks per k-row: a power of two
+    while (chunks < 2 * g.NB) chunks <<= 1;
+    g.NP = 4 * chunks;
+    // Tile width: a whole number of columns per column group, about 16 KB of rows in flight per
+    // tile, at most kPre float4 registers per thread.
+    int per_group = 4096 / (g.NP * g.KG);
+    if (per_group < 1) per_group = 1;
+    int tk = per_group * g.KG;
+    tk = (tk + 3) / 4 * 4;
+    while ((long long)n * (tk / 4) > (long long)kPre * kGramThreads && tk > 4) tk -= 4;
     g.TK = tk;
     g.entries = g.nblk * 64;
     size_t tiles = sizeof(float) * 2 * (size_t)g.TK * g.NP;
