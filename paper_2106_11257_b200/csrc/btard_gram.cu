@@ -172,6 +172,147 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
     if (tid == 0) a.ticket[p] = 0;
 }
 
+// ---- n <= 16: the Gram block on the tensor cores, straight from registers ------------------------
+// One warp owns 16 rows x 16 columns at a time.  In the m16n8k8 fragment layout the B operand of
+// R R^T is the A operand itself (lane (g, t) holds rows g, g+8 and the same four columns for both),
+// so nothing is staged in shared memory.  TF32 alone would lose the low 13 bits of every residual;
+// each value is split as hi + lo (both TF32) and hi.hi + hi.lo + lo.hi is accumulated, which keeps
+// products to about 2^-21.  The tensor core adds with truncation, so its accumulator only ever
+// holds one 16-column block (6 chained MMAs); blocks are summed on the fp32 pipe (round to
+// nearest) and moved to fp64 every 64 blocks.
+__device__ __forceinline__ uint32_t to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+constexpr int kMmaStepCols = 64;      // columns a warp takes per step (4 blocks of 16)
+
+__global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
+{
+    __shared__ double sh_tile[kGramThreads / 32][16][16];
+    __shared__ int sh_last;
+    const GramLaunch& a = k.a;
+    const int n = a.n, cpp = k.g.cpp, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const long long stride = a.stride, len = a.table[p].len;
+    const float* gp = a.g + (size_t)p * n * stride;
+    const float* vp = a.v0 + (size_t)p * stride;
+    long long c0 = stride * j / cpp, c1 = stride * (j + 1) / cpp;
+    if (j > 0) c0 &= ~31LL;
+    if (j + 1 < cpp) c1 &= ~31LL;
+
+    const bool row0 = g < n, row1 = g + 8 < n;
+    const float* p0 = gp + (size_t)g * stride;
+    const float* p1 = gp + (size_t)(g + 8) * stride;
+
+    float sum0[4] = {0.f, 0.f, 0.f, 0.f}, sum1[4] = {0.f, 0.f, 0.f, 0.f};     // fp32 running sums
+    double big0[4] = {0., 0., 0., 0.}, big1[4] = {0., 0., 0., 0.};
+    int since_flush = 0;
+
+    for (long long cs = c0 + (long long)warp * kMmaStepCols; cs < c1; cs += (long long)(kGramThreads / 32) * kMmaStepCols) {
+        float4 x0[4], x1[4], v4[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {                  // all loads of the step first
+            const long long col = cs + 16 * b + 4 * t;
+            const bool in = col < c1;
+            x0[b] = (in && row0) ? __ldcs(reinterpret_cast<const float4*>(p0 + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x1[b] = (in && row1) ? __ldcs(reinterpret_cast<const float4*>(p1 + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v4[b] = in ? *reinterpret_cast<const float4*>(vp + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const long long col = cs + 16 * b + 4 * t;
+            const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
+            const bool m2 = col + 2 < len && col < c1, m3 = col + 3 < len && col < c1;
+            // residuals of rows g and g+8 at this lane's four columns
+            const float r0[4] = {(m0 && row0) ? x0[b].x - v4[b].x : 0.f, (m1 && row0) ? x0[b].y - v4[b].y : 0.f,
+                                 (m2 && row0) ? x0[b].z - v4[b].z : 0.f, (m3 && row0) ? x0[b].w - v4[b].w : 0.f};
+            const float r1[4] = {(m0 && row1) ? x1[b].x - v4[b].x : 0.f, (m1 && row1) ? x1[b].y - v4[b].y : 0.f,
+                                 (m2 && row1) ? x1[b].z - v4[b].z : 0.f, (m3 && row1) ? x1[b].w - v4[b].w : 0.f};
+            uint32_t h0[4], h1[4], l0[4], l1[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                h0[q] = to_tf32(r0[q]);
+                h1[q] = to_tf32(r1[q]);
+                l0[q] = to_tf32(r0[q] - __uint_as_float(h0[q]));
+                l1[q] = to_tf32(r1[q] - __uint_as_float(h1[q]));
+            }
+            float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {           // two k-steps: columns (0,1) then (2,3) of the lane
+                const int qa = 2 * ks, qb = 2 * ks + 1;
+                const uint32_t ah[4] = {h0[qa], h1[qa], h0[qb], h1[qb]};
+                const uint32_t al[4] = {l0[qa], l1[qa], l0[qb], l1[qb]};
+                // columns 0..7 of G: B = rows g of R; columns 8..15: rows g+8
+                mma_tf32(d0, ah, h0[qa], h0[qb]);
+                mma_tf32(d0, ah, l0[qa], l0[qb]);
+                mma_tf32(d0, al, h0[qa], h0[qb]);
+                mma_tf32(d1, ah, h1[qa], h1[qb]);
+                mma_tf32(d1, ah, l1[qa], l1[qb]);
+                mma_tf32(d1, al, h1[qa], h1[qb]);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { sum0[q] += d0[q]; sum1[q] += d1[q]; }
+        }
+        if (++since_flush == 16) {                     // 64 blocks of 16 columns
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                big0[q] += (double)sum0[q]; big1[q] += (double)sum1[q];
+                sum0[q] = 0.f; sum1[q] = 0.f;
+            }
+            since_flush = 0;
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { big0[q] += (double)sum0[q]; big1[q] += (double)sum1[q]; }
+
+    // accumulator fragment: (row g, col 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1); d1 is 8 columns on
+    sh_tile[warp][g][2 * t] = big0[0];
+    sh_tile[warp][g][2 * t + 1] = big0[1];
+    sh_tile[warp][g + 8][2 * t] = big0[2];
+    sh_tile[warp][g + 8][2 * t + 1] = big0[3];
+    sh_tile[warp][g][8 + 2 * t] = big1[0];
+    sh_tile[warp][g][8 + 2 * t + 1] = big1[1];
+    sh_tile[warp][g + 8][8 + 2 * t] = big1[2];
+    sh_tile[warp][g + 8][8 + 2 * t + 1] = big1[3];
+    __syncthreads();
+    const int entries = k.g.entries, NB = k.g.NB;
+    double* slots = a.slots + (size_t)p * cpp * entries;
+    double* dst = slots + (size_t)j * entries;
+    for (int idx = tid; idx < entries; idx += kGramThreads) {
+        const int b = idx >> 6, e = idx & 63;
+        int bi, bj;
+        block_coords(b, NB, bi, bj);
+        const int r = 8 * bi + (e >> 3), c = 8 * bj + (e & 7);
+        double s = 0.0;
+        for (int w = 0; w < kGramThreads / 32; ++w) s += sh_tile[w][r][c];
+        dst[idx] = s;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sh_last = (atomicAdd(&a.ticket[p], 1u) == (unsigned)(cpp - 1));
+    __syncthreads();
+    if (!sh_last) return;
+    __threadfence();
+    double* out = a.gram + (size_t)p * entries;
+    for (int idx = tid; idx < entries; idx += kGramThreads) {
+        double s = 0.0;
+#pragma unroll 8
+        for (int c = 0; c < cpp; ++c) s += __ldcg(slots + (size_t)c * entries + idx);
+        out[idx] = s;
+    }
+    if (tid == 0) a.ticket[p] = 0;
+}
+
 // Sum over the threads of the CTA (fixed order).
 __device__ double block_sum(double x, double* red)
 {
@@ -302,6 +443,14 @@ GramGeometry gram_geometry(int n, int P, long long stride)
     if (c > most) c = most;
     if (c < 1) c = 1;
     g.cpp = (int)c;
+    if (n <= 16) {   // tensor-core kernel: whole waves of resident CTAs
+        int nb = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, gram_mma16_kernel, kGramThreads, 0) != cudaSuccess || nb < 1) {
+            (void)cudaGetLastError();
+            nb = 2;
+        }
+        g.cpp = choose_ctas_per_partition(P, stride >> 2, 16 * (kGramThreads / 32), sm_count() * nb);
+    }
     return g;
 }
 
@@ -311,7 +460,8 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     if (geo.smem > 48 * 1024)
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
     prof_begin(KIND_GRAM, st);
-    gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
+    if (a.n <= 16) gram_mma16_kernel<<<a.P * geo.cpp, kGramThreads, 0, st>>>(ga);
+    else gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
     prof_end(KIND_GRAM, st);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
