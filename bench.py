@@ -85,6 +85,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(ms, dist, device):
+    """The job is as slow as its slowest replica: MAX of a per-rank time over all ranks."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_rank, ms_step, world):
+    """Replicas only: every rank aggregates its own copy, the job's throughput is the sum."""
+    return world * bytes_per_rank / (ms_step * 1e-3) / 1e9
+
+
 def algorithmic_bytes(w, iters, gram=False):
     """Bytes the method must move for one aggregation: one init pass, one pass per update and one
     verification pass over each partition's [n][row_stride] rows, each with v read and written.
@@ -173,11 +188,8 @@ def run_ours(args):
     status = state["c"]["status"].cpu().numpy()
     in_bytes, alg_bytes, passes = algorithmic_bytes(w, iters, gram=(args.algo == "gram"))
     ms_step = ms_total / args.steps
-    if dist:
-        t = torch.tensor([ms_step], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-    value = world * in_bytes / (ms_step * 1e-3) / 1e9
+    ms_step = max_over_ranks(ms_step, dist, dev)
+    value = whole_job_value(in_bytes, ms_step, world)
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----------
     e2e = None
@@ -204,12 +216,9 @@ def run_ours(args):
             host_step()
         torch.cuda.synchronize()
         ms_e2e = (time.perf_counter() - t0) * 1e3 / k2
-        if dist:
-            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = max_over_ranks(ms_e2e, dist, dev)
         d2h = sum(hout[k].numel() * hout[k].element_size() for k in hout)
-        e2e = {"value": world * in_bytes / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+        e2e = {"value": whole_job_value(in_bytes, ms_e2e, world), "unit": UNIT,
                "ms_per_step": ms_e2e, "h2d_bytes_per_step": gh.numel() * 4, "d2h_bytes_per_step": d2h}
         del gh, scratch
 
