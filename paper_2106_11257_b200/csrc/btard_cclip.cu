@@ -370,9 +370,56 @@ __device__ __forceinline__ float key_value(uint32_t key)
     return __uint_as_float((key & 0x80000000u) ? (key & 0x7FFFFFFFu) : ~key);
 }
 
-// One thread sorts the n values of one column in registers with a bitonic network of N2 >= n
-// inputs (missing inputs are the largest key).
-template <int N2>
+// Batcher's odd-even merge sort as a comparator network on registers (N a power of two).  All
+// indices are compile-time constants, so when only the middle outputs are used the compiler drops
+// every comparator that does not feed them.
+template <int N>
+struct OddEvenNetwork {
+    template <int LO, int CNT, int R>
+    static __device__ __forceinline__ void merge(int (&k)[N])
+    {
+        constexpr int STEP = R * 2;
+        if constexpr (STEP < CNT) {
+            merge<LO, CNT, STEP>(k);
+            merge<LO + R, CNT, STEP>(k);
+#pragma unroll
+            for (int i = LO + R; i + R < LO + CNT; i += STEP) {
+                const int lo = min(k[i], k[i + R]), hi = max(k[i], k[i + R]);
+                k[i] = lo;
+                k[i + R] = hi;
+            }
+        } else {
+            const int lo = min(k[LO], k[LO + R]), hi = max(k[LO], k[LO + R]);
+            k[LO] = lo;
+            k[LO + R] = hi;
+        }
+    }
+    template <int LO, int CNT>
+    static __device__ __forceinline__ void sort(int (&k)[N])
+    {
+        if constexpr (CNT > 1) {
+            sort<LO, CNT / 2>(k);
+            sort<LO + CNT / 2, CNT / 2>(k);
+            merge<LO, CNT, 1>(k);
+        }
+    }
+};
+
+// Signed-integer image of a float whose integer order is the IEEE total order of the floats.
+__device__ __forceinline__ int signed_key(float f)
+{
+    const int b = __float_as_int(f);
+    return b ^ ((b >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float signed_key_value(int k)
+{
+    return __int_as_float(k ^ ((k >> 31) & 0x7fffffff));
+}
+
+// One thread takes the median of the n values of one column.  EXACT: n == N2 is known at compile
+// time (the two middle outputs are fixed registers and the network is pruned to them); otherwise
+// the column is padded to N2 inputs with the largest key and the middle is picked at run time.
+template <int N2, bool EXACT>
 __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float* v,
                                                           const PartEntry* table, long long stride,
                                                           int n)
@@ -384,34 +431,25 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
     float out = 0.0f;
     if (c < len) {
         const float* gp = g + (size_t)p * n * stride + c;
-        uint32_t key[N2];
+        int key[N2];
 #pragma unroll
-        for (int i = 0; i < N2; ++i) key[i] = (i < n) ? order_key(__ldcs(gp + (size_t)i * stride)) : 0xFFFFFFFFu;
+        for (int i = 0; i < N2; ++i)
+            key[i] = (EXACT || i < n) ? signed_key(__ldcs(gp + (size_t)i * stride)) : 0x7fffffff;
+        OddEvenNetwork<N2>::template sort<0, N2>(key);
+        int ka = 0, kb = 0;
+        if (EXACT) {
+            ka = key[(N2 - 1) / 2];
+            kb = key[N2 / 2];
+        } else {
+            // n is a run-time value: pick the two middle keys without dynamic register indexing.
+            const int ia = (n - 1) >> 1, ib = n >> 1;
 #pragma unroll
-        for (int kk = 2; kk <= N2; kk <<= 1) {
-#pragma unroll
-            for (int jj = kk >> 1; jj > 0; jj >>= 1) {
-#pragma unroll
-                for (int i = 0; i < N2; ++i) {
-                    const int l = i ^ jj;
-                    if (l > i) {
-                        const uint32_t lo = min(key[i], key[l]), hi = max(key[i], key[l]);
-                        const bool up = (i & kk) == 0;
-                        key[i] = up ? lo : hi;
-                        key[l] = up ? hi : lo;
-                    }
-                }
+            for (int i = 0; i < N2; ++i) {
+                if (i == ia) ka = key[i];
+                if (i == ib) kb = key[i];
             }
         }
-        // n is a run-time value: pick the two middle keys without dynamic register indexing.
-        uint32_t ka = 0, kb = 0;
-        const int ia = (n - 1) >> 1, ib = n >> 1;
-#pragma unroll
-        for (int i = 0; i < N2; ++i) {
-            if (i == ia) ka = key[i];
-            if (i == ib) kb = key[i];
-        }
-        out = (float)(((double)key_value(ka) + (double)key_value(kb)) * 0.5);
+        out = (float)(((double)signed_key_value(ka) + (double)signed_key_value(kb)) * 0.5);
     }
     v[(size_t)p * stride + c] = out;
 }
@@ -552,12 +590,18 @@ int launch_median_init(const float* g, float* v, const PartEntry* table, long lo
     const int threads = 128;
     dim3 grid((unsigned)((stride + threads - 1) / threads), (unsigned)P);
     prof_begin(KIND_MEDIAN, st);
-    if (n <= 2) median_sort_kernel<2><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n <= 4) median_sort_kernel<4><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n <= 8) median_sort_kernel<8><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n <= 16) median_sort_kernel<16><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n <= 32) median_sort_kernel<32><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n <= 64) median_sort_kernel<64><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    if (n == 1) median_sort_kernel<1, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n == 2) median_sort_kernel<2, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n == 4) median_sort_kernel<4, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n == 8) median_sort_kernel<8, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n == 16) median_sort_kernel<16, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n == 32) median_sort_kernel<32, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n == 64) median_sort_kernel<64, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n < 4) median_sort_kernel<4, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n < 8) median_sort_kernel<8, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n < 16) median_sort_kernel<16, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n < 32) median_sort_kernel<32, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    else if (n < 64) median_sort_kernel<64, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
     else median_rank_kernel<<<grid, threads, 0, st>>>(g, v, table, stride, n);
     prof_end(KIND_MEDIAN, st);
     BTARD_CUDA_TRY(cudaGetLastError());
