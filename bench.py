@@ -21,6 +21,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "CenteredClip+verify input GB/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the iteration kernel (ncu capture
+# summarised in profiles/cclip_pass_iter_config2.md); set to None whenever that kernel changes.
+ITER_TRAFFIC = {(2, "direct"): 798.7e6}
 UNIT = "GB/s"
 
 
@@ -166,8 +169,7 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    btard.profile_collect()
-    btard.profile_enable(True)
+    # Timed region: K steps, nothing but the library's own launches on the stream.
     launches0 = btard.kernel_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -179,9 +181,19 @@ def run_ours(args):
     if dist:
         dist.barrier()
     ms_total = e0.elapsed_time(e1)
-    btard.profile_enable(False)
-    prof = btard.profile_collect()
     launches = btard.kernel_launch_count() - launches0
+    # The same K steps once more with every kernel bracketed by CUDA events on the launching stream
+    # (per-kernel durations for the roofline).  Kept apart because an event between two launches
+    # stops them from running back to back: with the events the step is 3-15 % slower.
+    prof = None
+    if not args.no_kernel_events:
+        btard.profile_collect()
+        btard.profile_enable(True)
+        for _ in range(args.steps):
+            step()
+        torch.cuda.synchronize()
+        btard.profile_enable(False)
+        prof = btard.profile_collect()
     clocks = sampler.stop() if rank == 0 else None
 
     iters = state["c"]["iters"].cpu().numpy()
@@ -229,6 +241,8 @@ def run_ours(args):
 
     # ---- roofline of the dominant kernel (the CenteredClip iteration pass) -----------------------
     peak, peak_kind = measured_peaks()
+    if prof is None:
+        prof = {k: (0.0, 0) for k in btard.KERNEL_KINDS}
     iter_ms, iter_launches = prof["iter"]
     per_pass_bytes = n * stride * 4 * (1.0 + 2.0 / n)
     iter_bytes = args.steps * sum(int(i) for i in iters) * per_pass_bytes
@@ -270,6 +284,7 @@ def run_ours(args):
                    "passes_counted": ("1 Gram + 1 combine + 1 verify per partition" if args.algo == "gram"
                                       else "1 init + iters + 1 verify per partition"),
                    "l2": "input (%.0f MB) larger than L2 (126 MB), no flush" % (g.numel() * 4 / 1e6),
+                   "kernel_events": "per-kernel durations come from a second run of the same K steps",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
         "fraction_of_hbm_peak": value / world / peak, "hbm_peak_gbs": peak, "hbm_peak_kind": peak_kind,
         "gpu_launches": int(launches),
@@ -277,7 +292,8 @@ def run_ours(args):
         "e2e": e2e,
         "roofline": {"kernel": "cclip_pass_kernel<ITER>", "bound": "hbm", "achieved": achieved,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak if achieved else None, "traffic": None,
+                     "frac": achieved / peak if achieved else None,
+                     "traffic": ITER_TRAFFIC.get((args.config, args.algo)),
                      "launches": iter_launches, "avg_launch_ms": iter_ms / max(1, iter_launches),
                      "algorithmic_bytes_per_launch": per_pass_bytes * P,
                      "verify_kernel_gbs": ver_gbs},
@@ -347,6 +363,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--algo", default="direct", choices=["direct", "gram"])
     ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
+    ap.add_argument("--no-kernel-events", action="store_true",
+                    help="do not bracket the library's kernels with CUDA events (no roofline object)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
