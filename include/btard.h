@@ -53,14 +53,18 @@ extern "C" {
 #define BTARD_INIT_MEAN 2
 #define BTARD_INIT_COORD_MEDIAN 3   /* coordinate-wise median of the n rows                         */
 
-#define BTARD_ALGO_DIRECT 0         /* one pass over g per iteration                                */
+#define BTARD_ALGO_DIRECT 0         /* one pass over g per iteration, one kernel launch per pass    */
 #define BTARD_ALGO_GRAM 1           /* Gram matrix pass + iteration in coefficient space + combine  */
+#define BTARD_ALGO_DIRECT_RESIDENT 2 /* as DIRECT, but chunks of partitions that fit the L2 cache are
+                                       iterated inside one cooperative kernel with grid barriers;
+                                       falls back to DIRECT where a partition does not fit         */
 
 #define BTARD_STOP_FIXED_ITERS 0    /* exactly max_iters updates                                    */
 #define BTARD_STOP_EPS 1            /* stop once ||v^{l+1} - v^l||_2 <= eps, at most max_iters       */
 
 #define BTARD_STATUS_NOT_CONVERGED 1u   /* EPS mode: max_iters reached with the last step > eps     */
 #define BTARD_STATUS_NONFINITE_ROW 2u   /* a row with non-finite residual norm got weight 0         */
+#define BTARD_STATUS_WAIT_EXPIRED 4u    /* a bounded wait inside a kernel ran out: results invalid  */
 
 /*
  * Split(v, n) of App. D.1 ("Basic building blocks"): offsets and lengths of the P parts of a

@@ -83,6 +83,7 @@ int check_common(int n, int P, long long stride, const int64_t* part_len, const 
 struct CclipWorkspace {
     size_t table, slots, tot[2], flags, flags_bytes, v_lo, v_lo_bytes, total;
     size_t gslots, gram, coef;      // Gram variant only
+    size_t rslots, rflags, rflags_bytes;   // L2-resident variant
 };
 
 constexpr int kMaxGramPeers = 128;
@@ -109,6 +110,9 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, in
         w.gram = off; off = align_up(off + sizeof(double) * (size_t)P * gg.entries, 256);
         w.coef = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
     }
+    w.rslots = off; off = align_up(off + sizeof(double) * 2 * (size_t)kResidentMaxGrid * (n + 1), 256);
+    w.rflags_bytes = sizeof(unsigned long long) * ((size_t)P + 1);   // a barrier word per chunk, error flag
+    w.rflags = off; off = align_up(off + w.rflags_bytes, 256);
     w.total = off;
     return w;
 }
@@ -219,7 +223,9 @@ int btard_centered_clip(const btard_cclip_args* a)
         return BTARD_ERR_INVALID_ARG;
     if (a->stop_mode != BTARD_STOP_FIXED_ITERS && a->stop_mode != BTARD_STOP_EPS)
         return BTARD_ERR_INVALID_ARG;
-    if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM) return BTARD_ERR_INVALID_ARG;
+    if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM &&
+        a->algo != BTARD_ALGO_DIRECT_RESIDENT)
+        return BTARD_ERR_INVALID_ARG;
     if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (!aligned16(a->g) || !aligned16(a->v) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
         return BTARD_ERR_BAD_ALIGNMENT;
@@ -252,8 +258,10 @@ int btard_centered_clip(const btard_cclip_args* a)
     }
 
     // Init pass: v^0 and the residual norms at v^0 (slot buffer 0).
+    // Chunks of partitions that fit the L2 cache take the resident path below (0: none do).
+    const int chunk = (a->algo == BTARD_ALGO_DIRECT_RESIDENT) ? resident_chunk_partitions(n, a->row_stride) : 0;
     L.init_mode = a->init_mode;
-    if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
+    if (a->init_mode == BTARD_INIT_COORD_MEDIAN && chunk < 1) {
         rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
         if (rc != BTARD_OK) return rc;
         L.init_mode = BTARD_INIT_CALLER_V0;
@@ -284,6 +292,43 @@ int btard_centered_clip(const btard_cclip_args* a)
         if (rc != BTARD_OK) return rc;
         return launch_gram_finalize(L.tot_out, a->resid_norm, a->status, n, P, st);
     }
+    // Start pass and every update of a chunk in one resident kernel.
+    if (chunk >= 1) {
+        BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.rflags, 0, ws.rflags_bytes, st));
+        unsigned long long* bars = (unsigned long long*)(base + ws.rflags);
+        unsigned int* err = (unsigned int*)(bars + P);
+        bool ok = true;
+        int ci = 0;
+        for (int c0 = 0; c0 < P && ok; c0 += chunk, ++ci) {
+            const int Pc = (P - c0 < chunk) ? P - c0 : chunk;
+            CclipLaunch C = L;
+            C.g = a->g + (size_t)c0 * n * a->row_stride;
+            C.v = a->v + (size_t)c0 * a->row_stride;
+            if (L.v_lo) C.v_lo = L.v_lo + (size_t)c0 * a->row_stride;
+            C.table = L.table + c0;
+            C.iters = a->iters + c0; C.last_step = a->last_step_norm + c0;
+            C.resid_norm = a->resid_norm + (size_t)c0 * n; C.status = a->status + c0;
+            C.P = Pc;
+            C.init_mode = a->init_mode;
+            if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
+                rc = launch_median_init(C.g, C.v, C.table, a->row_stride, n, Pc, st);
+                if (rc != BTARD_OK) return rc;
+                C.init_mode = BTARD_INIT_CALLER_V0;
+            }
+            rc = launch_cclip_resident(C, geo, (double*)(base + ws.rslots), bars + ci, err, st);
+            if (rc != BTARD_OK) {
+                if (c0 == 0) ok = false;      // nothing done yet: take the streaming path instead
+                else return rc;
+            }
+        }
+        if (ok) return BTARD_OK;
+        if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {          // streaming path after all
+            rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
+            if (rc != BTARD_OK) return rc;
+            L.init_mode = BTARD_INIT_CALLER_V0;
+        }
+    }
+
     rc = launch_cclip_pass(L, geo, PASS_INIT, st);
     if (rc != BTARD_OK) return rc;
 

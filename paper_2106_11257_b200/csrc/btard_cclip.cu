@@ -338,6 +338,306 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     if (tid == 0) a.ticket[p] = 0;
 }
 
+// =================================================================================================
+// L2-resident variant: all updates of a chunk of partitions inside ONE cooperative kernel.
+//
+// B200 has 126 MB of L2; a chunk of partitions whose rows fit in it is read from HBM once (by the
+// start pass) and then every CenteredClip update streams it from L2 (measured 17-19 TB/s against
+// 6.5-7 TB/s from HBM).  That needs all updates of the chunk back to back with nothing else
+// flushing L2, i.e. one kernel whose CTAs all stay resident and meet at a grid-wide barrier between
+// updates.  The kernel is launched cooperatively (the runtime refuses the launch if the CTAs cannot
+// all be resident), every wait on the barrier is bounded, and a wait that expires sets an error
+// flag and status bit and makes every CTA leave.
+// =================================================================================================
+struct ResidentArgs {
+    CclipLaunch a;                  // chunk-relative pointers; a.P = partitions in the chunk
+    int RG, CL, cppc;               // cppc CTAs per partition of the chunk
+    double* rslots;                 // [2][P][cppc][n+1]
+    unsigned long long* barrier;    // low word: arrivals (monotonic), high word: finished partitions
+    unsigned int* error;            // set when a bounded wait expired
+};
+
+constexpr long long kBarrierSpinLimit = 8LL * 1000 * 1000;     // a few seconds of polling
+
+__device__ __forceinline__ unsigned long long ld_volatile_u64(const unsigned long long* p)
+{
+    unsigned long long v;
+    asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide barrier.  Returns true when every partition of the chunk has finished (or a wait ran
+// out): the caller then leaves the kernel; CTAs still on their way see the same word and leave too,
+// so nobody is left waiting for an arrival that will not come.
+__device__ bool grid_barrier(const ResidentArgs& k, unsigned& generation, unsigned add_finished, int* sh_flag)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        generation += 1;
+        const unsigned long long target = (unsigned long long)generation * gridDim.x;
+        const unsigned long long inc = 1ull + ((unsigned long long)add_finished << 32);
+        unsigned long long v = atomicAdd(k.barrier, inc) + inc;
+        long long spins = 0;
+        bool expired = false;
+        while ((v & 0xffffffffull) < target && (v >> 32) < (unsigned long long)k.a.P) {
+            v = ld_volatile_u64(k.barrier);
+            if (++spins > kBarrierSpinLimit) { expired = true; break; }
+        }
+        if (expired) {
+            atomicExch(k.error, 1u);
+            atomicAdd(k.barrier, (unsigned long long)k.a.P << 32);   // release everybody else
+        }
+        if (atomicAdd(k.error, 0u) != 0u) expired = true;
+        __threadfence();
+        *sh_flag = (expired || (v >> 32) >= (unsigned long long)k.a.P) ? 1 : 0;
+    } else {
+        generation += 1;
+    }
+    __syncthreads();
+    return *sh_flag != 0;
+}
+
+template <int R, bool COMP>
+__global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs k)
+{
+    extern __shared__ float4 sh_x[];                  // [2][RG][CL]
+    __shared__ double sh_sum[BTARD_MAX_PEERS + 1];
+    __shared__ float sh_w[BTARD_MAX_PEERS + 16];
+    __shared__ double sh_red[16][17];
+    __shared__ double sh_part[512 + BTARD_MAX_PEERS + 1];
+    __shared__ int sh_flag, sh_bar;
+
+    const CclipLaunch& a = k.a;
+    const int n = a.n, RG = k.RG, CL = k.CL, cppc = k.cppc, Pc = a.P;
+    const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
+    const bool active = (int)blockIdx.x < Pc * cppc;
+    const int p = active ? (int)blockIdx.x / cppc : 0, j = active ? (int)blockIdx.x % cppc : 0;
+    const long long stride = a.stride, len = a.table[p].len;
+    const double tau = a.table[p].tau;
+    const float* gp = a.g + (size_t)p * n * stride;
+    float* vp = a.v + (size_t)p * stride;
+    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
+    const float inv_n = 1.0f / (float)n;
+    const float* wrow = sh_w + rg * R;
+    const int per = n + 1;
+
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cppc, q1 = Q * (j + 1) / cppc;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cppc) q1 &= ~7LL;
+    const long long full_quads = len >> 2;
+    const long long ntiles = (q1 - q0 + CL - 1) / CL;
+
+    float acc[R];
+    float step_acc = 0.0f;
+
+    // One tile of CL quads.  INIT: v holds (or becomes) v^0 and the norms at v^0 are taken;
+    // otherwise one CenteredClip update.
+    auto tile = [&](auto init_tag, auto masked_tag, long long qb, int parity) {
+        constexpr bool INIT = decltype(init_tag)::value;
+        constexpr bool MASKED = decltype(masked_tag)::value;
+        const long long col = (qb + cl) * 4;
+        const bool valid = !MASKED || (qb + cl < q1);
+        const bool m0 = !MASKED || (valid && col < len), m1 = !MASKED || (valid && col + 1 < len);
+        const bool m2 = !MASKED || (valid && col + 2 < len), m3 = !MASKED || (valid && col + 3 < len);
+        float4 x[R];
+        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f), lo4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int i = rg * R + r;
+                x[r] = (i < n) ? __ldg(reinterpret_cast<const float4*>(gp + (size_t)i * stride + col))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (!INIT || a.init_mode == BTARD_INIT_CALLER_V0) v4 = *reinterpret_cast<const float4*>(vp + col);
+            if (COMP && !INIT) {
+                const uint2 lb = *reinterpret_cast<const uint2*>(lop + col);
+                lo4 = make_float4(bf16_value(lb.x & 0xFFFFu), bf16_value(lb.x >> 16),
+                                  bf16_value(lb.y & 0xFFFFu), bf16_value(lb.y >> 16));
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (!INIT) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = (x[r].x - v4.x) - lo4.x; x[r].y = (x[r].y - v4.y) - lo4.y;
+                x[r].z = (x[r].z - v4.z) - lo4.z; x[r].w = (x[r].w - v4.w) - lo4.w;
+            }
+        }
+        float4 vn = v4, dv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!INIT || a.init_mode == BTARD_INIT_MEAN) {
+            float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                if (!INIT) {
+                    const float wr = wrow[r];
+                    if (wr != 0.0f) {
+                        s4.x = fmaf(wr, x[r].x, s4.x); s4.y = fmaf(wr, x[r].y, s4.y);
+                        s4.z = fmaf(wr, x[r].z, s4.z); s4.w = fmaf(wr, x[r].w, s4.w);
+                    }
+                } else {
+                    s4.x += x[r].x; s4.y += x[r].y; s4.z += x[r].z; s4.w += x[r].w;
+                }
+            }
+            if (RG > 1) {
+                float4* buf = sh_x + (size_t)parity * RG * CL;
+                buf[rg * CL + cl] = s4;
+                __syncthreads();
+                s4 = buf[cl];
+                for (int q = 1; q < RG; ++q) {
+                    const float4 o = buf[q * CL + cl];
+                    s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
+                }
+            }
+            const float4 u = make_float4(s4.x * inv_n, s4.y * inv_n, s4.z * inv_n, s4.w * inv_n);
+            if (!INIT) {
+                if (COMP) {
+                    uint32_t b0, b1, b2, b3;
+                    float4 ln;
+                    two_sum_bf16(v4.x, lo4.x + u.x, vn.x, ln.x, b0);
+                    two_sum_bf16(v4.y, lo4.y + u.y, vn.y, ln.y, b1);
+                    two_sum_bf16(v4.z, lo4.z + u.z, vn.z, ln.z, b2);
+                    two_sum_bf16(v4.w, lo4.w + u.w, vn.w, ln.w, b3);
+                    if (!m0) b0 = 0;
+                    if (!m1) b1 = 0;
+                    if (!m2) b2 = 0;
+                    if (!m3) b3 = 0;
+                    dv = make_float4((vn.x - v4.x) + (ln.x - lo4.x), (vn.y - v4.y) + (ln.y - lo4.y),
+                                     (vn.z - v4.z) + (ln.z - lo4.z), (vn.w - v4.w) + (ln.w - lo4.w));
+                    if (rg == 0 && valid)
+                        *reinterpret_cast<uint2*>(lop + col) = make_uint2(b0 | (b1 << 16), b2 | (b3 << 16));
+                } else {
+                    vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+                    dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
+                }
+                if (rg == 0)
+                    step_acc += (m0 ? u.x * u.x : 0.f) + (m1 ? u.y * u.y : 0.f) +
+                                (m2 ? u.z * u.z : 0.f) + (m3 ? u.w * u.w : 0.f);
+            } else {
+                vn = u;
+            }
+        } else if (INIT && a.init_mode == BTARD_INIT_ZERO) {
+            vn = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (!m0) vn.x = 0.f;
+        if (!m1) vn.y = 0.f;
+        if (!m2) vn.z = 0.f;
+        if (!m3) vn.w = 0.f;
+        if (rg == 0 && valid) {
+            *reinterpret_cast<float4*>(vp + col) = vn;
+            if (COMP && INIT) *reinterpret_cast<uint2*>(lop + col) = make_uint2(0u, 0u);
+        }
+        if (INIT) dv = vn;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float dx = m0 ? x[r].x - dv.x : 0.f, dy = m1 ? x[r].y - dv.y : 0.f;
+            const float dz = m2 ? x[r].z - dv.z : 0.f, dw = m3 ? x[r].w - dv.w : 0.f;
+            acc[r] += fmaf(dx, dx, fmaf(dy, dy, fmaf(dz, dz, dw * dw)));
+        }
+    };
+
+    // All tiles of this CTA, then its partial sums into slot buffer `which`.
+    auto sweep = [&](auto init_tag, int which) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = 0.0f;
+        step_acc = 0.0f;
+        for (long long t = 0; t < ntiles; ++t) {
+            const long long qb = q0 + t * CL;
+            if (qb + CL <= q1 && qb + CL <= full_quads) tile(init_tag, std::false_type{}, qb, (int)(t & 1));
+            else tile(init_tag, std::true_type{}, qb, (int)(t & 1));
+        }
+        const int warp = tid >> 5, lane = tid & 31, wpg = CL >> 5;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const double s = warp_sum((double)acc[r]);
+            if (lane == 0) sh_red[warp][r] = s;
+        }
+        {
+            const double s = warp_sum((double)step_acc);
+            if (lane == 0) sh_red[warp][16] = s;
+        }
+        __syncthreads();
+        double* dst = k.rslots + (((size_t)which * Pc + p) * cppc + j) * per;
+        for (int i = tid; i <= n; i += blockDim.x) {
+            double s = 0.0;
+            if (i < n) {
+                const int g0 = (i / R) * wpg;
+                for (int q = 0; q < wpg; ++q) s += sh_red[g0 + q][i % R];
+            } else {
+                for (int q = 0; q < wpg; ++q) s += sh_red[q][16];
+            }
+            dst[i] = s;
+        }
+    };
+
+    unsigned generation = 0;
+    bool finished = !active;
+    if (active) {
+        if (j == 0 && tid == 0) a.status[p] = 0;
+        sweep(std::true_type{}, 0);
+    }
+    if (grid_barrier(k, generation, 0u, &sh_bar)) return;
+
+    for (int l = 0; l <= a.max_iters; ++l) {
+        unsigned add_finished = 0;
+        if (!finished) {
+            // Every CTA of the partition adds up the partition's slots itself, same grouping, same
+            // order: identical totals everywhere, and nobody waits for a designated reducer.
+            const double* slots = k.rslots + ((size_t)(l & 1) * Pc + p) * cppc * per;
+            int groups = blockDim.x / per;
+            if (groups < 1) groups = 1;
+            if (groups > cppc) groups = cppc;
+            for (int e = tid; e < groups * per; e += blockDim.x) {
+                const int cg = e / per, i = e - cg * per;
+                double s = 0.0;
+                for (int c = cg; c < cppc; c += groups) s += __ldcg(slots + (size_t)c * per + i);
+                sh_part[e] = s;
+            }
+            __syncthreads();
+            for (int i = tid; i < per; i += blockDim.x) {
+                double s = 0.0;
+                for (int cg = 0; cg < groups; ++cg) s += sh_part[cg * per + i];
+                sh_sum[i] = s;
+            }
+            if (tid == 0) sh_flag = 0;
+            __syncthreads();
+            const bool eps_mode = (a.stop_mode == BTARD_STOP_EPS);
+            const bool converged = eps_mode && l >= 1 && (sh_sum[n] <= a.eps2);
+            if (converged || l == a.max_iters) {
+                finished = true;
+                if (j == 0) {
+                    for (int i = tid; i < n; i += blockDim.x) a.resid_norm[(size_t)p * n + i] = sqrt(sh_sum[i]);
+                    if (tid == 0) {
+                        a.iters[p] = l;
+                        a.last_step[p] = sqrt(sh_sum[n]);
+                        unsigned st = 0;
+                        for (int i = 0; i < n; ++i)
+                            if (!isfinite(sh_sum[i])) st |= BTARD_STATUS_NONFINITE_ROW;
+                        if (eps_mode && !(sh_sum[n] <= a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
+                        atomicOr(&a.status[p], st);
+                    }
+                    add_finished = 1;
+                }
+            } else {
+                for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) {
+                    bool bad = false;
+                    sh_w[i] = (i < n) ? clip_weight(sh_sum[i], tau, bad) : 0.0f;
+                    if (bad) sh_flag = 1;
+                }
+                __syncthreads();
+                if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+                sweep(std::false_type{}, (l + 1) & 1);
+            }
+        }
+        if (grid_barrier(k, generation, add_finished, &sh_bar)) break;
+    }
+    if (active && j == 0 && tid == 0 && atomicAdd(k.error, 0u) != 0u)
+        atomicOr(&a.status[p], BTARD_STATUS_WAIT_EXPIRED);
+}
+
 // After the last pass: partitions still running take iters = max_iters.
 __global__ void cclip_finalize_kernel(const KernelArgs k)
 {
@@ -580,6 +880,63 @@ int launch_totals_to_norms(const double* tot, double* norm, int n, int P, cudaSt
 {
     totals_to_norms_kernel<<<P, 128, 0, st>>>(tot, norm, n);
     BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+// Resident CTAs per SM of the resident kernel (2 when no device can be asked).
+static int resident_ctas_per_sm(int R, bool comp, int threads, size_t smem)
+{
+    int nb = 0;
+    cudaError_t e;
+    if (R == 4) e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<4, true>, threads, smem)
+                         : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<4, false>, threads, smem);
+    else if (R == 8) e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<8, true>, threads, smem)
+                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<8, false>, threads, smem);
+    else e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<16, true>, threads, smem)
+                  : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<16, false>, threads, smem);
+    if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 0; }
+    return nb;
+}
+
+int resident_chunk_partitions(int n, long long stride)
+{
+    int dev = 0, l2 = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    if (!coop || l2 <= 0) return 0;
+    // rows + v (fp32 and bf16) of one partition against three quarters of the L2
+    const double part_bytes = (double)stride * (4.0 * n + 6.0);
+    return (int)(0.75 * (double)l2 / part_bytes);
+}
+
+int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, double* rslots,
+                          unsigned long long* barrier, unsigned int* error, cudaStream_t st)
+{
+    ResidentArgs ra{a, geo.RG, geo.CL, 0, rslots, barrier, error};
+    const bool comp = a.v_lo != nullptr;
+    const size_t smem = (geo.RG > 1) ? sizeof(float4) * 2 * geo.RG * geo.CL : 0;
+    const int occ = resident_ctas_per_sm(geo.R, comp, geo.threads, smem);
+    if (occ < 1) return BTARD_ERR_UNSUPPORTED;
+    int grid = sm_count() * occ;
+    if (grid > kResidentMaxGrid) grid = kResidentMaxGrid;
+    if (grid < a.P) return BTARD_ERR_UNSUPPORTED;
+    ra.cppc = grid / a.P;
+    const long long most = ((a.stride >> 2) + 7) / 8;          // at least one 128-byte line per CTA
+    if (ra.cppc > most) ra.cppc = (int)(most < 1 ? 1 : most);
+    void* args[] = {(void*)&ra};
+    const void* fn;
+    if (geo.R == 4) fn = comp ? (const void*)cclip_resident_kernel<4, true> : (const void*)cclip_resident_kernel<4, false>;
+    else if (geo.R == 8) fn = comp ? (const void*)cclip_resident_kernel<8, true> : (const void*)cclip_resident_kernel<8, false>;
+    else fn = comp ? (const void*)cclip_resident_kernel<16, true> : (const void*)cclip_resident_kernel<16, false>;
+    prof_begin(KIND_ITER, st);
+    cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(geo.threads), args, smem, st);
+    prof_end(KIND_ITER, st);
+    if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return BTARD_ERR_CUDA; }
     count_launch();
     return BTARD_OK;
 }

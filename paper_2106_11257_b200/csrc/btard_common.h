@@ -80,6 +80,12 @@ Geometry cclip_geometry(int n, int P, long long stride);
 int choose_ctas_per_partition(int P, long long quads, int CL, int slots);
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
+// L2-resident variant: how many partitions fit one chunk (0: not available on this device), and the
+// cooperative launch that runs the start pass and every update of one chunk.
+constexpr int kResidentMaxGrid = 148 * 8;
+int resident_chunk_partitions(int n, long long stride);
+int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, double* rslots,
+                          unsigned long long* barrier, unsigned int* error, cudaStream_t st);
 int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
                        int P, cudaStream_t st);
 // squared-norm totals -> norms, used when verification is asked to compute the norms itself.

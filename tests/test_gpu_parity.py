@@ -191,6 +191,40 @@ def test_peer_and_partition_indexing():
     assert np.allclose(cpu(r["v"]), ref["v"], rtol=1e-6)
 
 
+# ----------------------------------------------------------------------------- L2-resident variant
+@pytest.mark.parametrize("n", [1, 4, 16, 23, 64, 256])
+@pytest.mark.parametrize("init", [btard.INIT_ZERO, btard.INIT_MEAN, btard.INIT_COORD_MEDIAN,
+                                  btard.INIT_CALLER_V0])
+def test_resident_variant_matches_oracle(n, init):
+    """All updates of a chunk inside one cooperative kernel with grid barriers: same numbers."""
+    rng = np.random.default_rng(400 + n)
+    P, stride = 3, 5024
+    lens = np.array([5024, 4097, 0 if n % 2 else 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.5, 1.0, 2.0])
+    v0 = rng.standard_normal((P, stride)).astype(np.float32) if init == btard.INIT_CALLER_V0 else None
+    ref = oracle.centered_clip(g, tau, lens, init_mode=init, v0=v0, max_iters=6)
+    _, r = run_gpu_cclip(g, tau, lens, init_mode=init, v0=v0, max_iters=6, algo=btard.ALGO_DIRECT_RESIDENT)
+    check_cclip(r, ref, lens)
+    assert not (cpu(r["status"]) & 4).any()
+
+
+def test_resident_variant_eps_mode_and_chunks():
+    """Rows long enough that the partitions go through in several L2-sized chunks; eps stop with
+    partitions finishing at different updates."""
+    rng = np.random.default_rng(12)
+    P, n, stride = 5, 16, 600_000
+    lens = np.array([600_000, 599_999, 123_457, 600_000, 31])
+    g = make_case(rng, P, n, stride, lens, far_rows=5, scale=0.001)
+    tau = np.array([1.0, 0.5, 2.0, 1.0, 1.0])
+    ref = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN,
+                               stop_mode=oracle.STOP_EPS, max_iters=60, eps=1e-5)
+    _, r = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_COORD_MEDIAN, stop_mode=btard.STOP_EPS,
+                         max_iters=60, eps=1e-5, algo=btard.ALGO_DIRECT_RESIDENT)
+    check_cclip(r, ref, lens, eps_mode=True)
+    assert len(set(ref["iters"].tolist())) > 1
+
+
 # ----------------------------------------------------------------------------- Gram variant
 @pytest.mark.parametrize("n", [1, 3, 8, 16, 23, 64, 100, 128])
 @pytest.mark.parametrize("init", [btard.INIT_MEAN, btard.INIT_COORD_MEDIAN, btard.INIT_CALLER_V0])
