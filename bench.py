@@ -210,12 +210,14 @@ def run_ours(args):
         gh.copy_(g)
         scratch = torch.empty(btard.aggregate_host_scratch(n, P, stride, w.K), dtype=torch.uint8, device=dev)
         hout = None
+        copy_stream = torch.cuda.Stream()
 
         def host_step():
             nonlocal hout
             r = btard.aggregate_host(gh, w.tau, w.zseed, K=w.K, part_len=w.part_len,
                                      init_mode=w.init_mode, stop_mode=w.stop_mode,
-                                     max_iters=w.max_iters, eps=w.eps, scratch=scratch, out=hout)
+                                     max_iters=w.max_iters, eps=w.eps, scratch=scratch, out=hout,
+                                     copy_stream=copy_stream)
             hout = {k: r[k] for k in r if k != "scratch"}
         for _ in range(max(1, min(args.warmup, 2))):
             host_step()

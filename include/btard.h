@@ -184,7 +184,8 @@ BTARD_API int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t p
 /*
  * The same aggregation + verification with HOST buffers: copies g to the device, runs
  * btard_centered_clip (DIRECT) and btard_verify_projections, copies the results back and waits for
- * `stream`.  All device memory comes from device_scratch (sized by btard_aggregate_host_scratch).
+ * `stream` (and for copy_stream, which only carries copies this call queued).  All device memory
+ * comes from device_scratch (sized by btard_aggregate_host_scratch).
  * Host output pointers may be NULL to skip that copy, except v.  Pinned host memory makes the
  * copies asynchronous and fast; pageable memory works too.
  */
@@ -215,6 +216,11 @@ typedef struct {
     void* device_scratch;        /* device, 256-byte aligned */
     size_t device_scratch_bytes;
     void* stream;
+    void* copy_stream;           /* optional second cudaStream_t (NULL: none).  When given and different
+                                    from `stream`, the rows are copied in up to four chunks of partitions
+                                    on it while the kernels of the previous chunk run on `stream`; g must
+                                    then be pinned host memory for the overlap to happen.  The chunks
+                                    change no result: partitions are independent.                      */
 } btard_host_args;
 
 BTARD_API size_t btard_aggregate_host_scratch(const btard_host_args* args);

@@ -66,7 +66,8 @@ class HostArgs(C.Structure):
                 ("weight", C.c_void_p), ("dot", C.c_void_p), ("s", C.c_void_p),
                 ("s_sum", C.c_void_p), ("znorm2", C.c_void_p), ("resid_sum_norm", C.c_void_p),
                 ("status", C.c_void_p), ("device_scratch", C.c_void_p),
-                ("device_scratch_bytes", C.c_size_t), ("stream", C.c_void_p)]
+                ("device_scratch_bytes", C.c_size_t), ("stream", C.c_void_p),
+                ("copy_stream", C.c_void_p)]
 
 
 _lib = None
@@ -320,9 +321,10 @@ def aggregate_host_scratch(n, P, row_stride, K):
 
 def aggregate_host(g_host, tau, seed, K=1, part_len=None, init_mode=INIT_COORD_MEDIAN, v_host=None,
                    stop_mode=STOP_FIXED_ITERS, max_iters=1, eps=0.0, scratch=None, out=None,
-                   device="cuda", stream=None):
+                   device="cuda", stream=None, copy_stream=None):
     """Whole aggregation + verification from HOST tensors (ideally pinned); blocks until done.
-    Returns dict of host tensors."""
+    `copy_stream` (a second torch.cuda.Stream) lets the host-to-device copy of the next chunk of
+    partitions overlap the kernels of the current one.  Returns dict of host tensors."""
     torch = _torch()
     assert not g_host.is_cuda and g_host.dtype == torch.float32 and g_host.dim() == 3 and g_host.is_contiguous()
     P, n, stride = g_host.shape
@@ -351,7 +353,8 @@ def aggregate_host(g_host, tau, seed, K=1, part_len=None, init_mode=INIT_COORD_M
                  s_sum=o["s_sum"].data_ptr(), znorm2=o["znorm2"].data_ptr(),
                  resid_sum_norm=o["resid_sum_norm"].data_ptr(), status=o["status"].data_ptr(),
                  device_scratch=scratch.data_ptr(), device_scratch_bytes=scratch.numel(),
-                 stream=_stream_ptr(stream))
+                 stream=_stream_ptr(stream),
+                 copy_stream=C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None)
     with torch.cuda.device(scratch.device):
         _check(lib().btard_aggregate_host(C.byref(a)), "btard_aggregate_host")
     res = dict(o)

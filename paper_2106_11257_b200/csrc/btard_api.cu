@@ -485,33 +485,62 @@ int btard_aggregate_host(const btard_host_args* a)
     char* base = (char*)a->device_scratch;
     const size_t n = a->n_peers, P = a->n_partitions, S = (size_t)a->row_stride, K = a->n_z;
 
-    BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.g, a->g, sizeof(float) * P * n * S, cudaMemcpyHostToDevice, st));
+    // With a second stream the partitions go through in up to four chunks: the copy of the next
+    // chunk's rows runs on copy_stream while the kernels of the current chunk run on stream.
+    cudaStream_t cs = (cudaStream_t)a->copy_stream;
+    const bool piped = a->copy_stream != nullptr && a->copy_stream != a->stream && P > 1;
+    const size_t nchunks = piped ? (P < 4 ? P : 4) : 1;
+    cudaEvent_t ready[4] = {nullptr, nullptr, nullptr, nullptr};
+    auto drop_events = [&]() {
+        for (size_t c = 0; c < 4; ++c)
+            if (ready[c]) { cudaEventDestroy(ready[c]); ready[c] = nullptr; }
+    };
     if (a->init_mode == BTARD_INIT_CALLER_V0)
         BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.v, a->v, sizeof(float) * P * S, cudaMemcpyHostToDevice, st));
+    if (piped) {
+        for (size_t c = 0; c < nchunks; ++c) {
+            const size_t p0 = P * c / nchunks, p1 = P * (c + 1) / nchunks;
+            cudaError_t e = cudaEventCreateWithFlags(&ready[c], cudaEventDisableTiming);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(base + h.g + sizeof(float) * p0 * n * S, a->g + p0 * n * S,
+                                    sizeof(float) * (p1 - p0) * n * S, cudaMemcpyHostToDevice, cs);
+            if (e == cudaSuccess) e = cudaEventRecord(ready[c], cs);
+            if (e != cudaSuccess) { set_cuda_error(e); drop_events(); return BTARD_ERR_CUDA; }
+        }
+    } else {
+        BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.g, a->g, sizeof(float) * P * n * S, cudaMemcpyHostToDevice, st));
+    }
 
-    btard_cclip_args ca{};
-    ca.n_peers = a->n_peers; ca.n_partitions = a->n_partitions; ca.row_stride = a->row_stride;
-    ca.part_len = a->part_len; ca.g = (const float*)(base + h.g); ca.tau = a->tau;
-    ca.init_mode = a->init_mode; ca.algo = BTARD_ALGO_DIRECT; ca.stop_mode = a->stop_mode;
-    ca.max_iters = a->max_iters; ca.eps = a->eps; ca.v = (float*)(base + h.v);
-    ca.iters = (int32_t*)(base + h.iters); ca.last_step_norm = (double*)(base + h.last_step);
-    ca.resid_norm = (double*)(base + h.resid_norm); ca.status = (uint32_t*)(base + h.status_c);
-    ca.workspace = base + h.ws_c; ca.workspace_bytes = h.ws_c_bytes; ca.stream = a->stream;
-    rc = btard_centered_clip(&ca);
-    if (rc != BTARD_OK) return rc;
+    for (size_t c = 0; c < nchunks; ++c) {
+        const size_t p0 = P * c / nchunks, p1 = P * (c + 1) / nchunks;
+        if (piped) {
+            cudaError_t e = cudaStreamWaitEvent(st, ready[c], 0);
+            if (e != cudaSuccess) { set_cuda_error(e); drop_events(); return BTARD_ERR_CUDA; }
+        }
+        btard_cclip_args ca{};
+        ca.n_peers = a->n_peers; ca.n_partitions = (int32_t)(p1 - p0); ca.row_stride = a->row_stride;
+        ca.part_len = a->part_len + p0; ca.g = (const float*)(base + h.g) + p0 * n * S; ca.tau = a->tau + p0;
+        ca.init_mode = a->init_mode; ca.algo = BTARD_ALGO_DIRECT; ca.stop_mode = a->stop_mode;
+        ca.max_iters = a->max_iters; ca.eps = a->eps; ca.v = (float*)(base + h.v) + p0 * S;
+        ca.iters = (int32_t*)(base + h.iters) + p0; ca.last_step_norm = (double*)(base + h.last_step) + p0;
+        ca.resid_norm = (double*)(base + h.resid_norm) + p0 * n; ca.status = (uint32_t*)(base + h.status_c) + p0;
+        ca.workspace = base + h.ws_c; ca.workspace_bytes = h.ws_c_bytes; ca.stream = a->stream;
+        rc = btard_centered_clip(&ca);
+        if (rc != BTARD_OK) { drop_events(); return rc; }
 
-    btard_verify_args va{};
-    va.n_peers = a->n_peers; va.n_partitions = a->n_partitions; va.row_stride = a->row_stride;
-    va.part_len = a->part_len; va.g = ca.g; va.v = ca.v; va.tau = a->tau; va.seed = a->seed;
-    va.n_z = a->n_z; va.partition_base = 0; va.resid_norm_in = ca.resid_norm;
-    va.norm = (double*)(base + h.norm); va.weight = (double*)(base + h.weight);
-    va.dot = (double*)(base + h.dot); va.s = (double*)(base + h.s);
-    va.s_sum = (double*)(base + h.s_sum); va.znorm2 = (double*)(base + h.znorm2);
-    va.resid_sum_norm = (double*)(base + h.rsn); va.resid_sum = nullptr;
-    va.status = (uint32_t*)(base + h.status_v);
-    va.workspace = base + h.ws_v; va.workspace_bytes = h.ws_v_bytes; va.stream = a->stream;
-    rc = btard_verify_projections(&va);
-    if (rc != BTARD_OK) return rc;
+        btard_verify_args va{};
+        va.n_peers = a->n_peers; va.n_partitions = ca.n_partitions; va.row_stride = a->row_stride;
+        va.part_len = ca.part_len; va.g = ca.g; va.v = ca.v; va.tau = ca.tau; va.seed = a->seed;
+        va.n_z = a->n_z; va.partition_base = (int32_t)p0; va.resid_norm_in = ca.resid_norm;
+        va.norm = (double*)(base + h.norm) + p0 * n; va.weight = (double*)(base + h.weight) + p0 * n;
+        va.dot = (double*)(base + h.dot) + p0 * n * K; va.s = (double*)(base + h.s) + p0 * n * K;
+        va.s_sum = (double*)(base + h.s_sum) + p0 * K; va.znorm2 = (double*)(base + h.znorm2) + p0 * K;
+        va.resid_sum_norm = (double*)(base + h.rsn) + p0; va.resid_sum = nullptr;
+        va.status = (uint32_t*)(base + h.status_v) + p0;
+        va.workspace = base + h.ws_v; va.workspace_bytes = h.ws_v_bytes; va.stream = a->stream;
+        rc = btard_verify_projections(&va);
+        if (rc != BTARD_OK) { drop_events(); return rc; }
+    }
 
     auto back = [&](void* dst, size_t off, size_t bytes) -> cudaError_t {
         if (!dst) return cudaSuccess;
@@ -533,7 +562,9 @@ int btard_aggregate_host(const btard_host_args* a)
         BTARD_CUDA_TRY(cudaMemcpyAsync(sc.data(), base + h.status_c, sizeof(uint32_t) * P, cudaMemcpyDeviceToHost, st));
         BTARD_CUDA_TRY(cudaMemcpyAsync(sv.data(), base + h.status_v, sizeof(uint32_t) * P, cudaMemcpyDeviceToHost, st));
     }
-    BTARD_CUDA_TRY(cudaStreamSynchronize(st));
+    const cudaError_t sync_err = cudaStreamSynchronize(st);
+    drop_events();
+    BTARD_CUDA_TRY(sync_err);
     if (a->status)
         for (size_t p = 0; p < P; ++p) a->status[p] = sc[p] | sv[p];
     return BTARD_OK;

@@ -356,6 +356,12 @@ def test_aggregate_host_matches_device_path():
     for key in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm"):
         assert torch.equal(h[key], o[key].cpu()), key
     assert torch.equal(h["iters"], r["iters"].cpu())
+    # chunked, with the copies on a second stream: same numbers (z is keyed by the global partition)
+    h2 = btard.aggregate_host(gh, 1.0, 77, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                              max_iters=7, copy_stream=torch.cuda.Stream())
+    assert torch.equal(h2["iters"], h["iters"])
+    for key in ("v", "norm", "weight", "dot", "s", "znorm2"):      # other CTA grouping: last bits may differ
+        assert rel_l2(h2[key].numpy(), h[key].numpy()) <= 1e-6, key
 
 
 # ----------------------------------------------------------------------------- full-size configs
