@@ -203,6 +203,40 @@ def run_ours(args):
     ms_step = max_over_ranks(ms_step, dist, dev)
     value = whole_job_value(in_bytes, ms_step, world)
 
+    # ---- the other algorithm on the same tensor, for the side-by-side the configurations ask for ---
+    other = None
+    if args.side_by_side and w.n <= 128:
+        other_algo = btard.ALGO_DIRECT if args.algo == "gram" else btard.ALGO_GRAM
+        ws_o = torch.empty(btard.centered_clip_workspace(n, P, stride, w.stop_mode, other_algo),
+                           dtype=torch.uint8, device=dev)
+        v_o = torch.empty((P, stride), dtype=torch.float32, device=dev)
+        so = {}
+
+        def other_step():
+            r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=w.init_mode, v=v_o,
+                                    stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps,
+                                    algo=other_algo, workspace=ws_o, out=so.get("c"))
+            so["c"] = {k: r[k] for k in ("iters", "last_step_norm", "resid_norm", "status")}
+            o = btard.verify_projections(g, v_o, w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                         resid_norm_in=r["resid_norm"], workspace=ws_v, out=so.get("v"))
+            so["v"] = {k: o[k] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2",
+                                         "resid_sum_norm", "status")}
+        for _ in range(3):
+            other_step()
+        torch.cuda.synchronize()
+        k3 = max(3, min(args.steps, 10))
+        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        o0.record()
+        for _ in range(k3):
+            other_step()
+        o1.record()
+        torch.cuda.synchronize()
+        ms_o = max_over_ranks(o0.elapsed_time(o1) / k3, dist, dev)
+        diff = float((v_o - v).norm() / v.norm())
+        other = {"algo": "direct" if args.algo == "gram" else "gram", "ms_per_aggregation": ms_o,
+                 "rel_l2_difference_of_v": diff}
+        del ws_o, v_o
+
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----------
     e2e = None
     if not args.no_e2e and args.algo == "direct":
@@ -300,6 +334,8 @@ def run_ours(args):
                      "algorithmic_bytes_per_launch": per_pass_bytes * P,
                      "verify_kernel_gbs": ver_gbs},
         "kernels": kernels,
+        "ms_per_aggregation": ms_step,
+        "other_algorithm": other,
         "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line))
@@ -367,6 +403,8 @@ def main():
     ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not bracket the library's kernels with CUDA events (no roofline object)")
+    ap.add_argument("--no-side-by-side", dest="side_by_side", action="store_false",
+                    help="do not also time the other algorithm (direct / Gram) on the same tensor")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

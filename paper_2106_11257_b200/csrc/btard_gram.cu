@@ -396,6 +396,82 @@ __global__ void __launch_bounds__(kGramThreads) gram_iterate_kernel(const GArgs 
     }
 }
 
+// n <= 32: the same iteration by ONE warp per partition, lane i owning row i of G in registers.
+// Sums are butterfly shuffles (every lane gets the same value), so there is no barrier at all and
+// an update costs a few hundred cycles instead of six CTA-wide synchronisations.
+__device__ __forceinline__ double warp_allsum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+template <int N>   // 16 or 32: rows of G held per lane
+__global__ void __launch_bounds__(32) gram_iterate_warp_kernel(const GArgs k)
+{
+    const GramLaunch& a = k.a;
+    const int n = a.n, NB = k.g.NB, lane = threadIdx.x, p = blockIdx.x;
+    const double* src = a.gram + (size_t)p * k.g.entries;
+    double Grow[N];
+    const bool row = lane < n;
+#pragma unroll
+    for (int jj = 0; jj < N; ++jj) {
+        double val = 0.0;
+        if (row && jj < n) {
+            const int i0 = lane < jj ? lane : jj, j0 = lane < jj ? jj : lane;   // stored triangle: bi <= bj
+            const int bi = i0 >> 3, bj = j0 >> 3;
+            int blk = bj - bi;
+            for (int q = 0; q < bi; ++q) blk += NB - q;
+            // inside a diagonal block both orders are stored and equal; elsewhere (i0, j0) is stored
+            val = src[(size_t)blk * 64 + (i0 & 7) * 8 + (j0 & 7)];
+        }
+        Grow[jj] = val;
+    }
+    const double tau = a.table[p].tau;
+    double gii = 0.0;
+#pragma unroll
+    for (int jj = 0; jj < N; ++jj)
+        if (jj == lane) gii = Grow[jj];
+    const bool bad = row && !isfinite(gii);
+    const bool live = row && !bad;
+    double ai = 0.0, Gai = 0.0, step2 = 0.0;
+    int iters = 0;
+    for (int l = 0; l < a.max_iters; ++l) {
+        const double aGa = warp_allsum(live ? ai * Gai : 0.0);
+        double w = 0.0;
+        if (live) {
+            double rho2 = gii - 2.0 * Gai + aGa;
+            if (rho2 < 0.0) rho2 = 0.0;
+            const double rho = sqrt(rho2);
+            if (isfinite(rho)) w = (rho <= tau) ? 1.0 : tau / rho;
+        }
+        const double W = warp_allsum(w);
+        const double d = live ? (w - W * ai) / (double)n : 0.0;
+        double Gd = 0.0;
+#pragma unroll
+        for (int q = 0; q < N; ++q) {
+            const double dq = __shfl_sync(0xffffffffu, d, q);
+            if (dq != 0.0 && live) Gd += Grow[q] * dq;
+        }
+        step2 = warp_allsum(live ? d * Gd : 0.0);
+        ai += d;
+        Gai += Gd;
+        iters = l + 1;
+        if (a.stop_mode == BTARD_STOP_EPS && step2 <= a.eps2) break;
+    }
+    if (step2 < 0.0) step2 = 0.0;
+    if (row) a.coef[(size_t)p * n + lane] = ai;
+    const unsigned anybad = __ballot_sync(0xffffffffu, bad);
+    if (lane == 0) {
+        a.iters[p] = iters;
+        a.last_step[p] = sqrt(step2);
+        unsigned st = 0;
+        if (anybad) st |= BTARD_STATUS_NONFINITE_ROW;
+        if (a.stop_mode == BTARD_STOP_EPS && !(step2 <= a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
+        a.status[p] = st;
+    }
+}
+
 __global__ void gram_finalize_kernel(const double* tot, double* resid_norm, uint32_t* status, int n)
 {
     const int p = blockIdx.x;
@@ -475,7 +551,9 @@ int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream
     if (smem > 48 * 1024)
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_iterate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     prof_begin(KIND_COEF, st);
-    gram_iterate_kernel<<<a.P, kGramThreads, smem, st>>>(ga);
+    if (a.n <= 16) gram_iterate_warp_kernel<16><<<a.P, 32, 0, st>>>(ga);
+    else if (a.n <= 32) gram_iterate_warp_kernel<32><<<a.P, 32, 0, st>>>(ga);
+    else gram_iterate_kernel<<<a.P, kGramThreads, smem, st>>>(ga);
     prof_end(KIND_COEF, st);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
