@@ -144,7 +144,8 @@ def run_ours(args):
     g = w.g
     P, n, stride = g.shape
     dev = g.device
-    algo = btard.ALGO_GRAM if args.algo == "gram" else btard.ALGO_DIRECT
+    algo = {"direct": btard.ALGO_DIRECT, "gram": btard.ALGO_GRAM,
+            "cooperative": btard.ALGO_DIRECT_COOPERATIVE, "resident": btard.ALGO_DIRECT_RESIDENT}[args.algo]
     ws_c = torch.empty(btard.centered_clip_workspace(n, P, stride, w.stop_mode, algo), dtype=torch.uint8, device=dev)
     ws_v = torch.empty(btard.verify_projections_workspace(n, P, stride, w.K), dtype=torch.uint8, device=dev)
     v = torch.empty((P, stride), dtype=torch.float32, device=dev)
@@ -239,7 +240,7 @@ def run_ours(args):
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region ----------
     e2e = None
-    if not args.no_e2e and args.algo == "direct":
+    if not args.no_e2e and args.algo != "gram":
         gh = torch.empty(g.shape, dtype=torch.float32, pin_memory=True)
         gh.copy_(g)
         scratch = torch.empty(btard.aggregate_host_scratch(n, P, stride, w.K), dtype=torch.uint8, device=dev)
@@ -399,7 +400,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--algo", default="direct", choices=["direct", "gram"])
+    ap.add_argument("--algo", default="direct", choices=["direct", "gram", "cooperative", "resident"])
     ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not bracket the library's kernels with CUDA events (no roofline object)")

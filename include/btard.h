@@ -53,11 +53,15 @@ extern "C" {
 #define BTARD_INIT_MEAN 2
 #define BTARD_INIT_COORD_MEDIAN 3   /* coordinate-wise median of the n rows                         */
 
-#define BTARD_ALGO_DIRECT 0         /* one pass over g per iteration, one kernel launch per pass    */
+#define BTARD_ALGO_DIRECT 0         /* one pass over g per update, one kernel launch per update     */
 #define BTARD_ALGO_GRAM 1           /* Gram matrix pass + iteration in coefficient space + combine  */
-#define BTARD_ALGO_DIRECT_RESIDENT 2 /* as DIRECT, but chunks of partitions that fit the L2 cache are
-                                       iterated inside one cooperative kernel with grid barriers;
-                                       falls back to DIRECT where a partition does not fit         */
+#define BTARD_ALGO_DIRECT_RESIDENT 2 /* as DIRECT, but partitions go through in chunks that fit the L2
+                                       cache, all updates of a chunk inside one cooperative kernel
+                                       with grid barriers; where a partition does not fit: DIRECT   */
+#define BTARD_ALGO_DIRECT_COOPERATIVE 3 /* as DIRECT, but all updates of all partitions inside one
+                                       cooperative kernel: no launch per update and nothing runs
+                                       after the last partition converged; where the device cannot
+                                       launch it: DIRECT                                            */
 
 #define BTARD_STOP_FIXED_ITERS 0    /* exactly max_iters updates                                    */
 #define BTARD_STOP_EPS 1            /* stop once ||v^{l+1} - v^l||_2 <= eps, at most max_iters       */

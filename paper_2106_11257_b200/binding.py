@@ -10,7 +10,7 @@ import os
 import numpy as np
 
 INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
-ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT = 0, 1, 2
+ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT, ALGO_DIRECT_COOPERATIVE = 0, 1, 2, 3
 STOP_FIXED_ITERS, STOP_EPS = 0, 1
 SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1
 STATUS_NOT_CONVERGED, STATUS_NONFINITE_ROW = 1, 2

@@ -110,7 +110,9 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, in
         w.gram = off; off = align_up(off + sizeof(double) * (size_t)P * gg.entries, 256);
         w.coef = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
     }
-    w.rslots = off; off = align_up(off + sizeof(double) * 2 * (size_t)kResidentMaxGrid * (n + 1), 256);
+    size_t ritems = (size_t)P * geo.cpp;
+    if (ritems < (size_t)kResidentMaxGrid) ritems = kResidentMaxGrid;
+    w.rslots = off; off = align_up(off + sizeof(double) * 2 * ritems * (n + 1), 256);
     w.rflags_bytes = sizeof(unsigned long long) * ((size_t)P + 1);   // a barrier word per chunk, error flag
     w.rflags = off; off = align_up(off + w.rflags_bytes, 256);
     w.total = off;
@@ -224,7 +226,7 @@ int btard_centered_clip(const btard_cclip_args* a)
     if (a->stop_mode != BTARD_STOP_FIXED_ITERS && a->stop_mode != BTARD_STOP_EPS)
         return BTARD_ERR_INVALID_ARG;
     if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM &&
-        a->algo != BTARD_ALGO_DIRECT_RESIDENT)
+        a->algo != BTARD_ALGO_DIRECT_RESIDENT && a->algo != BTARD_ALGO_DIRECT_COOPERATIVE)
         return BTARD_ERR_INVALID_ARG;
     if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (!aligned16(a->g) || !aligned16(a->v) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
@@ -258,8 +260,11 @@ int btard_centered_clip(const btard_cclip_args* a)
     }
 
     // Init pass: v^0 and the residual norms at v^0 (slot buffer 0).
-    // Chunks of partitions that fit the L2 cache take the resident path below (0: none do).
-    const int chunk = (a->algo == BTARD_ALGO_DIRECT_RESIDENT) ? resident_chunk_partitions(n, a->row_stride) : 0;
+    // How the updates are driven: one cooperative kernel over everything (whole), one per L2-sized
+    // chunk of partitions (chunk >= 1), or one launch per update.
+    const int fit = resident_chunk_partitions(n, a->row_stride);         // partitions per L2 budget
+    const int chunk = (a->algo == BTARD_ALGO_DIRECT_RESIDENT) ? fit : 0;
+    const bool whole = (a->algo == BTARD_ALGO_DIRECT_COOPERATIVE) && cooperative_launch_supported();
     L.init_mode = a->init_mode;
     if (a->init_mode == BTARD_INIT_COORD_MEDIAN && chunk < 1) {
         rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
@@ -292,6 +297,15 @@ int btard_centered_clip(const btard_cclip_args* a)
         if (rc != BTARD_OK) return rc;
         return launch_gram_finalize(L.tot_out, a->resid_norm, a->status, n, P, st);
     }
+    if (whole) {
+        BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.rflags, 0, ws.rflags_bytes, st));
+        unsigned long long* bars = (unsigned long long*)(base + ws.rflags);
+        unsigned int* err = (unsigned int*)(bars + P);
+        rc = launch_cclip_resident(L, geo, geo.cpp, fit >= P ? 0 : 1, (double*)(base + ws.rslots), bars, err, st);
+        if (rc == BTARD_OK) return BTARD_OK;
+        // the cooperative launch was refused: nothing ran, take the launch-per-update path
+    }
+
     // Start pass and every update of a chunk in one resident kernel.
     if (chunk >= 1) {
         BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.rflags, 0, ws.rflags_bytes, st));
@@ -306,6 +320,7 @@ int btard_centered_clip(const btard_cclip_args* a)
             C.v = a->v + (size_t)c0 * a->row_stride;
             if (L.v_lo) C.v_lo = L.v_lo + (size_t)c0 * a->row_stride;
             C.table = L.table + c0;
+            C.done = L.done + c0;
             C.iters = a->iters + c0; C.last_step = a->last_step_norm + c0;
             C.resid_norm = a->resid_norm + (size_t)c0 * n; C.status = a->status + c0;
             C.P = Pc;
@@ -315,7 +330,7 @@ int btard_centered_clip(const btard_cclip_args* a)
                 if (rc != BTARD_OK) return rc;
                 C.init_mode = BTARD_INIT_CALLER_V0;
             }
-            rc = launch_cclip_resident(C, geo, (double*)(base + ws.rslots), bars + ci, err, st);
+            rc = launch_cclip_resident(C, geo, 0, 0, (double*)(base + ws.rslots), bars + ci, err, st);
             if (rc != BTARD_OK) {
                 if (c0 == 0) ok = false;      // nothing done yet: take the streaming path instead
                 else return rc;
@@ -449,6 +464,7 @@ HostScratch host_layout(const btard_host_args* a)
     btard_cclip_args ca{};
     ca.n_peers = a->n_peers; ca.n_partitions = a->n_partitions; ca.row_stride = a->row_stride;
     ca.stop_mode = BTARD_STOP_EPS;   // the larger of the two layouts
+    ca.algo = BTARD_ALGO_DIRECT_COOPERATIVE;
     h.ws_c_bytes = btard_centered_clip_workspace(&ca);
     btard_verify_args va{};
     va.n_peers = a->n_peers; va.n_partitions = a->n_partitions; va.row_stride = a->row_stride;
@@ -520,7 +536,9 @@ int btard_aggregate_host(const btard_host_args* a)
         btard_cclip_args ca{};
         ca.n_peers = a->n_peers; ca.n_partitions = (int32_t)(p1 - p0); ca.row_stride = a->row_stride;
         ca.part_len = a->part_len + p0; ca.g = (const float*)(base + h.g) + p0 * n * S; ca.tau = a->tau + p0;
-        ca.init_mode = a->init_mode; ca.algo = BTARD_ALGO_DIRECT; ca.stop_mode = a->stop_mode;
+        // eps mode: nothing should be launched after convergence, chunk by chunk
+        ca.init_mode = a->init_mode; ca.stop_mode = a->stop_mode;
+        ca.algo = (a->stop_mode == BTARD_STOP_EPS) ? BTARD_ALGO_DIRECT_COOPERATIVE : BTARD_ALGO_DIRECT;
         ca.max_iters = a->max_iters; ca.eps = a->eps; ca.v = (float*)(base + h.v) + p0 * S;
         ca.iters = (int32_t*)(base + h.iters) + p0; ca.last_step_norm = (double*)(base + h.last_step) + p0;
         ca.resid_norm = (double*)(base + h.resid_norm) + p0 * n; ca.status = (uint32_t*)(base + h.status_c) + p0;

@@ -351,7 +351,8 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 // =================================================================================================
 struct ResidentArgs {
     CclipLaunch a;                  // chunk-relative pointers; a.P = partitions in the chunk
-    int RG, CL, cppc;               // cppc CTAs per partition of the chunk
+    int RG, CL, cppc;               // cppc work items (column ranges) per partition of the chunk
+    int streaming;                  // 1: the chunk is larger than L2 (evict-first loads, alternating sweeps)
     double* rslots;                 // [2][P][cppc][n+1]
     unsigned long long* barrier;    // low word: arrivals (monotonic), high word: finished partitions
     unsigned int* error;            // set when a bounded wait expired
@@ -411,23 +412,36 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
     const CclipLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cppc = k.cppc, Pc = a.P;
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
-    const bool active = (int)blockIdx.x < Pc * cppc;
-    const int p = active ? (int)blockIdx.x / cppc : 0, j = active ? (int)blockIdx.x % cppc : 0;
-    const long long stride = a.stride, len = a.table[p].len;
-    const double tau = a.table[p].tau;
-    const float* gp = a.g + (size_t)p * n * stride;
-    float* vp = a.v + (size_t)p * stride;
-    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
+    const int items = Pc * cppc;                       // CTA b owns items b, b + gridDim.x, ...
+    const long long stride = a.stride;
     const float inv_n = 1.0f / (float)n;
     const float* wrow = sh_w + rg * R;
     const int per = n + 1;
-
     const long long Q = stride >> 2;
-    long long q0 = Q * j / cppc, q1 = Q * (j + 1) / cppc;
-    if (j > 0) q0 &= ~7LL;
-    if (j + 1 < cppc) q1 &= ~7LL;
-    const long long full_quads = len >> 2;
-    const long long ntiles = (q1 - q0 + CL - 1) / CL;
+    const uint64_t policy = policy_evict_first();
+
+    // the work item in hand
+    int p = 0, j = 0;
+    long long len = 0, q0 = 0, q1 = 0, full_quads = 0, ntiles = 0;
+    double tau = 0.0;
+    const float* gp = a.g;
+    float* vp = a.v;
+    unsigned short* lop = nullptr;
+    auto take_item = [&](int item) {
+        p = item / cppc;
+        j = item - p * cppc;
+        len = a.table[p].len;
+        tau = a.table[p].tau;
+        gp = a.g + (size_t)p * n * stride;
+        vp = a.v + (size_t)p * stride;
+        lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
+        q0 = Q * j / cppc;
+        q1 = Q * (j + 1) / cppc;
+        if (j > 0) q0 &= ~7LL;
+        if (j + 1 < cppc) q1 &= ~7LL;
+        full_quads = len >> 2;
+        ntiles = (q1 - q0 + CL - 1) / CL;
+    };
 
     float acc[R];
     float step_acc = 0.0f;
@@ -447,8 +461,9 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const int i = rg * R + r;
-                x[r] = (i < n) ? __ldg(reinterpret_cast<const float4*>(gp + (size_t)i * stride + col))
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float* src = gp + (size_t)i * stride + col;
+                x[r] = (i >= n) ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                : (k.streaming ? ld_policy(src, policy) : __ldg(reinterpret_cast<const float4*>(src)));
             }
             if (!INIT || a.init_mode == BTARD_INIT_CALLER_V0) v4 = *reinterpret_cast<const float4*>(vp + col);
             if (COMP && !INIT) {
@@ -539,13 +554,13 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
         }
     };
 
-    // All tiles of this CTA, then its partial sums into slot buffer `which`.
-    auto sweep = [&](auto init_tag, int which) {
+    // All tiles of the item in hand, then its partial sums into slot buffer `which`.
+    auto sweep = [&](auto init_tag, int which, bool backwards) {
 #pragma unroll
         for (int r = 0; r < R; ++r) acc[r] = 0.0f;
         step_acc = 0.0f;
         for (long long t = 0; t < ntiles; ++t) {
-            const long long qb = q0 + t * CL;
+            const long long qb = q0 + (backwards ? ntiles - 1 - t : t) * CL;
             if (qb + CL <= q1 && qb + CL <= full_quads) tile(init_tag, std::false_type{}, qb, (int)(t & 1));
             else tile(init_tag, std::true_type{}, qb, (int)(t & 1));
         }
@@ -574,18 +589,27 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
     };
 
     unsigned generation = 0;
-    bool finished = !active;
-    if (active) {
+    const int first = (int)blockIdx.x, hop = (int)gridDim.x;
+    const int mine = first < items ? (items - first + hop - 1) / hop : 0;    // items of this CTA
+    for (int m = 0; m < mine; ++m) {
+        take_item(first + m * hop);
         if (j == 0 && tid == 0) a.status[p] = 0;
-        sweep(std::true_type{}, 0);
+        sweep(std::true_type{}, 0, false);
+        __syncthreads();
     }
     if (grid_barrier(k, generation, 0u, &sh_bar)) return;
 
+    const bool eps_mode = (a.stop_mode == BTARD_STOP_EPS);
     for (int l = 0; l <= a.max_iters; ++l) {
         unsigned add_finished = 0;
-        if (!finished) {
-            // Every CTA of the partition adds up the partition's slots itself, same grouping, same
-            // order: identical totals everywhere, and nobody waits for a designated reducer.
+        // Larger than L2: consecutive updates sweep in opposite directions, so that an update
+        // starts on the lines the previous one read last.
+        const bool backwards = k.streaming && ((l & 1) == 0);
+        for (int m = 0; m < mine; ++m) {
+            take_item(first + (backwards ? mine - 1 - m : m) * hop);
+            if (a.done[p]) continue;                   // set in an earlier update, behind a barrier
+            // Every CTA holding an item of the partition adds up the partition's slots itself, same
+            // grouping, same order: identical totals everywhere, nobody waits for a reducer.
             const double* slots = k.rslots + ((size_t)(l & 1) * Pc + p) * cppc * per;
             int groups = blockDim.x / per;
             if (groups < 1) groups = 1;
@@ -604,10 +628,8 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
             }
             if (tid == 0) sh_flag = 0;
             __syncthreads();
-            const bool eps_mode = (a.stop_mode == BTARD_STOP_EPS);
             const bool converged = eps_mode && l >= 1 && (sh_sum[n] <= a.eps2);
             if (converged || l == a.max_iters) {
-                finished = true;
                 if (j == 0) {
                     for (int i = tid; i < n; i += blockDim.x) a.resid_norm[(size_t)p * n + i] = sqrt(sh_sum[i]);
                     if (tid == 0) {
@@ -618,8 +640,9 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
                             if (!isfinite(sh_sum[i])) st |= BTARD_STATUS_NONFINITE_ROW;
                         if (eps_mode && !(sh_sum[n] <= a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
                         atomicOr(&a.status[p], st);
+                        a.done[p] = 1;                 // read by the other CTAs after the next barrier
                     }
-                    add_finished = 1;
+                    add_finished += 1;
                 }
             } else {
                 for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) {
@@ -629,14 +652,19 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
                 }
                 __syncthreads();
                 if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
-                sweep(std::false_type{}, (l + 1) & 1);
+                sweep(std::false_type{}, (l + 1) & 1, backwards);
             }
+            __syncthreads();                           // shared memory is reused by the next item
         }
         if (grid_barrier(k, generation, add_finished, &sh_bar)) break;
     }
-    if (active && j == 0 && tid == 0 && atomicAdd(k.error, 0u) != 0u)
-        atomicOr(&a.status[p], BTARD_STATUS_WAIT_EXPIRED);
+    if (tid == 0 && atomicAdd(k.error, 0u) != 0u)
+        for (int m = 0; m < mine; ++m) {
+            take_item(first + m * hop);
+            if (j == 0) atomicOr(&a.status[p], BTARD_STATUS_WAIT_EXPIRED);
+        }
 }
+
 
 // After the last pass: partitions still running take iters = max_iters.
 __global__ void cclip_finalize_kernel(const KernelArgs k)
@@ -914,20 +942,27 @@ int resident_chunk_partitions(int n, long long stride)
     return (int)(0.75 * (double)l2 / part_bytes);
 }
 
-int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, double* rslots,
-                          unsigned long long* barrier, unsigned int* error, cudaStream_t st)
+int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, int items_per_partition,
+                          int streaming, double* rslots, unsigned long long* barrier,
+                          unsigned int* error, cudaStream_t st)
 {
-    ResidentArgs ra{a, geo.RG, geo.CL, 0, rslots, barrier, error};
+    ResidentArgs ra{a, geo.RG, geo.CL, 0, streaming, rslots, barrier, error};
     const bool comp = a.v_lo != nullptr;
     const size_t smem = (geo.RG > 1) ? sizeof(float4) * 2 * geo.RG * geo.CL : 0;
     const int occ = resident_ctas_per_sm(geo.R, comp, geo.threads, smem);
     if (occ < 1) return BTARD_ERR_UNSUPPORTED;
     int grid = sm_count() * occ;
     if (grid > kResidentMaxGrid) grid = kResidentMaxGrid;
-    if (grid < a.P) return BTARD_ERR_UNSUPPORTED;
-    ra.cppc = grid / a.P;
-    const long long most = ((a.stride >> 2) + 7) / 8;          // at least one 128-byte line per CTA
-    if (ra.cppc > most) ra.cppc = (int)(most < 1 ? 1 : most);
+    long long cppc = items_per_partition;
+    if (cppc < 1) {                                    // one item per resident CTA
+        if (grid < a.P) return BTARD_ERR_UNSUPPORTED;
+        cppc = grid / a.P;
+    }
+    const long long most = ((a.stride >> 2) + 7) / 8;          // at least one 128-byte line per item
+    if (cppc > most) cppc = most < 1 ? 1 : most;
+    if ((long long)a.P * cppc > kResidentMaxItems) return BTARD_ERR_UNSUPPORTED;
+    ra.cppc = (int)cppc;
+    if ((long long)grid > (long long)a.P * cppc) grid = (int)((long long)a.P * cppc);
     void* args[] = {(void*)&ra};
     const void* fn;
     if (geo.R == 4) fn = comp ? (const void*)cclip_resident_kernel<4, true> : (const void*)cclip_resident_kernel<4, false>;
@@ -939,6 +974,18 @@ int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, double* rsl
     if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); return BTARD_ERR_CUDA; }
     count_launch();
     return BTARD_OK;
+}
+
+// 1 when this device can launch cooperative kernels.
+int cooperative_launch_supported()
+{
+    int dev = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return coop;
 }
 
 int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,

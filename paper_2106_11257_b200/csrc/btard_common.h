@@ -83,9 +83,14 @@ int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_
 // L2-resident variant: how many partitions fit one chunk (0: not available on this device), and the
 // cooperative launch that runs the start pass and every update of one chunk.
 constexpr int kResidentMaxGrid = 148 * 8;
+constexpr long long kResidentMaxItems = 1LL << 20;
 int resident_chunk_partitions(int n, long long stride);
-int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, double* rslots,
-                          unsigned long long* barrier, unsigned int* error, cudaStream_t st);
+int cooperative_launch_supported();
+// items_per_partition < 1: one work item per resident CTA.  streaming != 0: the chunk does not fit
+// L2 (evict-first loads, alternating sweep direction).
+int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, int items_per_partition,
+                          int streaming, double* rslots, unsigned long long* barrier,
+                          unsigned int* error, cudaStream_t st);
 int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
                        int P, cudaStream_t st);
 // squared-norm totals -> norms, used when verification is asked to compute the norms itself.

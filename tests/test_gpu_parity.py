@@ -85,10 +85,11 @@ def make_case(rng, P, n, stride, lens, far_rows=0, scale=0.02):
     return g
 
 
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
 @pytest.mark.parametrize("n", [1, 3, 4, 7, 8, 16, 23, 64, 100, 256])
 @pytest.mark.parametrize("init", [btard.INIT_ZERO, btard.INIT_MEAN, btard.INIT_COORD_MEDIAN,
                                   btard.INIT_CALLER_V0])
-def test_fixed_iterations_match_oracle(n, init):
+def test_fixed_iterations_match_oracle(n, init, algo):
     rng = np.random.default_rng(100 + n)
     P, stride = 3, 5024
     lens = np.array([5024, 4097, 0 if n % 2 else 13])
@@ -98,8 +99,9 @@ def test_fixed_iterations_match_oracle(n, init):
     if init == btard.INIT_CALLER_V0:
         v0 = rng.standard_normal((P, stride)).astype(np.float32)
     ref = oracle.centered_clip(g, tau, lens, init_mode=init, v0=v0, max_iters=6)
-    _, r = run_gpu_cclip(g, tau, lens, init_mode=init, v0=v0, max_iters=6)
+    _, r = run_gpu_cclip(g, tau, lens, init_mode=init, v0=v0, max_iters=6, algo=algo)
     check_cclip(r, ref, lens)
+    assert not (cpu(r["status"]) & 4).any()
 
 
 def test_many_tiles_per_cta_and_many_ctas():
@@ -127,7 +129,8 @@ def test_config1_fixed_and_eps():
     assert cpu(r["status"])[0] == ref["status"][0] == 0
 
 
-def test_eps_mode_counts_and_cap_flag():
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
+def test_eps_mode_counts_and_cap_flag(algo):
     rng = np.random.default_rng(6)
     P, n, stride = 4, 8, 2048
     lens = np.array([2048, 2000, 1, 1027])
@@ -136,7 +139,7 @@ def test_eps_mode_counts_and_cap_flag():
         ref = oracle.centered_clip(g, 0.7, lens, init_mode=oracle.INIT_MEAN, stop_mode=oracle.STOP_EPS,
                                    max_iters=cap, eps=eps)
         _, r = run_gpu_cclip(g, 0.7, lens, init_mode=btard.INIT_MEAN, stop_mode=btard.STOP_EPS,
-                             max_iters=cap, eps=eps)
+                             max_iters=cap, eps=eps, algo=algo)
         check_cclip(r, ref, lens, eps_mode=True)
         same = cpu(r["iters"]) == ref["iters"]
         assert np.array_equal(cpu(r["status"])[same] & 1, ref["status"][same] & 1)
