@@ -99,7 +99,7 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, in
     w.slots = off; off = align_up(off + sizeof(double) * (size_t)P * geo.cpp * (n + 1), 256);
     w.tot[0] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
     w.tot[1] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
-    w.flags_bytes = sizeof(int) * 3 * (size_t)P;              // done[P], ticket[P], Gram ticket[P]
+    w.flags_bytes = sizeof(int) * (3 * (size_t)P + 1);        // done[P], ticket[P], Gram ticket[P], error
     w.flags = off; off = align_up(off + w.flags_bytes, 256);
     const bool gram = (algo == BTARD_ALGO_GRAM);
     w.v_lo_bytes = (stop_mode == BTARD_STOP_EPS && !gram) ? sizeof(unsigned short) * (size_t)P * stride : 0;
@@ -284,6 +284,7 @@ int btard_centered_clip(const btard_cclip_args* a)
         G.g = a->g; G.v0 = a->v; G.table = L.table;
         G.slots = (double*)(base + ws.gslots); G.gram = (double*)(base + ws.gram);
         G.ticket = (unsigned int*)(base + ws.flags) + 2 * P;
+        G.error = (unsigned int*)(base + ws.flags) + 3 * P;
         G.coef = (double*)(base + ws.coef);
         G.iters = a->iters; G.last_step = a->last_step_norm; G.status = a->status;
         G.stride = a->row_stride; G.n = n; G.P = P;
@@ -295,7 +296,7 @@ int btard_centered_clip(const btard_cclip_args* a)
         L.coef = G.coef;
         rc = launch_cclip_pass(L, geo, PASS_COMBINE, st);
         if (rc != BTARD_OK) return rc;
-        return launch_gram_finalize(L.tot_out, a->resid_norm, a->status, n, P, st);
+        return launch_gram_finalize(L.tot_out, a->resid_norm, a->status, n, P, G.error, st);
     }
     if (whole) {
         BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.rflags, 0, ws.rflags_bytes, st));

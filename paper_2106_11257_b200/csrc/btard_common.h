@@ -114,6 +114,7 @@ struct GramLaunch {
     double* slots;              // device [P][cpp][entries]
     double* gram;               // device [P][entries] summed blocks
     unsigned int* ticket;       // device [P]
+    unsigned int* error;        // device: set when a bounded wait in the Gram kernel expired
     double* coef;               // device [P][n] out of the coefficient iteration
     int32_t* iters;
     double* last_step;
@@ -128,7 +129,7 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st);
 int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st);
 // resid_norm from the totals of the combine pass
 int launch_gram_finalize(const double* tot, double* resid_norm, uint32_t* status, int n, int P,
-                         cudaStream_t st);
+                         const unsigned int* error, cudaStream_t st);
 
 // ---- verification (btard_verify.cu) -------------------------------------------------------------
 struct VerifyLaunch {

@@ -313,6 +313,233 @@ __global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
     if (tid == 0) a.ticket[p] = 0;
 }
 
+// ---- 17 <= n <= 64: the Gram block on the 5th-generation tensor cores (tcgen05 + TMEM) ----------
+// Per 32-column tile the CTA's threads form R = g - v0, split every value into TF32 hi + lo and write
+// both as K-major operand tiles (128-byte rows, 128-byte swizzle) into shared memory; one thread then
+// issues, per 8-column k-block, three tcgen05.mma (hi.hi, hi.lo, lo.hi) with M = 128 (rows n..127 are
+// zero), N = 64, accumulating G in 64 columns of tensor memory.  A and B descriptors point at the
+// same tiles: B = R.  Two stages alternate, an mbarrier per stage (armed by tcgen05.commit) tells when
+// the tensor core has finished reading it.  Because tensor-core accumulation truncates, the
+// accumulator is read back (tcgen05.ld) and restarted every 4 tiles; the read-back values are summed
+// on the fp32 pipe and turned into fp64 at the end.  Every wait is bounded; if one expires the CTA
+// raises the error flag, still frees its tensor memory and leaves.
+constexpr int kUmmaThreads = 128;
+constexpr int kUmmaTileCols = 32;                       // one 128-byte swizzle row of TF32
+constexpr int kUmmaTileBytes = 128 * 128;               // 128 rows x 128 bytes
+constexpr int kUmmaFlushTiles = 4;
+constexpr int kUmmaSpinLimit = 1 << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
+{
+    // K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; descriptor version 1 (sm_100)
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int spin = 0; spin < kUmmaSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, unsigned int* error)
+{
+    extern __shared__ __align__(1024) unsigned char sh_raw[];
+    __shared__ __align__(8) unsigned long long sh_mbar[2];
+    __shared__ uint32_t sh_tmem;
+    __shared__ int sh_last;
+    const GramLaunch& a = k.a;
+    const int n = a.n, cpp = k.g.cpp, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const long long stride = a.stride, len = a.table[p].len;
+    const float* gp = a.g + (size_t)p * n * stride;
+    const float* vp = a.v0 + (size_t)p * stride;
+    long long c0 = stride * j / cpp, c1 = stride * (j + 1) / cpp;
+    if (j > 0) c0 &= ~31LL;
+    if (j + 1 < cpp) c1 &= ~31LL;
+    const int ntiles = (int)((c1 - c0 + kUmmaTileCols - 1) / kUmmaTileCols);
+
+    // operand tiles: [stage][hi, lo][128 rows][128 bytes], 1024-byte aligned
+    unsigned char* tiles = (unsigned char*)(((uintptr_t)sh_raw + 1023) & ~(uintptr_t)1023);
+    for (int e = tid; e < 4 * kUmmaTileBytes / 16; e += kUmmaThreads)
+        reinterpret_cast<uint4*>(tiles)[e] = make_uint4(0u, 0u, 0u, 0u);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_mbar[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_mbar[1])));
+    }
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh_tmem)), "r"(64));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = sh_tmem;
+
+    // tf32 inputs, fp32 accumulate, K-major A and B, N = 64, M = 128
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+    const uint32_t tile_base = smem_u32(tiles);
+
+    float sum[64];
+#pragma unroll
+    for (int q = 0; q < 64; ++q) sum[q] = 0.0f;
+    int commits[2] = {0, 0};
+    bool failed = false;
+    int since_flush = 0;
+
+    // this thread's four 16-byte chunks of a tile: rows row0 + 16 i, chunk ch (4 columns)
+    const int row0 = tid >> 3, ch = tid & 7;
+    float4 x[4], v4;
+    auto fetch = [&](int t) {
+        const long long col = c0 + (long long)t * kUmmaTileCols + 4 * ch;
+        const bool in = col < c1;
+        v4 = in ? *reinterpret_cast<const float4*>(vp + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = row0 + 16 * i;
+            x[i] = (in && r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+
+    if (ntiles > 0) fetch(0);
+    for (int t = 0; t < ntiles && !failed; ++t) {
+        const int s = t & 1;
+        // the tensor core must be done with what it read from this stage two tiles ago
+        bool ok = true;
+        if (commits[s] > 0) ok = mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1));
+        if (__syncthreads_or(!ok)) { failed = true; break; }
+
+        const long long col = c0 + (long long)t * kUmmaTileCols + 4 * ch;
+        const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
+        const bool m2 = col + 2 < len && col < c1, m3 = col + 3 < len && col < c1;
+        unsigned char* hi_tile = tiles + (size_t)(2 * s) * kUmmaTileBytes;
+        unsigned char* lo_tile = hi_tile + kUmmaTileBytes;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = row0 + 16 * i;
+            if (r < n) {
+                const float r0 = m0 ? x[i].x - v4.x : 0.f, r1 = m1 ? x[i].y - v4.y : 0.f;
+                const float r2 = m2 ? x[i].z - v4.z : 0.f, r3 = m3 ? x[i].w - v4.w : 0.f;
+                const uint32_t h0 = to_tf32(r0), h1 = to_tf32(r1), h2 = to_tf32(r2), h3 = to_tf32(r3);
+                const uint32_t l0 = to_tf32(r0 - __uint_as_float(h0)), l1 = to_tf32(r1 - __uint_as_float(h1));
+                const uint32_t l2 = to_tf32(r2 - __uint_as_float(h2)), l3 = to_tf32(r3 - __uint_as_float(h3));
+                const int off = (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4);
+                *reinterpret_cast<uint4*>(hi_tile + off) = make_uint4(h0, h1, h2, h3);
+                *reinterpret_cast<uint4*>(lo_tile + off) = make_uint4(l0, l1, l2, l3);
+            }
+        }
+        if (t + 1 < ntiles) fetch(t + 1);              // next tile's loads fly during the MMAs
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t hi_addr = tile_base + (uint32_t)(2 * s) * kUmmaTileBytes;
+            const uint32_t lo_addr = hi_addr + kUmmaTileBytes;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {           // 8 TF32 = 32 bytes per k-block
+                const uint64_t dh = umma_desc(hi_addr + 32u * ks), dl = umma_desc(lo_addr + 32u * ks);
+                const uint32_t acc0 = (since_flush > 0 || ks > 0) ? 1u : 0u;
+                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+                             ::"r"(tmem), "l"(dh), "l"(dh), "r"(idesc), "r"(acc0) : "memory");
+                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+                             ::"r"(tmem), "l"(dh), "l"(dl), "r"(idesc), "r"(1u) : "memory");
+                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+                             ::"r"(tmem), "l"(dl), "l"(dh), "r"(idesc), "r"(1u) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                         ::"r"(smem_u32(&sh_mbar[s])) : "memory");
+        }
+        commits[s] += 1;
+        since_flush += 1;
+
+        if (since_flush == kUmmaFlushTiles || t + 1 == ntiles) {
+            // read the accumulator back: wait for the commit just issued (covers all earlier MMAs)
+            ok = mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1));
+            if (__syncthreads_or(!ok)) { failed = true; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (warp < 2) {                            // lanes 0..63 of tensor memory = rows of G
+                uint32_t d[64];
+                const uint32_t taddr = tmem + ((uint32_t)(32 * warp) << 16);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                    : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
+                      "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15]),
+                      "=r"(d[16]), "=r"(d[17]), "=r"(d[18]), "=r"(d[19]), "=r"(d[20]), "=r"(d[21]), "=r"(d[22]), "=r"(d[23]),
+                      "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
+                    : "r"(taddr));
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                    : "=r"(d[32]), "=r"(d[33]), "=r"(d[34]), "=r"(d[35]), "=r"(d[36]), "=r"(d[37]), "=r"(d[38]), "=r"(d[39]),
+                      "=r"(d[40]), "=r"(d[41]), "=r"(d[42]), "=r"(d[43]), "=r"(d[44]), "=r"(d[45]), "=r"(d[46]), "=r"(d[47]),
+                      "=r"(d[48]), "=r"(d[49]), "=r"(d[50]), "=r"(d[51]), "=r"(d[52]), "=r"(d[53]), "=r"(d[54]), "=r"(d[55]),
+                      "=r"(d[56]), "=r"(d[57]), "=r"(d[58]), "=r"(d[59]), "=r"(d[60]), "=r"(d[61]), "=r"(d[62]), "=r"(d[63])
+                    : "r"(taddr + 32u));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int q = 0; q < 64; ++q) sum[q] += __uint_as_float(d[q]);
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            since_flush = 0;
+        }
+    }
+    if (failed && tid == 0) atomicExch(error, 1u);
+
+    // leave tensor memory the way it was found
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64));
+    }
+
+    // row i = 32 warp + lane of G (warps 0, 1) -> fp64 matrix in shared memory -> this CTA's slot
+    double* sh_g = reinterpret_cast<double*>(tiles);     // [64][64], the operand tiles are dead now
+    __syncthreads();
+    if (warp < 2) {
+        const int i = 32 * warp + lane;
+#pragma unroll
+        for (int q = 0; q < 64; ++q) sh_g[i * 64 + q] = (double)sum[q];
+    }
+    __syncthreads();
+    const int entries = k.g.entries, NB = k.g.NB;
+    double* slots = a.slots + (size_t)p * cpp * entries;
+    double* dst = slots + (size_t)j * entries;
+    for (int idx = tid; idx < entries; idx += kUmmaThreads) {
+        const int b = idx >> 6, e = idx & 63;
+        int bi, bj;
+        block_coords(b, NB, bi, bj);
+        dst[idx] = sh_g[(8 * bi + (e >> 3)) * 64 + 8 * bj + (e & 7)];
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sh_last = (atomicAdd(&a.ticket[p], 1u) == (unsigned)(cpp - 1));
+    __syncthreads();
+    if (!sh_last) return;
+    __threadfence();
+    double* out = a.gram + (size_t)p * entries;
+    for (int idx = tid; idx < entries; idx += kUmmaThreads) {
+        double s = 0.0;
+#pragma unroll 8
+        for (int c = 0; c < cpp; ++c) s += __ldcg(slots + (size_t)c * entries + idx);
+        out[idx] = s;
+    }
+    if (tid == 0) a.ticket[p] = 0;
+}
+
 // Sum over the threads of the CTA (fixed order).
 __device__ double block_sum(double x, double* red)
 {
@@ -472,10 +699,12 @@ __global__ void __launch_bounds__(32) gram_iterate_warp_kernel(const GArgs k)
     }
 }
 
-__global__ void gram_finalize_kernel(const double* tot, double* resid_norm, uint32_t* status, int n)
+__global__ void gram_finalize_kernel(const double* tot, double* resid_norm, uint32_t* status, int n,
+                                     const unsigned int* error)
 {
     const int p = blockIdx.x;
     bool bad = false;
+    if (threadIdx.x == 0 && error && *error) atomicOr(&status[p], BTARD_STATUS_WAIT_EXPIRED);
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const double v = tot[(size_t)p * (n + 1) + i];
         resid_norm[(size_t)p * n + i] = sqrt(v);
@@ -526,6 +755,13 @@ GramGeometry gram_geometry(int n, int P, long long stride)
             nb = 2;
         }
         g.cpp = choose_ctas_per_partition(P, stride >> 2, 16 * (kGramThreads / 32), sm_count() * nb);
+    } else if (n <= 64) {   // tcgen05 kernel: 3 CTAs of 65 KB shared memory per SM
+        // fp32 read-back sums: at most 512 flushes of 128 columns per CTA before fp64
+        const long long cap_cols = 512LL * kUmmaFlushTiles * kUmmaTileCols;
+        long long cmin2 = (stride + cap_cols - 1) / cap_cols;
+        int c2 = choose_ctas_per_partition(P, stride >> 2, 8 * 32, sm_count() * 3);
+        if (c2 < cmin2) c2 = (int)cmin2;
+        g.cpp = c2;
     }
     return g;
 }
@@ -535,8 +771,12 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     GArgs ga{a, geo};
     if (geo.smem > 48 * 1024)
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
+    constexpr int umma_smem = 4 * kUmmaTileBytes + 1024;
+    if (a.n > 16 && a.n <= 64)
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, umma_smem));
     prof_begin(KIND_GRAM, st);
     if (a.n <= 16) gram_mma16_kernel<<<a.P * geo.cpp, kGramThreads, 0, st>>>(ga);
+    else if (a.n <= 64) gram_umma_kernel<<<a.P * geo.cpp, kUmmaThreads, umma_smem, st>>>(ga, a.error);
     else gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
     prof_end(KIND_GRAM, st);
     BTARD_CUDA_TRY(cudaGetLastError());
@@ -561,9 +801,9 @@ int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream
 }
 
 int launch_gram_finalize(const double* tot, double* resid_norm, uint32_t* status, int n, int P,
-                         cudaStream_t st)
+                         const unsigned int* error, cudaStream_t st)
 {
-    gram_finalize_kernel<<<P, 128, 0, st>>>(tot, resid_norm, status, n);
+    gram_finalize_kernel<<<P, 128, 0, st>>>(tot, resid_norm, status, n, error);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
     return BTARD_OK;
