@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     const VerifyLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL, nthr = blockDim.x;
+    const int cl_shift = 31 - __clz(CL);              // CL is a power of two
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
     const long long stride = a.stride, len = a.table[p].len;
     const double tau = a.table[p].tau;
@@ -97,14 +98,16 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
         // 1. this tile's block of z
         float4* zb = sh_z + (size_t)par * KT * CL;
         for (int idx = tid; idx < KT * CL; idx += nthr) {
-            const int kq = idx / CL, cq = idx % CL;
+            const int kq = idx >> cl_shift, cq = idx & (CL - 1);
             const long long col = (qb + cq) * 4;
             float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
             if (kq < a.kc && qb + cq < q1 && col < len) {
-                z = z_quad((uint32_t)(col >> 2), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
-                if (col + 1 >= len) z.y = 0.f;
-                if (col + 2 >= len) z.z = 0.f;
-                if (col + 3 >= len) z.w = 0.f;
+                z = z_quad((uint32_t)(qb + cq), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
+                if (col + 3 >= len) {                  // only the last quad of a ragged partition
+                    if (col + 1 >= len) z.y = 0.f;
+                    if (col + 2 >= len) z.z = 0.f;
+                    z.w = 0.f;
+                }
             }
             zb[kq * CL + cq] = z;
         }
@@ -130,12 +133,19 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
 #pragma unroll
             for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        if (m3) {                                      // whole quad inside the data: no predicates
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            x[r].x = m0 ? x[r].x - v4.x : 0.f;
-            x[r].y = m1 ? x[r].y - v4.y : 0.f;
-            x[r].z = m2 ? x[r].z - v4.z : 0.f;
-            x[r].w = m3 ? x[r].w - v4.w : 0.f;
+            for (int r = 0; r < R; ++r) {
+                x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = m0 ? x[r].x - v4.x : 0.f;
+                x[r].y = m1 ? x[r].y - v4.y : 0.f;
+                x[r].z = m2 ? x[r].z - v4.z : 0.f;
+                x[r].w = 0.f;
+            }
         }
         // 3. projections
 #pragma unroll
