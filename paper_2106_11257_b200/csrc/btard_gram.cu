@@ -316,8 +316,9 @@ __global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
 // ---- 17 <= n <= 64: the Gram block on the 5th-generation tensor cores (tcgen05 + TMEM) ----------
 // Per 32-column tile the CTA's threads form R = g - v0, split every value into TF32 hi + lo and write
 // both as K-major operand tiles (128-byte rows, 128-byte swizzle) into shared memory; one thread then
-// issues, per 8-column k-block, three tcgen05.mma (hi.hi, hi.lo, lo.hi) with M = 128 (rows n..127 are
-// zero), N = 64, accumulating G in 64 columns of tensor memory.  A and B descriptors point at the
+// issues, per 8-column k-block, three tcgen05.mma (hi.hi, hi.lo, lo.hi) with M = 64 (rows n..63 are
+// zero), N = 64, accumulating G in 64 columns of tensor memory (row m of G lives in lane
+// m % 16 + 32 (m / 16): sixteen rows in the lower half of each warp's quarter).  A and B descriptors point at the
 // same tiles: B = R.  Two stages alternate, an mbarrier per stage (armed by tcgen05.commit) tells when
 // the tensor core has finished reading it.  Because tensor-core accumulation truncates, the
 // accumulator is read back (tcgen05.ld) and restarted every 4 tiles; the read-back values are summed
@@ -325,7 +326,7 @@ __global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
 // raises the error flag, still frees its tensor memory and leaves.
 constexpr int kUmmaThreads = 128;
 constexpr int kUmmaTileCols = 32;                       // one 128-byte swizzle row of TF32
-constexpr int kUmmaTileBytes = 128 * 128;               // 128 rows x 128 bytes
+constexpr int kUmmaTileBytes = 64 * 128;                // 64 rows x 128 bytes
 constexpr int kUmmaFlushTiles = 4;
 constexpr int kUmmaSpinLimit = 1 << 22;
 
@@ -345,6 +346,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
+        __nanosleep(32);                               // do not burn issue slots while the tensor core works
     }
     return false;
 }
@@ -361,12 +363,15 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
     const long long stride = a.stride, len = a.table[p].len;
     const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v0 + (size_t)p * stride;
-    long long c0 = stride * j / cpp, c1 = stride * (j + 1) / cpp;
-    if (j > 0) c0 &= ~31LL;
-    if (j + 1 < cpp) c1 &= ~31LL;
-    const int ntiles = (int)((c1 - c0 + kUmmaTileCols - 1) / kUmmaTileCols);
+    // The CTAs of a partition take its 32-column tiles round-robin (tile j, j + cpp, ...): they are
+    // resident together, so at any moment they read neighbouring 128-byte pieces of the same rows and
+    // an open DRAM page is used whole instead of 128 bytes at a time.
+    const long long c1 = stride;
+    const long long all_tiles = (stride + kUmmaTileCols - 1) / kUmmaTileCols;
+    const int ntiles = (int)((all_tiles - j + cpp - 1) / cpp);      // tiles j + m cpp < all_tiles
+    auto tile_col = [&](int t) { return ((long long)j + (long long)t * cpp) * kUmmaTileCols; };
 
-    // operand tiles: [stage][hi, lo][128 rows][128 bytes], 1024-byte aligned
+    // operand tiles: [stage][hi, lo][64 rows][128 bytes], 1024-byte aligned
     unsigned char* tiles = (unsigned char*)(((uintptr_t)sh_raw + 1023) & ~(uintptr_t)1023);
     for (int e = tid; e < 4 * kUmmaTileBytes / 16; e += kUmmaThreads)
         reinterpret_cast<uint4*>(tiles)[e] = make_uint4(0u, 0u, 0u, 0u);
@@ -385,8 +390,8 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = sh_tmem;
 
-    // tf32 inputs, fp32 accumulate, K-major A and B, N = 64, M = 128
-    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+    // tf32 inputs, fp32 accumulate, K-major A and B, N = 64, M = 64
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((64u >> 3) << 17) | ((64u >> 4) << 24);
     const uint32_t tile_base = smem_u32(tiles);
 
     float sum[64];
@@ -395,13 +400,16 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
     int commits[2] = {0, 0};
     bool failed = false;
     int since_flush = 0;
+    __shared__ int sh_fail;
+    if (tid == 0) sh_fail = 0;
 
-    // this thread's four 16-byte chunks of a tile: rows row0 + 16 i, chunk ch (4 columns)
+    // this thread's four 16-byte chunks of a tile: rows row0 + 16 i, chunk ch (4 columns);
+    // the rows of the next two tiles are kept in flight in registers
     const int row0 = tid >> 3, ch = tid & 7;
-    float4 x[4], v4;
-    auto fetch = [&](int t) {
-        const long long col = c0 + (long long)t * kUmmaTileCols + 4 * ch;
-        const bool in = col < c1;
+    float4 xa[4], xb[4], va, vb;
+    auto fetch = [&](int t, float4 (&x)[4], float4& v4) {
+        const long long col = tile_col(t) + 4 * ch;
+        const bool in = t < ntiles && col < c1;
         v4 = in ? *reinterpret_cast<const float4*>(vp + col) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -410,16 +418,31 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     };
+    // 32 accumulator columns starting at column `first` of this warp's 32 lanes, added to sum
+    auto read_back = [&](uint32_t taddr, float* dst) {
+        uint32_t d[32];
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+            "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
+              "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15]),
+              "=r"(d[16]), "=r"(d[17]), "=r"(d[18]), "=r"(d[19]), "=r"(d[20]), "=r"(d[21]), "=r"(d[22]), "=r"(d[23]),
+              "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
+            : "r"(taddr));
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int q = 0; q < 32; ++q) dst[q] += __uint_as_float(d[q]);
+    };
 
-    if (ntiles > 0) fetch(0);
-    for (int t = 0; t < ntiles && !failed; ++t) {
+    fetch(0, xa, va);
+    fetch(1, xb, vb);
+    __syncthreads();
+    for (int t = 0; t < ntiles; ++t) {
         const int s = t & 1;
         // the tensor core must be done with what it read from this stage two tiles ago
-        bool ok = true;
-        if (commits[s] > 0) ok = mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1));
-        if (__syncthreads_or(!ok)) { failed = true; break; }
+        if (commits[s] > 0 && !mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1))) sh_fail = 1;
 
-        const long long col = c0 + (long long)t * kUmmaTileCols + 4 * ch;
+        const long long col = tile_col(t) + 4 * ch;
         const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
         const bool m2 = col + 2 < len && col < c1, m3 = col + 3 < len && col < c1;
         unsigned char* hi_tile = tiles + (size_t)(2 * s) * kUmmaTileBytes;
@@ -428,8 +451,8 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
         for (int i = 0; i < 4; ++i) {
             const int r = row0 + 16 * i;
             if (r < n) {
-                const float r0 = m0 ? x[i].x - v4.x : 0.f, r1 = m1 ? x[i].y - v4.y : 0.f;
-                const float r2 = m2 ? x[i].z - v4.z : 0.f, r3 = m3 ? x[i].w - v4.w : 0.f;
+                const float r0 = m0 ? xa[i].x - va.x : 0.f, r1 = m1 ? xa[i].y - va.y : 0.f;
+                const float r2 = m2 ? xa[i].z - va.z : 0.f, r3 = m3 ? xa[i].w - va.w : 0.f;
                 const uint32_t h0 = to_tf32(r0), h1 = to_tf32(r1), h2 = to_tf32(r2), h3 = to_tf32(r3);
                 const uint32_t l0 = to_tf32(r0 - __uint_as_float(h0)), l1 = to_tf32(r1 - __uint_as_float(h1));
                 const uint32_t l2 = to_tf32(r2 - __uint_as_float(h2)), l3 = to_tf32(r3 - __uint_as_float(h3));
@@ -438,10 +461,15 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
                 *reinterpret_cast<uint4*>(lo_tile + off) = make_uint4(l0, l1, l2, l3);
             }
         }
-        if (t + 1 < ntiles) fetch(t + 1);              // next tile's loads fly during the MMAs
+        // rotate the register queue and put tile t + 2 in flight
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xa[i] = xb[i];
+        va = vb;
+        fetch(t + 2, xb, vb);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
+        if (sh_fail) { failed = true; break; }         // a bounded wait ran out somewhere in the CTA
         if (tid == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t hi_addr = tile_base + (uint32_t)(2 * s) * kUmmaTileBytes;
@@ -465,31 +493,14 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
 
         if (since_flush == kUmmaFlushTiles || t + 1 == ntiles) {
             // read the accumulator back: wait for the commit just issued (covers all earlier MMAs)
-            ok = mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1));
-            if (__syncthreads_or(!ok)) { failed = true; break; }
+            if (!mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1))) sh_fail = 1;
+            __syncthreads();
+            if (sh_fail) { failed = true; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (warp < 2) {                            // lanes 0..63 of tensor memory = rows of G
-                uint32_t d[64];
+            {                                          // lanes 0..15 of every warp: rows 16 warp + lane
                 const uint32_t taddr = tmem + ((uint32_t)(32 * warp) << 16);
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                    : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
-                      "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15]),
-                      "=r"(d[16]), "=r"(d[17]), "=r"(d[18]), "=r"(d[19]), "=r"(d[20]), "=r"(d[21]), "=r"(d[22]), "=r"(d[23]),
-                      "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
-                    : "r"(taddr));
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                    : "=r"(d[32]), "=r"(d[33]), "=r"(d[34]), "=r"(d[35]), "=r"(d[36]), "=r"(d[37]), "=r"(d[38]), "=r"(d[39]),
-                      "=r"(d[40]), "=r"(d[41]), "=r"(d[42]), "=r"(d[43]), "=r"(d[44]), "=r"(d[45]), "=r"(d[46]), "=r"(d[47]),
-                      "=r"(d[48]), "=r"(d[49]), "=r"(d[50]), "=r"(d[51]), "=r"(d[52]), "=r"(d[53]), "=r"(d[54]), "=r"(d[55]),
-                      "=r"(d[56]), "=r"(d[57]), "=r"(d[58]), "=r"(d[59]), "=r"(d[60]), "=r"(d[61]), "=r"(d[62]), "=r"(d[63])
-                    : "r"(taddr + 32u));
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int q = 0; q < 64; ++q) sum[q] += __uint_as_float(d[q]);
+                read_back(taddr, sum);
+                read_back(taddr + 32u, sum + 32);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncthreads();
@@ -506,11 +517,11 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64));
     }
 
-    // row i = 32 warp + lane of G (warps 0, 1) -> fp64 matrix in shared memory -> this CTA's slot
+    // row i = 16 warp + lane of G (lanes 0..15) -> fp64 matrix in shared memory -> this CTA's slot
     double* sh_g = reinterpret_cast<double*>(tiles);     // [64][64], the operand tiles are dead now
     __syncthreads();
-    if (warp < 2) {
-        const int i = 32 * warp + lane;
+    if (lane < 16) {
+        const int i = 16 * warp + lane;
 #pragma unroll
         for (int q = 0; q < 64; ++q) sh_g[i * 64 + q] = (double)sum[q];
     }
@@ -755,7 +766,7 @@ GramGeometry gram_geometry(int n, int P, long long stride)
             nb = 2;
         }
         g.cpp = choose_ctas_per_partition(P, stride >> 2, 16 * (kGramThreads / 32), sm_count() * nb);
-    } else if (n <= 64) {   // tcgen05 kernel: 3 CTAs of 65 KB shared memory per SM
+    } else if (n <= 64) {   // tcgen05 kernel: 3 CTAs per SM (160 registers x 128 threads each)
         // fp32 read-back sums: at most 512 flushes of 128 columns per CTA before fp64
         const long long cap_cols = 512LL * kUmmaFlushTiles * kUmmaTileCols;
         long long cmin2 = (stride + cap_cols - 1) / cap_cols;
