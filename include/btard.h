@@ -151,6 +151,40 @@ BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* arg
 BTARD_API int btard_verify_projections(const btard_verify_args* args);
 
 /*
+ * The predicates of Verifications 1-3 (Alg. 6 lines 17-38) on the scalars peers broadcast.  For
+ * partition p (aggregated by peer p) and peer i:
+ *   Verification 1: norm_mismatch[p][i] = reported norm_ip differs from ||g_i(p) - v(p)||;
+ *   Verification 2: s_mismatch[p][i][k] = reported s_i^p differs from <z_k[p], Delta_i^p>;
+ *                   sum_violation[p][k] = sum_i (reported s_i^p) != 0   ("v(p) is wrong");
+ *   Verification 3: check[p][i] = ||g_i(p) - v(p)|| > Delta_max[p];  votes[p] = sum_i check[p][i];
+ *                   check_averaging[p] = votes[p] > n/2  (then CheckAveraging(p) is due).
+ * The paper compares exactly; here "differs" means |a - b| > rel_tol max(|a|, |b|) + abs_tol (NaN always
+ * differs) and the sum test is |sum_i s| > sum_tol sum_i |s|, so that all-zero tolerances give the
+ * paper's tests.  The library only evaluates the predicates; accusing and banning are the caller's.
+ * `norm` and `s` are what btard_verify_projections computed; `norm_reported` / `s_reported` are what
+ * the peers sent (either may be NULL: that test is skipped and, for the sum, the computed s is used).
+ * All arrays are device memory; outputs are one byte per flag.  One small kernel on `stream`;
+ * no workspace.
+ */
+typedef struct {
+    int32_t n_peers, n_partitions, n_z;
+    const double* norm;           /* device [P][n]    computed */
+    const double* norm_reported;  /* device [P][n]    or NULL  */
+    const double* s;              /* device [P][n][K] computed */
+    const double* s_reported;     /* device [P][n][K] or NULL  */
+    const double* delta_max;      /* device [P] (+inf or NaN: Verification 3 never fires) */
+    double rel_tol, abs_tol, sum_tol;
+    uint8_t* norm_mismatch;       /* device [P][n]    out */
+    uint8_t* s_mismatch;          /* device [P][n][K] out */
+    uint8_t* sum_violation;       /* device [P][K]    out */
+    uint8_t* check;               /* device [P][n]    out */
+    int32_t* votes;               /* device [P]       out */
+    uint8_t* check_averaging;     /* device [P]       out */
+    void* stream;
+} btard_checks_args;
+BTARD_API int btard_verification_checks(const btard_checks_args* args);
+
+/*
  * btard_verify_projections without caller-supplied scratch.  The paper has no counterpart: this is
  * a packaging variant of the call above, same arguments, same kernels, same outputs.
  *

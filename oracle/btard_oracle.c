@@ -397,6 +397,46 @@ int btard_oracle_verify(const float *g, int32_t n, int32_t P, int64_t stride,
     return rc_all;
 }
 
+/* ------------------------------------------------------------------------- */
+/* Verifications 1-3 on the broadcast scalars (Alg. 6 lines 17-38), for one     */
+/* partition.  "differs" is |a - b| > rel_tol max(|a|,|b|) + abs_tol (NaN        */
+/* differs); all-zero tolerances give the paper's exact tests.                   */
+/* ------------------------------------------------------------------------- */
+static int oracle_differs(double x, double y, double rel_tol, double abs_tol)
+{
+    double scale = fabs(x) > fabs(y) ? fabs(x) : fabs(y);
+    return !(fabs(x - y) <= rel_tol * scale + abs_tol);
+}
+
+void btard_oracle_checks_one(int32_t n, int32_t K, const double *norm, const double *norm_reported,
+                             const double *s, const double *s_reported, double delta_max,
+                             double rel_tol, double abs_tol, double sum_tol,
+                             uint8_t *norm_mismatch, uint8_t *s_mismatch, uint8_t *sum_violation,
+                             uint8_t *check, int32_t *votes, uint8_t *check_averaging)
+{
+    int32_t v = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        /* Verification 1: reported norm against the recomputed one */
+        norm_mismatch[i] = norm_reported ? (uint8_t)oracle_differs(norm_reported[i], norm[i], rel_tol, abs_tol) : 0;
+        /* Verification 3: is the aggregate farther than Delta_max from this peer's part? */
+        check[i] = (uint8_t)(norm[i] > delta_max);
+        v += check[i];
+        /* Verification 2, first test: reported inner products against the recomputed ones */
+        for (int32_t k = 0; k < K; ++k)
+            s_mismatch[i * K + k] =
+                s_reported ? (uint8_t)oracle_differs(s_reported[i * K + k], s[i * K + k], rel_tol, abs_tol) : 0;
+    }
+    /* Verification 2, second test: the broadcast inner products must sum to zero */
+    for (int32_t k = 0; k < K; ++k) {
+        const double *sv = s_reported ? s_reported : s;
+        double sum = 0.0, mag = 0.0;
+        for (int32_t i = 0; i < n; ++i) { sum += sv[i * K + k]; mag += fabs(sv[i * K + k]); }
+        sum_violation[k] = (uint8_t)(!(fabs(sum) <= sum_tol * mag));
+    }
+    *votes = v;
+    *check_averaging = (uint8_t)(2 * v > n);      /* more than n/2 peers voted */
+}
+
 int btard_oracle_max_threads(void)
 {
 #ifdef _OPENMP

@@ -169,3 +169,31 @@ def verify(g, v, tau, seed, K=1, part_len=None, norm_in=None, want_resid_sum=Fal
     if rs is not None:
         out["resid_sum"] = rs
     return out
+
+
+def checks(norm, s, delta_max, norm_reported=None, s_reported=None, rel_tol=0.0, abs_tol=0.0, sum_tol=0.0):
+    """Predicates of Verifications 1-3.  norm [P][n], s [P][n][K], delta_max [P] (float64)."""
+    norm = np.ascontiguousarray(norm, dtype=np.float64)
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    P, n, K = s.shape
+    dm = _per_part(delta_max, P, np.float64)
+    nr = None if norm_reported is None else np.ascontiguousarray(norm_reported, dtype=np.float64)
+    sr = None if s_reported is None else np.ascontiguousarray(s_reported, dtype=np.float64)
+    out = dict(norm_mismatch=np.zeros((P, n), np.uint8), s_mismatch=np.zeros((P, n, K), np.uint8),
+               sum_violation=np.zeros((P, K), np.uint8), check=np.zeros((P, n), np.uint8),
+               votes=np.zeros(P, np.int32), check_averaging=np.zeros(P, np.uint8))
+    lib = _load()
+    for p in range(P):
+        votes = C.c_int32(0)
+        ca = C.c_uint8(0)
+        lib.btard_oracle_checks_one(
+            C.c_int32(n), C.c_int32(K), _p(norm[p], C.c_double),
+            _p(nr[p], C.c_double) if nr is not None else None, _p(s[p], C.c_double),
+            _p(sr[p], C.c_double) if sr is not None else None, C.c_double(float(dm[p])),
+            C.c_double(rel_tol), C.c_double(abs_tol), C.c_double(sum_tol),
+            _p(out["norm_mismatch"][p], C.c_uint8), _p(out["s_mismatch"][p], C.c_uint8),
+            _p(out["sum_violation"][p], C.c_uint8), _p(out["check"][p], C.c_uint8),
+            C.byref(votes), C.byref(ca))
+        out["votes"][p] = votes.value
+        out["check_averaging"][p] = ca.value
+    return out

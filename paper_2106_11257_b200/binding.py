@@ -20,7 +20,7 @@ EXPORTS = [
     "btard_verify_projections_workspace", "btard_verify_projections", "btard_random_vector",
     "btard_aggregate_host_scratch", "btard_aggregate_host", "btard_last_cuda_error",
     "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
-    "btard_verify_projections_static",
+    "btard_verify_projections_static", "btard_verification_checks",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -70,6 +70,15 @@ class HostArgs(C.Structure):
                 ("copy_stream", C.c_void_p)]
 
 
+class ChecksArgs(C.Structure):
+    _fields_ = [("n_peers", C.c_int32), ("n_partitions", C.c_int32), ("n_z", C.c_int32),
+                ("norm", C.c_void_p), ("norm_reported", C.c_void_p), ("s", C.c_void_p),
+                ("s_reported", C.c_void_p), ("delta_max", C.c_void_p), ("rel_tol", C.c_double),
+                ("abs_tol", C.c_double), ("sum_tol", C.c_double), ("norm_mismatch", C.c_void_p),
+                ("s_mismatch", C.c_void_p), ("sum_violation", C.c_void_p), ("check", C.c_void_p),
+                ("votes", C.c_void_p), ("check_averaging", C.c_void_p), ("stream", C.c_void_p)]
+
+
 _lib = None
 
 
@@ -99,6 +108,8 @@ def lib():
         L.btard_verify_projections.argtypes = [C.POINTER(VerifyArgs)]
         L.btard_verify_projections_static.restype = C.c_int
         L.btard_verify_projections_static.argtypes = [C.POINTER(VerifyArgs)]
+        L.btard_verification_checks.restype = C.c_int
+        L.btard_verification_checks.argtypes = [C.POINTER(ChecksArgs)]
         L.btard_random_vector.restype = C.c_int
         L.btard_random_vector.argtypes = [C.c_uint64, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
                                           C.c_void_p]
@@ -301,6 +312,33 @@ def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in
     if rs is not None:
         res["resid_sum"] = rs
     return res
+
+
+def verification_checks(norm, s, delta_max, norm_reported=None, s_reported=None, rel_tol=0.0,
+                        abs_tol=0.0, sum_tol=0.0, stream=None):
+    """Predicates of Verifications 1-3 on CUDA float64 tensors norm [P][n], s [P][n][K], delta_max [P].
+    Returns dict of CUDA tensors: norm_mismatch, check [P][n] uint8; s_mismatch [P][n][K] uint8;
+    sum_violation [P][K] uint8; votes [P] int32; check_averaging [P] uint8."""
+    torch = _torch()
+    P, n, K = s.shape
+    dev = s.device
+    for t in (norm, s, delta_max, norm_reported, s_reported):
+        assert t is None or (t.is_cuda and t.dtype == torch.float64 and t.is_contiguous())
+    u8 = dict(dtype=torch.uint8, device=dev)
+    o = dict(norm_mismatch=torch.empty((P, n), **u8), s_mismatch=torch.empty((P, n, K), **u8),
+             sum_violation=torch.empty((P, K), **u8), check=torch.empty((P, n), **u8),
+             votes=torch.empty(P, dtype=torch.int32, device=dev), check_averaging=torch.empty(P, **u8))
+    a = ChecksArgs(n_peers=n, n_partitions=P, n_z=K, norm=norm.data_ptr(),
+                   norm_reported=norm_reported.data_ptr() if norm_reported is not None else None,
+                   s=s.data_ptr(), s_reported=s_reported.data_ptr() if s_reported is not None else None,
+                   delta_max=delta_max.data_ptr(), rel_tol=rel_tol, abs_tol=abs_tol, sum_tol=sum_tol,
+                   norm_mismatch=o["norm_mismatch"].data_ptr(), s_mismatch=o["s_mismatch"].data_ptr(),
+                   sum_violation=o["sum_violation"].data_ptr(), check=o["check"].data_ptr(),
+                   votes=o["votes"].data_ptr(), check_averaging=o["check_averaging"].data_ptr(),
+                   stream=_stream_ptr(stream))
+    with torch.cuda.device(dev):
+        _check(lib().btard_verification_checks(C.byref(a)), "btard_verification_checks")
+    return o
 
 
 def random_vector(seed, p, k, part_len, device="cuda", stream=None):

@@ -425,6 +425,18 @@ int btard_verify_projections(const btard_verify_args* a)
     return BTARD_OK;
 }
 
+int btard_verification_checks(const btard_checks_args* a)
+{
+    if (!a || a->n_peers < 1 || a->n_partitions < 1 || a->n_partitions > 65535 || a->n_z < 1)
+        return BTARD_ERR_INVALID_ARG;
+    if (a->n_peers > BTARD_MAX_PEERS || a->n_z > BTARD_MAX_Z) return BTARD_ERR_UNSUPPORTED;
+    if (!a->norm || !a->s || !a->delta_max || !a->norm_mismatch || !a->s_mismatch || !a->sum_violation ||
+        !a->check || !a->votes || !a->check_averaging)
+        return BTARD_ERR_INVALID_ARG;
+    if (!(a->rel_tol >= 0.0) || !(a->abs_tol >= 0.0) || !(a->sum_tol >= 0.0)) return BTARD_ERR_INVALID_ARG;
+    return launch_checks(*a, (cudaStream_t)a->stream);
+}
+
 int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t part_len, float* z_out,
                         void* stream)
 {

@@ -155,6 +155,7 @@ struct VerifyGeometry {
 
 VerifyGeometry verify_geometry(int n, int P, long long stride, int K);
 int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t st);
+int launch_checks(const btard_checks_args& a, cudaStream_t st);
 int launch_random_vector(uint64_t seed, int p, int k, long long len, float* z, cudaStream_t st);
 
 }  // namespace btard

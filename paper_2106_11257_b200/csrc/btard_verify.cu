@@ -259,6 +259,48 @@ __global__ void verify_finalize_kernel(const VArgs k, int KT)
     if (a.k0 == 0 && threadIdx.x == 0) a.resid_sum_norm[p] = sqrt(sh_v[n * KT + KT]);
 }
 
+// Verifications 1-3 on broadcast scalars (Alg. 6 lines 17-38): one CTA per partition.
+__device__ __forceinline__ bool differs(double x, double y, double rel_tol, double abs_tol)
+{
+    const double scale = fmax(fabs(x), fabs(y));
+    return !(fabs(x - y) <= rel_tol * scale + abs_tol);      // NaN anywhere: differs
+}
+
+__global__ void checks_kernel(const btard_checks_args a)
+{
+    __shared__ int sh_votes;
+    const int p = blockIdx.x, n = a.n_peers, K = a.n_z;
+    if (threadIdx.x == 0) sh_votes = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const double nv = a.norm[(size_t)p * n + i];
+        a.norm_mismatch[(size_t)p * n + i] =
+            a.norm_reported ? (uint8_t)differs(a.norm_reported[(size_t)p * n + i], nv, a.rel_tol, a.abs_tol) : (uint8_t)0;
+        const bool far = nv > a.delta_max[p];
+        a.check[(size_t)p * n + i] = (uint8_t)far;
+        if (far) atomicAdd(&sh_votes, 1);
+    }
+    for (int e = threadIdx.x; e < n * K; e += blockDim.x) {
+        const size_t at = (size_t)p * n * K + e;
+        a.s_mismatch[at] = a.s_reported ? (uint8_t)differs(a.s_reported[at], a.s[at], a.rel_tol, a.abs_tol) : (uint8_t)0;
+    }
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        const double* sv = a.s_reported ? a.s_reported : a.s;
+        double sum = 0.0, mag = 0.0;
+        for (int i = 0; i < n; ++i) {
+            const double v = sv[((size_t)p * n + i) * K + k];
+            sum += v;
+            mag += fabs(v);
+        }
+        a.sum_violation[(size_t)p * K + k] = (uint8_t)(!(fabs(sum) <= a.sum_tol * mag));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        a.votes[p] = sh_votes;
+        a.check_averaging[p] = (uint8_t)(2 * sh_votes > n);
+    }
+}
+
 __global__ void random_vector_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t p, uint32_t kz,
                                      long long len, float* z)
 {
@@ -360,6 +402,14 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
     }
     if (rc != BTARD_OK) return rc;
     verify_finalize_kernel<<<a.P, 128, sizeof(double) * vg.slots, st>>>(va, vg.KT);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_checks(const btard_checks_args& a, cudaStream_t st)
+{
+    checks_kernel<<<a.n_partitions, 128, 0, st>>>(a);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
     return BTARD_OK;

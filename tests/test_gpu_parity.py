@@ -342,6 +342,48 @@ def test_wrong_aggregate_is_exposed_on_the_gpu_too():
     assert np.all(np.abs(sb) > 10 * np.abs(sg))
 
 
+def test_verification_checks_are_bit_exact():
+    """Integer/boolean outputs: same fp64 inputs, same fp64 comparisons, identical flags."""
+    rng = np.random.default_rng(15)
+    P, n, K = 7, 23, 3
+    norm = np.abs(rng.standard_normal((P, n))) * 2
+    s = rng.standard_normal((P, n, K))
+    s[:, -1, :] = -s[:, :-1, :].sum(axis=1)                       # sums to ~0 up to rounding
+    nr = norm.copy(); sr = s.copy()
+    nr[1, 3] *= 1 + 1e-9; nr[2, 0] = np.nan; sr[4, 5, 1] += 1e-7; sr[6, :, 0] += 0.01
+    dmax = np.array([0.5, 1.0, 1.5, 2.0, np.inf, 0.0, 1.3])
+    for tol in (dict(), dict(rel_tol=1e-8, abs_tol=1e-12, sum_tol=1e-9), dict(rel_tol=1e-3, sum_tol=1e-2)):
+        for rep in (dict(), dict(norm_reported=nr, s_reported=sr)):
+            ref = oracle.checks(norm, s, dmax, **rep, **tol)
+            dev = {k: torch.from_numpy(v).cuda() for k, v in rep.items()}
+            out = btard.verification_checks(torch.from_numpy(norm).cuda(), torch.from_numpy(s).cuda(),
+                                            torch.from_numpy(dmax).cuda(), **dev, **tol)
+            torch.cuda.synchronize()
+            for key in ref:
+                assert np.array_equal(cpu(out[key]), ref[key]), (key, tol, list(rep))
+
+
+def test_checks_on_library_outputs_catch_a_shifted_aggregate():
+    w = workloads.make_workload(1)
+    g = w.g.cuda()
+    r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
+                            stop_mode=btard.STOP_EPS, max_iters=500, eps=1e-7)
+    good = btard.verify_projections(g, r["v"], w.tau, 0, K=2, part_len=w.part_len, resid_norm_in=r["resid_norm"])
+    dmax = torch.tensor([5.0], dtype=torch.float64, device="cuda")
+    ok = btard.verification_checks(good["norm"], good["s"], dmax, sum_tol=1e-4)
+    bad = btard.verify_projections(g, r["v"] + 1.0, w.tau, 0, K=2, part_len=w.part_len)
+    flagged = btard.verification_checks(bad["norm"], bad["s"], dmax, sum_tol=1e-4)
+    torch.cuda.synchronize()
+    assert not cpu(ok["sum_violation"]).any() and cpu(ok["check_averaging"])[0] == 0
+    assert cpu(flagged["sum_violation"]).all() and cpu(flagged["check_averaging"])[0] == 1
+    # a peer that misreports its inner product is singled out
+    sr = good["s"].clone(); sr[0, 2, 1] += 0.5
+    acc = btard.verification_checks(good["norm"], good["s"], dmax, s_reported=sr, rel_tol=1e-9, sum_tol=1e-4)
+    torch.cuda.synchronize()
+    assert cpu(acc["s_mismatch"]).sum() == 1 and cpu(acc["s_mismatch"])[0, 2, 1] == 1
+    assert cpu(acc["sum_violation"])[0, 1] == 1
+
+
 # ----------------------------------------------------------------------------- host-buffer path
 def test_aggregate_host_matches_device_path():
     rng = np.random.default_rng(10)

@@ -431,3 +431,49 @@ def test_empty_partition_projects_to_zero():
     out = oracle.verify(g, v, 1.0, seed=1, K=2, part_len=np.array([0, 8]))
     assert np.all(out["s"][0] == 0) and np.all(out["s_sum"][0] == 0) and np.all(out["znorm2"][0] == 0)
     assert np.all(np.isfinite(out["s"]))
+
+
+# ----------------------------------------------------------------------------- Verifications 1-3
+def test_check_predicates_follow_alg6():
+    """Alg. 6: norm_ji != ||.|| (V1), s_j^i != <z, Delta> and sum_i s_i != 0 (V2),
+    check_ij = [norm > Delta_max] with CheckAveraging when more than n/2 peers vote (V3)."""
+    norm = np.array([[1.0, 2.0, 5.0, 0.5, 7.0]])
+    s = np.array([[[0.25], [-0.75], [0.5], [-0.125], [0.125]]])        # sums to exactly 0
+    out = oracle.checks(norm, s, [1.5])
+    assert out["check"].tolist() == [[0, 1, 1, 0, 1]] and out["votes"][0] == 3
+    assert out["check_averaging"][0] == 1                              # 3 > 5/2
+    assert out["sum_violation"][0, 0] == 0 and not out["norm_mismatch"].any() and not out["s_mismatch"].any()
+    out = oracle.checks(norm, s, [2.0])                                # strict ">": 2.0 is not far
+    assert out["check"].tolist() == [[0, 0, 1, 0, 1]] and out["check_averaging"][0] == 0
+    out = oracle.checks(norm[:, :4], s[:, :4], [0.75])                 # n = 4: 2 votes is not > n/2
+    assert out["votes"][0] == 3 and out["check_averaging"][0] == 1
+    out = oracle.checks(norm[:, :4], s[:, :4], [1.5])
+    assert out["votes"][0] == 2 and out["check_averaging"][0] == 0
+    # a peer misreports its norm and its inner product; the broadcast sum no longer vanishes
+    nr = norm.copy(); nr[0, 3] = 0.5000001
+    sr = s.copy(); sr[0, 1, 0] = -0.7
+    out = oracle.checks(norm, s, [1.5], norm_reported=nr, s_reported=sr)
+    assert out["norm_mismatch"].tolist() == [[0, 0, 0, 1, 0]]
+    assert out["s_mismatch"][0, :, 0].tolist() == [0, 1, 0, 0, 0] and out["sum_violation"][0, 0] == 1
+    # tolerances: the same discrepancies pass when allowed for
+    out = oracle.checks(norm, s, [1.5], norm_reported=nr, s_reported=sr, rel_tol=0.1, sum_tol=0.1)
+    assert not out["norm_mismatch"].any() and not out["s_mismatch"].any() and not out["sum_violation"].any()
+    # NaN reports always differ; Delta_max = inf never fires
+    nr[0, 0] = np.nan
+    out = oracle.checks(norm, s, [np.inf], norm_reported=nr, rel_tol=1.0)
+    assert out["norm_mismatch"][0, 0] == 1 and out["votes"][0] == 0
+
+
+def test_checks_flag_an_aggregation_attack_end_to_end():
+    """Aggregation attack (App. C): the aggregator returns a shifted v.  Honest peers' inner products
+    then do not sum to zero (V2), and if the shift is large most peers see norm > Delta_max (V3)."""
+    x, r = _converged_case()
+    tau = 1.0
+    good = oracle.verify(x, r["v"].astype(np.float32), tau, seed=3, K=2)
+    dmax = float(np.sort(good["norm"][0])[x.shape[0] // 2 - 1] * 1.5)   # most honest peers are within it
+    ok = oracle.checks(good["norm"], good["s"], [dmax], sum_tol=1e-5)
+    assert not ok["sum_violation"].any() and ok["check_averaging"][0] == 0
+    bad_v = (r["v"] + 3.0).astype(np.float32)
+    bad = oracle.verify(x, bad_v, tau, seed=3, K=2)
+    flagged = oracle.checks(bad["norm"], bad["s"], [dmax], sum_tol=1e-5)
+    assert flagged["sum_violation"].all() and flagged["check_averaging"][0] == 1
