@@ -63,6 +63,15 @@ extern "C" {
                                        after the last partition converged; where the device cannot
                                        launch it: DIRECT                                            */
 
+/* Aggregation rule.  The paper's experiments (Sec. 4.1) compare CenteredClip with plain averaging,
+   the coordinate-wise median and the geometric median; they run on the same streaming kernels. */
+#define BTARD_RULE_CENTERED_CLIP 0     /* App. D.2 eq. (CenteredClip)                                 */
+#define BTARD_RULE_GEOMETRIC_MEDIAN 1  /* Weiszfeld: v <- sum_i x_i/rho_i / sum_i 1/rho_i, rho_i =
+                                          max(||x_i - v||, tau[p]): tau is the distance floor, > 0;
+                                          same stop rules; DIRECT algorithms only                    */
+#define BTARD_RULE_MEAN 2              /* v = (1/n) sum_i x_i, one pass, iters = 0                    */
+#define BTARD_RULE_COORD_MEDIAN 3      /* coordinate-wise median, iters = 0                           */
+
 #define BTARD_STOP_FIXED_ITERS 0    /* exactly max_iters updates                                    */
 #define BTARD_STOP_EPS 1            /* stop once ||v^{l+1} - v^l||_2 <= eps, at most max_iters       */
 
@@ -105,6 +114,7 @@ typedef struct {
     void* workspace;             /* device, 256-byte aligned                                        */
     size_t workspace_bytes;
     void* stream;                /* cudaStream_t                                                    */
+    int32_t rule;                /* BTARD_RULE_*; 0 = CenteredClip                                  */
 } btard_cclip_args;
 
 /* Bytes of workspace btard_centered_clip needs for these arguments (0 on invalid arguments).

@@ -219,14 +219,46 @@ static double residual_norm(const float *x, const double *v, int64_t len)
     return sqrt(acc);
 }
 
+#define ORACLE_RULE_CENTERED_CLIP 0
+#define ORACLE_RULE_GEOMETRIC_MEDIAN 1   /* Weiszfeld's iteration; the baseline "geometric median" of Sec. 4.1 */
+#define ORACLE_RULE_MEAN 2               /* plain averaging (All-Reduce baseline of Sec. 4.1)                   */
+#define ORACLE_RULE_COORD_MEDIAN 3       /* coordinate-wise median baseline of Sec. 4.1                          */
+
+int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t stride, int64_t len,
+                               double tau, int32_t init_mode, const float *v0,
+                               int32_t stop_mode, int32_t max_iters, double eps,
+                               double *v, double *resid_norm, int32_t *iters,
+                               double *last_step_norm, uint32_t *status);
+
 int btard_oracle_centered_clip_one(const float *g, int32_t n, int64_t stride, int64_t len,
                                    double tau, int32_t init_mode, const float *v0,
                                    int32_t stop_mode, int32_t max_iters, double eps,
                                    double *v, double *resid_norm, int32_t *iters,
                                    double *last_step_norm, uint32_t *status)
 {
+    return btard_oracle_aggregate_one(ORACLE_RULE_CENTERED_CLIP, g, n, stride, len, tau, init_mode, v0,
+                                      stop_mode, max_iters, eps, v, resid_norm, iters, last_step_norm,
+                                      status);
+}
+
+/*
+ * One partition under one of the aggregation rules the paper compares (Sec. 4.1).
+ *   CENTERED_CLIP:    App. D.2 eq. (CenteredClip), w_i = min{1, tau / rho_i}, v += (1/n) sum_i w_i r_i.
+ *   GEOMETRIC_MEDIAN: Weiszfeld, v <- sum_i x_i / rho_i / sum_i 1 / rho_i with rho_i floored at tau,
+ *                     written as v += sum_i (1/rho_i) r_i / sum_i (1/rho_i); same stop rules.
+ *   MEAN / COORD_MEDIAN: v is the mean / coordinate-wise median of the rows; no update, iters = 0.
+ */
+int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t stride, int64_t len,
+                               double tau, int32_t init_mode, const float *v0,
+                               int32_t stop_mode, int32_t max_iters, double eps,
+                               double *v, double *resid_norm, int32_t *iters,
+                               double *last_step_norm, uint32_t *status)
+{
     if (n < 1 || len < 0 || stride < len || max_iters < 1) return -1;
     if (!(tau >= 0.0)) return -1;
+    if (rule == ORACLE_RULE_GEOMETRIC_MEDIAN && !(tau > 0.0 && isfinite(tau))) return -1;
+    if (rule == ORACLE_RULE_MEAN) { init_mode = ORACLE_INIT_MEAN; max_iters = 0; stop_mode = ORACLE_STOP_FIXED; }
+    if (rule == ORACLE_RULE_COORD_MEDIAN) { init_mode = ORACLE_INIT_COORD_MEDIAN; max_iters = 0; stop_mode = ORACLE_STOP_FIXED; }
     uint32_t st = 0;
     /* v^0: the paper leaves the starting point open (App. D.2, "a sequence {v_l}"). */
     if (init_mode == ORACLE_INIT_CALLER) {
@@ -250,8 +282,20 @@ int btard_oracle_centered_clip_one(const float *g, int32_t n, int64_t stride, in
     double step = 0.0;
     int32_t done = 0;
     for (int32_t l = 0; l < max_iters; ++l) {
-        for (int32_t i = 0; i < n; ++i)
-            w[i] = clip_weight(residual_norm(g + (int64_t)i * stride, v, len), tau, &st);
+        if (rule == ORACLE_RULE_GEOMETRIC_MEDIAN) {
+            double total = 0.0;
+            for (int32_t i = 0; i < n; ++i) {
+                double rho = residual_norm(g + (int64_t)i * stride, v, len);
+                if (!isfinite(rho)) { st |= ORACLE_STATUS_NONFINITE_ROW; w[i] = 0.0; }
+                else w[i] = 1.0 / (rho > tau ? rho : tau);
+                total += w[i];
+            }
+            /* scaled so that the common update below, (1/n) sum_i w_i r_i, is the Weiszfeld step */
+            for (int32_t i = 0; i < n; ++i) w[i] = total > 0.0 ? n * w[i] / total : 0.0;
+        } else {
+            for (int32_t i = 0; i < n; ++i)
+                w[i] = clip_weight(residual_norm(g + (int64_t)i * stride, v, len), tau, &st);
+        }
         for (int64_t c = 0; c < len; ++c) u[c] = 0.0;
         for (int32_t i = 0; i < n; ++i) {
             if (w[i] == 0.0) continue;                  /* weight 0: the row is left out */
@@ -348,6 +392,29 @@ int btard_oracle_verify_one(const float *g, int32_t n, int64_t stride, int64_t l
 /* OpenMP, when enabled, runs whole partitions on different cores and changes  */
 /* no arithmetic.  v is [P][stride] doubles (entries past part_len[p] are 0).  */
 /* ------------------------------------------------------------------------- */
+int btard_oracle_aggregate(int32_t rule, const float *g, int32_t n, int32_t P, int64_t stride,
+                           const int64_t *part_len, const double *tau, int32_t init_mode,
+                           const float *v0, int32_t stop_mode, int32_t max_iters, double eps,
+                           double *v, double *resid_norm, int32_t *iters, double *last_step_norm,
+                           uint32_t *status)
+{
+    int rc_all = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t p = 0; p < P; ++p) {
+        double *vp = v + (int64_t)p * stride;
+        for (int64_t c = 0; c < stride; ++c) vp[c] = 0.0;
+        int rc = btard_oracle_aggregate_one(
+            rule, g + (int64_t)p * n * stride, n, stride, part_len[p], tau[p], init_mode,
+            v0 ? v0 + (int64_t)p * stride : NULL, stop_mode, max_iters, eps, vp,
+            resid_norm + (int64_t)p * n, iters + p, last_step_norm + p, status + p);
+        if (rc) {
+#pragma omp atomic write
+            rc_all = rc;
+        }
+    }
+    return rc_all;
+}
+
 int btard_oracle_centered_clip(const float *g, int32_t n, int32_t P, int64_t stride,
                                const int64_t *part_len, const double *tau, int32_t init_mode,
                                const float *v0 /* [P][stride] or NULL */, int32_t stop_mode,

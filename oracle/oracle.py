@@ -14,6 +14,7 @@ INIT_CALLER, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
 STOP_FIXED, STOP_EPS = 0, 1
 SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1
 STATUS_NOT_CONVERGED, STATUS_NONFINITE_ROW = 1, 2
+RULE_CENTERED_CLIP, RULE_GEOMETRIC_MEDIAN, RULE_MEAN, RULE_COORD_MEDIAN = 0, 1, 2, 3
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "btard_oracle.c")
@@ -94,7 +95,7 @@ def _per_part(x, P, dtype):
 
 
 def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v0=None, stop_mode=STOP_FIXED,
-                  max_iters=1, eps=0.0):
+                  max_iters=1, eps=0.0, rule=RULE_CENTERED_CLIP):
     """Batched CenteredClip.  g: [P][n][stride] fp32 (or [n][stride]).
 
     Returns dict(v [P][stride] f64, resid_norm [P][n], iters [P], last_step_norm [P], status [P]).
@@ -110,8 +111,8 @@ def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v0=None, stop_mode
     it = np.zeros(P, dtype=np.int32)
     ls = np.zeros(P, dtype=np.float64)
     st = np.zeros(P, dtype=np.uint32)
-    rc = _load().btard_oracle_centered_clip(
-        _p(g, C.c_float), C.c_int32(n), C.c_int32(P), C.c_int64(stride), _p(ln, C.c_int64),
+    rc = _load().btard_oracle_aggregate(
+        C.c_int32(rule), _p(g, C.c_float), C.c_int32(n), C.c_int32(P), C.c_int64(stride), _p(ln, C.c_int64),
         _p(tau, C.c_double), C.c_int32(init_mode), _p(v0, C.c_float), C.c_int32(stop_mode),
         C.c_int32(max_iters), C.c_double(eps), _p(v, C.c_double), _p(rn, C.c_double),
         _p(it, C.c_int32), _p(ls, C.c_double), _p(st, C.c_uint32))

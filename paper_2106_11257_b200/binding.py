@@ -12,6 +12,7 @@ import numpy as np
 INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
 ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT, ALGO_DIRECT_COOPERATIVE = 0, 1, 2, 3
 STOP_FIXED_ITERS, STOP_EPS = 0, 1
+RULE_CENTERED_CLIP, RULE_GEOMETRIC_MEDIAN, RULE_MEAN, RULE_COORD_MEDIAN = 0, 1, 2, 3
 SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1
 STATUS_NOT_CONVERGED, STATUS_NONFINITE_ROW = 1, 2
 
@@ -43,7 +44,7 @@ class CclipArgs(C.Structure):
                 ("max_iters", C.c_int32), ("eps", C.c_double), ("v", C.c_void_p),
                 ("iters", C.c_void_p), ("last_step_norm", C.c_void_p), ("resid_norm", C.c_void_p),
                 ("status", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("stream", C.c_void_p)]
+                ("stream", C.c_void_p), ("rule", C.c_int32)]
 
 
 class VerifyArgs(C.Structure):
@@ -188,7 +189,8 @@ def centered_clip_workspace(n, P, row_stride, stop_mode=STOP_EPS, algo=ALGO_DIRE
 
 
 def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v=None, stop_mode=STOP_FIXED_ITERS,
-                  max_iters=1, eps=0.0, algo=ALGO_DIRECT, workspace=None, out=None, stream=None):
+                  max_iters=1, eps=0.0, algo=ALGO_DIRECT, workspace=None, out=None, stream=None,
+                  rule=RULE_CENTERED_CLIP):
     """g: CUDA float32 [P][n][row_stride].  Returns dict of CUDA tensors
     (v, iters, last_step_norm, resid_norm, status).  Asynchronous on the current stream."""
     torch = _torch()
@@ -215,7 +217,7 @@ def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v=None, stop_mode=
                   iters=o["iters"].data_ptr(), last_step_norm=o["last_step_norm"].data_ptr(),
                   resid_norm=o["resid_norm"].data_ptr(), status=o["status"].data_ptr(),
                   workspace=workspace.data_ptr(), workspace_bytes=workspace.numel(),
-                  stream=_stream_ptr(stream))
+                  stream=_stream_ptr(stream), rule=rule)
     with torch.cuda.device(dev):
         _check(lib().btard_centered_clip(C.byref(a)), "btard_centered_clip")
     res = dict(o)

@@ -229,6 +229,11 @@ int btard_centered_clip(const btard_cclip_args* a)
         a->algo != BTARD_ALGO_DIRECT_RESIDENT && a->algo != BTARD_ALGO_DIRECT_COOPERATIVE)
         return BTARD_ERR_INVALID_ARG;
     if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
+    if (a->rule < BTARD_RULE_CENTERED_CLIP || a->rule > BTARD_RULE_COORD_MEDIAN) return BTARD_ERR_INVALID_ARG;
+    if (a->rule != BTARD_RULE_CENTERED_CLIP && a->algo == BTARD_ALGO_GRAM) return BTARD_ERR_UNSUPPORTED;
+    if (a->rule == BTARD_RULE_GEOMETRIC_MEDIAN)
+        for (int p = 0; p < a->n_partitions; ++p)
+            if (!(a->tau[p] > 0.0) || std::isinf(a->tau[p])) return BTARD_ERR_INVALID_ARG;
     if (!aligned16(a->g) || !aligned16(a->v) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
         return BTARD_ERR_BAD_ALIGNMENT;
 
@@ -249,6 +254,7 @@ int btard_centered_clip(const btard_cclip_args* a)
     L.status = a->status;
     L.stride = a->row_stride; L.n = n; L.P = P;
     L.stop_mode = a->stop_mode; L.max_iters = a->max_iters; L.eps2 = a->eps * a->eps;
+    L.rule = a->rule;
     double* tot[2] = {(double*)(base + ws.tot[0]), (double*)(base + ws.tot[1])};
 
     rc = upload_table((PartEntry*)(base + ws.table), P, a->part_len, a->tau, st);
@@ -260,6 +266,20 @@ int btard_centered_clip(const btard_cclip_args* a)
     }
 
     // Init pass: v^0 and the residual norms at v^0 (slot buffer 0).
+    if (a->rule == BTARD_RULE_MEAN || a->rule == BTARD_RULE_COORD_MEDIAN) {
+        L.init_mode = BTARD_INIT_MEAN;
+        if (a->rule == BTARD_RULE_COORD_MEDIAN) {
+            rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
+            if (rc != BTARD_OK) return rc;
+            L.init_mode = BTARD_INIT_CALLER_V0;
+        }
+        L.tot_in = nullptr; L.tot_out = tot[0]; L.l = 0;
+        rc = launch_cclip_pass(L, geo, PASS_INIT, st);          // v and the residual norms at v
+        if (rc != BTARD_OK) return rc;
+        L.tot_in = tot[0]; L.max_iters = 0; L.stop_mode = BTARD_STOP_FIXED_ITERS;
+        return launch_cclip_finalize(L, geo, st);
+    }
+
     // How the updates are driven: one cooperative kernel over everything (whole), one per L2-sized
     // chunk of partitions (chunk >= 1), or one launch per update.
     const int fit = resident_chunk_partitions(n, a->row_stride);         // partitions per L2 budget

@@ -52,6 +52,37 @@ __device__ __forceinline__ float clip_weight(double norm2, double tau, bool& non
     return (float)(tau / rho);
 }
 
+// Weights of the rows for the next update, from their squared residual norms (all threads call it;
+// it ends with the CTA synchronised).  CenteredClip: min{1, tau / rho}.  Geometric median (Weiszfeld):
+// n (1/rho_i) / sum_j (1/rho_j), rho floored at tau, so that (1/n) sum_i w_i (x_i - v) is the
+// Weiszfeld step.  Rows with a non-finite norm get 0 and raise *sh_flag.  scratch: n doubles.
+__device__ void row_weights(const double* sh_sum, float* sh_w, int n, double tau, int rule, int* sh_flag,
+                            double* scratch)
+{
+    const int tid = threadIdx.x;
+    if (rule == BTARD_RULE_GEOMETRIC_MEDIAN) {
+        for (int i = tid; i < n; i += blockDim.x) {
+            const double rho = sqrt(sh_sum[i]);
+            double inv = 0.0;
+            if (isfinite(rho)) inv = 1.0 / fmax(rho, tau);
+            else *sh_flag = 1;
+            scratch[i] = inv;
+        }
+        __syncthreads();
+        double total = 0.0;
+        for (int i = 0; i < n; ++i) total += scratch[i];           // same order in every thread
+        for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x)
+            sh_w[i] = (i < n && total > 0.0) ? (float)((double)n * scratch[i] / total) : 0.0f;
+    } else {
+        for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) {
+            bool bad = false;
+            sh_w[i] = (i < n) ? clip_weight(sh_sum[i], tau, bad) : 0.0f;
+            if (bad) *sh_flag = 1;
+        }
+    }
+    __syncthreads();
+}
+
 struct KernelArgs {
     CclipLaunch a;
     int RG, CL, tiles, cpp;
@@ -132,12 +163,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
         if (tid == 0) sh_flag = 0;
         __syncthreads();
-        for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) {
-            bool bad = false;
-            sh_w[i] = (i < n) ? clip_weight(sh_sum[i], tau, bad) : 0.0f;
-            if (bad) sh_flag = 1;
-        }
-        __syncthreads();
+        row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, sh_part);
         if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
     } else if (MODE == PASS_COMBINE) {
         // v = v0 + sum_i a_i (x_i - v0): the update formula with weights n a_i.
@@ -645,12 +671,7 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
                     add_finished += 1;
                 }
             } else {
-                for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) {
-                    bool bad = false;
-                    sh_w[i] = (i < n) ? clip_weight(sh_sum[i], tau, bad) : 0.0f;
-                    if (bad) sh_flag = 1;
-                }
-                __syncthreads();
+                row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, sh_part);
                 if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
                 sweep(std::false_type{}, (l + 1) & 1, backwards);
             }

@@ -74,6 +74,7 @@ struct CclipLaunch {
     int stop_mode, max_iters;
     double eps2;
     int init_mode;            // PASS_INIT
+    int rule;                 // BTARD_RULE_*: how the row weights follow from the norms
 };
 
 Geometry cclip_geometry(int n, int P, long long stride);

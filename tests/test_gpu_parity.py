@@ -228,6 +228,45 @@ def test_resident_variant_eps_mode_and_chunks():
     assert len(set(ref["iters"].tolist())) > 1
 
 
+# ----------------------------------------------------------------------------- baseline aggregators
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE, btard.ALGO_DIRECT_RESIDENT])
+@pytest.mark.parametrize("n", [3, 16, 64])
+def test_geometric_median_rule_matches_oracle(n, algo):
+    rng = np.random.default_rng(500 + n)
+    P, stride = 3, 5024
+    lens = np.array([5024, 4097, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    floor = np.array([1e-3, 1e-6, 0.5])
+    for stop, iters, eps in ((btard.STOP_FIXED_ITERS, 8, 0.0), (btard.STOP_EPS, 200, 1e-5)):
+        ref = oracle.centered_clip(g, floor, lens, init_mode=oracle.INIT_MEAN, stop_mode=stop,
+                                   max_iters=iters, eps=eps, rule=oracle.RULE_GEOMETRIC_MEDIAN)
+        _, r = run_gpu_cclip(g, floor, lens, init_mode=btard.INIT_MEAN, stop_mode=stop, max_iters=iters,
+                             eps=eps, algo=algo, rule=btard.RULE_GEOMETRIC_MEDIAN)
+        check_cclip(r, ref, lens, eps_mode=(stop == btard.STOP_EPS))
+
+
+@pytest.mark.parametrize("n", [1, 4, 16, 23, 64, 100])
+def test_mean_and_coordinate_median_rules_match_oracle(n):
+    rng = np.random.default_rng(600 + n)
+    P, stride = 3, 5024
+    lens = np.array([5024, 4097, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    for rule, orule in ((btard.RULE_MEAN, oracle.RULE_MEAN), (btard.RULE_COORD_MEDIAN, oracle.RULE_COORD_MEDIAN)):
+        ref = oracle.centered_clip(g, 1.0, lens, rule=orule)
+        _, r = run_gpu_cclip(g, 1.0, lens, rule=rule)
+        check_cclip(r, ref, lens)
+        assert (cpu(r["iters"]) == 0).all()
+
+
+def test_geometric_median_rule_rejects_a_zero_floor_and_gram():
+    g = torch.zeros((1, 4, 64), device="cuda")
+    with pytest.raises(btard.BtardError):
+        btard.centered_clip(g, 0.0, init_mode=btard.INIT_ZERO, rule=btard.RULE_GEOMETRIC_MEDIAN)
+    with pytest.raises(btard.BtardError) as e:
+        btard.centered_clip(g, 1.0, init_mode=btard.INIT_ZERO, rule=btard.RULE_GEOMETRIC_MEDIAN, algo=btard.ALGO_GRAM)
+    assert e.value.code == -5
+
+
 # ----------------------------------------------------------------------------- Gram variant
 @pytest.mark.parametrize("n", [1, 3, 8, 16, 23, 64, 100, 128])
 @pytest.mark.parametrize("init", [btard.INIT_MEAN, btard.INIT_COORD_MEDIAN, btard.INIT_CALLER_V0])

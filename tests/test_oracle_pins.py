@@ -477,3 +477,54 @@ def test_checks_flag_an_aggregation_attack_end_to_end():
     bad = oracle.verify(x, bad_v, tau, seed=3, K=2)
     flagged = oracle.checks(bad["norm"], bad["s"], [dmax], sum_tol=1e-5)
     assert flagged["sum_violation"].all() and flagged["check_averaging"][0] == 1
+
+
+# ----------------------------------------------------------------------------- baseline aggregators
+def test_geometric_median_closed_forms():
+    """Weiszfeld's iteration: the Fermat point of an equilateral triangle is its centroid; the
+    geometric median of collinear points (odd count) is the middle point; one point is itself."""
+    tri = np.array([[0.0, 0.0], [4.0, 0.0], [2.0, 2.0 * math.sqrt(3.0)]], dtype=np.float32)
+    r = oracle.centered_clip(tri, 1e-9, init_mode=oracle.INIT_ZERO, stop_mode=oracle.STOP_EPS,
+                             max_iters=1000, eps=1e-13, rule=oracle.RULE_GEOMETRIC_MEDIAN)
+    assert np.allclose(r["v"][0], tri.astype(np.float64).mean(0), atol=1e-9) and r["status"][0] == 0
+    line = np.array([[-3.0, -6.0], [0.5, 1.0], [1.0, 2.0], [7.0, 14.0], [2.0, 4.0]], dtype=np.float32)
+    r = oracle.centered_clip(line, 1e-12, init_mode=oracle.INIT_MEAN, stop_mode=oracle.STOP_EPS,
+                             max_iters=20000, eps=1e-14, rule=oracle.RULE_GEOMETRIC_MEDIAN)
+    assert np.allclose(r["v"][0], [1.0, 2.0], atol=1e-6)
+    one = np.array([[3.0, -1.0, 2.0]], dtype=np.float32)
+    r = oracle.centered_clip(one, 1e-6, init_mode=oracle.INIT_ZERO, max_iters=1, rule=oracle.RULE_GEOMETRIC_MEDIAN)
+    assert np.allclose(r["v"][0], one[0], atol=1e-15)
+
+
+def test_geometric_median_optimality_and_centered_clip_limit():
+    """At the geometric median the unit vectors to the points cancel; that is also the fixed-point
+    equation of CenteredClip when tau is below every distance (App. D.2: tau -> 0)."""
+    rng = np.random.default_rng(21)
+    x = rand_rows(rng, 9, 40, 2.0)
+    r = oracle.centered_clip(x, 1e-9, init_mode=oracle.INIT_COORD_MEDIAN, stop_mode=oracle.STOP_EPS,
+                             max_iters=5000, eps=1e-13, rule=oracle.RULE_GEOMETRIC_MEDIAN)
+    v = r["v"][0]
+    d = x.astype(np.float64) - v
+    unit = d / np.linalg.norm(d, axis=1, keepdims=True)
+    assert np.linalg.norm(unit.sum(0)) < 1e-9
+    tau = 1e-3
+    lhs, rho, w = clipped_residual_sum(x, v, tau)
+    assert rho.min() > tau and np.linalg.norm(lhs) < 1e-11           # v solves the CenteredClip equation
+    # one Weiszfeld step from v0, against its textbook form sum x_i/rho_i / sum 1/rho_i
+    v0 = rng.standard_normal(40).astype(np.float32)
+    r1 = oracle.centered_clip(x, 1e-9, init_mode=oracle.INIT_CALLER, v0=v0[None], max_iters=1,
+                              rule=oracle.RULE_GEOMETRIC_MEDIAN)
+    rho0 = np.linalg.norm(x.astype(np.float64) - v0, axis=1)
+    assert np.allclose(r1["v"][0], (x.astype(np.float64) / rho0[:, None]).sum(0) / (1 / rho0).sum(), atol=1e-13)
+
+
+def test_mean_and_coordinate_median_rules():
+    rng = np.random.default_rng(22)
+    g = rng.standard_normal((2, 6, 33)).astype(np.float32)
+    lens = np.array([33, 20])
+    for rule, fn in ((oracle.RULE_MEAN, np.mean), (oracle.RULE_COORD_MEDIAN, np.median)):
+        r = oracle.centered_clip(g, 1.0, part_len=lens, rule=rule, max_iters=7)
+        for p in range(2):
+            ref = fn(g[p][:, :lens[p]].astype(np.float64), axis=0)
+            assert np.allclose(r["v"][p, :lens[p]], ref, atol=1e-15) and r["iters"][p] == 0
+            assert np.allclose(r["resid_norm"][p], np.linalg.norm(g[p][:, :lens[p]] - ref, axis=1), rtol=1e-12)
