@@ -161,6 +161,31 @@ BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* arg
 BTARD_API int btard_verify_projections(const btard_verify_args* args);
 
 /*
+ * Per-part gradient clipping of BTARD-Clipped-SGD (Alg. 9 and the paragraph after it):
+ *     g~_i(l) = min{1, lambda / ||g_i(l)||_2} g_i(l)
+ * applied IN PLACE to g [P][n][row_stride] (row i of slab l is g_i(l)) before it is aggregated.
+ * lambda: host [P] (the paper uses one lambda_k per step; per-part values are allowed), >= 0, +inf = no
+ * clipping.  Outputs: row_norm [P][n] = ||g_i(l)||_2 before clipping, factor [P][n] = the multiplier
+ * applied (1 when the row is left untouched; 0 for a row with a non-finite norm, which is set to zero
+ * and flagged in status).  Two passes over g (norms, then rescaling of the clipped rows only).
+ */
+typedef struct {
+    int32_t n_peers, n_partitions;
+    int64_t row_stride;
+    const int64_t* part_len;     /* host [P] */
+    const double* lambda;        /* host [P] */
+    float* g;                    /* device [P][n][row_stride], modified in place */
+    double* row_norm;            /* device [P][n] out */
+    double* factor;              /* device [P][n] out */
+    uint32_t* status;            /* device [P] out */
+    void* workspace;             /* device, 256-byte aligned */
+    size_t workspace_bytes;
+    void* stream;
+} btard_preclip_args;
+BTARD_API size_t btard_preclip_workspace(const btard_preclip_args* args);
+BTARD_API int btard_preclip(const btard_preclip_args* args);
+
+/*
  * The predicates of Verifications 1-3 (Alg. 6 lines 17-38) on the scalars peers broadcast.  For
  * partition p (aggregated by peer p) and peer i:
  *   Verification 1: norm_mismatch[p][i] = reported norm_ip differs from ||g_i(p) - v(p)||;

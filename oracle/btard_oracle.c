@@ -504,6 +504,24 @@ void btard_oracle_checks_one(int32_t n, int32_t K, const double *norm, const dou
     *check_averaging = (uint8_t)(2 * v > n);      /* more than n/2 peers voted */
 }
 
+/* ------------------------------------------------------------------------- */
+/* Per-part clipping of BTARD-Clipped-SGD (Alg. 9 and the paragraph after it):  */
+/*   g~_i(l) = min{1, lambda / ||g_i(l)||} g_i(l).  One row; a row whose norm is */
+/*   not finite is set to zero (factor 0).                                      */
+/* ------------------------------------------------------------------------- */
+void btard_oracle_preclip_row(const float *x, int64_t len, double lambda, double *out, double *norm,
+                              double *factor)
+{
+    double acc = 0.0;
+    for (int64_t c = 0; c < len; ++c) acc += (double)x[c] * (double)x[c];
+    double nrm = sqrt(acc), f;
+    if (!isfinite(nrm)) f = 0.0;
+    else f = (nrm <= lambda) ? 1.0 : lambda / nrm;
+    for (int64_t c = 0; c < len; ++c) out[c] = (f == 0.0) ? 0.0 : f * (double)x[c];
+    *norm = nrm;
+    *factor = f;
+}
+
 int btard_oracle_max_threads(void)
 {
 #ifdef _OPENMP

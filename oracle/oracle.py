@@ -198,3 +198,23 @@ def checks(norm, s, delta_max, norm_reported=None, s_reported=None, rel_tol=0.0,
         out["votes"][p] = votes.value
         out["check_averaging"][p] = ca.value
     return out
+
+
+def preclip(g, lam, part_len=None):
+    """Per-part clipping.  Returns dict(g [P][n][stride] float64, row_norm, factor [P][n])."""
+    g = _as_g(g)
+    P, n, stride = g.shape
+    ln = _per_part(stride if part_len is None else part_len, P, np.int64)
+    lam = _per_part(lam, P, np.float64)
+    out = np.zeros((P, n, stride), dtype=np.float64)
+    norm = np.zeros((P, n))
+    fac = np.zeros((P, n))
+    lib = _load()
+    for p in range(P):
+        for i in range(n):
+            nr, f = C.c_double(0.0), C.c_double(0.0)
+            lib.btard_oracle_preclip_row(_p(g[p, i], C.c_float), C.c_int64(int(ln[p])),
+                                         C.c_double(float(lam[p])), _p(out[p, i], C.c_double),
+                                         C.byref(nr), C.byref(f))
+            norm[p, i], fac[p, i] = nr.value, f.value
+    return dict(g=out, row_norm=norm, factor=fac)

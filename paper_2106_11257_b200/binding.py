@@ -21,7 +21,8 @@ EXPORTS = [
     "btard_verify_projections_workspace", "btard_verify_projections", "btard_random_vector",
     "btard_aggregate_host_scratch", "btard_aggregate_host", "btard_last_cuda_error",
     "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
-    "btard_verify_projections_static", "btard_verification_checks",
+    "btard_verify_projections_static", "btard_verification_checks", "btard_preclip_workspace",
+    "btard_preclip",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -71,6 +72,13 @@ class HostArgs(C.Structure):
                 ("copy_stream", C.c_void_p)]
 
 
+class PreclipArgs(C.Structure):
+    _fields_ = [("n_peers", C.c_int32), ("n_partitions", C.c_int32), ("row_stride", C.c_int64),
+                ("part_len", C.c_void_p), ("lambda_", C.c_void_p), ("g", C.c_void_p),
+                ("row_norm", C.c_void_p), ("factor", C.c_void_p), ("status", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p)]
+
+
 class ChecksArgs(C.Structure):
     _fields_ = [("n_peers", C.c_int32), ("n_partitions", C.c_int32), ("n_z", C.c_int32),
                 ("norm", C.c_void_p), ("norm_reported", C.c_void_p), ("s", C.c_void_p),
@@ -109,6 +117,10 @@ def lib():
         L.btard_verify_projections.argtypes = [C.POINTER(VerifyArgs)]
         L.btard_verify_projections_static.restype = C.c_int
         L.btard_verify_projections_static.argtypes = [C.POINTER(VerifyArgs)]
+        L.btard_preclip_workspace.restype = C.c_size_t
+        L.btard_preclip_workspace.argtypes = [C.POINTER(PreclipArgs)]
+        L.btard_preclip.restype = C.c_int
+        L.btard_preclip.argtypes = [C.POINTER(PreclipArgs)]
         L.btard_verification_checks.restype = C.c_int
         L.btard_verification_checks.argtypes = [C.POINTER(ChecksArgs)]
         L.btard_random_vector.restype = C.c_int
@@ -314,6 +326,31 @@ def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in
     if rs is not None:
         res["resid_sum"] = rs
     return res
+
+
+def preclip(g, lam, part_len=None, stream=None):
+    """In-place per-part clipping g_i(l) <- min{1, lam/||g_i(l)||} g_i(l) of a CUDA float32 tensor
+    [P][n][row_stride].  Returns dict(row_norm, factor [P][n] float64, status [P])."""
+    torch = _torch()
+    assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
+    P, n, stride = g.shape
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    lam_h = _host_arr(lam, P, np.float64)
+    dev = g.device
+    o = dict(row_norm=torch.empty((P, n), dtype=torch.float64, device=dev),
+             factor=torch.empty((P, n), dtype=torch.float64, device=dev),
+             status=torch.empty(P, dtype=torch.int32, device=dev))
+    a = PreclipArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
+                    lambda_=lam_h.ctypes.data, g=g.data_ptr(), row_norm=o["row_norm"].data_ptr(),
+                    factor=o["factor"].data_ptr(), status=o["status"].data_ptr(), stream=_stream_ptr(stream))
+    need = int(lib().btard_preclip_workspace(C.byref(a)))
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    a.workspace = ws.data_ptr()
+    a.workspace_bytes = ws.numel()
+    with torch.cuda.device(dev):
+        _check(lib().btard_preclip(C.byref(a)), "btard_preclip")
+    o["workspace"] = ws
+    return o
 
 
 def verification_checks(norm, s, delta_max, norm_reported=None, s_reported=None, rel_tol=0.0,

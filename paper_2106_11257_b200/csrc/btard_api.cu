@@ -445,6 +445,34 @@ int btard_verify_projections(const btard_verify_args* a)
     return BTARD_OK;
 }
 
+size_t btard_preclip_workspace(const btard_preclip_args* a)
+{
+    if (!a || a->n_peers < 1 || a->n_peers > BTARD_MAX_PEERS || a->n_partitions < 1 || a->row_stride < 4)
+        return 0;
+    const int chunks = preclip_chunks(a->n_peers, a->n_partitions, a->row_stride);
+    return align_up(sizeof(PartEntry) * (size_t)a->n_partitions, 256) +
+           align_up(sizeof(double) * (size_t)a->n_peers * a->n_partitions * chunks, 256);
+}
+
+int btard_preclip(const btard_preclip_args* a)
+{
+    if (!a) return BTARD_ERR_INVALID_ARG;
+    int rc = check_common(a->n_peers, a->n_partitions, a->row_stride, a->part_len, a->lambda);
+    if (rc != BTARD_OK) return rc;
+    if (!a->g || !a->row_norm || !a->factor || !a->status || !a->workspace) return BTARD_ERR_INVALID_ARG;
+    if (!aligned16(a->g) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return BTARD_ERR_BAD_ALIGNMENT;
+    if (a->workspace_bytes < btard_preclip_workspace(a)) return BTARD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)a->stream;
+    char* base = (char*)a->workspace;
+    PartEntry* table = (PartEntry*)base;
+    rc = upload_table(table, a->n_partitions, a->part_len, a->lambda, st);    // lambda rides in the tau field
+    if (rc != BTARD_OK) return rc;
+    double* slots = (double*)(base + align_up(sizeof(PartEntry) * (size_t)a->n_partitions, 256));
+    const int chunks = preclip_chunks(a->n_peers, a->n_partitions, a->row_stride);
+    return launch_preclip(a->g, table, slots, a->row_norm, a->factor, a->status, a->row_stride,
+                          a->n_peers, a->n_partitions, chunks, st);
+}
+
 int btard_verification_checks(const btard_checks_args* a)
 {
     if (!a || a->n_peers < 1 || a->n_partitions < 1 || a->n_partitions > 65535 || a->n_z < 1)

@@ -132,6 +132,11 @@ int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream
 int launch_gram_finalize(const double* tot, double* resid_norm, uint32_t* status, int n, int P,
                          const unsigned int* error, cudaStream_t st);
 
+// ---- per-part gradient clipping (btard_preclip.cu) ----------------------------------------------
+int preclip_chunks(int n, int P, long long stride);
+int launch_preclip(float* g, const PartEntry* table, double* slots, double* row_norm, double* factor,
+                   uint32_t* status, long long stride, int n, int P, int chunks, cudaStream_t st);
+
 // ---- verification (btard_verify.cu) -------------------------------------------------------------
 struct VerifyLaunch {
     const float* g;

@@ -267,6 +267,33 @@ def test_geometric_median_rule_rejects_a_zero_floor_and_gram():
     assert e.value.code == -5
 
 
+# ----------------------------------------------------------------------------- Clipped-SGD pre-clip
+@pytest.mark.parametrize("n,stride", [(4, 1024), (16, 100_000), (64, 5024)])
+def test_preclip_matches_oracle(n, stride):
+    rng = np.random.default_rng(700 + n)
+    P = 3
+    lens = np.array([stride, stride - 27, 13])
+    g = (rng.standard_normal((P, n, stride)) * 0.01).astype(np.float32)
+    g[:, ::3] *= 50.0                                              # every third peer is far too long
+    g[1, 1, 7] = np.inf
+    lam = np.array([1.0, 2.0, np.inf])
+    ref = oracle.preclip(g, lam, part_len=lens)
+    gd = torch.from_numpy(g.copy()).cuda()
+    out = btard.preclip(gd, lam, part_len=lens)
+    torch.cuda.synchronize()
+    got = cpu(gd)
+    for p in range(P):
+        L = lens[p]
+        fin = np.isfinite(ref["row_norm"][p])
+        assert rel_l2(cpu(out["row_norm"])[p][fin], ref["row_norm"][p][fin]) <= 1e-6
+        assert np.array_equal(np.isfinite(cpu(out["row_norm"])[p]), fin)
+        assert rel_l2(cpu(out["factor"])[p], ref["factor"][p]) <= 1e-6
+        assert rel_l2(got[p, :, :L], ref["g"][p, :, :L]) <= 1e-6
+        untouched = ref["factor"][p] == 1.0
+        assert np.array_equal(got[p, untouched, :L], g[p, untouched, :L])   # bit for bit
+    assert cpu(out["status"])[1] & btard.STATUS_NONFINITE_ROW and np.all(got[1, 1, :lens[1]] == 0)
+
+
 # ----------------------------------------------------------------------------- Gram variant
 @pytest.mark.parametrize("n", [1, 3, 8, 16, 23, 64, 100, 128])
 @pytest.mark.parametrize("init", [btard.INIT_MEAN, btard.INIT_COORD_MEDIAN, btard.INIT_CALLER_V0])

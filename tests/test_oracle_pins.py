@@ -528,3 +528,30 @@ def test_mean_and_coordinate_median_rules():
             ref = fn(g[p][:, :lens[p]].astype(np.float64), axis=0)
             assert np.allclose(r["v"][p, :lens[p]], ref, atol=1e-15) and r["iters"][p] == 0
             assert np.allclose(r["resid_norm"][p], np.linalg.norm(g[p][:, :lens[p]] - ref, axis=1), rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- Clipped-SGD pre-clip
+def test_preclip_closed_forms():
+    """g~ = min{1, lambda/||g||} g (Alg. 9): short rows are untouched, long rows land on the sphere of
+    radius lambda with their direction kept; lambda = inf is the identity."""
+    rng = np.random.default_rng(30)
+    g = rng.standard_normal((2, 4, 40)).astype(np.float32)
+    g[0, 1] *= 100; g[1, 3] *= 1e-3
+    lens = np.array([40, 25])
+    out = oracle.preclip(g, [3.0, 3.0], part_len=lens)
+    for p in range(2):
+        for i in range(4):
+            x = g[p, i, :lens[p]].astype(np.float64)
+            nrm = np.linalg.norm(x)
+            assert abs(out["row_norm"][p, i] - nrm) < 1e-12
+            y = out["g"][p, i, :lens[p]]
+            if nrm <= 3.0:
+                assert out["factor"][p, i] == 1.0 and np.array_equal(y, x)
+            else:
+                assert abs(np.linalg.norm(y) - 3.0) < 1e-12 and np.allclose(y / 3.0, x / nrm, atol=1e-15)
+            assert np.all(out["g"][p, i, lens[p]:] == 0)
+    ident = oracle.preclip(g, np.inf, part_len=lens)
+    assert np.array_equal(ident["g"][0], g[0].astype(np.float64)) and np.all(ident["factor"] == 1.0)
+    bad = g.copy(); bad[0, 2, 5] = np.nan
+    out = oracle.preclip(bad, 3.0, part_len=lens)
+    assert out["factor"][0, 2] == 0.0 and np.all(out["g"][0, 2] == 0)
