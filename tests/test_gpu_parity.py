@@ -526,17 +526,26 @@ def test_config2_and_4_gram_mode_full_size_sampled():
     _full_config(4, sample=[17], algo=btard.ALGO_GRAM)
 
 
-def test_config5_shape_sampled():
-    """Config 5 at a quarter of its length (16 GiB of rows): fixed 20 iterations and the Gram variant
-    side by side, one partition checked against the oracle."""
-    w = workloads.make_workload(5, device="cuda", d=1 << 26)
+def test_config5_full_size_sampled():
+    """Config 5 at full size (64 GiB of rows): fixed 20 iterations and the Gram variant side by side,
+    one 1 GiB partition checked against the oracle, then the verification pass (K = 4) on it."""
+    free, _ = torch.cuda.mem_get_info()
+    d = 1 << 28 if free > 90 * (1 << 30) else 1 << 26              # smaller boards: a quarter of the length
+    w = workloads.make_workload(5, device="cuda", d=d)
+    p = 41
+    gp = cpu(w.g[p:p + 1])
+    lens = w.part_len[p:p + 1]
+    ref = oracle.centered_clip(gp, w.tau[p], lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=20)
     for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
         r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
                                 stop_mode=btard.STOP_FIXED_ITERS, max_iters=20, algo=algo)
         torch.cuda.synchronize()
-        p = 41
-        gp = cpu(w.g[p:p + 1])
-        ref = oracle.centered_clip(gp, w.tau[p], w.part_len[p:p + 1], init_mode=oracle.INIT_COORD_MEDIAN,
-                                   max_iters=20)
         sub = {k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}
-        check_cclip(sub, ref, w.part_len[p:p + 1])
+        check_cclip(sub, ref, lens)
+    o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                 resid_norm_in=r["resid_norm"])
+    torch.cuda.synchronize()
+    refv = oracle.verify(gp, cpu(r["v"][p:p + 1]), w.tau[p], w.zseed, K=w.K, part_len=lens,
+                         norm_in=cpu(r["resid_norm"][p:p + 1]), first_partition=p)
+    subo = {k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm")}
+    check_verify(subo, refv, w.K)
