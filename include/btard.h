@@ -90,6 +90,21 @@ BTARD_API int btard_partition_layout(int64_t d, int32_t P, int32_t mode, int32_t
                            int64_t* part_offset, int64_t* part_len, int64_t* row_stride);
 
 /*
+ * Split and Merge of App. D.1 as device copies.  btard_split_gradients turns the n gradient vectors
+ * grads [n][d] into the slab tensor g [P][n][row_stride] (row i of slab p = part p of peer i, padding
+ * columns zero): with all peers on one GPU this is what the all-to-all of Alg. 2 lines 3-4 delivers.
+ * btard_merge_partitions concatenates the aggregated parts v [P][row_stride] into out [d] (Alg. 2 line 9).
+ * part_offset / part_len: host [P] as returned by btard_partition_layout; table: device scratch of
+ * 16 * P bytes.  All tensors device memory; asynchronous on `stream`.
+ */
+BTARD_API int btard_split_gradients(int64_t d, int32_t n_peers, int32_t n_partitions, int64_t row_stride,
+                                    const int64_t* part_offset, const int64_t* part_len,
+                                    const float* grads, float* g, void* table, void* stream);
+BTARD_API int btard_merge_partitions(int64_t d, int32_t n_partitions, int64_t row_stride,
+                                     const int64_t* part_offset, const int64_t* part_len,
+                                     const float* v, float* out, void* table, void* stream);
+
+/*
  * CenteredClip, App. D.2 eq. (CenteredClip), on all P partitions at once:
  *     v^{l+1} = v^l + (1/n) sum_i (x_i - v^l) min{1, tau / ||x_i - v^l||_2},   x_i = g[p][i][:].
  * A row whose residual norm is not finite takes weight 0 and is left out of the sum.

@@ -22,7 +22,7 @@ EXPORTS = [
     "btard_aggregate_host_scratch", "btard_aggregate_host", "btard_last_cuda_error",
     "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
     "btard_verify_projections_static", "btard_verification_checks", "btard_preclip_workspace",
-    "btard_preclip",
+    "btard_preclip", "btard_split_gradients", "btard_merge_partitions",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -326,6 +326,45 @@ def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in
     if rs is not None:
         res["resid_sum"] = rs
     return res
+
+
+def split_gradients(grads, P, mode=SPLIT_CEIL_PAD, align_elems=32, stream=None):
+    """grads: CUDA float32 [n][d] -> (g [P][n][row_stride], part_offset, part_len)."""
+    torch = _torch()
+    assert grads.is_cuda and grads.dtype == torch.float32 and grads.dim() == 2 and grads.is_contiguous()
+    n, d = grads.shape
+    off, ln, stride = partition_layout(d, P, mode, align_elems)
+    g = torch.empty((P, n, stride), dtype=torch.float32, device=grads.device)
+    table = torch.empty(16 * P, dtype=torch.uint8, device=grads.device)
+    L = lib()
+    L.btard_split_gradients.restype = C.c_int
+    L.btard_split_gradients.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    with torch.cuda.device(grads.device):
+        _check(L.btard_split_gradients(d, n, P, stride, off.ctypes.data, ln.ctypes.data, grads.data_ptr(),
+                                       g.data_ptr(), table.data_ptr(), _stream_ptr(stream)),
+               "btard_split_gradients")
+    return g, off, ln
+
+
+def merge_partitions(v, d, part_offset, part_len, stream=None):
+    """v: CUDA float32 [P][row_stride] -> out [d]."""
+    torch = _torch()
+    assert v.is_cuda and v.dtype == torch.float32 and v.dim() == 2 and v.is_contiguous()
+    P, stride = v.shape
+    out = torch.empty(d, dtype=torch.float32, device=v.device)
+    table = torch.empty(16 * P, dtype=torch.uint8, device=v.device)
+    off = np.ascontiguousarray(part_offset, dtype=np.int64)
+    ln = np.ascontiguousarray(part_len, dtype=np.int64)
+    L = lib()
+    L.btard_merge_partitions.restype = C.c_int
+    L.btard_merge_partitions.argtypes = [C.c_int64, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_void_p]
+    with torch.cuda.device(v.device):
+        _check(L.btard_merge_partitions(d, P, stride, off.ctypes.data, ln.ctypes.data, v.data_ptr(),
+                                        out.data_ptr(), table.data_ptr(), _stream_ptr(stream)),
+               "btard_merge_partitions")
+    return out
 
 
 def preclip(g, lam, part_len=None, stream=None):

@@ -445,6 +445,40 @@ int btard_verify_projections(const btard_verify_args* a)
     return BTARD_OK;
 }
 
+namespace {
+int upload_pack_table(void* table, int P, int64_t d, int64_t stride, const int64_t* off, const int64_t* len,
+                      cudaStream_t st)
+{
+    if (P < 1 || P > 65535 || !off || !len || !table || d < 0 || stride < 1) return BTARD_ERR_INVALID_ARG;
+    std::vector<long long> host(2 * (size_t)P);
+    for (int p = 0; p < P; ++p) {
+        if (off[p] < 0 || len[p] < 0 || len[p] > stride || off[p] + len[p] > d) return BTARD_ERR_INVALID_ARG;
+        host[2 * p] = off[p];
+        host[2 * p + 1] = len[p];
+    }
+    BTARD_CUDA_TRY(cudaMemcpyAsync(table, host.data(), sizeof(long long) * 2 * P, cudaMemcpyHostToDevice, st));
+    return BTARD_OK;
+}
+}  // namespace
+
+int btard_split_gradients(int64_t d, int32_t n, int32_t P, int64_t stride, const int64_t* off,
+                          const int64_t* len, const float* grads, float* g, void* table, void* stream)
+{
+    if (n < 1 || !grads || !g) return BTARD_ERR_INVALID_ARG;
+    int rc = upload_pack_table(table, P, d, stride, off, len, (cudaStream_t)stream);
+    if (rc != BTARD_OK) return rc;
+    return launch_split(grads, g, table, d, stride, n, P, (cudaStream_t)stream);
+}
+
+int btard_merge_partitions(int64_t d, int32_t P, int64_t stride, const int64_t* off, const int64_t* len,
+                           const float* v, float* out, void* table, void* stream)
+{
+    if (!v || !out) return BTARD_ERR_INVALID_ARG;
+    int rc = upload_pack_table(table, P, d, stride, off, len, (cudaStream_t)stream);
+    if (rc != BTARD_OK) return rc;
+    return launch_merge(v, out, table, stride, P, (cudaStream_t)stream);
+}
+
 size_t btard_preclip_workspace(const btard_preclip_args* a)
 {
     if (!a || a->n_peers < 1 || a->n_peers > BTARD_MAX_PEERS || a->n_partitions < 1 || a->row_stride < 4)

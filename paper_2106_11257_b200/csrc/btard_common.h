@@ -137,6 +137,11 @@ int preclip_chunks(int n, int P, long long stride);
 int launch_preclip(float* g, const PartEntry* table, double* slots, double* row_norm, double* factor,
                    uint32_t* status, long long stride, int n, int P, int chunks, cudaStream_t st);
 
+// ---- Split / Merge copies (btard_pack.cu); table_dev: device {offset, len}[P] as two int64 each ---
+int launch_split(const float* grads, float* g, const void* table_dev, long long d, long long stride,
+                 int n, int P, cudaStream_t st);
+int launch_merge(const float* v, float* out, const void* table_dev, long long stride, int P, cudaStream_t st);
+
 // ---- verification (btard_verify.cu) -------------------------------------------------------------
 struct VerifyLaunch {
     const float* g;

@@ -267,6 +267,30 @@ def test_geometric_median_rule_rejects_a_zero_floor_and_gram():
     assert e.value.code == -5
 
 
+# ----------------------------------------------------------------------------- Split / Merge
+@pytest.mark.parametrize("mode", [btard.SPLIT_PAPER, btard.SPLIT_CEIL_PAD])
+@pytest.mark.parametrize("n,d,P", [(4, 1024, 1), (5, 100_003, 7), (3, 10, 4), (16, 1_000_001, 16)])
+def test_split_and_merge_are_exact_copies(n, d, P, mode):
+    """Split(v, n) / Merge (App. D.1): bit-exact against plain slicing with the oracle's layout."""
+    rng = np.random.default_rng(d)
+    grads = rng.standard_normal((n, d)).astype(np.float32)
+    g, off, ln = btard.split_gradients(torch.from_numpy(grads).cuda(), P, mode=mode)
+    o_off, o_ln, o_stride = oracle.partition_layout(d, P, mode, 32)
+    assert np.array_equal(off, o_off) and np.array_equal(ln, o_ln) and g.shape[2] == max(o_stride, 32)
+    got = cpu(g)
+    for p in range(P):
+        assert np.array_equal(got[p, :, :ln[p]], grads[:, off[p]:off[p] + ln[p]])
+        assert np.all(got[p, :, ln[p]:] == 0)
+    # aggregate with tau = inf (the mean) and merge: the average gradient, as plain All-Reduce would give
+    r = btard.centered_clip(g, np.inf, part_len=ln, init_mode=btard.INIT_ZERO, max_iters=1)
+    merged = cpu(btard.merge_partitions(r["v"], d, off, ln))
+    assert rel_l2(merged, grads.astype(np.float64).mean(0)) < 1e-6
+    v = torch.from_numpy(rng.standard_normal((P, g.shape[2])).astype(np.float32)).cuda()
+    out = cpu(btard.merge_partitions(v, d, off, ln))
+    for p in range(P):
+        assert np.array_equal(out[off[p]:off[p] + ln[p]], cpu(v)[p, :ln[p]])
+
+
 # ----------------------------------------------------------------------------- Clipped-SGD pre-clip
 @pytest.mark.parametrize("n,stride", [(4, 1024), (16, 100_000), (64, 5024)])
 def test_preclip_matches_oracle(n, stride):
