@@ -90,6 +90,21 @@ BTARD_API int btard_partition_layout(int64_t d, int32_t P, int32_t mode, int32_t
                            int64_t* part_offset, int64_t* part_len, int64_t* row_stride);
 
 /*
+ * Commitments of Alg. 2 lines 2 and 6 (hash(g_i[j]) and hash(g^_i), broadcast before the parts travel).
+ * The paper asks only for "a cryptographic hash"; this library fixes SHA-256 (FIPS 180-4) in a two-level
+ * tree so that one part is hashed by many threads:
+ *     H(row) = SHA256( SHA256(chunk_0) || SHA256(chunk_1) || ... || LE64(byte length) ),
+ * chunks = consecutive 4096-byte pieces of the row's first 4 * part_len bytes (float32 as stored).
+ * x: device [P][rows_per_part][row_stride] — pass g with rows_per_part = n for the peers' parts, or v
+ * with rows_per_part = 1 for the aggregates.  digests: device [P][rows_per_part][32] bytes out.
+ * Workspace from btard_hash_partitions_workspace.  Asynchronous on `stream`.
+ */
+BTARD_API size_t btard_hash_partitions_workspace(int32_t n_partitions, int32_t rows_per_part, int64_t row_stride);
+BTARD_API int btard_hash_partitions(int32_t n_partitions, int32_t rows_per_part, int64_t row_stride,
+                                    const int64_t* part_len /* host [P] */, const float* x,
+                                    uint8_t* digests, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Split and Merge of App. D.1 as device copies.  btard_split_gradients turns the n gradient vectors
  * grads [n][d] into the slab tensor g [P][n][row_stride] (row i of slab p = part p of peer i, padding
  * columns zero): with all peers on one GPU this is what the all-to-all of Alg. 2 lines 3-4 delivers.

@@ -10,5 +10,5 @@ from .oracle import (  # noqa: F401
     INIT_CALLER, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN, STOP_FIXED, STOP_EPS,
     SPLIT_PAPER, SPLIT_CEIL_PAD, RULE_CENTERED_CLIP, RULE_GEOMETRIC_MEDIAN, RULE_MEAN, RULE_COORD_MEDIAN, STATUS_NOT_CONVERGED, STATUS_NONFINITE_ROW,
     build, philox4x32_10, random_vector, partition_layout, centered_clip, verify,
-    max_threads, checks, preclip,
+    max_threads, checks, preclip, sha256, commitment,
 )

@@ -522,6 +522,77 @@ void btard_oracle_preclip_row(const float *x, int64_t len, double lambda, double
     *factor = f;
 }
 
+/* ------------------------------------------------------------------------- */
+/* Commitments (Alg. 2 lines 2 and 6): SHA-256 (FIPS 180-4), byte oriented, and  */
+/* the two-level tree over 4096-byte chunks that the library defines:            */
+/*   H(row) = SHA256(SHA256(chunk_0) || ... || SHA256(chunk_m-1) || LE64(bytes)). */
+/* ------------------------------------------------------------------------- */
+static const uint32_t sha_k[64] = {
+    0x428a2f98u, 0x71374491u, 0xb5c0fbcfu, 0xe9b5dba5u, 0x3956c25bu, 0x59f111f1u, 0x923f82a4u, 0xab1c5ed5u,
+    0xd807aa98u, 0x12835b01u, 0x243185beu, 0x550c7dc3u, 0x72be5d74u, 0x80deb1feu, 0x9bdc06a7u, 0xc19bf174u,
+    0xe49b69c1u, 0xefbe4786u, 0x0fc19dc6u, 0x240ca1ccu, 0x2de92c6fu, 0x4a7484aau, 0x5cb0a9dcu, 0x76f988dau,
+    0x983e5152u, 0xa831c66du, 0xb00327c8u, 0xbf597fc7u, 0xc6e00bf3u, 0xd5a79147u, 0x06ca6351u, 0x14292967u,
+    0x27b70a85u, 0x2e1b2138u, 0x4d2c6dfcu, 0x53380d13u, 0x650a7354u, 0x766a0abbu, 0x81c2c92eu, 0x92722c85u,
+    0xa2bfe8a1u, 0xa81a664bu, 0xc24b8b70u, 0xc76c51a3u, 0xd192e819u, 0xd6990624u, 0xf40e3585u, 0x106aa070u,
+    0x19a4c116u, 0x1e376c08u, 0x2748774cu, 0x34b0bcb5u, 0x391c0cb3u, 0x4ed8aa4au, 0x5b9cca4fu, 0x682e6ff3u,
+    0x748f82eeu, 0x78a5636fu, 0x84c87814u, 0x8cc70208u, 0x90befffau, 0xa4506cebu, 0xbef9a3f7u, 0xc67178f2u};
+
+static uint32_t ror32(uint32_t x, int n) { return (x >> n) | (x << (32 - n)); }
+
+static void sha256_block(uint32_t h[8], const unsigned char *blk)
+{
+    uint32_t w[64];
+    for (int i = 0; i < 16; ++i)
+        w[i] = ((uint32_t)blk[4 * i] << 24) | ((uint32_t)blk[4 * i + 1] << 16) | ((uint32_t)blk[4 * i + 2] << 8) | blk[4 * i + 3];
+    for (int i = 16; i < 64; ++i) {
+        uint32_t s0 = ror32(w[i - 15], 7) ^ ror32(w[i - 15], 18) ^ (w[i - 15] >> 3);
+        uint32_t s1 = ror32(w[i - 2], 17) ^ ror32(w[i - 2], 19) ^ (w[i - 2] >> 10);
+        w[i] = w[i - 16] + s0 + w[i - 7] + s1;
+    }
+    uint32_t a = h[0], b = h[1], c = h[2], d = h[3], e = h[4], f = h[5], g = h[6], hh = h[7];
+    for (int i = 0; i < 64; ++i) {
+        uint32_t t1 = hh + (ror32(e, 6) ^ ror32(e, 11) ^ ror32(e, 25)) + ((e & f) ^ (~e & g)) + sha_k[i] + w[i];
+        uint32_t t2 = (ror32(a, 2) ^ ror32(a, 13) ^ ror32(a, 22)) + ((a & b) ^ (a & c) ^ (b & c));
+        hh = g; g = f; f = e; e = d + t1; d = c; c = b; b = a; a = t1 + t2;
+    }
+    h[0] += a; h[1] += b; h[2] += c; h[3] += d; h[4] += e; h[5] += f; h[6] += g; h[7] += hh;
+}
+
+void btard_oracle_sha256(const unsigned char *msg, int64_t len, unsigned char out[32])
+{
+    uint32_t h[8] = {0x6a09e667u, 0xbb67ae85u, 0x3c6ef372u, 0xa54ff53au,
+                     0x510e527fu, 0x9b05688cu, 0x1f83d9abu, 0x5be0cd19u};
+    int64_t at = 0;
+    for (; at + 64 <= len; at += 64) sha256_block(h, msg + at);
+    unsigned char tail[128];
+    int64_t rest = len - at;
+    memset(tail, 0, sizeof tail);
+    memcpy(tail, msg + at, (size_t)rest);
+    tail[rest] = 0x80;
+    int blocks = (rest + 1 + 8 <= 64) ? 1 : 2;
+    uint64_t bits = (uint64_t)len * 8u;
+    for (int i = 0; i < 8; ++i) tail[64 * blocks - 1 - i] = (unsigned char)(bits >> (8 * i));
+    for (int b = 0; b < blocks; ++b) sha256_block(h, tail + 64 * b);
+    for (int i = 0; i < 8; ++i) {
+        out[4 * i] = (unsigned char)(h[i] >> 24); out[4 * i + 1] = (unsigned char)(h[i] >> 16);
+        out[4 * i + 2] = (unsigned char)(h[i] >> 8); out[4 * i + 3] = (unsigned char)h[i];
+    }
+}
+
+void btard_oracle_commitment(const float *row, int64_t len, unsigned char out[32])
+{
+    const int64_t bytes = 4 * len, chunk = 4096;
+    const int64_t m = (bytes + chunk - 1) / chunk;
+    unsigned char *cat = (unsigned char *)malloc((size_t)(32 * m + 8));
+    for (int64_t c = 0; c < m; ++c) {
+        int64_t nb = bytes - c * chunk < chunk ? bytes - c * chunk : chunk;
+        btard_oracle_sha256((const unsigned char *)row + c * chunk, nb, cat + 32 * c);
+    }
+    for (int i = 0; i < 8; ++i) cat[32 * m + i] = (unsigned char)((uint64_t)bytes >> (8 * i));
+    btard_oracle_sha256(cat, 32 * m + 8, out);
+    free(cat);
+}
+
 int btard_oracle_max_threads(void)
 {
 #ifdef _OPENMP

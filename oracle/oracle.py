@@ -218,3 +218,26 @@ def preclip(g, lam, part_len=None):
                                          C.byref(nr), C.byref(f))
             norm[p, i], fac[p, i] = nr.value, f.value
     return dict(g=out, row_norm=norm, factor=fac)
+
+
+def sha256(data):
+    """SHA-256 of a bytes object by the oracle's own implementation."""
+    buf = np.frombuffer(bytes(data), dtype=np.uint8).copy() if len(data) else np.zeros(1, np.uint8)
+    out = np.zeros(32, dtype=np.uint8)
+    _load().btard_oracle_sha256(_p(buf, C.c_uint8), C.c_int64(len(data)), _p(out, C.c_uint8))
+    return out.tobytes()
+
+
+def commitment(x, part_len=None):
+    """Tree SHA-256 of every row of x [P][rows][stride] (or [P][stride]): uint8 [P][rows][32]."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    if x.ndim == 2:
+        x = x[:, None, :]
+    P, rows, stride = x.shape
+    ln = _per_part(stride if part_len is None else part_len, P, np.int64)
+    out = np.zeros((P, rows, 32), dtype=np.uint8)
+    lib = _load()
+    for p in range(P):
+        for i in range(rows):
+            lib.btard_oracle_commitment(_p(x[p, i], C.c_float), C.c_int64(int(ln[p])), _p(out[p, i], C.c_uint8))
+    return out

@@ -23,6 +23,7 @@ EXPORTS = [
     "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
     "btard_verify_projections_static", "btard_verification_checks", "btard_preclip_workspace",
     "btard_preclip", "btard_split_gradients", "btard_merge_partitions",
+    "btard_hash_partitions_workspace", "btard_hash_partitions",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -364,6 +365,29 @@ def merge_partitions(v, d, part_offset, part_len, stream=None):
         _check(L.btard_merge_partitions(d, P, stride, off.ctypes.data, ln.ctypes.data, v.data_ptr(),
                                         out.data_ptr(), table.data_ptr(), _stream_ptr(stream)),
                "btard_merge_partitions")
+    return out
+
+
+def hash_partitions(x, part_len=None, stream=None):
+    """Tree SHA-256 commitment of every row of a CUDA float32 tensor [P][rows][row_stride] (g) or
+    [P][row_stride] (v).  Returns a CUDA uint8 tensor [P][rows][32]."""
+    torch = _torch()
+    if x.dim() == 2:
+        x = x.unsqueeze(1)
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 3 and x.is_contiguous()
+    P, rows, stride = x.shape
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    L = lib()
+    L.btard_hash_partitions_workspace.restype = C.c_size_t
+    L.btard_hash_partitions_workspace.argtypes = [C.c_int32, C.c_int32, C.c_int64]
+    L.btard_hash_partitions.restype = C.c_int
+    L.btard_hash_partitions.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_size_t, C.c_void_p]
+    ws = torch.empty(int(L.btard_hash_partitions_workspace(P, rows, stride)), dtype=torch.uint8, device=x.device)
+    out = torch.empty((P, rows, 32), dtype=torch.uint8, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(L.btard_hash_partitions(P, rows, stride, ln.ctypes.data, x.data_ptr(), out.data_ptr(),
+                                       ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "btard_hash_partitions")
     return out
 
 

@@ -479,6 +479,33 @@ int btard_merge_partitions(int64_t d, int32_t P, int64_t stride, const int64_t* 
     return launch_merge(v, out, table, stride, P, (cudaStream_t)stream);
 }
 
+size_t btard_hash_partitions_workspace(int32_t P, int32_t rows_per_part, int64_t stride)
+{
+    if (P < 1 || rows_per_part < 1 || stride < 1) return 0;
+    return align_up(sizeof(PartEntry) * (size_t)P, 256) +
+           align_up(sizeof(uint32_t) * 8 * (size_t)P * rows_per_part * hash_max_leaves(stride), 256);
+}
+
+int btard_hash_partitions(int32_t P, int32_t rows_per_part, int64_t stride, const int64_t* part_len,
+                          const float* x, uint8_t* digests, void* workspace, size_t workspace_bytes,
+                          void* stream)
+{
+    if (P < 1 || rows_per_part < 1 || stride < 1 || !part_len || !x || !digests || !workspace)
+        return BTARD_ERR_INVALID_ARG;
+    if ((long long)P * rows_per_part > 0x7fffffffLL / 2) return BTARD_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return BTARD_ERR_BAD_ALIGNMENT;
+    if (workspace_bytes < btard_hash_partitions_workspace(P, rows_per_part, stride)) return BTARD_ERR_WORKSPACE_TOO_SMALL;
+    std::vector<double> zeros((size_t)P, 0.0);
+    for (int p = 0; p < P; ++p)
+        if (part_len[p] < 0 || part_len[p] > stride) return BTARD_ERR_INVALID_ARG;
+    char* base = (char*)workspace;
+    int rc = upload_table((PartEntry*)base, P, part_len, zeros.data(), (cudaStream_t)stream);
+    if (rc != BTARD_OK) return rc;
+    uint32_t* leaves = (uint32_t*)(base + align_up(sizeof(PartEntry) * (size_t)P, 256));
+    return launch_hash_rows(x, (const PartEntry*)base, leaves, digests, stride, rows_per_part,
+                            P * rows_per_part, (cudaStream_t)stream);
+}
+
 size_t btard_preclip_workspace(const btard_preclip_args* a)
 {
     if (!a || a->n_peers < 1 || a->n_peers > BTARD_MAX_PEERS || a->n_partitions < 1 || a->row_stride < 4)

@@ -142,6 +142,11 @@ int launch_split(const float* grads, float* g, const void* table_dev, long long 
                  int n, int P, cudaStream_t st);
 int launch_merge(const float* v, float* out, const void* table_dev, long long stride, int P, cudaStream_t st);
 
+// ---- commitments (btard_hash.cu): tree SHA-256 of every row of a [rows][stride] tensor ----------
+int hash_max_leaves(long long stride);
+int launch_hash_rows(const float* x, const PartEntry* table, uint32_t* leaves, unsigned char* out,
+                     long long stride, int rows_per_part, int rows, cudaStream_t st);
+
 // ---- verification (btard_verify.cu) -------------------------------------------------------------
 struct VerifyLaunch {
     const float* g;

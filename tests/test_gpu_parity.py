@@ -291,6 +291,26 @@ def test_split_and_merge_are_exact_copies(n, d, P, mode):
         assert np.array_equal(out[off[p]:off[p] + ln[p]], cpu(v)[p, :ln[p]])
 
 
+# ----------------------------------------------------------------------------- commitments
+@pytest.mark.parametrize("rows,stride,lens", [(4, 1024, [1024]), (16, 100_000, [100_000, 99_973, 1]),
+                                               (3, 2048, [2047, 1025, 0, 14]), (1, 698_400, [698_373, 698_367])])
+def test_commitments_are_bit_exact(rows, stride, lens):
+    rng = np.random.default_rng(stride + rows)
+    P = len(lens)
+    x = rng.standard_normal((P, rows, stride)).astype(np.float32)
+    ref = oracle.commitment(x, np.array(lens))
+    out = cpu(btard.hash_partitions(torch.from_numpy(x).cuda(), np.array(lens)))
+    assert np.array_equal(out, ref)
+
+
+def test_commitment_of_an_aggregate_changes_with_one_bit():
+    v = torch.randn((2, 4096), device="cuda")
+    a = cpu(btard.hash_partitions(v))
+    v2 = v.clone(); v2[1, 4095] = torch.nextafter(v2[1, 4095], torch.tensor(10.0, device="cuda"))
+    b = cpu(btard.hash_partitions(v2))
+    assert np.array_equal(a[0], b[0]) and not np.array_equal(a[1], b[1])
+
+
 # ----------------------------------------------------------------------------- Clipped-SGD pre-clip
 @pytest.mark.parametrize("n,stride", [(4, 1024), (16, 100_000), (64, 5024)])
 def test_preclip_matches_oracle(n, stride):

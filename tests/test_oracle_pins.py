@@ -555,3 +555,38 @@ def test_preclip_closed_forms():
     bad = g.copy(); bad[0, 2, 5] = np.nan
     out = oracle.preclip(bad, 3.0, part_len=lens)
     assert out["factor"][0, 2] == 0.0 and np.all(out["g"][0, 2] == 0)
+
+
+# ----------------------------------------------------------------------------- commitments
+def test_sha256_against_published_answers_and_hashlib():
+    """FIPS 180-4 examples ("abc", the empty message, the 448-bit message) and hashlib on messages whose
+    lengths straddle every padding case."""
+    import hashlib
+    assert oracle.sha256(b"abc").hex() == "ba7816bf8f01cfea414140de5dae2223b00361a396177a9cb410ff61f20015ad"
+    assert oracle.sha256(b"").hex() == "e3b0c44298fc1c149afbf4c8996fb92427ae41e4649b934ca495991b7852b855"
+    assert oracle.sha256(b"abcdbcdecdefdefgefghfghighijhijkijkljklmklmnlmnomnopnopq").hex() == \
+        "248d6a61d20638b8e5c026930c3e6039a33ce45964ff2167f6ecedd419db06c1"
+    rng = np.random.default_rng(40)
+    for n in (1, 3, 55, 56, 57, 63, 64, 65, 119, 120, 128, 4095, 4096, 4097, 100_000):
+        m = rng.integers(0, 256, n, dtype=np.uint8).tobytes()
+        assert oracle.sha256(m) == hashlib.sha256(m).digest(), n
+
+
+def test_commitment_is_the_stated_tree_of_sha256():
+    import hashlib
+    rng = np.random.default_rng(41)
+    x = rng.standard_normal((2, 3, 2600)).astype(np.float32)
+    lens = np.array([2600, 1023])
+    out = oracle.commitment(x, lens)
+    for p in range(2):
+        for i in range(3):
+            raw = x[p, i, :lens[p]].tobytes()
+            cat = b"".join(hashlib.sha256(raw[o:o + 4096]).digest() for o in range(0, len(raw), 4096))
+            assert out[p, i].tobytes() == hashlib.sha256(cat + len(raw).to_bytes(8, "little")).digest()
+    empty = oracle.commitment(x[:1, :1], np.array([0]))
+    assert empty[0, 0].tobytes() == hashlib.sha256((0).to_bytes(8, "little")).digest()
+    # a one-bit change anywhere, or padding content, must / must not change the commitment
+    y = x.copy(); y[1, 2, 1022] = np.nextafter(y[1, 2, 1022], np.float32(10))
+    z = x.copy(); z[1, 2, 1023:] = 7.0
+    assert not np.array_equal(oracle.commitment(y, lens)[1, 2], out[1, 2])
+    assert np.array_equal(oracle.commitment(z, lens), out)
