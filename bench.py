@@ -145,7 +145,8 @@ def run_ours(args):
     P, n, stride = g.shape
     dev = g.device
     algo = {"direct": btard.ALGO_DIRECT, "gram": btard.ALGO_GRAM,
-            "cooperative": btard.ALGO_DIRECT_COOPERATIVE, "resident": btard.ALGO_DIRECT_RESIDENT}[args.algo]
+            "cooperative": btard.ALGO_DIRECT_COOPERATIVE, "resident": btard.ALGO_DIRECT_RESIDENT,
+            "staged": btard.ALGO_DIRECT_STAGED}[args.algo]
     ws_c = torch.empty(btard.centered_clip_workspace(n, P, stride, w.stop_mode, algo), dtype=torch.uint8, device=dev)
     ws_v = torch.empty(btard.verify_projections_workspace(n, P, stride, w.K), dtype=torch.uint8, device=dev)
     v = torch.empty((P, stride), dtype=torch.float32, device=dev)
@@ -400,7 +401,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--algo", default="direct", choices=["direct", "gram", "cooperative", "resident"])
+    ap.add_argument("--algo", default="direct", choices=["direct", "gram", "cooperative", "resident", "staged"])
     ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not bracket the library's kernels with CUDA events (no roofline object)")

@@ -63,6 +63,11 @@ extern "C" {
                                        after the last partition converged; where the device cannot
                                        launch it: DIRECT                                            */
 
+#define BTARD_ALGO_DIRECT_STAGED 4  /* as DIRECT, but for n_peers <= 16 and row_stride a multiple of 32
+                                       the update pass is fed by bulk asynchronous copies through a
+                                       ring of shared-memory stages instead of loads into registers;
+                                       other shapes: DIRECT                                         */
+
 /* Aggregation rule.  The paper's experiments (Sec. 4.1) compare CenteredClip with plain averaging,
    the coordinate-wise median and the geometric median; they run on the same streaming kernels. */
 #define BTARD_RULE_CENTERED_CLIP 0     /* App. D.2 eq. (CenteredClip)                                 */

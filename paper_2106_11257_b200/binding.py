@@ -10,7 +10,7 @@ import os
 import numpy as np
 
 INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
-ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT, ALGO_DIRECT_COOPERATIVE = 0, 1, 2, 3
+ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT, ALGO_DIRECT_COOPERATIVE, ALGO_DIRECT_STAGED = 0, 1, 2, 3, 4
 STOP_FIXED_ITERS, STOP_EPS = 0, 1
 RULE_CENTERED_CLIP, RULE_GEOMETRIC_MEDIAN, RULE_MEAN, RULE_COORD_MEDIAN = 0, 1, 2, 3
 SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1

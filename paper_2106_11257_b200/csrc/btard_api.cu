@@ -96,13 +96,16 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, in
     CclipWorkspace w{};
     size_t off = 0;
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
-    w.slots = off; off = align_up(off + sizeof(double) * (size_t)P * geo.cpp * (n + 1), 256);
+    const bool gram = (algo == BTARD_ALGO_GRAM);
+    const bool comp = (stop_mode == BTARD_STOP_EPS && !gram);
+    const StagedGeometry sg = cclip_staged_geometry(n, P, stride, comp);
+    const int cpp = (sg.ok && sg.g.cpp > geo.cpp) ? sg.g.cpp : geo.cpp;
+    w.slots = off; off = align_up(off + sizeof(double) * (size_t)P * cpp * (n + 1), 256);
     w.tot[0] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
     w.tot[1] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
     w.flags_bytes = sizeof(int) * (3 * (size_t)P + 1);        // done[P], ticket[P], Gram ticket[P], error
     w.flags = off; off = align_up(off + w.flags_bytes, 256);
-    const bool gram = (algo == BTARD_ALGO_GRAM);
-    w.v_lo_bytes = (stop_mode == BTARD_STOP_EPS && !gram) ? sizeof(unsigned short) * (size_t)P * stride : 0;
+    w.v_lo_bytes = comp ? sizeof(unsigned short) * (size_t)P * stride : 0;
     w.v_lo = off; off = align_up(off + w.v_lo_bytes, 256);
     if (gram && n <= kMaxGramPeers) {
         const GramGeometry gg = gram_geometry(n, P, stride);
@@ -226,7 +229,8 @@ int btard_centered_clip(const btard_cclip_args* a)
     if (a->stop_mode != BTARD_STOP_FIXED_ITERS && a->stop_mode != BTARD_STOP_EPS)
         return BTARD_ERR_INVALID_ARG;
     if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM &&
-        a->algo != BTARD_ALGO_DIRECT_RESIDENT && a->algo != BTARD_ALGO_DIRECT_COOPERATIVE)
+        a->algo != BTARD_ALGO_DIRECT_RESIDENT && a->algo != BTARD_ALGO_DIRECT_COOPERATIVE &&
+        a->algo != BTARD_ALGO_DIRECT_STAGED)
         return BTARD_ERR_INVALID_ARG;
     if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (a->rule < BTARD_RULE_CENTERED_CLIP || a->rule > BTARD_RULE_COORD_MEDIAN) return BTARD_ERR_INVALID_ARG;
@@ -369,9 +373,11 @@ int btard_centered_clip(const btard_cclip_args* a)
     if (rc != BTARD_OK) return rc;
 
     // Update l reads the totals in buffer l % 2 and writes buffer (l + 1) % 2.
+    StagedGeometry sg = cclip_staged_geometry(n, P, a->row_stride, L.v_lo != nullptr);
+    if (a->algo != BTARD_ALGO_DIRECT_STAGED) sg.ok = 0;
     for (int l = 0; l < a->max_iters; ++l) {
         L.l = l; L.tot_in = tot[l & 1]; L.tot_out = tot[(l + 1) & 1];
-        rc = launch_cclip_pass(L, geo, PASS_ITER, st);
+        rc = sg.ok ? launch_cclip_staged(L, sg, st) : launch_cclip_pass(L, geo, PASS_ITER, st);
         if (rc != BTARD_OK) return rc;
     }
     L.tot_in = tot[a->max_iters & 1];

@@ -36,6 +36,12 @@ __device__ __forceinline__ uint64_t policy_evict_first()
     return pol;
 }
 
+__device__ __forceinline__ uint64_t policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
 __device__ __forceinline__ double warp_sum(double x)
 {
 #pragma unroll
@@ -89,21 +95,21 @@ struct KernelArgs {
 };
 
 // Records the end state of a partition (called by one CTA of it).
-__device__ void finish_partition(const KernelArgs& k, int p, const double* sums, int iters_done,
+__device__ void finish_partition(const CclipLaunch& a, int p, const double* sums, int iters_done,
                                  bool eps_mode)
 {
-    const int n = k.a.n;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) k.a.resid_norm[(size_t)p * n + i] = sqrt(sums[i]);
+    const int n = a.n;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) a.resid_norm[(size_t)p * n + i] = sqrt(sums[i]);
     if (threadIdx.x == 0) {
         const double step2 = sums[n];
-        k.a.iters[p] = iters_done;
-        k.a.last_step[p] = sqrt(step2);
+        a.iters[p] = iters_done;
+        a.last_step[p] = sqrt(step2);
         unsigned st = 0;
         for (int i = 0; i < n; ++i)
             if (!isfinite(sums[i])) st |= BTARD_STATUS_NONFINITE_ROW;
-        if (eps_mode && !(step2 <= k.a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
-        atomicOr(&k.a.status[p], st);
-        k.a.done[p] = 1;
+        if (eps_mode && !(step2 <= a.eps2)) st |= BTARD_STATUS_NOT_CONVERGED;
+        atomicOr(&a.status[p], st);
+        a.done[p] = 1;
     }
 }
 
@@ -125,6 +131,41 @@ __device__ __forceinline__ void two_sum_bf16(float v, float s, float& hi, float&
     lo = bf16_value(lo_bits);
 }
 
+// Two fp32 values in one 64-bit register, and the packed arithmetic on them.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// 128-bit loads as two packed pairs: read-only rows with an eviction policy; v with a policy.
+__device__ __forceinline__ void ld_row_pairs(const float* p, uint64_t policy, uint64_t& lo, uint64_t& hi)
+{
+    asm volatile("ld.global.nc.L2::cache_hint.v2.b64 {%0, %1}, [%2], %3;" : "=l"(lo), "=l"(hi) : "l"(p), "l"(policy));
+}
+
 // COMP (PASS_ITER only): v is carried as hi + lo, hi the fp32 output vector and lo a bf16 correction
 // in the workspace, so that the update and the stop test do not drown in the rounding of v.
 template <int R, int MODE, bool COMP>
@@ -136,6 +177,8 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     __shared__ double sh_red[16][17];
     __shared__ double sh_part[512 + BTARD_MAX_PEERS + 1];
     __shared__ int sh_flag;
+    __shared__ float sh_wsum;                         // sum of the clip weights (PASS_ITER)
+    __shared__ __align__(8) float2 sh_w2[(MODE == PASS_ITER) ? BTARD_MAX_PEERS + 16 : 1];   // (w_i, w_i)
 
     const CclipLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
@@ -158,13 +201,19 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         __syncthreads();
         const bool converged = (a.stop_mode == BTARD_STOP_EPS) && a.l >= 1 && (sh_sum[n] <= a.eps2);
         if (converged) {                              // same decision in every CTA of the partition
-            if (j == 0) finish_partition(k, p, sh_sum, a.l, true);
+            if (j == 0) finish_partition(k.a, p, sh_sum, a.l, true);
             return;
         }
         if (tid == 0) sh_flag = 0;
         __syncthreads();
         row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, sh_part);
-        if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+        if (tid == 0) {
+            float w = 0.0f;
+            for (int i = 0; i < n; ++i) w += sh_w[i];
+            sh_wsum = w;
+            if (j == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+        }
+        __syncthreads();
     } else if (MODE == PASS_COMBINE) {
         // v = v0 + sum_i a_i (x_i - v0): the update formula with weights n a_i.
         for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x)
@@ -175,6 +224,12 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     }
     (void)tau;
     const float* wrow = sh_w + rg * R;                // this thread's R clip weights
+    bool skip_rows = false;                           // some row has weight 0 and must be left out
+    if (MODE == PASS_ITER) {
+        for (int i = tid; i < BTARD_MAX_PEERS + 16; i += blockDim.x) sh_w2[i] = make_float2(sh_w[i], sh_w[i]);
+        skip_rows = sh_flag != 0;
+        __syncthreads();
+    }
 
     float acc[R];
 #pragma unroll
@@ -193,6 +248,10 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     if (j + 1 < cpp) q1 &= ~7LL;
     const long long full_quads = len >> 2;             // quads that lie entirely inside the data
 
+    // v is read and written by every update pass: its loads ask L2 to keep the lines and its stores are
+    // marked streaming (measured: fewer DRAM bytes and a shorter pass than with default accesses).
+    constexpr bool KEEPV = (MODE == PASS_ITER);
+    const uint64_t keep = policy_evict_last();
     // One tile: CL quads starting at quad qb.  MASKED = false when every lane's quad is inside both
     // the CTA's range and the data, so no predicate is needed.
     auto tile = [&](auto masked_tag, long long qb, int parity, uint64_t policy) {
@@ -210,10 +269,14 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
                 const int i = rg * R + r;
                 x[r] = (i < n) ? ld_policy(gp + (size_t)i * stride + col, policy) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            if (MODE != PASS_INIT || a.init_mode == BTARD_INIT_CALLER_V0)
-                v4 = *reinterpret_cast<const float4*>(vp + col);
+            if (MODE != PASS_INIT || a.init_mode == BTARD_INIT_CALLER_V0) {
+                if (KEEPV) asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;" : "=f"(v4.x), "=f"(v4.y), "=f"(v4.z), "=f"(v4.w) : "l"(vp + col), "l"(keep));
+                else v4 = *reinterpret_cast<const float4*>(vp + col);
+            }
             if (COMP) {
-                const uint2 lb = *reinterpret_cast<const uint2*>(lop + col);
+                uint2 lb;
+                if (KEEPV) asm volatile("ld.global.L2::cache_hint.v2.u32 {%0, %1}, [%2], %3;" : "=r"(lb.x), "=r"(lb.y) : "l"(lop + col), "l"(keep));
+                else lb = *reinterpret_cast<const uint2*>(lop + col);
                 lo4 = make_float4(bf16_value(lb.x & 0xFFFFu), bf16_value(lb.x >> 16),
                                   bf16_value(lb.y & 0xFFFFu), bf16_value(lb.y >> 16));
             }
@@ -270,8 +333,10 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
                     if (!m3) b3 = 0;
                     dv = make_float4((vn.x - v4.x) + (ln.x - lo4.x), (vn.y - v4.y) + (ln.y - lo4.y),
                                      (vn.z - v4.z) + (ln.z - lo4.z), (vn.w - v4.w) + (ln.w - lo4.w));
-                    if (rg == 0 && valid)
-                        *reinterpret_cast<uint2*>(lop + col) = make_uint2(b0 | (b1 << 16), b2 | (b3 << 16));
+                    if (rg == 0 && valid) {
+                        if (KEEPV) __stcs(reinterpret_cast<uint2*>(lop + col), make_uint2(b0 | (b1 << 16), b2 | (b3 << 16)));
+                        else *reinterpret_cast<uint2*>(lop + col) = make_uint2(b0 | (b1 << 16), b2 | (b3 << 16));
+                    }
                 } else {
                     vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
                     dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
@@ -289,7 +354,10 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         if (!m1) vn.y = 0.f;
         if (!m2) vn.z = 0.f;
         if (!m3) vn.w = 0.f;
-        if (MODE != PASS_NORMS && rg == 0 && valid) *reinterpret_cast<float4*>(vp + col) = vn;
+        if (MODE != PASS_NORMS && rg == 0 && valid) {
+            if (KEEPV) __stcs(reinterpret_cast<float4*>(vp + col), vn);
+            else *reinterpret_cast<float4*>(vp + col) = vn;
+        }
         if (MODE == PASS_INIT) dv = vn;                // x still holds the rows themselves
 
 #pragma unroll
@@ -300,6 +368,88 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
     };
 
+    // Interior tile of an update pass when no row has to be left out: the same update on (column,
+    // column + 1) pairs with the packed fp32 instructions of sm_100 (add/sub/mul/fma .f32x2, the IEEE
+    // results of two scalar operations each).  d = x - v_hi; s += w d; r = d - e with e = v_lo + (move
+    // of v).  The low-order part of v enters the column sums once, as -v_lo * sum_i w_i.
+    auto fast_tile = [&](long long qb, int parity, uint64_t policy) {
+        const long long col = (qb + cl) * 4;
+        uint64_t xa[R], xb[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int i = rg * R + r;
+            if (i < n) ld_row_pairs(gp + (size_t)i * stride + col, policy, xa[r], xb[r]);
+            else { xa[r] = 0ull; xb[r] = 0ull; }
+        }
+        float4 v4;
+        asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                     : "=f"(v4.x), "=f"(v4.y), "=f"(v4.z), "=f"(v4.w) : "l"(vp + col), "l"(keep));
+        float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (COMP) {
+            uint2 lb;
+            asm volatile("ld.global.L2::cache_hint.v2.u32 {%0, %1}, [%2], %3;" : "=r"(lb.x), "=r"(lb.y) : "l"(lop + col), "l"(keep));
+            lo4 = make_float4(bf16_value(lb.x & 0xFFFFu), bf16_value(lb.x >> 16),
+                              bf16_value(lb.y & 0xFFFFu), bf16_value(lb.y >> 16));
+        }
+        const uint64_t va = pack2(v4.x, v4.y), vb = pack2(v4.z, v4.w);
+        uint64_t sa = 0ull, sb = 0ull;
+        const uint64_t* w2 = reinterpret_cast<const uint64_t*>(sh_w2) + rg * R;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            xa[r] = sub2(xa[r], va);
+            xb[r] = sub2(xb[r], vb);
+            const uint64_t w = w2[r];
+            sa = fma2(w, xa[r], sa);
+            sb = fma2(w, xb[r], sb);
+        }
+        float4 s4;
+        unpack2(sa, s4.x, s4.y);
+        unpack2(sb, s4.z, s4.w);
+        if (RG > 1) {                                  // add the row groups' partial column sums
+            float4* buf = sh_x + (size_t)parity * RG * CL;
+            buf[rg * CL + cl] = s4;
+            __syncthreads();
+            s4 = buf[cl];
+            for (int q = 1; q < RG; ++q) {
+                const float4 o = buf[q * CL + cl];
+                s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
+            }
+        }
+        if (COMP) {
+            const float nw = -sh_wsum;
+            s4.x = fmaf(nw, lo4.x, s4.x); s4.y = fmaf(nw, lo4.y, s4.y);
+            s4.z = fmaf(nw, lo4.z, s4.z); s4.w = fmaf(nw, lo4.w, s4.w);
+        }
+        const float4 u = make_float4(s4.x * inv_n, s4.y * inv_n, s4.z * inv_n, s4.w * inv_n);
+        float4 vn, e4;                                 // new v_hi; v_lo + what the represented v moved by
+        if (COMP) {
+            uint32_t b0, b1, b2, b3;
+            float4 ln;
+            two_sum_bf16(v4.x, lo4.x + u.x, vn.x, ln.x, b0);
+            two_sum_bf16(v4.y, lo4.y + u.y, vn.y, ln.y, b1);
+            two_sum_bf16(v4.z, lo4.z + u.z, vn.z, ln.z, b2);
+            two_sum_bf16(v4.w, lo4.w + u.w, vn.w, ln.w, b3);
+            e4 = make_float4((vn.x - v4.x) + ln.x, (vn.y - v4.y) + ln.y, (vn.z - v4.z) + ln.z, (vn.w - v4.w) + ln.w);
+            if (rg == 0) __stcs(reinterpret_cast<uint2*>(lop + col), make_uint2(b0 | (b1 << 16), b2 | (b3 << 16)));
+        } else {
+            vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+            e4 = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
+        }
+        if (rg == 0) {
+            step_acc += (u.x * u.x + u.y * u.y) + (u.z * u.z + u.w * u.w);
+            __stcs(reinterpret_cast<float4*>(vp + col), vn);
+        }
+        const uint64_t ea = pack2(e4.x, e4.y), eb = pack2(e4.z, e4.w);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {                  // residuals at the new v
+            const uint64_t da = sub2(xa[r], ea), db = sub2(xb[r], eb);
+            const uint64_t q2 = fma2(db, db, mul2(da, da));
+            float q0f, q1f;
+            unpack2(q2, q0f, q1f);
+            acc[r] += q0f + q1f;
+        }
+    };
+
     // The rows are marked evict-first in L2: nothing is read twice within a pass, and what is
     // still resident when the next pass starts (it starts where this one ends) is a bonus.
     // Measured: pinning the tail with evict-last instead was slower for every budget tried.
@@ -307,8 +457,14 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const uint64_t pol = policy_evict_first();
     for (long long t = 0; t < ntiles; ++t) {
         const long long qb = q0 + (rev ? ntiles - 1 - t : t) * CL;
-        if (qb + CL <= q1 && qb + CL <= full_quads) tile(std::false_type{}, qb, (int)(t & 1), pol);
-        else tile(std::true_type{}, qb, (int)(t & 1), pol);
+        const bool inner = (qb + CL <= q1 && qb + CL <= full_quads);
+        if (MODE == PASS_ITER) {
+            if (inner && !skip_rows) fast_tile(qb, (int)(t & 1), pol);
+            else tile(std::true_type{}, qb, (int)(t & 1), pol);
+        } else {
+            if (inner) tile(std::false_type{}, qb, (int)(t & 1), pol);
+            else tile(std::true_type{}, qb, (int)(t & 1), pol);
+        }
     }
 
     // CTA reduction: lanes of a warp share a row group, so a warp reduces R rows at once.
@@ -348,6 +504,346 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     int groups = blockDim.x / per;
     if (groups < 1) groups = 1;
     if (groups > cpp) groups = cpp;
+    for (int e = tid; e < groups * per; e += blockDim.x) {
+        const int cg = e / per, i = e - cg * per;
+        double s = 0.0;
+        for (int c = cg; c < cpp; c += groups) s += __ldcg(slots + (size_t)c * per + i);
+        sh_part[e] = s;
+    }
+    __syncthreads();
+    double* tot = a.tot_out + (size_t)p * per;
+    for (int i = tid; i < per; i += blockDim.x) {
+        double s = 0.0;
+        for (int cg = 0; cg < groups; ++cg) s += sh_part[cg * per + i];
+        tot[i] = s;
+    }
+    if (tid == 0) a.ticket[p] = 0;
+}
+
+// =================================================================================================
+// Staged iteration pass for n <= 16 (all rows of a column in one thread).  Same update as
+// cclip_pass_kernel<R, PASS_ITER, COMP>, but the rows reach the SM through bulk asynchronous copies
+// (one per row and tile, plus v and its low-order part) into a ring of shared-memory stages.  Per
+// stage an mbarrier counts the bytes that landed and a counter the warps that have moved their part
+// of the tile into registers; the warp that arrives last refills the stage with the tile S steps
+// ahead.  No CTA-wide barrier sits inside the loop, and the bytes in flight do not depend on the
+// registers of the threads.  Every wait is bounded; a wait that runs out sets
+// BTARD_STATUS_WAIT_EXPIRED, all loops end, and the CTA goes on to its epilogue.
+//
+// A consumer thread owns 2 columns and works on (column, column + 1) pairs with the packed fp32
+// instructions of sm_100 (add/sub/mul/fma .f32x2: the same IEEE results as two scalar operations).
+// Per element: d = x - v_hi; s += w d; r = d - e with e = v_lo + (move of v); |r|^2.  The low-order
+// part of v enters the column sum once, as -v_lo * sum_i w_i.
+// =================================================================================================
+constexpr int kMaxStages = 4;
+constexpr unsigned kStageWaitLimit = 1u << 22;
+constexpr int kStagedConsumerWarps = 8;
+constexpr int kStagedThreads = 32 * kStagedConsumerWarps;
+constexpr int kStagedMaxTilesPerCta = 128;        // a thread's fp32 running sums get one term per tile
+constexpr int kStagedTileQuads = 16 * kStagedConsumerWarps;      // 2 columns per consumer thread: 128 quads
+
+struct StagedArgs {
+    CclipLaunch a;
+    int cpp, stages;
+    unsigned stage_bytes;           // multiple of 128
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
+{
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// false: the wait ran out (or another warp's did: give_up, when given, points at a non-zero flag)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity, const volatile int* give_up)
+{
+    for (unsigned spins = 0; spins < kStageWaitLimit; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 1023u) == 1023u && give_up && *give_up) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_load_hint(void* dst, const void* src, unsigned bytes, uint64_t* bar, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy) : "memory");
+}
+
+template <int R, bool COMP>
+__global__ void __launch_bounds__(kStagedThreads, 2) cclip_iter_staged_kernel(const StagedArgs k)
+{
+    extern __shared__ __align__(128) unsigned char sh_raw[];   // the stages
+    __shared__ double sh_sum[BTARD_MAX_PEERS + 1];             // totals in; slot sums of the last CTA out
+    __shared__ float sh_w[BTARD_MAX_PEERS + 16];
+    __shared__ __align__(8) float2 sh_w2[16];                  // (w_i, w_i)
+    __shared__ double sh_red[16][17];
+    __shared__ __align__(8) uint64_t sh_full[kMaxStages];
+    __shared__ int sh_taken[kMaxStages];                       // warps that hold their part of the stage's tile
+    __shared__ int sh_flag, sh_expired, sh_issued;
+    __shared__ float sh_wsum;
+
+    const CclipLaunch& a = k.a;
+    constexpr int CL = kStagedTileQuads;
+    const int n = a.n, cpp = k.cpp, S = k.stages;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool rev = (a.l & 1) == 0;
+    const int bid = rev ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+    const int p = bid / cpp, j = bid % cpp;
+    const long long stride = a.stride;
+
+    if (a.done[p]) return;
+
+    const float* gp = a.g + (size_t)p * n * stride;
+    float* vp = a.v + (size_t)p * stride;
+    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
+    const float inv_n = 1.0f / (float)n;
+
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cpp) q1 &= ~7LL;
+    const int ntiles = (int)((q1 - q0 + CL - 1) / CL);
+    constexpr unsigned row_bytes = (unsigned)CL * 16u;    // one row of a full tile
+    const uint64_t pol = policy_evict_first();
+    // v is read and written by every pass: its loads ask L2 to keep the lines, its stores are marked
+    // streaming (measured: 7 us per pass faster than default or evict-last stores of the same lines).
+    const uint64_t keep = policy_evict_last();
+    const volatile int* give_up = &sh_expired;
+
+    // One warp fills stage (t % S) with tile t of the sweep: n rows, v and (COMP) the bf16 part.
+    auto issue = [&](int t) {
+        const long long qb = q0 + (long long)(rev ? ntiles - 1 - t : t) * CL;
+        const long long rest = q1 - qb;
+        const unsigned nq = (unsigned)(rest < CL ? rest : CL);
+        unsigned char* st = sh_raw + (size_t)(t % S) * k.stage_bytes;
+        uint64_t* bar = &sh_full[t % S];
+        if (lane == 0) {
+            const unsigned total = nq * 16u * (unsigned)(n + 1) + (COMP ? nq * 8u : 0u);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(total) : "memory");
+        }
+        __syncwarp();
+        if (lane < n) bulk_load_hint(st + (size_t)lane * row_bytes, gp + (size_t)lane * stride + qb * 4, nq * 16u, bar, pol);
+        else if (lane == n) bulk_load_hint(st + (size_t)n * row_bytes, vp + qb * 4, nq * 16u, bar, keep);
+        else if (COMP && lane == n + 1) bulk_load_hint(st + (size_t)(n + 1) * row_bytes, lop + qb * 4, nq * 8u, bar, keep);
+        __syncwarp();
+    };
+
+    // The first copies leave before anything else is read, so that the totals, the stop test and the
+    // clip weights below overlap with their flight.
+    if (warp == 0) {
+        if (lane == 0) {
+            sh_flag = 0; sh_expired = 0;
+            for (int s = 0; s < S; ++s) {
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&sh_full[s])));
+                sh_taken[s] = 0;
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        int issued = 0;
+        for (; issued < S && issued < ntiles; ++issued) issue(issued);
+        if (lane == 0) sh_issued = issued;
+    }
+    {
+        const double* src = a.tot_in + (size_t)p * (n + 1);
+        for (int i = tid; i <= n; i += blockDim.x) sh_sum[i] = __ldcg(src + i);
+        __syncthreads();
+        const bool converged = (a.stop_mode == BTARD_STOP_EPS) && a.l >= 1 && (sh_sum[n] <= a.eps2);
+        if (converged) {                              // same decision in every CTA of the partition
+            // the copies already issued must have landed before the CTA gives its shared memory back
+            if (tid < S && tid < ntiles) (void)mbar_wait_bounded(&sh_full[tid], 0u, nullptr);
+            __syncthreads();
+            if (j == 0) finish_partition(a, p, sh_sum, a.l, true);
+            return;
+        }
+    }
+    const long long len = a.table[p].len;
+    const double tau = a.table[p].tau;
+    const long long full_quads = len >> 2;
+
+    // Clip weights of this update (the first copies are already on their way).
+    row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, &sh_red[0][0]);
+    if (tid < 16) sh_w2[tid] = make_float2(sh_w[tid], sh_w[tid]);
+    if (tid == 0) {
+        float w = 0.0f;
+        for (int i = 0; i < n; ++i) w += sh_w[i];
+        sh_wsum = w;
+        if (j == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+    }
+    __syncthreads();
+    const bool skip_rows = sh_flag != 0;              // some row has a non-finite norm: leave it out
+    const float wsum = sh_wsum;
+
+    uint64_t acc2[R];                                 // per row: squared residuals of the two columns
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc2[r] = 0ull;
+    float step_acc = 0.0f;
+
+    {
+        const int ct = tid;                           // consumer thread: columns 2 ct, 2 ct + 1 of the tile
+        for (int t = 0; t < ntiles; ++t) {
+            const int s = t % S;
+            const long long qb = q0 + (long long)(rev ? ntiles - 1 - t : t) * CL;
+            const unsigned char* st = sh_raw + (size_t)s * k.stage_bytes;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&sh_full[s], (unsigned)((t / S) & 1), give_up));
+            if (!ok) { if (lane == 0) sh_expired = 1; break; }
+            const long long col = qb * 4 + 2 * ct;
+            const bool fast = !skip_rows && (qb + CL <= q1) && (qb + CL <= full_quads);
+            uint64_t x2[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                x2[r] = (r < n) ? reinterpret_cast<const uint64_t*>(st + (size_t)r * row_bytes)[ct] : 0ull;
+            const uint64_t v2 = reinterpret_cast<const uint64_t*>(st + (size_t)n * row_bytes)[ct];
+            uint32_t lob = 0;
+            if (COMP) lob = reinterpret_cast<const uint32_t*>(st + (size_t)(n + 1) * row_bytes)[ct];
+            // This warp's part of the tile is in registers.  The last warp to say so refills the stage.
+            __syncwarp();
+            int before = 0;
+            if (lane == 0) {
+                __threadfence_block();
+                before = atomicAdd(&sh_taken[s], 1);
+            }
+            before = __shfl_sync(0xffffffffu, before, 0);
+            if (before == kStagedConsumerWarps - 1 && t + S < ntiles) {
+                if (lane == 0) {
+                    sh_taken[s] = 0;
+                    atomicMax(&sh_issued, t + S + 1);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                issue(t + S);
+            }
+
+            float vx, vy;
+            unpack2(v2, vx, vy);
+            const float lx = bf16_value(lob & 0xFFFFu), ly = bf16_value(lob >> 16);
+            if (fast) {
+                uint64_t s2 = 0ull, t2 = 0ull;         // even and odd rows: two shorter dependency chains
+#pragma unroll
+                for (int r = 0; r < R; r += 2) {
+                    x2[r] = sub2(x2[r], v2);
+                    x2[r + 1] = sub2(x2[r + 1], v2);
+                    s2 = fma2(*reinterpret_cast<const uint64_t*>(&sh_w2[r]), x2[r], s2);
+                    t2 = fma2(*reinterpret_cast<const uint64_t*>(&sh_w2[r + 1]), x2[r + 1], t2);
+                }
+                float ux, uy, tx, ty;
+                unpack2(s2, ux, uy);
+                unpack2(t2, tx, ty);
+                ux += tx; uy += ty;
+                if (COMP) { ux = fmaf(-wsum, lx, ux); uy = fmaf(-wsum, ly, uy); }
+                ux *= inv_n; uy *= inv_n;
+                float nx, ny, ex, ey;
+                if (COMP) {
+                    uint32_t b0, b1;
+                    float l0, l1;
+                    two_sum_bf16(vx, lx + ux, nx, l0, b0);
+                    two_sum_bf16(vy, ly + uy, ny, l1, b1);
+                    ex = (nx - vx) + l0; ey = (ny - vy) + l1;
+                    __stcs(reinterpret_cast<uint32_t*>(lop + col), b0 | (b1 << 16));
+                } else {
+                    nx = vx + ux; ny = vy + uy;
+                    ex = nx - vx; ey = ny - vy;
+                }
+                step_acc += ux * ux + uy * uy;
+                __stcs(reinterpret_cast<float2*>(vp + col), make_float2(nx, ny));
+                const uint64_t e2 = pack2(ex, ey);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const uint64_t d2 = sub2(x2[r], e2);
+                    acc2[r] = fma2(d2, d2, acc2[r]);
+                }
+            } else {
+                // ragged tile, or rows to leave out: scalar, with masks
+                const bool valid = (qb + (ct >> 1) < q1);
+                const bool m0 = valid && col < len, m1 = valid && col + 1 < len;
+                float sx = 0.f, sy = 0.f;
+                float dx[R], dy[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float ax, ay;
+                    unpack2(x2[r], ax, ay);
+                    dx[r] = (valid && r < n) ? ax - vx : 0.f;
+                    dy[r] = (valid && r < n) ? ay - vy : 0.f;
+                    const float wr = sh_w[r];
+                    if (wr != 0.0f) { sx = fmaf(wr, dx[r], sx); sy = fmaf(wr, dy[r], sy); }
+                }
+                float ux = sx, uy = sy;
+                if (COMP) { ux = fmaf(-wsum, lx, ux); uy = fmaf(-wsum, ly, uy); }
+                ux *= inv_n; uy *= inv_n;
+                float nx, ny, ex, ey;
+                if (COMP) {
+                    uint32_t b0, b1;
+                    float l0, l1;
+                    two_sum_bf16(vx, lx + ux, nx, l0, b0);
+                    two_sum_bf16(vy, ly + uy, ny, l1, b1);
+                    ex = (nx - vx) + l0; ey = (ny - vy) + l1;
+                    if (!m0) b0 = 0;
+                    if (!m1) b1 = 0;
+                    if (valid) __stcs(reinterpret_cast<uint32_t*>(lop + col), b0 | (b1 << 16));
+                } else {
+                    nx = vx + ux; ny = vy + uy;
+                    ex = nx - vx; ey = ny - vy;
+                }
+                step_acc += (m0 ? ux * ux : 0.f) + (m1 ? uy * uy : 0.f);
+                if (!m0) nx = 0.f;
+                if (!m1) ny = 0.f;
+                if (valid) __stcs(reinterpret_cast<float2*>(vp + col), make_float2(nx, ny));
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float rx = m0 ? dx[r] - ex : 0.f, ry = m1 ? dy[r] - ey : 0.f;
+                    const uint64_t d2 = pack2(rx, ry);
+                    acc2[r] = fma2(d2, d2, acc2[r]);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (sh_expired) {
+        // Copies of tiles nobody consumed may still be landing: one more bounded wait per stage
+        // before the CTA ends.
+        const int last = sh_issued - 1;
+        if (tid < S && last >= tid) {
+            const int ts = last - ((last - tid) % S);
+            (void)mbar_wait_bounded(&sh_full[tid], (unsigned)((ts / S) & 1), nullptr);
+        }
+        if (tid == 0) atomicOr(&a.status[p], BTARD_STATUS_WAIT_EXPIRED);
+        __syncthreads();
+    }
+
+    // CTA reduction, slots, and the last CTA of the partition adds the slots up: as in the
+    // register-fed pass.
+    {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            float a0, a1;
+            unpack2(acc2[r], a0, a1);
+            const double s = warp_sum((double)a0 + (double)a1);
+            if (lane == 0) sh_red[warp][r] = s;
+        }
+        const double s = warp_sum((double)step_acc);
+        if (lane == 0) sh_red[warp][16] = s;
+    }
+    __syncthreads();
+    double* slots = a.slots + (size_t)p * cpp * (n + 1);
+    double* dst = slots + (size_t)j * (n + 1);
+    for (int i = tid; i <= n; i += blockDim.x) {
+        double s = 0.0;
+        const int c = (i < n) ? i : 16;
+        for (int q = 0; q < kStagedConsumerWarps; ++q) s += sh_red[q][c];
+        dst[i] = s;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sh_flag = (atomicAdd(&a.ticket[p], 1u) == (unsigned)(cpp - 1));
+    __syncthreads();
+    if (!sh_flag) return;
+    __threadfence();
+    const int per = n + 1;
+    double* sh_part = sh_sum;                          // the totals read at the start are dead by now
+    int groups = blockDim.x / per;
+    if (groups > cpp) groups = cpp;
+    if (groups * per > BTARD_MAX_PEERS + 1) groups = (BTARD_MAX_PEERS + 1) / per;
     for (int e = tid; e < groups * per; e += blockDim.x) {
         const int cg = e / per, i = e - cg * per;
         double s = 0.0;
@@ -697,7 +1193,7 @@ __global__ void cclip_finalize_kernel(const KernelArgs k)
     const double* src = a.tot_in + (size_t)p * (n + 1);
     for (int i = threadIdx.x; i <= n; i += blockDim.x) sh_sum[i] = src[i];
     __syncthreads();
-    finish_partition(k, p, sh_sum, a.max_iters, a.stop_mode == BTARD_STOP_EPS);
+    finish_partition(k.a, p, sh_sum, a.max_iters, a.stop_mode == BTARD_STOP_EPS);
 }
 
 __global__ void totals_to_norms_kernel(const double* tot, double* norm, int n)
@@ -864,6 +1360,77 @@ static int iter_ctas_per_sm(int R, int threads, size_t smem)
     else e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_pass_kernel<16, PASS_ITER, true>, threads, smem);
     if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 2; }
     return nb;
+}
+
+// Staged iteration kernel (n <= 16): stages of n rows + v (+ bf16 part) of 128 quads each, two CTAs
+// per SM, as many stages as their share of the shared memory holds (2 to 4).
+StagedGeometry cclip_staged_geometry(int n, int P, long long stride, bool comp)
+{
+    StagedGeometry sg{};
+    sg.ok = 0;
+    if (n > 16 || (stride & 31) != 0) return sg;
+    Geometry& g = sg.g;
+    g.R = (n <= 4) ? 4 : (n <= 8) ? 8 : 16;
+    g.RG = 1;
+    g.CL = kStagedTileQuads;
+    g.threads = kStagedThreads;
+    g.tiles = 0;
+    const size_t row_bytes = (size_t)g.CL * 16;
+    sg.stage_bytes = (unsigned)align_up((size_t)(n + 1) * row_bytes + (comp ? row_bytes / 2 : 0), 128);
+    int dev = 0, smem_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        smem_sm = 233472;                              // sm_100 figure, for sizing without a device
+    }
+    const long long room = (long long)smem_sm / 2 - 6144 - 1024;   // static arrays, per-CTA reserve
+    int stages = (int)(room / (long long)sg.stage_bytes);
+    if (stages < 2) return sg;
+    if (stages > kMaxStages) stages = kMaxStages;
+    sg.stages = stages;
+    sg.smem = (size_t)stages * sg.stage_bytes;
+    g.slots = sm_count() * 2;
+    // One wave of resident CTAs when that keeps at least nine slots in ten busy (every CTA pays its
+    // prologue, pipeline fill and epilogue once), else whole waves as for the register-fed pass.
+    const long long quads = stride >> 2;
+    long long one = g.slots / P;
+    const long long most = (quads + 7) / 8;
+    if (one > most) one = most;
+    const bool one_wave = one >= 1 && one * P * 10 >= (long long)g.slots * 9 &&
+                          quads <= one * (long long)(kStagedMaxTilesPerCta - 1) * g.CL;
+    g.cpp = one_wave ? (int)one : choose_ctas_per_partition(P, quads, g.CL, g.slots);
+    sg.ok = 1;
+    return sg;
+}
+
+template <int R>
+static int launch_staged_r(const StagedArgs& sa, size_t smem, int grid, cudaStream_t st)
+{
+    const bool comp = sa.a.v_lo != nullptr;
+    if (sa.a.l == 0) {                                 // first update of an aggregation
+        const int most = 113 * 1024;
+        cudaError_t e = comp ? cudaFuncSetAttribute(cclip_iter_staged_kernel<R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most)
+                             : cudaFuncSetAttribute(cclip_iter_staged_kernel<R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+        if (e != cudaSuccess) { set_cuda_error(e); return BTARD_ERR_CUDA; }
+    }
+    prof_begin(KIND_ITER, st);
+    if (comp) cclip_iter_staged_kernel<R, true><<<grid, kStagedThreads, smem, st>>>(sa);
+    else cclip_iter_staged_kernel<R, false><<<grid, kStagedThreads, smem, st>>>(sa);
+    prof_end(KIND_ITER, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int launch_cclip_staged(const CclipLaunch& a, const StagedGeometry& sg, cudaStream_t st)
+{
+    StagedArgs sa{a, sg.g.cpp, sg.stages, sg.stage_bytes};
+    const int grid = a.P * sg.g.cpp;
+    switch (sg.g.R) {
+        case 4: return launch_staged_r<4>(sa, sg.smem, grid, st);
+        case 8: return launch_staged_r<8>(sa, sg.smem, grid, st);
+        default: return launch_staged_r<16>(sa, sg.smem, grid, st);
+    }
 }
 
 // CTAs per partition: the smallest count that respects the bound on tiles per CTA, then the count

@@ -81,6 +81,16 @@ Geometry cclip_geometry(int n, int P, long long stride);
 int choose_ctas_per_partition(int P, long long quads, int CL, int slots);
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
+// Iteration pass fed by bulk asynchronous copies through shared-memory stages (ok = 0: this shape
+// takes the register-fed pass instead).
+struct StagedGeometry {
+    Geometry g;
+    int ok, stages;
+    unsigned stage_bytes;
+    size_t smem;
+};
+StagedGeometry cclip_staged_geometry(int n, int P, long long stride, bool comp);
+int launch_cclip_staged(const CclipLaunch& a, const StagedGeometry& sg, cudaStream_t st);
 // L2-resident variant: how many partitions fit one chunk (0: not available on this device), and the
 // cooperative launch that runs the start pass and every update of one chunk.
 constexpr int kResidentMaxGrid = 148 * 8;

@@ -85,7 +85,7 @@ def make_case(rng, P, n, stride, lens, far_rows=0, scale=0.02):
     return g
 
 
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED, btard.ALGO_DIRECT_COOPERATIVE])
 @pytest.mark.parametrize("n", [1, 3, 4, 7, 8, 16, 23, 64, 100, 256])
 @pytest.mark.parametrize("init", [btard.INIT_ZERO, btard.INIT_MEAN, btard.INIT_COORD_MEDIAN,
                                   btard.INIT_CALLER_V0])
@@ -104,15 +104,17 @@ def test_fixed_iterations_match_oracle(n, init, algo):
     assert not (cpu(r["status"]) & 4).any()
 
 
-def test_many_tiles_per_cta_and_many_ctas():
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED])
+@pytest.mark.parametrize("stop", [btard.STOP_FIXED_ITERS, btard.STOP_EPS])
+def test_many_tiles_per_cta_and_many_ctas(algo, stop):
     """One long partition: several CTAs, each with many tiles, plus a ragged last tile."""
     rng = np.random.default_rng(5)
     P, n, stride = 2, 16, 1_000_032
     lens = np.array([1_000_001, 999_999])
     g = make_case(rng, P, n, stride, lens, far_rows=5, scale=0.001)
-    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4)
-    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=4)
-    check_cclip(r, ref, lens)
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4, stop_mode=stop, eps=1e-9)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=4, algo=algo, stop_mode=stop, eps=1e-9)
+    check_cclip(r, ref, lens, eps_mode=(stop == btard.STOP_EPS))
 
 
 def test_config1_fixed_and_eps():
@@ -129,7 +131,7 @@ def test_config1_fixed_and_eps():
     assert cpu(r["status"])[0] == ref["status"][0] == 0
 
 
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED, btard.ALGO_DIRECT_COOPERATIVE])
 def test_eps_mode_counts_and_cap_flag(algo):
     rng = np.random.default_rng(6)
     P, n, stride = 4, 8, 2048
@@ -160,16 +162,18 @@ def test_special_radii():
     assert np.all(v[1] == 0)                                               # tau = 0: never moves
 
 
-def test_non_finite_rows_take_weight_zero():
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED])
+@pytest.mark.parametrize("stride", [1024, 40_000])
+def test_non_finite_rows_take_weight_zero(algo, stride):
     rng = np.random.default_rng(8)
-    P, n, stride = 2, 6, 1024
-    lens = np.array([1024, 1024])
+    P, n = 2, 6
+    lens = np.array([stride, stride - 3])
     g = make_case(rng, P, n, stride, lens)
     g[0, 2, 17] = np.nan
     g[1, 4, 900] = np.inf
     g[1, 0, 3] = -np.inf
     ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_ZERO, max_iters=4)
-    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_ZERO, max_iters=4)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_ZERO, max_iters=4, algo=algo)
     v = cpu(r["v"])
     assert np.all(np.isfinite(v))
     for p in range(P):
@@ -229,7 +233,8 @@ def test_resident_variant_eps_mode_and_chunks():
 
 
 # ----------------------------------------------------------------------------- baseline aggregators
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE, btard.ALGO_DIRECT_RESIDENT])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED, btard.ALGO_DIRECT_COOPERATIVE,
+                                  btard.ALGO_DIRECT_RESIDENT])
 @pytest.mark.parametrize("n", [3, 16, 64])
 def test_geometric_median_rule_matches_oracle(n, algo):
     rng = np.random.default_rng(500 + n)
