@@ -193,6 +193,40 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const long long len = a.table[p].len;
     const double tau = a.table[p].tau;
 
+    const float* gp = a.g + (size_t)p * n * stride;
+    float* vp = a.v + (size_t)p * stride;
+    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
+    const float inv_n = 1.0f / (float)n;
+
+    // This CTA's share of the partition, in groups of 4 columns ("quads"), cut on 128-byte lines.
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cpp) q1 &= ~7LL;
+    const long long full_quads = len >> 2;             // quads that lie entirely inside the data
+    const long long ntiles = (q1 - q0 + CL - 1) / CL;
+    // The rows are marked evict-first in L2: nothing is read twice within a pass, and what is
+    // still resident when the next pass starts (it starts where this one ends) is a bonus.
+    // Measured: pinning the tail with evict-last instead was slower for every budget tried.
+    const uint64_t pol = policy_evict_first();
+
+    // Update passes are launched back to back with programmatic dependent launch: this grid may start
+    // while the previous pass is still draining.  Until griddepcontrol.wait returns, only memory that
+    // no pass writes is touched: the partition table and the rows of g.  The rows of the first tile
+    // are asked into L2 here, so that they are on their way while the previous pass finishes and
+    // while the clip weights are worked out below.  (done[p] only ever goes from 0 to 1 between the
+    // start pass and here, so a 1 read early is final and a 0 is checked again after the wait.)
+    if (MODE == PASS_ITER) {
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        if (ntiles > 0 && tid < n && !*reinterpret_cast<const volatile int*>(a.done + p)) {
+            const long long qb = q0 + (rev ? ntiles - 1 : 0) * CL;
+            const long long rest = q1 - qb;
+            const unsigned bytes = (unsigned)(rest < CL ? rest : CL) * 16u;
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gp + (size_t)tid * stride + qb * 4), "r"(bytes) : "memory");
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+
     if (MODE == PASS_ITER) {
         if (a.done[p]) return;
         // Totals the previous pass left behind: squared norms at the current v, and its squared step.
@@ -235,18 +269,6 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 #pragma unroll
     for (int r = 0; r < R; ++r) acc[r] = 0.0f;
     float step_acc = 0.0f;
-
-    const float* gp = a.g + (size_t)p * n * stride;
-    float* vp = a.v + (size_t)p * stride;
-    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
-    const float inv_n = 1.0f / (float)n;
-
-    // This CTA's share of the partition, in groups of 4 columns ("quads"), cut on 128-byte lines.
-    const long long Q = stride >> 2;
-    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
-    if (j > 0) q0 &= ~7LL;
-    if (j + 1 < cpp) q1 &= ~7LL;
-    const long long full_quads = len >> 2;             // quads that lie entirely inside the data
 
     // v is read and written by every update pass: its loads ask L2 to keep the lines and its stores are
     // marked streaming (measured: fewer DRAM bytes and a shorter pass than with default accesses).
@@ -450,11 +472,6 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
     };
 
-    // The rows are marked evict-first in L2: nothing is read twice within a pass, and what is
-    // still resident when the next pass starts (it starts where this one ends) is a bonus.
-    // Measured: pinning the tail with evict-last instead was slower for every budget tried.
-    const long long ntiles = (q1 - q0 + CL - 1) / CL;
-    const uint64_t pol = policy_evict_first();
     for (long long t = 0; t < ntiles; ++t) {
         const long long qb = q0 + (rev ? ntiles - 1 - t : t) * CL;
         const bool inner = (qb + CL <= q1 && qb + CL <= full_quads);
@@ -1335,10 +1352,20 @@ int launch_pass_r(const KernelArgs& ka, int mode, int threads, size_t smem, int 
     prof_begin(kind, st);
     switch (mode) {
         case PASS_INIT: cclip_pass_kernel<R, PASS_INIT, false><<<grid, threads, smem, st>>>(ka); break;
-        case PASS_ITER:
-            if (ka.a.v_lo) cclip_pass_kernel<R, PASS_ITER, true><<<grid, threads, smem, st>>>(ka);
-            else cclip_pass_kernel<R, PASS_ITER, false><<<grid, threads, smem, st>>>(ka);
+        case PASS_ITER: {
+            // programmatic dependent launch: the grid may be set up while the pass before it drains
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)threads);
+            cfg.dynamicSmemBytes = smem; cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            cudaError_t e = ka.a.v_lo ? cudaLaunchKernelEx(&cfg, cclip_pass_kernel<R, PASS_ITER, true>, ka)
+                                      : cudaLaunchKernelEx(&cfg, cclip_pass_kernel<R, PASS_ITER, false>, ka);
+            if (e != cudaSuccess) { set_cuda_error(e); (void)cudaGetLastError(); prof_end(kind, st); return BTARD_ERR_CUDA; }
             break;
+        }
         case PASS_COMBINE: cclip_pass_kernel<R, PASS_COMBINE, false><<<grid, threads, smem, st>>>(ka); break;
         default: cclip_pass_kernel<R, PASS_NORMS, false><<<grid, threads, smem, st>>>(ka); break;
     }
