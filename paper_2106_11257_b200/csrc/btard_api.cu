@@ -16,6 +16,18 @@ void set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 // ---- optional kernel timing ---------------------------------------------------------------------
+// Size of the L2 cache of the current device in bytes (B200's when no device can be asked).
+static long long l2_bytes()
+{
+    int dev = 0, l2 = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0) {
+        (void)cudaGetLastError();
+        return 126LL << 20;
+    }
+    return l2;
+}
+
 namespace {
 struct ProfRecord { int kind; cudaEvent_t a, b; };
 std::mutex g_prof_mu;
@@ -268,6 +280,7 @@ int btard_centered_clip(const btard_cclip_args* a)
         L.v_lo = (unsigned short*)(base + ws.v_lo);
         BTARD_CUDA_TRY(cudaMemsetAsync(L.v_lo, 0, ws.v_lo_bytes, st));
     }
+    L.v_fits_l2 = (double)P * (double)a->row_stride * (L.v_lo ? 6.0 : 4.0) <= 0.6 * (double)l2_bytes();
 
     // Init pass: v^0 and the residual norms at v^0 (slot buffer 0).
     if (a->rule == BTARD_RULE_MEAN || a->rule == BTARD_RULE_COORD_MEDIAN) {

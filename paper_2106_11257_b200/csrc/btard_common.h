@@ -27,6 +27,9 @@ struct Geometry {
 };
 
 constexpr int kMaxTilesPerCta = 64;   // bounds the length of every fp32 running sum (256 terms)
+// CenteredClip passes add one term per tile and row to a thread's fp32 running sums (the term is the
+// sum of 4 squares), so twice as many tiles keep the sums as short.
+constexpr int kMaxTilesPerPass = 128;
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -75,10 +78,11 @@ struct CclipLaunch {
     double eps2;
     int init_mode;            // PASS_INIT
     int rule;                 // BTARD_RULE_*: how the row weights follow from the norms
+    int v_fits_l2;            // v (and its bf16 part) of all partitions takes at most 60 % of the L2
 };
 
 Geometry cclip_geometry(int n, int P, long long stride);
-int choose_ctas_per_partition(int P, long long quads, int CL, int slots);
+int choose_ctas_per_partition(int P, long long quads, int CL, int slots, int max_tiles = kMaxTilesPerCta);
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
 // Iteration pass fed by bulk asynchronous copies through shared-memory stages (ok = 0: this shape
