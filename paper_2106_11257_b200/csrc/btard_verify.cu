@@ -95,6 +95,26 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
 
     int par = 0;
     for (long long qb = q0; qb < q1; qb += CL, par ^= 1) {
+        // 0. this thread's rows and columns are requested first, so that they are in flight while the
+        //    block of z is generated
+        const long long col = (qb + cl) * 4;
+        const bool valid = qb + cl < q1;
+        const bool m0 = valid && col < len, m1 = valid && col + 1 < len;
+        const bool m2 = valid && col + 2 < len, m3 = valid && col + 3 < len;
+        float4 x[R];
+        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int i = rg * R + r;
+                x[r] = (i < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)i * stride + col))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            v4 = *reinterpret_cast<const float4*>(vp + col);
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         // 1. this tile's block of z
         float4* zb = sh_z + (size_t)par * KT * CL;
         for (int idx = tid; idx < KT * CL; idx += nthr) {
@@ -115,24 +135,6 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
         if (first_chunk && qb > q0) consume_sums(qb - CL, par ^ 1);
 
         // 2. residuals of this thread's rows and columns
-        const long long col = (qb + cl) * 4;
-        const bool valid = qb + cl < q1;
-        const bool m0 = valid && col < len, m1 = valid && col + 1 < len;
-        const bool m2 = valid && col + 2 < len, m3 = valid && col + 3 < len;
-        float4 x[R];
-        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) {
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int i = rg * R + r;
-                x[r] = (i < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)i * stride + col))
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            v4 = *reinterpret_cast<const float4*>(vp + col);
-        } else {
-#pragma unroll
-            for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
         if (m3) {                                      // whole quad inside the data: no predicates
 #pragma unroll
             for (int r = 0; r < R; ++r) {
