@@ -181,6 +181,7 @@ struct VerifyGeometry {
     Geometry g;
     int KT;      // z vectors per launch (compile-time choice)
     int slots;   // doubles per CTA in part_out
+    int own_z;   // n <= 16 and K <= 2: each thread draws the z of its own columns (verify_rows_kernel)
 };
 
 VerifyGeometry verify_geometry(int n, int P, long long stride, int K);

@@ -211,6 +211,145 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     }
 }
 
+// n <= 16 and at most two directions per launch: one thread holds every row of its 4 columns (R >= n
+// rows x 4 columns in registers, as in the CenteredClip passes), so it draws the z quads of those
+// columns itself.  Each quad of z is still generated exactly once per launch, nothing is staged in
+// shared memory and the tile loop has no barrier.  Same per-CTA slot layout as verify_kernel.
+template <int R, int KT>
+__global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
+{
+    __shared__ float sh_w[16];
+    __shared__ double sh_red[8][R * KT + KT + 1];
+
+    const VerifyLaunch& a = k.a;
+    const int n = a.n, cpp = k.cpp;
+    constexpr int CL = 256;
+    const int tid = threadIdx.x;
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const long long stride = a.stride, len = a.table[p].len;
+    const double tau = a.table[p].tau;
+
+    if (tid < 16) {
+        float w = 0.0f;
+        if (tid < n) {
+            const double rho = a.norm_in[(size_t)p * n + tid];
+            if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+        }
+        sh_w[tid] = w;
+    }
+    __syncthreads();
+
+    float acc[R][KT];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int q = 0; q < KT; ++q) acc[r][q] = 0.0f;
+    float zz[KT];
+#pragma unroll
+    for (int q = 0; q < KT; ++q) zz[q] = 0.0f;
+    float rs2 = 0.0f;
+
+    // This CTA's share of the partition in groups of 4 columns, cut on 128-byte lines.
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cpp) q1 &= ~7LL;
+    const float* gp = a.g + (size_t)p * n * stride;
+    const float* vp = a.v + (size_t)p * stride;
+    float* rsp = a.resid_sum ? a.resid_sum + (size_t)p * stride : nullptr;
+    const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
+    const uint32_t pg = (uint32_t)(a.p_base + p);
+
+    for (long long qb = q0 + tid; qb < q1; qb += CL) {
+        const long long col = qb * 4;
+        float4 x[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            x[r] = (r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
+        // this thread's quads of z, drawn while the rows are on their way
+        float4 z[KT];
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            z[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (q < a.kc && col < len) {
+                z[q] = z_quad((uint32_t)qb, pg, (uint32_t)(a.k0 + q), a.seed_lo, a.seed_hi);
+                if (col + 3 >= len) {                  // only the last quad of a ragged partition
+                    if (col + 1 >= len) z[q].y = 0.f;
+                    if (col + 2 >= len) z[q].z = 0.f;
+                    z[q].w = 0.f;
+                }
+            }
+        }
+        if (col + 3 < len) {                           // whole quad inside the data: no predicates
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
+            }
+        } else {
+            const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = m0 ? x[r].x - v4.x : 0.f;
+                x[r].y = m1 ? x[r].y - v4.y : 0.f;
+                x[r].z = m2 ? x[r].z - v4.z : 0.f;
+                x[r].w = 0.f;
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            zz[q] += fmaf(z[q].x, z[q].x, fmaf(z[q].y, z[q].y, fmaf(z[q].z, z[q].z, z[q].w * z[q].w)));
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                acc[r][q] += fmaf(x[r].x, z[q].x, fmaf(x[r].y, z[q].y, fmaf(x[r].z, z[q].z, x[r].w * z[q].w)));
+        }
+        if (first_chunk) {                             // clipped-residual sum of these 4 columns
+            float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float wr = sh_w[r];
+                if (wr != 0.0f) {                      // weight 0: the row is left out, not multiplied
+                    s4.x = fmaf(wr, x[r].x, s4.x);
+                    s4.y = fmaf(wr, x[r].y, s4.y);
+                    s4.z = fmaf(wr, x[r].z, s4.z);
+                    s4.w = fmaf(wr, x[r].w, s4.w);
+                }
+            }
+            rs2 += fmaf(s4.x, s4.x, fmaf(s4.y, s4.y, fmaf(s4.z, s4.z, s4.w * s4.w)));
+            if (rsp) *reinterpret_cast<float4*>(rsp + col) = s4;
+        }
+    }
+
+    // CTA reduction
+    const int warp = tid >> 5, lane = tid & 31;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            const double s = warp_sum((double)acc[r][q]);
+            if (lane == 0) sh_red[warp][r * KT + q] = s;
+        }
+#pragma unroll
+    for (int q = 0; q < KT; ++q) {
+        const double s = warp_sum((double)zz[q]);
+        if (lane == 0) sh_red[warp][R * KT + q] = s;
+    }
+    {
+        const double s = warp_sum((double)rs2);
+        if (lane == 0) sh_red[warp][R * KT + KT] = s;
+    }
+    __syncthreads();
+    double* dst = a.part_out + ((size_t)p * cpp + j) * k.slots;
+    const int total = n * KT + KT + 1;
+    for (int e = tid; e < total; e += CL) {
+        const int col = (e < n * KT) ? e : R * KT + (e - n * KT);   // rows, then znorm2, then the resid-sum slot
+        double s = 0.0;
+        for (int u = 0; u < 8; ++u) s += sh_red[u][col];
+        dst[e] = s;
+    }
+}
+
 // Sums the CTA slots of a partition in a fixed order and writes the outputs of z indices
 // k0 .. k0+kc-1 (and, with the first chunk, the per-row and per-partition values).
 __global__ void verify_finalize_kernel(const VArgs k, int KT)
@@ -361,12 +500,51 @@ int verify_ctas_per_sm(int R, int KT, int threads, size_t smem)
     return nb;
 }
 
+template <int R>
+int launch_rows_r(const VArgs& va, int KT, int grid, cudaStream_t st)
+{
+    prof_begin(KIND_VERIFY, st);
+    if (KT == 1) verify_rows_kernel<R, 1><<<grid, 256, 0, st>>>(va);
+    else verify_rows_kernel<R, 2><<<grid, 256, 0, st>>>(va);
+    prof_end(KIND_VERIFY, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
+}
+
+int rows_ctas_per_sm(int R, int KT)
+{
+    int nb = 0;
+    cudaError_t e;
+    if (R == 4) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 1>, 256, 0)
+                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 2>, 256, 0);
+    else if (R == 8) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 1>, 256, 0)
+                                   : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 2>, 256, 0);
+    else e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 1>, 256, 0)
+                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 2>, 256, 0);
+    if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 2; }
+    return nb;
+}
+
 }  // namespace
 
 VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
 {
     VerifyGeometry vg;
     Geometry& g = vg.g;
+    vg.own_z = (n <= 16 && K <= 2) ? 1 : 0;
+    if (vg.own_z) {                  // every row of a column in one thread: z drawn in registers
+        g.R = (n <= 4) ? 4 : (n <= 8) ? 8 : 16;
+        g.RG = 1;
+        g.CL = 256;
+        g.threads = 256;
+        g.tiles = 0;
+        vg.KT = K;
+        g.slots = sm_count() * rows_ctas_per_sm(g.R, K);
+        g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, g.slots);
+        vg.slots = n * K + K + 1;
+        return vg;
+    }
     g.R = (n <= 16) ? 4 : 8;
     g.RG = (n + g.R - 1) / g.R;
     g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 4) ? 64 : 32;
@@ -397,6 +575,13 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
     const size_t smem = sizeof(float4) * (2 * (size_t)vg.KT * g.CL + 2 * (size_t)g.RG * g.CL);
     const int grid = a.P * g.cpp;
     int rc;
+    if (vg.own_z) {
+        switch (g.R) {
+            case 4: rc = launch_rows_r<4>(va, vg.KT, grid, st); break;
+            case 8: rc = launch_rows_r<8>(va, vg.KT, grid, st); break;
+            default: rc = launch_rows_r<16>(va, vg.KT, grid, st); break;
+        }
+    } else
     switch (g.R) {
         case 4: rc = launch_r<4>(va, vg.KT, g.threads, smem, grid, st); break;
         case 8: rc = launch_r<8>(va, vg.KT, g.threads, smem, grid, st); break;

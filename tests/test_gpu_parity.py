@@ -395,8 +395,8 @@ def check_verify(out, ref, K):
         assert abs(cpu(out["resid_sum_norm"])[p] - ref["resid_sum_norm"][p]) <= RTOL * rscale
 
 
-@pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (5, 3), (16, 8), (16, 1), (23, 4), (64, 4), (64, 8),
-                                 (64, 11), (100, 2), (200, 5)])
+@pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (4, 2), (5, 3), (8, 2), (13, 2), (16, 8), (16, 1), (16, 2),
+                                 (23, 4), (64, 4), (64, 8), (64, 11), (100, 2), (200, 5)])
 def test_verify_matches_oracle(n, K):
     rng = np.random.default_rng(200 + n + K)
     P, stride = 3, 5024
