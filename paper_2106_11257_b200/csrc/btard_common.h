@@ -121,6 +121,7 @@ struct GramGeometry {
     int cpp;       // CTAs per partition
     int entries;   // doubles per Gram slot = 64 nblk
     size_t smem;   // dynamic shared memory of the Gram kernel
+    int umma;      // 17 <= n <= 64 and the rows can be described by a tensor map: tcgen05 kernel
 };
 struct GramLaunch {
     const float* g;

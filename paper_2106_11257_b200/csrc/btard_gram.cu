@@ -11,6 +11,8 @@
 // G is a dense contraction over the columns.  It is computed here on the fp32 FMA pipes: the
 // products of residuals that differ by orders of magnitude (attacked rows) must stay accurate to
 // about 1e-6 relative for the subtraction above, which rules out single-pass TF32.
+#include <cuda.h>
+
 #include "btard_common.h"
 
 namespace btard {
@@ -180,11 +182,14 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
 // products to about 2^-21.  The tensor core adds with truncation, so its accumulator only ever
 // holds one 16-column block (6 chained MMAs); blocks are summed on the fp32 pipe (round to
 // nearest) and moved to fp64 every 64 blocks.
-__device__ __forceinline__ uint32_t to_tf32(float x)
+// r = hi + lo with hi on the TF32 grid: round to nearest (ties away from zero, as cvt.rna does for finite
+// values) by adding half a TF32 unit to the magnitude bits and clearing the 13 low bits; lo = r - hi is
+// exact in fp32 and is handed to the tensor core as it is, which reads only its TF32 part (an error of
+// 2^-21 |r| at most, of either sign).  Two integer instructions and one subtraction; a NaN stays a NaN in lo.
+__device__ __forceinline__ void split_tf32(float r, uint32_t& hi, uint32_t& lo)
 {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
+    hi = (__float_as_uint(r) + 0x1000u) & 0xFFFFE000u;
+    lo = __float_as_uint(r - __uint_as_float(hi));
 }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
@@ -241,10 +246,8 @@ __global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
             uint32_t h0[4], h1[4], l0[4], l1[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                h0[q] = to_tf32(r0[q]);
-                h1[q] = to_tf32(r1[q]);
-                l0[q] = to_tf32(r0[q] - __uint_as_float(h0[q]));
-                l1[q] = to_tf32(r1[q] - __uint_as_float(h1[q]));
+                split_tf32(r0[q], h0[q], l0[q]);
+                split_tf32(r1[q], h1[q], l1[q]);
             }
             float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -313,22 +316,10 @@ __global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
     if (tid == 0) a.ticket[p] = 0;
 }
 
-// ---- 17 <= n <= 64: the Gram block on the 5th-generation tensor cores (tcgen05 + TMEM) ----------
-// Per 32-column tile the CTA's threads form R = g - v0, split every value into TF32 hi + lo and write
-// both as K-major operand tiles (128-byte rows, 128-byte swizzle) into shared memory; one thread then
-// issues, per 8-column k-block, three tcgen05.mma (hi.hi, hi.lo, lo.hi) with M = 64 (rows n..63 are
-// zero), N = 64, accumulating G in 64 columns of tensor memory (row m of G lives in lane
-// m % 16 + 32 (m / 16): sixteen rows in the lower half of each warp's quarter).  A and B descriptors point at the
-// same tiles: B = R.  Two stages alternate, an mbarrier per stage (armed by tcgen05.commit) tells when
-// the tensor core has finished reading it.  Because tensor-core accumulation truncates, the
-// accumulator is read back (tcgen05.ld) and restarted every 4 tiles; the read-back values are summed
-// on the fp32 pipe and turned into fp64 at the end.  Every wait is bounded; if one expires the CTA
-// raises the error flag, still frees its tensor memory and leaves.
-constexpr int kUmmaThreads = 128;
+// ---- constants and helpers of the tcgen05 kernel below ------------------------------------------
 constexpr int kUmmaTileCols = 32;                       // one 128-byte swizzle row of TF32
 constexpr int kUmmaTileBytes = 64 * 128;                // 64 rows x 128 bytes
 constexpr int kUmmaFlushTiles = 4;
-constexpr int kUmmaSpinLimit = 1 << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -339,49 +330,123 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
            (1ull << 46) | (2ull << 61);
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// ---- 17 <= n <= 64: the Gram block on the 5th-generation tensor cores, work split by warp role ----
+// Per 32-column tile of a partition:
+//   loader         one thread issues one tensor copy (the partition's n rows x 128 bytes, described by a
+//                  2-d tensor map over g) and one bulk copy of v0 into a ring of raw stages; an mbarrier
+//                  per stage counts the bytes that landed;
+//   4 producer     warp w takes tiles w, w + 4, ...: reads the raw tile, forms R = g - v0, splits every
+//     warps        value into TF32 hi + lo and writes a 128-row K-major operand tile [hi rows 0..63; lo
+//                  rows 0..63] (128-byte rows, 128-byte swizzle) into its operand stage;
+//   issuing warp   one thread issues, per 8-column k-block, ONE tcgen05.mma with M = 128, N = 64:
+//                  A = the whole operand tile, B = its hi half, so rows 0..63 of the accumulator gather
+//                  hi hi^T and rows 64..127 gather lo hi^T;  G = top + bottom + bottom^T (hi lo^T is the
+//                  transpose of lo hi^T) is formed once, in fp64, at the end.
+// Stages are handed over through mbarriers only (raw full: bytes landed; raw empty and operand full: one
+// arrival of the producer warp that owns the tile; operand empty: a tcgen05.commit); nothing in the loop
+// synchronises the CTA.  Tensor-core accumulation truncates, so two accumulators of 64 tensor-memory
+// columns alternate every kUmmaFlushTiles tiles: the producer warps (they own the four lane quarters)
+// read one back and add it to fp32 sums in registers while the tensor core fills the other.  Every wait
+// is bounded in time and also ends when another warp has given up; a CTA that gave up raises the error
+// flag, waits (bounded) for its copies in flight and for the tensor core, frees its tensor memory and
+// leaves.  Shared-memory traffic (TMA write + read of the raw tile, write of the operand tile, operand
+// reads of the tensor core: 57 KB per 8 KB of rows) is what bounds this kernel, not HBM.
+constexpr int kWsProducerWarps = 4;
+constexpr int kWsIssueWarp = kWsProducerWarps;           // warp index of the MMA issuer
+constexpr int kWsLoadWarp = kWsProducerWarps + 1;        // warp index of the loader
+constexpr int kWsThreads = 32 * (kWsProducerWarps + 2);
+constexpr int kWsOpStages = 4;
+constexpr int kWsOpBytes = 2 * kUmmaTileBytes;           // hi tile, then lo tile: 128 rows x 128 bytes
+constexpr int kWsRawStages = 5;
+constexpr int kWsRawBytes = 65 * 128;                    // 64 rows + v0, 128 bytes each
+constexpr int kWsTmemCols = 128;                         // two accumulators of 64 columns
+constexpr int kWsSmem = kWsOpStages * kWsOpBytes + kWsRawStages * kWsRawBytes + 1024;
+static_assert(kUmmaFlushTiles == kWsProducerWarps, "one tile per producer warp and accumulator group");
+static_assert(kWsOpStages >= kWsProducerWarps, "every producer warp needs an operand stage of its own");
+
+// Bounded wait on an mbarrier phase: first a plain test, then try_wait with a suspend-time hint (the
+// thread sleeps in hardware until the phase completes or the hint runs out).  The bound is on elapsed
+// clock cycles (about two seconds), whatever the hardware makes of the hint.
+constexpr long long kWsWaitCycles = 4000000000LL;
+__device__ __forceinline__ bool mbar_wait_or_quit(uint32_t bar, uint32_t parity, const volatile int* quit)
 {
-    for (int spin = 0; spin < kUmmaSpinLimit; ++spin) {
-        uint32_t done;
-        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    uint32_t done;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    const long long start = clock64();
+    for (;;) {
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
         if (done) return true;
-        __nanosleep(32);                               // do not burn issue slots while the tensor core works
+        if ((quit && *quit) || clock64() - start > kWsWaitCycles) return false;
     }
-    return false;
+}
+// 128-bit shared-memory accesses by 32-bit shared address (the address space is explicit, so these are
+// always single 128-bit shared loads and stores)
+__device__ __forceinline__ float4 lds128(uint32_t addr)
+{
+    float4 r;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr) : "memory");
+    return r;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-__global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, unsigned int* error)
+// ROWS_FULL: n == 64, no row predicate anywhere.
+template <bool ROWS_FULL>
+__global__ void __launch_bounds__(kWsThreads, 2) gram_umma_ws_kernel(const GArgs k, unsigned int* error,
+                                                                      const __grid_constant__ CUtensorMap g_map)
 {
     extern __shared__ __align__(1024) unsigned char sh_raw[];
-    __shared__ __align__(8) unsigned long long sh_mbar[2];
+    __shared__ __align__(8) unsigned long long sh_op_full[kWsOpStages], sh_op_empty[kWsOpStages];
+    __shared__ __align__(8) unsigned long long sh_raw_full[kWsRawStages], sh_raw_empty[kWsRawStages];
+    __shared__ __align__(8) unsigned long long sh_acc_full[2], sh_acc_empty[2], sh_drain;
     __shared__ uint32_t sh_tmem;
     __shared__ int sh_last;
+    __shared__ int sh_fail;
     const GramLaunch& a = k.a;
     const int n = a.n, cpp = k.g.cpp, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
     const long long stride = a.stride, len = a.table[p].len;
-    const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v0 + (size_t)p * stride;
-    // The CTAs of a partition take its 32-column tiles round-robin (tile j, j + cpp, ...): they are
-    // resident together, so at any moment they read neighbouring 128-byte pieces of the same rows and
-    // an open DRAM page is used whole instead of 128 bytes at a time.
-    const long long c1 = stride;
+    // The CTAs of a partition take its 32-column tiles round-robin (tile j, j + cpp, ...): resident
+    // together, they read neighbouring 128-byte pieces of the same rows, so an open DRAM page is used whole.
     const long long all_tiles = (stride + kUmmaTileCols - 1) / kUmmaTileCols;
     const int ntiles = (int)((all_tiles - j + cpp - 1) / cpp);      // tiles j + m cpp < all_tiles
+    const int ngroups = (ntiles + kUmmaFlushTiles - 1) / kUmmaFlushTiles;
     auto tile_col = [&](int t) { return ((long long)j + (long long)t * cpp) * kUmmaTileCols; };
 
-    // operand tiles: [stage][hi, lo][64 rows][128 bytes], 1024-byte aligned
-    unsigned char* tiles = (unsigned char*)(((uintptr_t)sh_raw + 1023) & ~(uintptr_t)1023);
-    for (int e = tid; e < 4 * kUmmaTileBytes / 16; e += kUmmaThreads)
-        reinterpret_cast<uint4*>(tiles)[e] = make_uint4(0u, 0u, 0u, 0u);
+    unsigned char* ops = (unsigned char*)(((uintptr_t)sh_raw + 1023) & ~(uintptr_t)1023);   // operand stages
+    unsigned char* raws = ops + kWsOpStages * kWsOpBytes;                                     // raw stages
+    for (int e = tid; e < kWsOpStages * kWsOpBytes / 16; e += kWsThreads)
+        reinterpret_cast<uint4*>(ops)[e] = make_uint4(0u, 0u, 0u, 0u);       // rows n .. 63 stay zero
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_mbar[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_mbar[1])));
+        for (int s = 0; s < kWsOpStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_op_full[s])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_op_empty[s])));
+        }
+        for (int s = 0; s < kWsRawStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_raw_full[s])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_raw_empty[s])));
+        }
+        for (int q = 0; q < 2; ++q) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_acc_full[q])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh_acc_empty[q])), "r"(kWsProducerWarps));
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh_drain)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        sh_fail = 0;
     }
-    if (warp == 0) {
+    if (warp == kWsIssueWarp) {
         __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh_tmem)), "r"(64));
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh_tmem)), "r"(kWsTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -389,139 +454,193 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = sh_tmem;
+    const volatile int* quit = &sh_fail;
 
-    // tf32 inputs, fp32 accumulate, K-major A and B, N = 64, M = 64
-    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((64u >> 3) << 17) | ((64u >> 4) << 24);
-    const uint32_t tile_base = smem_u32(tiles);
-
-    float sum[64];
+    float sum[64];                                     // producer threads: row 32 warp + lane of the accumulator
 #pragma unroll
     for (int q = 0; q < 64; ++q) sum[q] = 0.0f;
-    int commits[2] = {0, 0};
-    bool failed = false;
-    int since_flush = 0;
-    __shared__ int sh_fail;
-    if (tid == 0) sh_fail = 0;
+    int issued = 0;                                    // loader: tiles whose copies have been issued
 
-    // this thread's four 16-byte chunks of a tile: rows row0 + 16 i, chunk ch (4 columns);
-    // the rows of the next two tiles are kept in flight in registers
-    const int row0 = tid >> 3, ch = tid & 7;
-    float4 xa[4], xb[4], va, vb;
-    auto fetch = [&](int t, float4 (&x)[4], float4& v4) {
-        const long long col = tile_col(t) + 4 * ch;
-        const bool in = t < ntiles && col < c1;
-        v4 = in ? *reinterpret_cast<const float4*>(vp + col) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int r = row0 + 16 * i;
-            x[i] = (in && r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
-                                 : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    };
-    // 32 accumulator columns starting at column `first` of this warp's 32 lanes, added to sum
-    auto read_back = [&](uint32_t taddr, float* dst) {
-        uint32_t d[32];
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-            "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-            : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
-              "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15]),
-              "=r"(d[16]), "=r"(d[17]), "=r"(d[18]), "=r"(d[19]), "=r"(d[20]), "=r"(d[21]), "=r"(d[22]), "=r"(d[23]),
-              "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
-            : "r"(taddr));
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int q = 0; q < 32; ++q) dst[q] += __uint_as_float(d[q]);
-    };
+    if (warp < kWsProducerWarps) {
+        // ---------------- producers: warp w turns tiles w, w + 4, ... into operand tiles, whole tiles ----------------
+        // lane = (q, ch): rows q + 4 m (m = 0 .. 15), 16-byte chunk ch of each; eight lanes cover one
+        // 128-byte row, so the reads and the swizzled writes are free of bank conflicts
+        const int q = lane >> 3, ch = lane & 7;
+        const uint32_t raw_lane = (uint32_t)(q * 128 + 16 * ch);
+        const uint32_t ops_addr = smem_u32(ops), raws_addr = smem_u32(raws);
+        const uint32_t op_even = (uint32_t)(q * 128 + ((ch ^ q) << 4));               // rows 8 u + q
+        const uint32_t op_odd = (uint32_t)((q + 4) * 128 + ((ch ^ (q + 4)) << 4));   // rows 8 u + 4 + q
+        bool ok = true;
+        int next_read = 0;                             // next accumulator group to read back
 
-    fetch(0, xa, va);
-    fetch(1, xb, vb);
-    __syncthreads();
-    for (int t = 0; t < ntiles; ++t) {
-        const int s = t & 1;
-        // the tensor core must be done with what it read from this stage two tiles ago
-        if (commits[s] > 0 && !mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1))) sh_fail = 1;
-
-        const long long col = tile_col(t) + 4 * ch;
-        const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
-        const bool m2 = col + 2 < len && col < c1, m3 = col + 3 < len && col < c1;
-        unsigned char* hi_tile = tiles + (size_t)(2 * s) * kUmmaTileBytes;
-        unsigned char* lo_tile = hi_tile + kUmmaTileBytes;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int r = row0 + 16 * i;
-            if (r < n) {
-                const float r0 = m0 ? xa[i].x - va.x : 0.f, r1 = m1 ? xa[i].y - va.y : 0.f;
-                const float r2 = m2 ? xa[i].z - va.z : 0.f, r3 = m3 ? xa[i].w - va.w : 0.f;
-                const uint32_t h0 = to_tf32(r0), h1 = to_tf32(r1), h2 = to_tf32(r2), h3 = to_tf32(r3);
-                const uint32_t l0 = to_tf32(r0 - __uint_as_float(h0)), l1 = to_tf32(r1 - __uint_as_float(h1));
-                const uint32_t l2 = to_tf32(r2 - __uint_as_float(h2)), l3 = to_tf32(r3 - __uint_as_float(h3));
-                const int off = (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4);
-                *reinterpret_cast<uint4*>(hi_tile + off) = make_uint4(h0, h1, h2, h3);
-                *reinterpret_cast<uint4*>(lo_tile + off) = make_uint4(l0, l1, l2, l3);
-            }
-        }
-        // rotate the register queue and put tile t + 2 in flight
-#pragma unroll
-        for (int i = 0; i < 4; ++i) xa[i] = xb[i];
-        va = vb;
-        fetch(t + 2, xb, vb);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (sh_fail) { failed = true; break; }         // a bounded wait ran out somewhere in the CTA
-        if (tid == 0) {
+        auto read_back = [&](int grp) -> bool {
+            const int qa = grp & 1;
+            if (!mbar_wait_or_quit(smem_u32(&sh_acc_full[qa]), (uint32_t)((grp >> 1) & 1), quit)) return false;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t hi_addr = tile_base + (uint32_t)(2 * s) * kUmmaTileBytes;
-            const uint32_t lo_addr = hi_addr + kUmmaTileBytes;
+            const uint32_t taddr = tmem + ((uint32_t)(32 * warp) << 16) + (uint32_t)(64 * qa);
+            uint32_t d[64];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {           // 8 TF32 = 32 bytes per k-block
-                const uint64_t dh = umma_desc(hi_addr + 32u * ks), dl = umma_desc(lo_addr + 32u * ks);
-                const uint32_t acc0 = (since_flush > 0 || ks > 0) ? 1u : 0u;
-                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
-                             ::"r"(tmem), "l"(dh), "l"(dh), "r"(idesc), "r"(acc0) : "memory");
-                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
-                             ::"r"(tmem), "l"(dh), "l"(dl), "r"(idesc), "r"(1u) : "memory");
-                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
-                             ::"r"(tmem), "l"(dl), "l"(dh), "r"(idesc), "r"(1u) : "memory");
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                         ::"r"(smem_u32(&sh_mbar[s])) : "memory");
-        }
-        commits[s] += 1;
-        since_flush += 1;
-
-        if (since_flush == kUmmaFlushTiles || t + 1 == ntiles) {
-            // read the accumulator back: wait for the commit just issued (covers all earlier MMAs)
-            if (!mbar_wait(smem_u32(&sh_mbar[s]), (uint32_t)((commits[s] - 1) & 1))) sh_fail = 1;
-            __syncthreads();
-            if (sh_fail) { failed = true; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            {                                          // lanes 0..15 of every warp: rows 16 warp + lane
-                const uint32_t taddr = tmem + ((uint32_t)(32 * warp) << 16);
-                read_back(taddr, sum);
-                read_back(taddr + 32u, sum + 32);
-            }
+            for (int h = 0; h < 4; ++h)                // four loads in flight, one wait
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                    : "=r"(d[16 * h + 0]), "=r"(d[16 * h + 1]), "=r"(d[16 * h + 2]), "=r"(d[16 * h + 3]),
+                      "=r"(d[16 * h + 4]), "=r"(d[16 * h + 5]), "=r"(d[16 * h + 6]), "=r"(d[16 * h + 7]),
+                      "=r"(d[16 * h + 8]), "=r"(d[16 * h + 9]), "=r"(d[16 * h + 10]), "=r"(d[16 * h + 11]),
+                      "=r"(d[16 * h + 12]), "=r"(d[16 * h + 13]), "=r"(d[16 * h + 14]), "=r"(d[16 * h + 15])
+                    : "r"(taddr + 16u * h));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int e = 0; e < 64; ++e) sum[e] += __uint_as_float(d[e]);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncthreads();
-            since_flush = 0;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh_acc_empty[qa]));
+            return true;
+        };
+
+        for (int t = warp; t < ntiles && ok; t += kWsProducerWarps) {
+            const int rs = t % kWsRawStages;
+            if (!mbar_wait_or_quit(smem_u32(&sh_raw_full[rs]), (uint32_t)((t / kWsRawStages) & 1), quit)) { ok = false; break; }
+            const int s = t % kWsOpStages, use = t / kWsOpStages;
+            if (use > 0) {                             // the tensor core must be done reading this stage
+                if (!mbar_wait_or_quit(smem_u32(&sh_op_empty[s]), (uint32_t)((use - 1) & 1), quit)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            }
+            const uint32_t raw = raws_addr + (uint32_t)rs * kWsRawBytes + raw_lane;
+            const uint32_t hi_tile = ops_addr + (uint32_t)s * kWsOpBytes;
+            const float4 v4 = lds128(raws_addr + (uint32_t)rs * kWsRawBytes + 64 * 128 + 16 * ch);
+            const long long col = tile_col(t) + 4 * ch;
+            const bool inside = col + 3 < len;         // chunk inside the data: no predicates
+            const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float4 x[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int m = 8 * half + i;        // row q + 4 m
+                    if (ROWS_FULL || q + 4 * m < n) x[i] = lds128(raw + m * 512);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int m = 8 * half + i;
+                    if (ROWS_FULL || q + 4 * m < n) {
+                        float r0 = x[i].x - v4.x, r1 = x[i].y - v4.y, r2 = x[i].z - v4.z, r3 = x[i].w - v4.w;
+                        if (!inside) {                 // ragged end: what lies beyond len (stale bytes included) is 0
+                            r0 = m0 ? r0 : 0.f; r1 = m1 ? r1 : 0.f; r2 = m2 ? r2 : 0.f; r3 = 0.f;
+                        }
+                        uint32_t h0, h1, h2, h3, l0, l1, l2, l3;
+                        split_tf32(r0, h0, l0); split_tf32(r1, h1, l1); split_tf32(r2, h2, l2); split_tf32(r3, h3, l3);
+                        const uint32_t off = (uint32_t)((m >> 1) * 1024) + ((m & 1) ? op_odd : op_even);
+                        sts128(hi_tile + off, h0, h1, h2, h3);
+                        sts128(hi_tile + kUmmaTileBytes + off, l0, l1, l2, l3);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh_raw_empty[rs]));       // the loader may refill the raw stage
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh_op_full[s]));
+            // every producer warp fills one tile of each group of kUmmaFlushTiles; with its tile of a group
+            // done, it reads back the groups before it while this one is multiplied
+            const int grp = t / kUmmaFlushTiles;
+            while (ok && next_read < grp) {
+                ok = read_back(next_read);
+                ++next_read;
+            }
+        }
+        while (ok && next_read < ngroups) {
+            ok = read_back(next_read);
+            ++next_read;
+        }
+        if (!ok) sh_fail = 1;
+    } else if (warp == kWsIssueWarp) {
+        if (lane == 0) {
+            // ---------------- the thread that issues the MMAs ----------------
+            // tf32 inputs, fp32 accumulate, K-major A and B, N = 64, M = 128
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t op_base = smem_u32(ops);
+            bool ok = true;
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int s = t % kWsOpStages, use = t / kWsOpStages;
+                const int grp = t / kUmmaFlushTiles, first = (t % kUmmaFlushTiles == 0);
+                const uint32_t acc = tmem + (uint32_t)(64 * (grp & 1));
+                if (first && grp >= 2)                 // the producers must have read this accumulator back
+                    ok = mbar_wait_or_quit(smem_u32(&sh_acc_empty[grp & 1]), (uint32_t)(((grp >> 1) - 1) & 1), quit);
+                if (ok) ok = mbar_wait_or_quit(smem_u32(&sh_op_full[s]), (uint32_t)(use & 1), quit);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tile_addr = op_base + (uint32_t)s * kWsOpBytes;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {       // 8 TF32 = 32 bytes per k-block
+                    const uint64_t d = umma_desc(tile_addr + 32u * ks);     // A: 128 rows; B: its first 64
+                    const uint32_t acc0 = (!first || ks > 0) ? 1u : 0u;
+                    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+                                 ::"r"(acc), "l"(d), "l"(d), "r"(idesc), "r"(acc0) : "memory");
+                }
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(smem_u32(&sh_op_empty[s])) : "memory");
+                if ((t + 1) % kUmmaFlushTiles == 0 || t + 1 == ntiles)
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                                 ::"r"(smem_u32(&sh_acc_full[grp & 1])) : "memory");
+            }
+            if (!ok) sh_fail = 1;
+        }
+    } else {
+        // ---------------- loader: one tensor copy (n rows x 128 bytes) and one copy of v0 per tile ----------------
+        if (lane == 0) {
+            uint64_t pol;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+            bool ok = true;
+            for (int t = 0; t < ntiles; ++t) {
+                const int rs = t % kWsRawStages, use = t / kWsRawStages;
+                if (use > 0) ok = mbar_wait_or_quit(smem_u32(&sh_raw_empty[rs]), (uint32_t)((use - 1) & 1), quit);
+                if (!ok) break;
+                const long long c = tile_col(t);
+                const long long rest = stride - c;
+                const unsigned vbytes = (unsigned)(rest < kUmmaTileCols ? rest : kUmmaTileCols) * 4u;   // multiple of 16
+                unsigned char* dst = raws + (size_t)rs * kWsRawBytes;
+                const uint32_t bar = smem_u32(&sh_raw_full[rs]);
+                // the tensor copy always delivers the whole box (columns beyond the row end arrive as zeros)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((unsigned)n * 128u + vbytes) : "memory");
+                asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                             ::"r"(smem_u32(dst)), "l"(&g_map), "r"((int)c), "r"(p * n), "r"(bar), "l"(pol) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_u32(dst + 64 * 128)), "l"(vp + c), "r"(vbytes), "r"(bar) : "memory");
+                issued = t + 1;
+            }
+            if (!ok) sh_fail = 1;
         }
     }
-    if (failed && tid == 0) atomicExch(error, 1u);
-
-    // leave tensor memory the way it was found
+    __syncwarp();
+    __syncthreads();
+    const bool failed = sh_fail != 0;
+    if (failed) {
+        if (warp == kWsLoadWarp && lane == 0) {
+            // copies still in flight must land before the shared memory goes away
+            for (int t = (issued > kWsRawStages ? issued - kWsRawStages : 0); t < issued; ++t)
+                (void)mbar_wait_or_quit(smem_u32(&sh_raw_full[t % kWsRawStages]), (uint32_t)((t / kWsRawStages) & 1), nullptr);
+        }
+        if (warp == kWsIssueWarp && lane == 0) {
+            // and the tensor core must be idle before its memory goes away
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                         ::"r"(smem_u32(&sh_drain)) : "memory");
+            (void)mbar_wait_or_quit(smem_u32(&sh_drain), 0u, nullptr);
+            atomicExch(error, 1u);
+        }
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 0) {
+    if (warp == kWsIssueWarp) {
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kWsTmemCols));
     }
 
-    // row i = 16 warp + lane of G (lanes 0..15) -> fp64 matrix in shared memory -> this CTA's slot
-    double* sh_g = reinterpret_cast<double*>(tiles);     // [64][64], the operand tiles are dead now
-    __syncthreads();
-    if (lane < 16) {
-        const int i = 16 * warp + lane;
+    // accumulator row 32 warp + lane -> fp64 [128][64] in shared memory (the stages are dead now);
+    // G = top + bottom + bottom^T -> this CTA's slot
+    double* sh_g = reinterpret_cast<double*>(ops);
+    if (warp < kWsProducerWarps) {
+        const int i = 32 * warp + lane;
 #pragma unroll
         for (int q = 0; q < 64; ++q) sh_g[i * 64 + q] = (double)sum[q];
     }
@@ -529,11 +648,12 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
     const int entries = k.g.entries, NB = k.g.NB;
     double* slots = a.slots + (size_t)p * cpp * entries;
     double* dst = slots + (size_t)j * entries;
-    for (int idx = tid; idx < entries; idx += kUmmaThreads) {
+    for (int idx = tid; idx < entries; idx += kWsThreads) {
         const int b = idx >> 6, e = idx & 63;
         int bi, bj;
         block_coords(b, NB, bi, bj);
-        dst[idx] = sh_g[(8 * bi + (e >> 3)) * 64 + 8 * bj + (e & 7)];
+        const int r = 8 * bi + (e >> 3), c = 8 * bj + (e & 7);
+        dst[idx] = sh_g[r * 64 + c] + (sh_g[(64 + r) * 64 + c] + sh_g[(64 + c) * 64 + r]);
     }
     __threadfence();
     __syncthreads();
@@ -542,7 +662,7 @@ __global__ void __launch_bounds__(kUmmaThreads) gram_umma_kernel(const GArgs k, 
     if (!sh_last) return;
     __threadfence();
     double* out = a.gram + (size_t)p * entries;
-    for (int idx = tid; idx < entries; idx += kUmmaThreads) {
+    for (int idx = tid; idx < entries; idx += kWsThreads) {
         double s = 0.0;
 #pragma unroll 8
         for (int c = 0; c < cpp; ++c) s += __ldcg(slots + (size_t)c * entries + idx);
@@ -724,11 +844,45 @@ __global__ void gram_finalize_kernel(const double* tot, double* resid_norm, uint
     if (bad) atomicOr(&status[p], BTARD_STATUS_NONFINITE_ROW);
 }
 
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn()
+{
+    static const EncodeTiledFn fn = [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            ptr = nullptr;
+        }
+        return (EncodeTiledFn)ptr;
+    }();
+    return fn;
+}
+
+// g [P][n][stride] as a 2-d tensor of P n rows; one box = the n rows of a partition x 32 columns.
+bool encode_rows_map(CUtensorMap* map, const float* g, int n, int P, long long stride)
+{
+    const EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)stride, (cuuint64_t)P * (cuuint64_t)n};
+    const cuuint64_t strides[1] = {(cuuint64_t)stride * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)kUmmaTileCols, (cuuint32_t)n};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(g), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 GramGeometry gram_geometry(int n, int P, long long stride)
 {
     GramGeometry g;
+    g.umma = 0;
     g.NB = (n + 7) / 8;
     g.nblk = g.NB * (g.NB + 1) / 2;
     g.KG = kGramThreads / g.nblk;
@@ -766,11 +920,13 @@ GramGeometry gram_geometry(int n, int P, long long stride)
             nb = 2;
         }
         g.cpp = choose_ctas_per_partition(P, stride >> 2, 16 * (kGramThreads / 32), sm_count() * nb);
-    } else if (n <= 64) {   // tcgen05 kernel: 3 CTAs per SM (160 registers x 128 threads each)
+    } else if (n <= 64 && stride >= kUmmaTileCols && stride < (1LL << 31) && encode_tiled_fn() != nullptr) {
+        // tcgen05 kernel: 2 CTAs per SM (about 100 KB of shared memory each)
+        g.umma = 1;
         // fp32 read-back sums: at most 512 flushes of 128 columns per CTA before fp64
         const long long cap_cols = 512LL * kUmmaFlushTiles * kUmmaTileCols;
         long long cmin2 = (stride + cap_cols - 1) / cap_cols;
-        int c2 = choose_ctas_per_partition(P, stride >> 2, 8 * 32, sm_count() * 3);
+        int c2 = choose_ctas_per_partition(P, stride >> 2, 8 * 32, sm_count() * 2);
         if (c2 < cmin2) c2 = (int)cmin2;
         g.cpp = c2;
     }
@@ -782,12 +938,16 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     GArgs ga{a, geo};
     if (geo.smem > 48 * 1024)
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
-    constexpr int umma_smem = 4 * kUmmaTileBytes + 1024;
-    if (a.n > 16 && a.n <= 64)
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, umma_smem));
+    CUtensorMap map;
+    if (geo.umma) {
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
+        if (!encode_rows_map(&map, a.g, a.n, a.P, a.stride)) { set_cuda_error(cudaErrorInvalidValue); return BTARD_ERR_CUDA; }
+    }
     prof_begin(KIND_GRAM, st);
     if (a.n <= 16) gram_mma16_kernel<<<a.P * geo.cpp, kGramThreads, 0, st>>>(ga);
-    else if (a.n <= 64) gram_umma_kernel<<<a.P * geo.cpp, kUmmaThreads, umma_smem, st>>>(ga, a.error);
+    else if (geo.umma && a.n == 64) gram_umma_ws_kernel<true><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
+    else if (geo.umma) gram_umma_ws_kernel<false><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
     else gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
     prof_end(KIND_GRAM, st);
     BTARD_CUDA_TRY(cudaGetLastError());
