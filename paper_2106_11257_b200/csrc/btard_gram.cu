@@ -8,9 +8,12 @@
 // So the tensor is read once to build G (this file), the iteration runs on n x n numbers in fp64,
 // and one more pass forms v = v0 + sum_j a_j R_j (the combine mode of the streaming kernel).
 //
-// G is a dense contraction over the columns.  It is computed here on the fp32 FMA pipes: the
-// products of residuals that differ by orders of magnitude (attacked rows) must stay accurate to
-// about 1e-6 relative for the subtraction above, which rules out single-pass TF32.
+// G is a dense contraction over the columns, but a thin one (n <= 128 rows against hundreds of thousands
+// of columns read once), and the products of residuals that differ by orders of magnitude (attacked rows)
+// must stay accurate to about 1e-6 relative for the subtraction above, which rules out single-pass TF32.
+// Three kernels, by n: n <= 16 exact fp32 products with all rows of a column in one thread; 17..64 on the
+// tcgen05 tensor cores with a TF32 hi/lo split (three products, one instruction); 65..128 fp32 FMA on
+// 8 x 8 register blocks from shared memory.
 #include <cuda.h>
 
 #include "btard_common.h"
@@ -174,14 +177,6 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
     if (tid == 0) a.ticket[p] = 0;
 }
 
-// ---- n <= 16: the Gram block on the tensor cores, straight from registers ------------------------
-// One warp owns 16 rows x 16 columns at a time.  In the m16n8k8 fragment layout the B operand of
-// R R^T is the A operand itself (lane (g, t) holds rows g, g+8 and the same four columns for both),
-// so nothing is staged in shared memory.  TF32 alone would lose the low 13 bits of every residual;
-// each value is split as hi + lo (both TF32) and hi.hi + hi.lo + lo.hi is accumulated, which keeps
-// products to about 2^-21.  The tensor core adds with truncation, so its accumulator only ever
-// holds one 16-column block (6 chained MMAs); blocks are summed on the fp32 pipe (round to
-// nearest) and moved to fp64 every 64 blocks.
 // r = hi + lo with hi on the TF32 grid: round to nearest (ties away from zero, as cvt.rna does for finite
 // values) by adding half a TF32 unit to the magnitude bits and clearing the 13 low bits; lo = r - hi is
 // exact in fp32 and is handed to the tensor core as it is, which reads only its TF32 part (an error of
@@ -191,114 +186,124 @@ __device__ __forceinline__ void split_tf32(float r, uint32_t& hi, uint32_t& lo)
     hi = (__float_as_uint(r) + 0x1000u) & 0xFFFFE000u;
     lo = __float_as_uint(r - __uint_as_float(hi));
 }
-__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
-constexpr int kMmaStepCols = 64;      // columns a warp takes per step (4 blocks of 16)
+// ---- n <= 16 on the fp32 pipes: every row of a column pair in one thread ---------------------------
+// A thread owns 2 columns of every tile of its CTA.  Its R >= n row values (and v0) of the next
+// kRowsStages - 1 tiles are on their way into shared memory as 8-byte asynchronous copies (cp.async; a
+// thread reads back only what it copied itself, so a wait on its own copy groups is all the
+// synchronisation there is), which keeps about 100 KB per SM in flight without holding registers.  The
+// thread forms the residuals of the current tile and adds the R (R + 1) / 2 products per column to fp32
+// running sums: 8.5 fused multiply-adds per element at R = 16, exact fp32 products, no splitting.  The
+// running sums are short: every kRowsFlushTiles tiles a warp adds its lanes' sums (shuffles) and moves
+// the result to fp64 in shared memory.
+constexpr int kRowsThreads = 256;
+constexpr int kRowsFlushTiles = 32;
+constexpr int kRowsStages = 3;
+constexpr int kRowsTile = 2 * kRowsThreads;              // columns per tile
 
-__global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
+template <int R>
+__host__ __device__ constexpr int rows_stage_bytes() { return (R + 1) * kRowsTile * 4; }   // R rows and v0
+
+template <int R>
+__global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs k)
 {
-    __shared__ double sh_tile[kGramThreads / 32][16][16];
+    constexpr int NP = R * (R + 1) / 2;
+    constexpr int STAGE = rows_stage_bytes<R>();
+    extern __shared__ __align__(16) unsigned char sh_stage[];          // [kRowsStages][R + 1][kRowsTile] floats
+    __shared__ double sh_acc[kRowsThreads / 32][NP];
     __shared__ int sh_last;
     const GramLaunch& a = k.a;
     const int n = a.n, cpp = k.g.cpp, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = lane >> 2, t = lane & 3;
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
     const long long stride = a.stride, len = a.table[p].len;
     const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v0 + (size_t)p * stride;
+    // columns of this CTA, cut on 128-byte lines
     long long c0 = stride * j / cpp, c1 = stride * (j + 1) / cpp;
     if (j > 0) c0 &= ~31LL;
     if (j + 1 < cpp) c1 &= ~31LL;
+    const int ntiles = (int)((c1 - c0 + kRowsTile - 1) / kRowsTile);
 
-    const bool row0 = g < n, row1 = g + 8 < n;
-    const float* p0 = gp + (size_t)g * stride;
-    const float* p1 = gp + (size_t)(g + 8) * stride;
+    for (int e = lane; e < NP; e += 32) sh_acc[warp][e] = 0.0;
+    __syncwarp();
+    float acc[NP];
+#pragma unroll
+    for (int e = 0; e < NP; ++e) acc[e] = 0.0f;
 
-    float sum0[4] = {0.f, 0.f, 0.f, 0.f}, sum1[4] = {0.f, 0.f, 0.f, 0.f};     // fp32 running sums
-    double big0[4] = {0., 0., 0., 0.}, big1[4] = {0., 0., 0., 0.};
+    const uint32_t my_base = (uint32_t)__cvta_generic_to_shared(sh_stage) + 8u * (uint32_t)tid;
+    // copies of tile t into stage t % kRowsStages (one group per tile, empty groups keep the count uniform)
+    auto issue = [&](int t) {
+        const long long col = c0 + (long long)t * kRowsTile + 2 * tid;
+        if (t < ntiles && col < c1) {                  // row_stride is a multiple of 4: a pair is in or out whole
+            const uint32_t dst = my_base + (uint32_t)(t % kRowsStages) * STAGE;
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (r < n)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)r * (kRowsTile * 4)),
+                                 "l"(gp + (size_t)r * stride + col) : "memory");
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)R * (kRowsTile * 4)),
+                         "l"(vp + col) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto flush = [&]() {
+#pragma unroll
+        for (int e = 0; e < NP; ++e) {
+            float sv = acc[e];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sv += __shfl_down_sync(0xffffffffu, sv, o);
+            if (lane == 0) sh_acc[warp][e] += (double)sv;
+            acc[e] = 0.0f;
+        }
+    };
+
+#pragma unroll
+    for (int t = 0; t < kRowsStages - 1; ++t) issue(t);
     int since_flush = 0;
-
-    for (long long cs = c0 + (long long)warp * kMmaStepCols; cs < c1; cs += (long long)(kGramThreads / 32) * kMmaStepCols) {
-        float4 x0[4], x1[4], v4[4];
+    for (int t = 0; t < ntiles; ++t) {
+        issue(t + kRowsStages - 1);                    // into the stage this thread emptied one tile ago
+        asm volatile("cp.async.wait_group %0;" ::"n"(kRowsStages - 1) : "memory");   // tile t has landed
+        const long long col = c0 + (long long)t * kRowsTile + 2 * tid;
+        const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
+        const uint32_t src = my_base + (uint32_t)(t % kRowsStages) * STAGE;
+        float2 x[R], v2;
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v2.x), "=f"(v2.y) : "r"(src + (uint32_t)R * (kRowsTile * 4)) : "memory");
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {                  // all loads of the step first
-            const long long col = cs + 16 * b + 4 * t;
-            const bool in = col < c1;
-            x0[b] = (in && row0) ? __ldcs(reinterpret_cast<const float4*>(p0 + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            x1[b] = (in && row1) ? __ldcs(reinterpret_cast<const float4*>(p1 + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            v4[b] = in ? *reinterpret_cast<const float4*>(vp + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int r = 0; r < R; ++r)
+            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x[r].x), "=f"(x[r].y) : "r"(src + (uint32_t)r * (kRowsTile * 4)) : "memory");
+#pragma unroll
+        for (int r = 0; r < R; ++r) {                  // residuals; what was never copied reads as 0
+            x[r].x = (m0 && r < n) ? x[r].x - v2.x : 0.f;
+            x[r].y = (m1 && r < n) ? x[r].y - v2.y : 0.f;
         }
+        int e = 0;
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const long long col = cs + 16 * b + 4 * t;
-            const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
-            const bool m2 = col + 2 < len && col < c1, m3 = col + 3 < len && col < c1;
-            // residuals of rows g and g+8 at this lane's four columns
-            const float r0[4] = {(m0 && row0) ? x0[b].x - v4[b].x : 0.f, (m1 && row0) ? x0[b].y - v4[b].y : 0.f,
-                                 (m2 && row0) ? x0[b].z - v4[b].z : 0.f, (m3 && row0) ? x0[b].w - v4[b].w : 0.f};
-            const float r1[4] = {(m0 && row1) ? x1[b].x - v4[b].x : 0.f, (m1 && row1) ? x1[b].y - v4[b].y : 0.f,
-                                 (m2 && row1) ? x1[b].z - v4[b].z : 0.f, (m3 && row1) ? x1[b].w - v4[b].w : 0.f};
-            uint32_t h0[4], h1[4], l0[4], l1[4];
+        for (int i = 0; i < R; ++i)
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                split_tf32(r0[q], h0[q], l0[q]);
-                split_tf32(r1[q], h1[q], l1[q]);
-            }
-            float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {           // two k-steps: columns (0,1) then (2,3) of the lane
-                const int qa = 2 * ks, qb = 2 * ks + 1;
-                const uint32_t ah[4] = {h0[qa], h1[qa], h0[qb], h1[qb]};
-                const uint32_t al[4] = {l0[qa], l1[qa], l0[qb], l1[qb]};
-                // columns 0..7 of G: B = rows g of R; columns 8..15: rows g+8
-                mma_tf32(d0, ah, h0[qa], h0[qb]);
-                mma_tf32(d0, ah, l0[qa], l0[qb]);
-                mma_tf32(d0, al, h0[qa], h0[qb]);
-                mma_tf32(d1, ah, h1[qa], h1[qb]);
-                mma_tf32(d1, ah, l1[qa], l1[qb]);
-                mma_tf32(d1, al, h1[qa], h1[qb]);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { sum0[q] += d0[q]; sum1[q] += d1[q]; }
-        }
-        if (++since_flush == 16) {                     // 64 blocks of 16 columns
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                big0[q] += (double)sum0[q]; big1[q] += (double)sum1[q];
-                sum0[q] = 0.f; sum1[q] = 0.f;
-            }
-            since_flush = 0;
-        }
+            for (int q = i; q < R; ++q, ++e)
+                acc[e] = fmaf(x[i].y, x[q].y, fmaf(x[i].x, x[q].x, acc[e]));
+        if (++since_flush == kRowsFlushTiles) { flush(); since_flush = 0; }
     }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) { big0[q] += (double)sum0[q]; big1[q] += (double)sum1[q]; }
-
-    // accumulator fragment: (row g, col 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1); d1 is 8 columns on
-    sh_tile[warp][g][2 * t] = big0[0];
-    sh_tile[warp][g][2 * t + 1] = big0[1];
-    sh_tile[warp][g + 8][2 * t] = big0[2];
-    sh_tile[warp][g + 8][2 * t + 1] = big0[3];
-    sh_tile[warp][g][8 + 2 * t] = big1[0];
-    sh_tile[warp][g][8 + 2 * t + 1] = big1[1];
-    sh_tile[warp][g + 8][8 + 2 * t] = big1[2];
-    sh_tile[warp][g + 8][8 + 2 * t + 1] = big1[3];
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    flush();
     __syncthreads();
+
+    // pair (i <= q) sits at i R - i (i - 1) / 2 + (q - i); the slot holds whole 8 x 8 blocks
     const int entries = k.g.entries, NB = k.g.NB;
     double* slots = a.slots + (size_t)p * cpp * entries;
     double* dst = slots + (size_t)j * entries;
-    for (int idx = tid; idx < entries; idx += kGramThreads) {
+    for (int idx = tid; idx < entries; idx += kRowsThreads) {
         const int b = idx >> 6, e = idx & 63;
         int bi, bj;
         block_coords(b, NB, bi, bj);
-        const int r = 8 * bi + (e >> 3), c = 8 * bj + (e & 7);
-        double s = 0.0;
-        for (int w = 0; w < kGramThreads / 32; ++w) s += sh_tile[w][r][c];
-        dst[idx] = s;
+        int r = 8 * bi + (e >> 3), c = 8 * bj + (e & 7);
+        if (r > c) { const int sw = r; r = c; c = sw; }
+        double sv = 0.0;
+        if (c < R) {
+            const int at = r * R - r * (r - 1) / 2 + (c - r);
+            for (int w = 0; w < kRowsThreads / 32; ++w) sv += sh_acc[w][at];
+        }
+        dst[idx] = sv;
     }
     __threadfence();
     __syncthreads();
@@ -307,11 +312,11 @@ __global__ void __launch_bounds__(kGramThreads) gram_mma16_kernel(const GArgs k)
     if (!sh_last) return;
     __threadfence();
     double* out = a.gram + (size_t)p * entries;
-    for (int idx = tid; idx < entries; idx += kGramThreads) {
-        double s = 0.0;
+    for (int idx = tid; idx < entries; idx += kRowsThreads) {
+        double sv = 0.0;
 #pragma unroll 8
-        for (int c = 0; c < cpp; ++c) s += __ldcg(slots + (size_t)c * entries + idx);
-        out[idx] = s;
+        for (int c = 0; c < cpp; ++c) sv += __ldcg(slots + (size_t)c * entries + idx);
+        out[idx] = sv;
     }
     if (tid == 0) a.ticket[p] = 0;
 }
@@ -913,13 +918,9 @@ GramGeometry gram_geometry(int n, int P, long long stride)
     if (c > most) c = most;
     if (c < 1) c = 1;
     g.cpp = (int)c;
-    if (n <= 16) {   // tensor-core kernel: whole waves of resident CTAs
-        int nb = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, gram_mma16_kernel, kGramThreads, 0) != cudaSuccess || nb < 1) {
-            (void)cudaGetLastError();
-            nb = 2;
-        }
-        g.cpp = choose_ctas_per_partition(P, stride >> 2, 16 * (kGramThreads / 32), sm_count() * nb);
+    if (n <= 16) {   // fp32 kernel with all rows in one thread: one CTA per SM, whole waves; the running
+                     // sums are flushed inside the kernel, so a CTA may take any number of tiles
+        g.cpp = choose_ctas_per_partition(P, stride >> 2, kRowsTile / 4, sm_count(), 1 << 20);
     } else if (n <= 64 && stride >= kUmmaTileCols && stride < (1LL << 31) && encode_tiled_fn() != nullptr) {
         // tcgen05 kernel: 2 CTAs per SM (about 100 KB of shared memory each)
         g.umma = 1;
@@ -938,6 +939,10 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     GArgs ga{a, geo};
     if (geo.smem > 48 * 1024)
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
+    if (a.n <= 16) {
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
+    }
     CUtensorMap map;
     if (geo.umma) {
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
@@ -945,7 +950,9 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
         if (!encode_rows_map(&map, a.g, a.n, a.P, a.stride)) { set_cuda_error(cudaErrorInvalidValue); return BTARD_ERR_CUDA; }
     }
     prof_begin(KIND_GRAM, st);
-    if (a.n <= 16) gram_mma16_kernel<<<a.P * geo.cpp, kGramThreads, 0, st>>>(ga);
+    if (a.n <= 4) gram_rows_kernel<4><<<a.P * geo.cpp, kRowsThreads, kRowsStages * rows_stage_bytes<4>(), st>>>(ga);
+    else if (a.n <= 8) gram_rows_kernel<8><<<a.P * geo.cpp, kRowsThreads, kRowsStages * rows_stage_bytes<8>(), st>>>(ga);
+    else if (a.n <= 16) gram_rows_kernel<16><<<a.P * geo.cpp, kRowsThreads, kRowsStages * rows_stage_bytes<16>(), st>>>(ga);
     else if (geo.umma && a.n == 64) gram_umma_ws_kernel<true><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
     else if (geo.umma) gram_umma_ws_kernel<false><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
     else gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
