@@ -197,14 +197,15 @@ __device__ __forceinline__ void split_tf32(float r, uint32_t& hi, uint32_t& lo)
 // running sums are short: every kRowsFlushTiles tiles a warp adds its lanes' sums (shuffles) and moves
 // the result to fp64 in shared memory.
 constexpr int kRowsThreads = 256;
-constexpr int kRowsFlushTiles = 32;
+constexpr int kRowsFlushTiles = 64;
 constexpr int kRowsStages = 3;
 constexpr int kRowsTile = 2 * kRowsThreads;              // columns per tile
 
 template <int R>
 __host__ __device__ constexpr int rows_stage_bytes() { return (R + 1) * kRowsTile * 4; }   // R rows and v0
 
-template <int R>
+// FULL: n == R, no row predicate anywhere.
+template <int R, bool FULL>
 __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs k)
 {
     constexpr int NP = R * (R + 1) / 2;
@@ -238,7 +239,7 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
             const uint32_t dst = my_base + (uint32_t)(t % kRowsStages) * STAGE;
 #pragma unroll
             for (int r = 0; r < R; ++r)
-                if (r < n)
+                if (FULL || r < n)
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)r * (kRowsTile * 4)),
                                  "l"(gp + (size_t)r * stride + col) : "memory");
             asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)R * (kRowsTile * 4)),
@@ -271,10 +272,16 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
 #pragma unroll
         for (int r = 0; r < R; ++r)
             asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x[r].x), "=f"(x[r].y) : "r"(src + (uint32_t)r * (kRowsTile * 4)) : "memory");
+        // residuals; what was never copied (rows >= n, columns beyond the CTA's range or the data) reads as 0
+        if (FULL && c0 + (long long)(t + 1) * kRowsTile <= (len < c1 ? len : c1)) {       // whole tile inside
 #pragma unroll
-        for (int r = 0; r < R; ++r) {                  // residuals; what was never copied reads as 0
-            x[r].x = (m0 && r < n) ? x[r].x - v2.x : 0.f;
-            x[r].y = (m1 && r < n) ? x[r].y - v2.y : 0.f;
+            for (int r = 0; r < R; ++r) { x[r].x -= v2.x; x[r].y -= v2.y; }
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = (m0 && (FULL || r < n)) ? x[r].x - v2.x : 0.f;
+                x[r].y = (m1 && (FULL || r < n)) ? x[r].y - v2.y : 0.f;
+            }
         }
         int e = 0;
 #pragma unroll
@@ -940,8 +947,10 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     if (geo.smem > 48 * 1024)
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
     if (a.n <= 16) {
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
     }
     CUtensorMap map;
     if (geo.umma) {
@@ -950,9 +959,15 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
         if (!encode_rows_map(&map, a.g, a.n, a.P, a.stride)) { set_cuda_error(cudaErrorInvalidValue); return BTARD_ERR_CUDA; }
     }
     prof_begin(KIND_GRAM, st);
-    if (a.n <= 4) gram_rows_kernel<4><<<a.P * geo.cpp, kRowsThreads, kRowsStages * rows_stage_bytes<4>(), st>>>(ga);
-    else if (a.n <= 8) gram_rows_kernel<8><<<a.P * geo.cpp, kRowsThreads, kRowsStages * rows_stage_bytes<8>(), st>>>(ga);
-    else if (a.n <= 16) gram_rows_kernel<16><<<a.P * geo.cpp, kRowsThreads, kRowsStages * rows_stage_bytes<16>(), st>>>(ga);
+    if (a.n <= 16) {
+        const int grid = a.P * geo.cpp;
+        if (a.n == 16) gram_rows_kernel<16, true><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<16>(), st>>>(ga);
+        else if (a.n > 8) gram_rows_kernel<16, false><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<16>(), st>>>(ga);
+        else if (a.n == 8) gram_rows_kernel<8, true><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<8>(), st>>>(ga);
+        else if (a.n > 4) gram_rows_kernel<8, false><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<8>(), st>>>(ga);
+        else if (a.n == 4) gram_rows_kernel<4, true><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<4>(), st>>>(ga);
+        else gram_rows_kernel<4, false><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<4>(), st>>>(ga);
+    }
     else if (geo.umma && a.n == 64) gram_umma_ws_kernel<true><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
     else if (geo.umma) gram_umma_ws_kernel<false><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
     else gram_kernel<<<a.P * geo.cpp, kGramThreads, geo.smem, st>>>(ga);
