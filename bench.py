@@ -111,7 +111,8 @@ def algorithmic_bytes(w, iters, gram=False):
     n, stride = w.n, w.row_stride
     per_pass = n * stride * 4 * (1.0 + 2.0 / n)
     input_only = n * stride * 4
-    passes = [3 for _ in iters] if gram else [2 + int(i) for i in iters]
+    fused = gram and n <= 16 and w.K <= 2            # combine and verification in one pass
+    passes = [2 if fused else 3 for _ in iters] if gram else [2 + int(i) for i in iters]
     return sum(passes) * input_only, sum(passes) * per_pass, passes
 
 
@@ -152,15 +153,28 @@ def run_ours(args):
     v = torch.empty((P, stride), dtype=torch.float32, device=dev)
     state = {}
 
+    ckeys = ("iters", "last_step_norm", "resid_norm", "status")
+    vkeys = ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm", "status")
+
+    def aggregate(which, vbuf, ws, st):
+        """One aggregation + verification with algorithm `which`; the Gram variant goes through the one-call
+        entry point (combine and verification passes fused where the library can)."""
+        if which == btard.ALGO_GRAM:
+            r, o = btard.centered_clip_verify(g, w.tau, w.zseed, K=w.K, part_len=w.part_len, init_mode=w.init_mode,
+                                              v=vbuf, stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps,
+                                              algo=which, workspaces=(ws, ws_v),
+                                              out=(st.get("c"), st.get("v")) if st else None)
+        else:
+            r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=w.init_mode, v=vbuf,
+                                    stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps, algo=which,
+                                    workspace=ws, out=st.get("c"))
+            o = btard.verify_projections(g, vbuf, w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                         resid_norm_in=r["resid_norm"], workspace=ws_v, out=st.get("v"))
+        st["c"] = {k: r[k] for k in ckeys}
+        st["v"] = {k: o[k] for k in vkeys}
+
     def step():
-        r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=w.init_mode, v=v,
-                                stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps, algo=algo,
-                                workspace=ws_c, out=state.get("c"))
-        state["c"] = {k: r[k] for k in ("iters", "last_step_norm", "resid_norm", "status")}
-        o = btard.verify_projections(g, v, w.tau, w.zseed, K=w.K, part_len=w.part_len,
-                                     resid_norm_in=r["resid_norm"], workspace=ws_v, out=state.get("v"))
-        state["v"] = {k: o[k] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2",
-                                        "resid_sum_norm", "status")}
+        aggregate(algo, v, ws_c, state)
 
     for _ in range(args.warmup):
         step()
@@ -215,14 +229,7 @@ def run_ours(args):
         so = {}
 
         def other_step():
-            r = btard.centered_clip(g, w.tau, part_len=w.part_len, init_mode=w.init_mode, v=v_o,
-                                    stop_mode=w.stop_mode, max_iters=w.max_iters, eps=w.eps,
-                                    algo=other_algo, workspace=ws_o, out=so.get("c"))
-            so["c"] = {k: r[k] for k in ("iters", "last_step_norm", "resid_norm", "status")}
-            o = btard.verify_projections(g, v_o, w.tau, w.zseed, K=w.K, part_len=w.part_len,
-                                         resid_norm_in=r["resid_norm"], workspace=ws_v, out=so.get("v"))
-            so["v"] = {k: o[k] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2",
-                                         "resid_sum_norm", "status")}
+            aggregate(other_algo, v_o, ws_o, so)
         for _ in range(3):
             other_step()
         torch.cuda.synchronize()
@@ -319,7 +326,8 @@ def run_ours(args):
                    "max_iters": w.max_iters, "eps": w.eps, "K": w.K,
                    "iters_per_partition": [int(i) for i in iters],
                    "not_converged_partitions": int((status & 1).sum()),
-                   "passes_counted": ("1 Gram + 1 combine + 1 verify per partition" if args.algo == "gram"
+                   "passes_counted": (("1 Gram + 1 combine-and-verify per partition" if (w.n <= 16 and w.K <= 2)
+                                       else "1 Gram + 1 combine + 1 verify per partition") if args.algo == "gram"
                                       else "1 init + iters + 1 verify per partition"),
                    "l2": "input (%.0f MB) larger than L2 (126 MB), no flush" % (g.numel() * 4 / 1e6),
                    "kernel_events": "per-kernel durations come from a second run of the same K steps",

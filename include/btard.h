@@ -196,6 +196,20 @@ BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* arg
 BTARD_API int btard_verify_projections(const btard_verify_args* args);
 
 /*
+ * Aggregation and verification of Alg. 2 line 5 and Alg. 6 lines 6-14 in one call: the same results as
+ * btard_centered_clip(clip) followed by btard_verify_projections(verify) on the aggregate it returned.
+ * `verify` supplies the seed, n_z, partition_base, its outputs and its own workspace; its g, v, part_len,
+ * tau, resid_norm_in and stream are taken from `clip` (what it holds there is ignored), and its n_peers,
+ * n_partitions and row_stride must equal clip's.  Both workspaces are sized by the two *_workspace()
+ * queries as for the separate calls.
+ * What the one call buys: with BTARD_ALGO_GRAM, n_peers <= 16 and n_z <= 2 the pass that forms v from
+ * the coefficients and the verification pass are one read of g instead of two (the clip weights inside
+ * that pass come from the Gram matrix, the reported norms and weights from the pass itself; they agree
+ * to rounding).  Every other combination runs the two calls back to back.
+ */
+BTARD_API int btard_centered_clip_verify(const btard_cclip_args* clip, const btard_verify_args* verify);
+
+/*
  * Per-part gradient clipping of BTARD-Clipped-SGD (Alg. 9 and the paragraph after it):
  *     g~_i(l) = min{1, lambda / ||g_i(l)||_2} g_i(l)
  * applied IN PLACE to g [P][n][row_stride] (row i of slab l is g_i(l)) before it is aggregated.

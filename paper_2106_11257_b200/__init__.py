@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     STATUS_NONFINITE_ROW, BtardError, lib, library_path, partition_layout, centered_clip,
     centered_clip_workspace, verify_projections, verify_projections_workspace, random_vector,
     aggregate_host, aggregate_host_scratch, kernel_launch_count, last_cuda_error, EXPORTS,
-    profile_enable, profile_collect, KERNEL_KINDS, verify_projections_static, verification_checks, preclip, split_gradients, merge_partitions, hash_partitions,
+    profile_enable, profile_collect, KERNEL_KINDS, verify_projections_static, verification_checks, preclip, centered_clip_verify, split_gradients, merge_partitions, hash_partitions,
 )

@@ -23,7 +23,7 @@ EXPORTS = [
     "btard_kernel_launch_count", "btard_profile_enable", "btard_profile_collect",
     "btard_verify_projections_static", "btard_verification_checks", "btard_preclip_workspace",
     "btard_preclip", "btard_split_gradients", "btard_merge_partitions",
-    "btard_hash_partitions_workspace", "btard_hash_partitions",
+    "btard_hash_partitions_workspace", "btard_hash_partitions", "btard_centered_clip_verify",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -118,6 +118,8 @@ def lib():
         L.btard_verify_projections.argtypes = [C.POINTER(VerifyArgs)]
         L.btard_verify_projections_static.restype = C.c_int
         L.btard_verify_projections_static.argtypes = [C.POINTER(VerifyArgs)]
+        L.btard_centered_clip_verify.restype = C.c_int
+        L.btard_centered_clip_verify.argtypes = [C.POINTER(CclipArgs), C.POINTER(VerifyArgs)]
         L.btard_preclip_workspace.restype = C.c_size_t
         L.btard_preclip_workspace.argtypes = [C.POINTER(PreclipArgs)]
         L.btard_preclip.restype = C.c_int
@@ -288,6 +290,66 @@ def verify_projections(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None, 
         res["resid_sum"] = rs
     res["workspace"] = workspace
     return res
+
+
+def centered_clip_verify(g, tau, seed, K=1, part_len=None, init_mode=INIT_ZERO, v=None,
+                         stop_mode=STOP_FIXED_ITERS, max_iters=1, eps=0.0, algo=ALGO_DIRECT, partition_base=0,
+                         want_resid_sum=False, workspaces=None, out=None, stream=None):
+    """btard_centered_clip_verify: aggregation and verification in one call.  Returns (clip, verify), the
+    dicts that centered_clip and verify_projections return.  workspaces / out: optional pairs to reuse."""
+    torch = _torch()
+    assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
+    P, n, stride = g.shape
+    ln = _host_arr(stride if part_len is None else part_len, P, np.int64)
+    tau_h = _host_arr(tau, P, np.float64)
+    dev = g.device
+    if v is None:
+        assert init_mode != INIT_CALLER_V0, "CALLER_V0 needs v"
+        v = torch.empty((P, stride), dtype=torch.float32, device=dev)
+    assert v.is_cuda and v.dtype == torch.float32 and v.is_contiguous() and v.numel() == P * stride
+    f64 = dict(dtype=torch.float64, device=dev)
+    oc, ov = out if out is not None else (None, None)
+    if oc is None:
+        oc = dict(iters=torch.empty(P, dtype=torch.int32, device=dev), last_step_norm=torch.empty(P, **f64),
+                  resid_norm=torch.empty((P, n), **f64), status=torch.empty(P, dtype=torch.int32, device=dev))
+    if ov is None:
+        ov = dict(norm=torch.empty((P, n), **f64), weight=torch.empty((P, n), **f64),
+                  dot=torch.empty((P, n, K), **f64), s=torch.empty((P, n, K), **f64),
+                  s_sum=torch.empty((P, K), **f64), znorm2=torch.empty((P, K), **f64),
+                  resid_sum_norm=torch.empty(P, **f64), status=torch.empty(P, dtype=torch.int32, device=dev))
+    rs = None
+    if want_resid_sum:
+        rs = ov.get("resid_sum")
+        if rs is None:
+            rs = torch.zeros((P, stride), dtype=torch.float32, device=dev)
+    wc, wv = workspaces if workspaces is not None else (None, None)
+    if wc is None:
+        wc = torch.empty(centered_clip_workspace(n, P, stride, stop_mode, algo), dtype=torch.uint8, device=dev)
+    if wv is None:
+        wv = torch.empty(verify_projections_workspace(n, P, stride, K), dtype=torch.uint8, device=dev)
+    ca = CclipArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
+                   g=g.data_ptr(), tau=tau_h.ctypes.data, init_mode=init_mode, algo=algo,
+                   stop_mode=stop_mode, max_iters=max_iters, eps=eps, v=v.data_ptr(),
+                   iters=oc["iters"].data_ptr(), last_step_norm=oc["last_step_norm"].data_ptr(),
+                   resid_norm=oc["resid_norm"].data_ptr(), status=oc["status"].data_ptr(),
+                   workspace=wc.data_ptr(), workspace_bytes=wc.numel(), stream=_stream_ptr(stream),
+                   rule=RULE_CENTERED_CLIP)
+    va = VerifyArgs(n_peers=n, n_partitions=P, row_stride=stride, seed=int(seed), n_z=K,
+                    partition_base=partition_base,
+                    norm=ov["norm"].data_ptr(), weight=ov["weight"].data_ptr(), dot=ov["dot"].data_ptr(),
+                    s=ov["s"].data_ptr(), s_sum=ov["s_sum"].data_ptr(), znorm2=ov["znorm2"].data_ptr(),
+                    resid_sum_norm=ov["resid_sum_norm"].data_ptr(),
+                    resid_sum=rs.data_ptr() if rs is not None else None, status=ov["status"].data_ptr(),
+                    workspace=wv.data_ptr(), workspace_bytes=wv.numel())
+    with torch.cuda.device(dev):
+        _check(lib().btard_centered_clip_verify(C.byref(ca), C.byref(va)), "btard_centered_clip_verify")
+    rc, rv = dict(oc), dict(ov)
+    rc["v"] = v
+    rc["workspace"] = wc
+    if rs is not None:
+        rv["resid_sum"] = rs
+    rv["workspace"] = wv
+    return rc, rv
 
 
 def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None,

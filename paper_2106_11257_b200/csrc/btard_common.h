@@ -176,7 +176,28 @@ struct VerifyLaunch {
     int n, P, K, k0, kc;      // this launch covers z indices k0 .. k0+kc-1
     int p_base;
     uint32_t seed_lo, seed_hi;
+    // Fused with the combine pass of the Gram variant (n <= 16, K <= 2 only): v holds v0 on entry and
+    // receives v = v0 + sum_j coef_j (x_j - v0); the norms come out of this pass (norm_in is not read).
+    int combine;
+    float* v_out;                 // == v
+    const double* coef;           // device [P][n]
+    const double* gram;           // device [P][gram_entries] blocks of G = (g - v0)(g - v0)^T
+    int gram_entries, gram_nb;
+    double* resid_norm_out;       // device [P][n]: the aggregation's resid_norm output
+    uint32_t* cclip_status;       // device [P]: the aggregation's status word (bits are OR-ed in)
+    const unsigned int* gram_error;   // device: a bounded wait of the Gram kernel expired
 };
+
+// Where entry (i, j) of a partition's Gram matrix sits: upper-triangular 8 x 8 blocks, NB = ceil(n / 8)
+// blocks per side, a diagonal block stored whole.
+__host__ __device__ inline int gram_entry_index(int NB, int i, int j)
+{
+    const int i0 = i < j ? i : j, j0 = i < j ? j : i;
+    const int bi = i0 >> 3, bj = j0 >> 3;
+    int blk = bj - bi;
+    for (int q = 0; q < bi; ++q) blk += NB - q;
+    return blk * 64 + (i0 & 7) * 8 + (j0 & 7);
+}
 
 struct VerifyGeometry {
     Geometry g;

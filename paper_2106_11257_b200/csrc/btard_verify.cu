@@ -215,11 +215,18 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
 // rows x 4 columns in registers, as in the CenteredClip passes), so it draws the z quads of those
 // columns itself.  Each quad of z is still generated exactly once per launch, nothing is staged in
 // shared memory and the tile loop has no barrier.  Same per-CTA slot layout as verify_kernel.
-template <int R, int KT>
+// COMBINE: the pass also forms v = v0 + sum_j a_j (x_j - v0) from the coefficients of the Gram variant
+// (the combine pass and the verification pass in one read of the rows): v holds v0 on entry, every
+// thread rewrites its own 4 columns, and the squared residual norms at the new v are one more set of
+// per-row sums (slot entries behind the others).  The clip weights that the clipped-residual sum needs
+// before the norms of this pass exist come from the Gram matrix: rho_i^2 = G_ii - 2 (G a)_i + a^T G a.
+template <int R, int KT, bool COMBINE>
 __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
 {
     __shared__ float sh_w[16];
-    __shared__ double sh_red[8][R * KT + KT + 1];
+    __shared__ float sh_c[16];                      // COMBINE: coefficients a_j
+    __shared__ double sh_ga[17];                    // COMBINE: (G a)_i, then a^T G a
+    __shared__ double sh_red[8][R * KT + KT + 1 + (COMBINE ? R : 0)];
 
     const VerifyLaunch& a = k.a;
     const int n = a.n, cpp = k.cpp;
@@ -229,7 +236,38 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
     const long long stride = a.stride, len = a.table[p].len;
     const double tau = a.table[p].tau;
 
-    if (tid < 16) {
+    if (COMBINE) {
+        const double* G = a.gram + (size_t)p * a.gram_entries;
+        const double* cf = a.coef + (size_t)p * n;
+        if (tid < 16) {
+            double ga = 0.0;
+            if (tid < n)
+                for (int q = 0; q < n; ++q) {
+                    const double cq = cf[q];
+                    if (cq != 0.0) ga += G[gram_entry_index(a.gram_nb, tid, q)] * cq;   // weight-0 rows are skipped
+                }
+            sh_ga[tid] = ga;
+            sh_c[tid] = (tid < n) ? (float)cf[tid] : 0.0f;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double aga = 0.0;
+            for (int q = 0; q < n; ++q)
+                if (cf[q] != 0.0) aga += cf[q] * sh_ga[q];
+            sh_ga[16] = aga;
+        }
+        __syncthreads();
+        if (tid < 16) {
+            float w = 0.0f;
+            if (tid < n) {
+                double rho2 = G[gram_entry_index(a.gram_nb, tid, tid)] - 2.0 * sh_ga[tid] + sh_ga[16];
+                if (rho2 < 0.0) rho2 = 0.0;
+                const double rho = sqrt(rho2);
+                if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+            }
+            sh_w[tid] = w;
+        }
+    } else if (tid < 16) {
         float w = 0.0f;
         if (tid < n) {
             const double rho = a.norm_in[(size_t)p * n + tid];
@@ -239,6 +277,9 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
     }
     __syncthreads();
 
+    float nacc[COMBINE ? R : 1];                       // COMBINE: squared residual norms at the new v
+#pragma unroll
+    for (int r = 0; r < (COMBINE ? R : 1); ++r) nacc[r] = 0.0f;
     float acc[R][KT];
 #pragma unroll
     for (int r = 0; r < R; ++r)
@@ -297,6 +338,30 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
                 x[r].w = 0.f;
             }
         }
+        if (COMBINE) {
+            // x holds the residuals at v0: move v by u = sum_j a_j (x_j - v0), then the residuals by what v
+            // really moved (the rounded difference), and add up the squared norms at the new v
+            float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float cr = sh_c[r];
+                if (cr != 0.0f) {                      // coefficient 0: the row is left out, not multiplied
+                    u.x = fmaf(cr, x[r].x, u.x); u.y = fmaf(cr, x[r].y, u.y);
+                    u.z = fmaf(cr, x[r].z, u.z); u.w = fmaf(cr, x[r].w, u.w);
+                }
+            }
+            const float4 vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+            const float4 dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
+            const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len, m3 = col + 3 < len;
+            *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) =
+                make_float4(m0 ? vn.x : 0.f, m1 ? vn.y : 0.f, m2 ? vn.z : 0.f, m3 ? vn.w : 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = m0 ? x[r].x - dv.x : 0.f; x[r].y = m1 ? x[r].y - dv.y : 0.f;
+                x[r].z = m2 ? x[r].z - dv.z : 0.f; x[r].w = m3 ? x[r].w - dv.w : 0.f;
+                nacc[r] += fmaf(x[r].x, x[r].x, fmaf(x[r].y, x[r].y, fmaf(x[r].z, x[r].z, x[r].w * x[r].w)));
+            }
+        }
 #pragma unroll
         for (int q = 0; q < KT; ++q) {
             zz[q] += fmaf(z[q].x, z[q].x, fmaf(z[q].y, z[q].y, fmaf(z[q].z, z[q].z, z[q].w * z[q].w)));
@@ -339,11 +404,19 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
         const double s = warp_sum((double)rs2);
         if (lane == 0) sh_red[warp][R * KT + KT] = s;
     }
+    if (COMBINE) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const double s = warp_sum((double)nacc[r]);
+            if (lane == 0) sh_red[warp][R * KT + KT + 1 + r] = s;
+        }
+    }
     __syncthreads();
     double* dst = a.part_out + ((size_t)p * cpp + j) * k.slots;
-    const int total = n * KT + KT + 1;
+    // slot: [n KT] dots, [KT] znorm2, the resid-sum slot, then (COMBINE) [n] squared norms
+    const int total = n * KT + KT + 1 + (COMBINE ? n : 0);
     for (int e = tid; e < total; e += CL) {
-        const int col = (e < n * KT) ? e : R * KT + (e - n * KT);   // rows, then znorm2, then the resid-sum slot
+        const int col = (e < n * KT) ? e : R * KT + (e - n * KT);
         double s = 0.0;
         for (int u = 0; u < 8; ++u) s += sh_red[u][col];
         dst[e] = s;
@@ -358,17 +431,18 @@ __global__ void verify_finalize_kernel(const VArgs k, int KT)
     __shared__ float sh_wf[BTARD_MAX_PEERS];
     const VerifyLaunch& a = k.a;
     const int p = blockIdx.x, n = a.n, K = a.K;
-    const int total = n * KT + KT + 1;
+    const int total = n * KT + KT + 1 + (a.combine ? n : 0);
     const double* src = a.part_out + (size_t)p * k.cpp * k.slots;
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
         double s = 0.0;
         for (int c = 0; c < k.cpp; ++c) s += src[(size_t)c * k.slots + e];
         sh_v[e] = s;
     }
+    if (a.combine) __syncthreads();                  // the norms below come from the sums above
     const double tau = a.table[p].tau;
     bool bad = false;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const double rho = a.norm_in[(size_t)p * n + i];
+        const double rho = a.combine ? sqrt(sh_v[n * KT + KT + 1 + i]) : a.norm_in[(size_t)p * n + i];
         float w = 0.0f;
         if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
         else bad = true;
@@ -377,10 +451,15 @@ __global__ void verify_finalize_kernel(const VArgs k, int KT)
             a.norm[(size_t)p * n + i] = rho;
             a.weight[(size_t)p * n + i] = (double)w;
         }
+        if (a.combine) a.resid_norm_out[(size_t)p * n + i] = rho;
     }
     if (a.k0 == 0 && threadIdx.x == 0) a.status[p] = 0;
     __syncthreads();
     if (bad) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
+    if (a.combine) {                                 // what the aggregation's own last kernel would have reported
+        if (bad) atomicOr(&a.cclip_status[p], BTARD_STATUS_NONFINITE_ROW);
+        if (threadIdx.x == 0 && a.gram_error && *a.gram_error) atomicOr(&a.cclip_status[p], BTARD_STATUS_WAIT_EXPIRED);
+    }
     for (int e = threadIdx.x; e < n * a.kc; e += blockDim.x) {
         const int i = e / a.kc, q = e % a.kc;
         const double d = sh_v[i * KT + q];
@@ -504,8 +583,13 @@ template <int R>
 int launch_rows_r(const VArgs& va, int KT, int grid, cudaStream_t st)
 {
     prof_begin(KIND_VERIFY, st);
-    if (KT == 1) verify_rows_kernel<R, 1><<<grid, 256, 0, st>>>(va);
-    else verify_rows_kernel<R, 2><<<grid, 256, 0, st>>>(va);
+    if (va.a.combine) {
+        if (KT == 1) verify_rows_kernel<R, 1, true><<<grid, 256, 0, st>>>(va);
+        else verify_rows_kernel<R, 2, true><<<grid, 256, 0, st>>>(va);
+    } else {
+        if (KT == 1) verify_rows_kernel<R, 1, false><<<grid, 256, 0, st>>>(va);
+        else verify_rows_kernel<R, 2, false><<<grid, 256, 0, st>>>(va);
+    }
     prof_end(KIND_VERIFY, st);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
@@ -516,12 +600,12 @@ int rows_ctas_per_sm(int R, int KT)
 {
     int nb = 0;
     cudaError_t e;
-    if (R == 4) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 1>, 256, 0)
-                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 2>, 256, 0);
-    else if (R == 8) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 1>, 256, 0)
-                                   : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 2>, 256, 0);
-    else e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 1>, 256, 0)
-                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 2>, 256, 0);
+    if (R == 4) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 1, false>, 256, 0)
+                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 2, false>, 256, 0);
+    else if (R == 8) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 1, false>, 256, 0)
+                                   : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 2, false>, 256, 0);
+    else e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 1, false>, 256, 0)
+                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 2, false>, 256, 0);
     if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 2; }
     return nb;
 }
@@ -542,7 +626,7 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
         vg.KT = K;
         g.slots = sm_count() * rows_ctas_per_sm(g.R, K);
         g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, g.slots);
-        vg.slots = n * K + K + 1;
+        vg.slots = n * K + K + 1 + n;      // room for the squared norms of the fused combine pass
         return vg;
     }
     g.R = (n <= 16) ? 4 : 8;

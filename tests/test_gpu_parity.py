@@ -427,6 +427,49 @@ def test_verify_matches_oracle(n, K):
     check_verify(out2, ref2, K)
 
 
+@pytest.mark.parametrize("algo", [btard.ALGO_GRAM, btard.ALGO_DIRECT])
+@pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (7, 2), (16, 1), (16, 2), (16, 3), (23, 1), (64, 2)])
+def test_one_call_aggregation_and_verification(n, K, algo):
+    """btard_centered_clip_verify against the oracle's aggregation followed by its verification.  With the
+    Gram variant, n <= 16 and K <= 2 the combine and verification passes are one kernel; the other
+    shapes take the two calls back to back.  A third of the rows are 100x farther than the rest."""
+    rng = np.random.default_rng(500 + 7 * n + K)
+    P, stride = 3, 40_032                     # several CTAs per partition, many tiles, a ragged tail
+    lens = np.array([40_032, 33_001, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.5, 1.0, 2.0])
+    seed = 0x5EED0000 + n
+    refc = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=9)
+    gd = torch.from_numpy(g).cuda()
+    rc, rv = btard.centered_clip_verify(gd, tau, seed, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                        max_iters=9, algo=algo, partition_base=2, want_resid_sum=True)
+    torch.cuda.synchronize()
+    check_cclip(rc, refc, lens)
+    # the oracle verifies the aggregate the GPU produced (fp32), with the norms the GPU reported
+    v32 = cpu(rc["v"])
+    refv = oracle.verify(g, v32, tau, seed, K=K, part_len=lens, first_partition=2, want_resid_sum=True)
+    check_verify(rv, refv, K)
+    for p in range(P):
+        L = lens[p]
+        scale = (refv["weight"][p] * refv["norm"][p]).sum()
+        assert np.linalg.norm(cpu(rv["resid_sum"])[p, :L] - refv["resid_sum"][p, :L]) <= RTOL * scale
+    assert np.array_equal(cpu(rc["status"]), np.zeros(P, dtype=np.int32))
+
+
+def test_one_call_reports_a_non_finite_row():
+    rng = np.random.default_rng(77)
+    P, n, stride = 2, 8, 4096
+    lens = np.array([4096, 4001])
+    g = make_case(rng, P, n, stride, lens)
+    g[1, 3, 17] = np.inf
+    rc, rv = btard.centered_clip_verify(torch.from_numpy(g).cuda(), 1.0, 5, K=1, part_len=lens,
+                                        init_mode=btard.INIT_MEAN, max_iters=4, algo=btard.ALGO_GRAM)
+    torch.cuda.synchronize()
+    assert cpu(rc["status"])[1] & btard.STATUS_NONFINITE_ROW and not cpu(rc["status"])[0] & btard.STATUS_NONFINITE_ROW
+    assert cpu(rv["status"])[1] & btard.STATUS_NONFINITE_ROW
+    assert cpu(rv["weight"])[1, 3] == 0.0
+
+
 def test_verify_partition_base_keys_z():
     rng = np.random.default_rng(9)
     P, n, stride, K = 2, 4, 1024, 2
