@@ -111,8 +111,7 @@ def algorithmic_bytes(w, iters, gram=False):
     n, stride = w.n, w.row_stride
     per_pass = n * stride * 4 * (1.0 + 2.0 / n)
     input_only = n * stride * 4
-    fused = gram and n <= 16 and w.K <= 2            # combine and verification in one pass
-    passes = [2 if fused else 3 for _ in iters] if gram else [2 + int(i) for i in iters]
+    passes = [2 for _ in iters] if gram else [2 + int(i) for i in iters]   # Gram: combine and verification are one pass
     return sum(passes) * input_only, sum(passes) * per_pass, passes
 
 
@@ -326,8 +325,7 @@ def run_ours(args):
                    "max_iters": w.max_iters, "eps": w.eps, "K": w.K,
                    "iters_per_partition": [int(i) for i in iters],
                    "not_converged_partitions": int((status & 1).sum()),
-                   "passes_counted": (("1 Gram + 1 combine-and-verify per partition" if (w.n <= 16 and w.K <= 2)
-                                       else "1 Gram + 1 combine + 1 verify per partition") if args.algo == "gram"
+                   "passes_counted": ("1 Gram + 1 combine-and-verify per partition" if args.algo == "gram"
                                       else "1 init + iters + 1 verify per partition"),
                    "l2": "input (%.0f MB) larger than L2 (126 MB), no flush" % (g.numel() * 4 / 1e6),
                    "kernel_events": "per-kernel durations come from a second run of the same K steps",

@@ -202,10 +202,10 @@ BTARD_API int btard_verify_projections(const btard_verify_args* args);
  * tau, resid_norm_in and stream are taken from `clip` (what it holds there is ignored), and its n_peers,
  * n_partitions and row_stride must equal clip's.  Both workspaces are sized by the two *_workspace()
  * queries as for the separate calls.
- * What the one call buys: with BTARD_ALGO_GRAM, n_peers <= 16 and n_z <= 2 the pass that forms v from
- * the coefficients and the verification pass are one read of g instead of two (the clip weights inside
- * that pass come from the Gram matrix, the reported norms and weights from the pass itself; they agree
- * to rounding).  Every other combination runs the two calls back to back.
+ * What the one call buys: with BTARD_ALGO_GRAM the pass that forms v from the coefficients and the
+ * verification pass are one read of g instead of two (the clip weights inside that pass come from the
+ * Gram matrix, the reported norms and weights from the pass itself; they agree to rounding).  The other
+ * algorithms run the two calls back to back.
  */
 BTARD_API int btard_centered_clip_verify(const btard_cclip_args* clip, const btard_verify_args* verify);
 

@@ -231,7 +231,8 @@ size_t btard_centered_clip_workspace(const btard_cclip_args* a)
 static int check_verify_args(const btard_verify_args* a);
 static bool fusable(const btard_cclip_args* c, const btard_verify_args* v)
 {
-    return c->algo == BTARD_ALGO_GRAM && c->rule == BTARD_RULE_CENTERED_CLIP && c->n_peers <= 16 && v->n_z <= 2;
+    (void)v;
+    return c->algo == BTARD_ALGO_GRAM && c->rule == BTARD_RULE_CENTERED_CLIP;
 }
 static int launch_fused_verify(const btard_cclip_args* c, const btard_verify_args* v, const PartEntry* table,
                                const double* coef, const double* gram, const GramGeometry& gg,
@@ -446,7 +447,7 @@ static int launch_fused_verify(const btard_cclip_args* c, const btard_verify_arg
     const VerifyGeometry vg = verify_geometry(n, P, c->row_stride, K);
     const Geometry cg = cclip_geometry(n, P, c->row_stride);
     const VerifyWorkspace ws = verify_ws_layout(n, P, vg, cg);
-    if (!vg.own_z || a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
+    if (a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
     char* base = (char*)a->workspace;
     VerifyLaunch V{};
     V.g = c->g; V.v = c->v; V.v_out = c->v; V.table = table; V.norm_in = nullptr;
@@ -456,10 +457,19 @@ static int launch_fused_verify(const btard_cclip_args* c, const btard_verify_arg
     V.znorm2 = a->znorm2; V.resid_sum_norm = a->resid_sum_norm; V.status = a->status;
     V.stride = c->row_stride; V.n = n; V.P = P; V.K = K; V.p_base = a->partition_base;
     V.seed_lo = (uint32_t)a->seed; V.seed_hi = (uint32_t)(a->seed >> 32);
-    V.k0 = 0; V.kc = K;
-    V.combine = 1; V.coef = coef; V.gram = gram; V.gram_entries = gg.entries; V.gram_nb = gg.NB;
+    V.coef = coef; V.gram = gram; V.gram_entries = gg.entries; V.gram_nb = gg.NB;
     V.resid_norm_out = c->resid_norm; V.cclip_status = c->status; V.gram_error = gram_error;
-    return launch_verify(V, vg, st);
+    // The first group of directions carries the combine; further groups (K beyond what one launch
+    // holds) are plain verification launches on the v and the norms the first one left.
+    for (int k0 = 0; k0 < K; k0 += vg.KT) {
+        V.k0 = k0;
+        V.kc = (K - k0 < vg.KT) ? K - k0 : vg.KT;
+        V.combine = (k0 == 0) ? 1 : 0;
+        V.norm_in = (k0 == 0) ? nullptr : c->resid_norm;
+        const int rc = launch_verify(V, vg, st);
+        if (rc != BTARD_OK) return rc;
+    }
+    return BTARD_OK;
 }
 
 int btard_centered_clip_verify(const btard_cclip_args* c, const btard_verify_args* v)

@@ -26,12 +26,17 @@ struct VArgs {
 };
 
 // slot layout per CTA: [n*KT] dots (row-major i, k), [KT] znorm2, [1] squared norm of resid_sum
-template <int R, int KT>
+// COMBINE: as in verify_rows_kernel, the pass first forms v = v0 + sum_j a_j (x_j - v0) from the
+// coefficients of the Gram variant.  The row groups' partial moves of v are exchanged through shared
+// memory before the CTA barrier that the z block needs anyway, so the tile loop keeps one barrier.
+template <int R, int KT, bool COMBINE>
 __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
 {
-    extern __shared__ float4 sh_dyn[];   // z: [2][KT][CL], then column sums: [2][RG][CL]
+    extern __shared__ float4 sh_dyn[];   // z: [2][KT][CL], column sums: [2][RG][CL], (COMBINE) moves of v: [2][RG][CL]
     __shared__ float sh_w[BTARD_MAX_PEERS];
-    __shared__ double sh_red[16][R * KT + KT + 1];
+    __shared__ float sh_c[COMBINE ? BTARD_MAX_PEERS : 1];          // coefficients a_j
+    __shared__ double sh_ga[COMBINE ? BTARD_MAX_PEERS + 1 : 1];    // (G a)_i, then a^T G a
+    __shared__ double sh_red[16][R * KT + KT + 1 + (COMBINE ? R : 0)];
 
     const VerifyLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
@@ -42,19 +47,54 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     const double tau = a.table[p].tau;
     float4* sh_z = sh_dyn;
     float4* sh_s = sh_dyn + 2 * KT * CL;
+    float4* sh_u = sh_s + 2 * RG * CL;
 
-    for (int i = tid; i < n; i += nthr) {
-        const double rho = a.norm_in[(size_t)p * n + i];
-        float w = 0.0f;
-        if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
-        sh_w[i] = w;
+    if (COMBINE) {
+        // clip weights from the Gram matrix: rho_i^2 = G_ii - 2 (G a)_i + a^T G a (rows with a_j = 0 are skipped)
+        const double* G = a.gram + (size_t)p * a.gram_entries;
+        const double* cf = a.coef + (size_t)p * n;
+        for (int i = tid; i < n; i += nthr) {
+            double ga = 0.0;
+            for (int q = 0; q < n; ++q) {
+                const double cq = cf[q];
+                if (cq != 0.0) ga += G[gram_entry_index(a.gram_nb, i, q)] * cq;
+            }
+            sh_ga[i] = ga;
+            sh_c[i] = (float)cf[i];
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double aga = 0.0;
+            for (int q = 0; q < n; ++q)
+                if (cf[q] != 0.0) aga += cf[q] * sh_ga[q];
+            sh_ga[n] = aga;
+        }
+        __syncthreads();
+        for (int i = tid; i < n; i += nthr) {
+            double rho2 = G[gram_entry_index(a.gram_nb, i, i)] - 2.0 * sh_ga[i] + sh_ga[n];
+            if (rho2 < 0.0) rho2 = 0.0;
+            const double rho = sqrt(rho2);
+            float w = 0.0f;
+            if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+            sh_w[i] = w;
+        }
+    } else {
+        for (int i = tid; i < n; i += nthr) {
+            const double rho = a.norm_in[(size_t)p * n + i];
+            float w = 0.0f;
+            if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+            sh_w[i] = w;
+        }
     }
     __syncthreads();
     float w[R];
+    float cw[COMBINE ? R : 1];                         // this thread's coefficients
+    float nacc[COMBINE ? R : 1];                       // squared residual norms at the new v
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         const int i = rg * R + r;
         w[r] = (i < n) ? sh_w[i] : 0.0f;
+        if (COMBINE) { cw[r] = (i < n) ? sh_c[i] : 0.0f; nacc[r] = 0.0f; }
     }
 
     float acc[R][KT];
@@ -131,11 +171,46 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
             }
             zb[kq * CL + cq] = z;
         }
+        if (COMBINE) {
+            // residuals at v0 and this row group's share of the move of v, published before the barrier
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = m0 ? x[r].x - v4.x : 0.f; x[r].y = m1 ? x[r].y - v4.y : 0.f;
+                x[r].z = m2 ? x[r].z - v4.z : 0.f; x[r].w = m3 ? x[r].w - v4.w : 0.f;
+            }
+            float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                if (cw[r] != 0.0f) {                   // coefficient 0: the row is left out, not multiplied
+                    u.x = fmaf(cw[r], x[r].x, u.x); u.y = fmaf(cw[r], x[r].y, u.y);
+                    u.z = fmaf(cw[r], x[r].z, u.z); u.w = fmaf(cw[r], x[r].w, u.w);
+                }
+            }
+            sh_u[(size_t)par * RG * CL + rg * CL + cl] = u;
+        }
         __syncthreads();
         if (first_chunk && qb > q0) consume_sums(qb - CL, par ^ 1);
 
         // 2. residuals of this thread's rows and columns
-        if (m3) {                                      // whole quad inside the data: no predicates
+        if (COMBINE) {
+            const float4* ub = sh_u + (size_t)par * RG * CL;
+            float4 u = ub[cl];
+            for (int q = 1; q < RG; ++q) {
+                const float4 o = ub[q * CL + cl];
+                u.x += o.x; u.y += o.y; u.z += o.z; u.w += o.w;
+            }
+            const float4 vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+            const float4 dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);   // what v really moved by
+            if (rg == 0 && valid)
+                *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) =
+                    make_float4(m0 ? vn.x : 0.f, m1 ? vn.y : 0.f, m2 ? vn.z : 0.f, m3 ? vn.w : 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r].x = m0 ? x[r].x - dv.x : 0.f; x[r].y = m1 ? x[r].y - dv.y : 0.f;
+                x[r].z = m2 ? x[r].z - dv.z : 0.f; x[r].w = m3 ? x[r].w - dv.w : 0.f;
+                nacc[r] += fmaf(x[r].x, x[r].x, fmaf(x[r].y, x[r].y, fmaf(x[r].z, x[r].z, x[r].w * x[r].w)));
+            }
+        } else if (m3) {                               // whole quad inside the data: no predicates
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
@@ -194,18 +269,30 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
         const double s = warp_sum((double)rs2);
         if (lane == 0) sh_red[warp][R * KT + KT] = s;
     }
+    if (COMBINE) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const double s = warp_sum((double)nacc[r]);
+            if (lane == 0) sh_red[warp][R * KT + KT + 1 + r] = s;
+        }
+    }
     __syncthreads();
     double* dst = a.part_out + ((size_t)p * cpp + j) * k.slots;
-    const int total = n * KT + KT + 1;
+    // slot: [n KT] dots, [KT] znorm2, the resid-sum slot, then (COMBINE) [n] squared norms
+    const int total = n * KT + KT + 1 + (COMBINE ? n : 0);
     for (int e = tid; e < total; e += nthr) {
         double s = 0.0;
         if (e < n * KT) {
             const int i = e / KT, q = e % KT;
             const int g0 = (i / R) * wpg;
             for (int u = 0; u < wpg; ++u) s += sh_red[g0 + u][(i % R) * KT + q];
-        } else {
+        } else if (e < n * KT + KT + 1) {
             const int q = e - n * KT;                  // znorm2 slots, then the resid-sum slot
             for (int u = 0; u < wpg; ++u) s += sh_red[u][R * KT + q];
+        } else {
+            const int i = e - (n * KT + KT + 1);       // squared norm of row i at the new v
+            const int g0 = (i / R) * wpg;
+            for (int u = 0; u < wpg; ++u) s += sh_red[g0 + u][R * KT + KT + 1 + (i % R)];
         }
         dst[e] = s;
     }
@@ -537,7 +624,8 @@ template <int R, int KT>
 int launch_rk(const VArgs& va, int threads, size_t smem, int grid, cudaStream_t st)
 {
     prof_begin(KIND_VERIFY, st);
-    verify_kernel<R, KT><<<grid, threads, smem, st>>>(va);
+    if (va.a.combine) verify_kernel<R, KT, true><<<grid, threads, smem, st>>>(va);
+    else verify_kernel<R, KT, false><<<grid, threads, smem, st>>>(va);
     prof_end(KIND_VERIFY, st);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
@@ -560,11 +648,11 @@ template <int R>
 int occ_r(int KT, int threads, size_t smem, int* nb)
 {
     cudaError_t e = cudaErrorInvalidValue;
-    if (KT == 1) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 1>, threads, smem);
-    else if (KT == 2) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 2>, threads, smem);
+    if (KT == 1) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 1, false>, threads, smem);
+    else if (KT == 2) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 2, false>, threads, smem);
     if constexpr (R <= 8) {
-        if (KT == 4) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 4>, threads, smem);
-        else if (KT == 8) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 8>, threads, smem);
+        if (KT == 4) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 4, false>, threads, smem);
+        else if (KT == 8) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 8, false>, threads, smem);
     }
     return (int)e;
 }
@@ -648,7 +736,7 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, g.threads, smem);
     g.slots = slots;
     g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, slots);
-    vg.slots = n * kt + kt + 1;
+    vg.slots = n * kt + kt + 1 + n;             // room for the squared norms of the fused combine pass
     return vg;
 }
 
@@ -656,7 +744,7 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
 {
     const Geometry& g = vg.g;
     VArgs va{a, g.RG, g.CL, g.tiles, g.cpp, vg.slots};
-    const size_t smem = sizeof(float4) * (2 * (size_t)vg.KT * g.CL + 2 * (size_t)g.RG * g.CL);
+    const size_t smem = sizeof(float4) * (2 * (size_t)vg.KT * g.CL + (a.combine ? 4 : 2) * (size_t)g.RG * g.CL);
     const int grid = a.P * g.cpp;
     int rc;
     if (vg.own_z) {

@@ -428,11 +428,14 @@ def test_verify_matches_oracle(n, K):
 
 
 @pytest.mark.parametrize("algo", [btard.ALGO_GRAM, btard.ALGO_DIRECT])
-@pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (7, 2), (16, 1), (16, 2), (16, 3), (23, 1), (64, 2)])
+@pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (7, 2), (16, 1), (16, 2), (16, 3), (16, 8), (23, 1), (64, 2),
+                                 (64, 4), (64, 11), (100, 2)])
 def test_one_call_aggregation_and_verification(n, K, algo):
     """btard_centered_clip_verify against the oracle's aggregation followed by its verification.  With the
-    Gram variant, n <= 16 and K <= 2 the combine and verification passes are one kernel; the other
-    shapes take the two calls back to back.  A third of the rows are 100x farther than the rest."""
+    Gram variant the combine and verification passes are one kernel (all rows of a column in one thread
+    for n <= 16 and K <= 2, row groups with a shared z block otherwise; K = 11 needs a second, plain
+    launch); the direct algorithm takes the two calls back to back.  A third of the rows are 100x
+    farther than the rest."""
     rng = np.random.default_rng(500 + 7 * n + K)
     P, stride = 3, 40_032                     # several CTAs per partition, many tiles, a ragged tail
     lens = np.array([40_032, 33_001, 13])
