@@ -173,10 +173,17 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
         }
         if (COMBINE) {
             // residuals at v0 and this row group's share of the move of v, published before the barrier
+            if (m3) {                                  // whole quad inside the data: no predicates
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                x[r].x = m0 ? x[r].x - v4.x : 0.f; x[r].y = m1 ? x[r].y - v4.y : 0.f;
-                x[r].z = m2 ? x[r].z - v4.z : 0.f; x[r].w = m3 ? x[r].w - v4.w : 0.f;
+                for (int r = 0; r < R; ++r) {
+                    x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    x[r].x = m0 ? x[r].x - v4.x : 0.f; x[r].y = m1 ? x[r].y - v4.y : 0.f;
+                    x[r].z = m2 ? x[r].z - v4.z : 0.f; x[r].w = 0.f;
+                }
             }
             float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -204,12 +211,21 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
             if (rg == 0 && valid)
                 *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) =
                     make_float4(m0 ? vn.x : 0.f, m1 ? vn.y : 0.f, m2 ? vn.z : 0.f, m3 ? vn.w : 0.f);
+            if (m3) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                x[r].x = m0 ? x[r].x - dv.x : 0.f; x[r].y = m1 ? x[r].y - dv.y : 0.f;
-                x[r].z = m2 ? x[r].z - dv.z : 0.f; x[r].w = m3 ? x[r].w - dv.w : 0.f;
-                nacc[r] += fmaf(x[r].x, x[r].x, fmaf(x[r].y, x[r].y, fmaf(x[r].z, x[r].z, x[r].w * x[r].w)));
+                for (int r = 0; r < R; ++r) {
+                    x[r].x -= dv.x; x[r].y -= dv.y; x[r].z -= dv.z; x[r].w -= dv.w;
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    x[r].x = m0 ? x[r].x - dv.x : 0.f; x[r].y = m1 ? x[r].y - dv.y : 0.f;
+                    x[r].z = m2 ? x[r].z - dv.z : 0.f; x[r].w = 0.f;
+                }
             }
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                nacc[r] += fmaf(x[r].x, x[r].x, fmaf(x[r].y, x[r].y, fmaf(x[r].z, x[r].z, x[r].w * x[r].w)));
         } else if (m3) {                               // whole quad inside the data: no predicates
 #pragma unroll
             for (int r = 0; r < R; ++r) {
