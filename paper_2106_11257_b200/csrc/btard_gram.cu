@@ -804,26 +804,37 @@ __global__ void __launch_bounds__(32) gram_iterate_warp_kernel(const GArgs k)
         if (jj == lane) gii = Grow[jj];
     const bool bad = row && !isfinite(gii);
     const bool live = row && !bad;
+    // One update is a chain of dependent double-precision operations, so the chain is kept short: one
+    // reciprocal square root instead of a square root and a division (tau / rho = tau rsqrt(rho^2)), a
+    // multiplication by 1/n, and four partial sums for G d.
+    const double tau2 = tau * tau, inv_n = 1.0 / (double)n;
     double ai = 0.0, Gai = 0.0, step2 = 0.0;
+    double aGa = 0.0;              // a^T G a, carried along: (a + d)^T G (a + d) = a^T G a + 2 d^T G a + d^T G d
     int iters = 0;
     for (int l = 0; l < a.max_iters; ++l) {
-        const double aGa = warp_allsum(live ? ai * Gai : 0.0);
         double w = 0.0;
         if (live) {
             double rho2 = gii - 2.0 * Gai + aGa;
             if (rho2 < 0.0) rho2 = 0.0;
-            const double rho = sqrt(rho2);
-            if (isfinite(rho)) w = (rho <= tau) ? 1.0 : tau / rho;
+            if (isfinite(rho2)) w = (rho2 <= tau2) ? 1.0 : tau * rsqrt(rho2);
         }
         const double W = warp_allsum(w);
-        const double d = live ? (w - W * ai) / (double)n : 0.0;
-        double Gd = 0.0;
+        const double d = live ? (w - W * ai) * inv_n : 0.0;
+        double part[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
         for (int q = 0; q < N; ++q) {
             const double dq = __shfl_sync(0xffffffffu, d, q);
-            if (dq != 0.0 && live) Gd += Grow[q] * dq;
+            if (dq != 0.0 && live) part[q & 3] += Grow[q] * dq;     // weight-0 rows are skipped, not multiplied
         }
-        step2 = warp_allsum(live ? d * Gd : 0.0);
+        const double Gd = (part[0] + part[1]) + (part[2] + part[3]);
+        double dGa = live ? d * Gai : 0.0;             // both sums ride the same butterfly
+        step2 = live ? d * Gd : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            step2 += __shfl_xor_sync(0xffffffffu, step2, o);
+            dGa += __shfl_xor_sync(0xffffffffu, dGa, o);
+        }
+        aGa += 2.0 * dGa + step2;
         ai += d;
         Gai += Gd;
         iters = l + 1;
