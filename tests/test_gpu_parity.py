@@ -459,6 +459,34 @@ def test_one_call_aggregation_and_verification(n, K, algo):
     assert np.array_equal(cpu(rc["status"]), np.zeros(P, dtype=np.int32))
 
 
+@pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
+def test_empty_partition_in_every_path(n, K):
+    """A partition without coordinates (possible when d < P): v stays 0, norms and projections are
+    empty sums, s is 0 and not 0/0; in the separate calls, the Gram variant and the one-call entry."""
+    rng = np.random.default_rng(900 + n + K)
+    P, stride = 3, 4096
+    lens = np.array([4096, 0, 17])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.5, 1.0, 2.0])
+    gd = torch.from_numpy(g).cuda()
+    refc = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=5)
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
+        _, r = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=5, algo=algo)
+        check_cclip(r, refc, lens)
+        v32 = cpu(r["v"])
+        refv = oracle.verify(g, v32, tau, 3, K=K, part_len=lens)
+        out = btard.verify_projections(gd, r["v"], tau, 3, K=K, part_len=lens, resid_norm_in=r["resid_norm"])
+        torch.cuda.synchronize()
+        check_verify(out, refv, K)
+        assert np.all(cpu(out["s"])[1] == 0.0) and np.all(cpu(out["znorm2"])[1] == 0.0)
+        rc, rv = btard.centered_clip_verify(gd, tau, 3, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                            max_iters=5, algo=algo)
+        torch.cuda.synchronize()
+        check_cclip(rc, refc, lens)
+        check_verify(rv, oracle.verify(g, cpu(rc["v"]), tau, 3, K=K, part_len=lens), K)
+        assert np.all(cpu(rv["s"])[1] == 0.0)
+
+
 def test_one_call_reports_a_non_finite_row():
     rng = np.random.default_rng(77)
     P, n, stride = 2, 8, 4096
