@@ -599,17 +599,23 @@ def test_aggregate_host_matches_device_path():
 
 
 # ----------------------------------------------------------------------------- full-size configs
-def _full_config(cfg, sample, max_iters=None, stop=None, algo=None):
+def _full_config(cfg, sample, max_iters=None, stop=None, algo=None, one_call=False):
     """Runs configuration `cfg` at full size on the GPU in the benchmark's launch configuration and
-    compares the sampled partitions with the oracle."""
+    compares the sampled partitions with the oracle.  one_call: through btard_centered_clip_verify, as
+    the benchmark does for the Gram variant."""
     w = workloads.make_workload(cfg, device="cuda")
     stop_mode = w.stop_mode if stop is None else stop
     iters = w.max_iters if max_iters is None else max_iters
-    r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
-                            stop_mode=stop_mode, max_iters=iters, eps=w.eps,
-                            algo=btard.ALGO_DIRECT if algo is None else algo)
-    o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
-                                 resid_norm_in=r["resid_norm"])
+    if one_call:
+        r, o = btard.centered_clip_verify(w.g, w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                          init_mode=btard.INIT_COORD_MEDIAN, stop_mode=stop_mode, max_iters=iters,
+                                          eps=w.eps, algo=btard.ALGO_DIRECT if algo is None else algo)
+    else:
+        r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
+                                stop_mode=stop_mode, max_iters=iters, eps=w.eps,
+                                algo=btard.ALGO_DIRECT if algo is None else algo)
+        o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                     resid_norm_in=r["resid_norm"])
     torch.cuda.synchronize()
     for p in sample:
         gp = cpu(w.g[p:p + 1])
@@ -649,6 +655,13 @@ def test_config2_and_4_gram_mode_full_size_sampled():
     _full_config(4, sample=[17], algo=btard.ALGO_GRAM)
 
 
+def test_gram_one_call_full_size_sampled():
+    """The Gram variant through the one-call entry point (fused combine-and-verify pass) at full size."""
+    _full_config(2, sample=[11], max_iters=20, stop=btard.STOP_FIXED_ITERS, algo=btard.ALGO_GRAM, one_call=True)
+    _full_config(3, sample=[6], algo=btard.ALGO_GRAM, one_call=True)
+    _full_config(4, sample=[40], algo=btard.ALGO_GRAM, one_call=True)
+
+
 def test_config5_full_size_sampled():
     """Config 5 at full size (64 GiB of rows): fixed 20 iterations and the Gram variant side by side,
     one 1 GiB partition checked against the oracle, then the verification pass (K = 4) on it."""
@@ -672,3 +685,13 @@ def test_config5_full_size_sampled():
                          norm_in=cpu(r["resid_norm"][p:p + 1]), first_partition=p)
     subo = {k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm")}
     check_verify(subo, refv, w.K)
+    # and the Gram variant through the one-call entry point (combine and verification in one pass)
+    r, o = btard.centered_clip_verify(w.g, w.tau, w.zseed, K=w.K, part_len=w.part_len,
+                                      init_mode=btard.INIT_COORD_MEDIAN, stop_mode=btard.STOP_FIXED_ITERS,
+                                      max_iters=20, algo=btard.ALGO_GRAM)
+    torch.cuda.synchronize()
+    check_cclip({k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}, ref, lens)
+    refv = oracle.verify(gp, cpu(r["v"][p:p + 1]), w.tau[p], w.zseed, K=w.K, part_len=lens,
+                         norm_in=cpu(r["resid_norm"][p:p + 1]), first_partition=p)
+    check_verify({k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm")},
+                 refv, w.K)
