@@ -743,6 +743,15 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
         g.CL = 32;
         g.threads = g.RG * g.CL;
     }
+    if (n > 16 && n <= 64 && K <= 2) {
+        // few directions: the accumulators of 16 rows per thread fit in registers, and fewer row groups
+        // exchange column sums (measured at n = 64, K = 1: 0.725 ms against 0.761 ms with 8 rows per
+        // thread; fused with the combine pass 1.10 ms against 1.23 ms)
+        g.R = 16;
+        g.RG = (n + 15) / 16;
+        g.CL = (g.RG >= 4) ? 32 : 64;
+        g.threads = g.RG * g.CL;
+    }
     int kt = 1;
     while (kt < K && kt < 8) kt <<= 1;
     if (g.R == 16 && kt > 2) kt = 2;          // 16 rows per thread: keep the accumulators in registers
