@@ -23,18 +23,32 @@ def up_to_date():
 
 
 def build(force=False, verbose=False):
+    """Compiles every translation unit on its own (in parallel) and links them into libbtard.so.  The
+    objects live in a temporary folder; only the library stays."""
     if not force and up_to_date():
         return LIB
+    import concurrent.futures
+    import shutil
+    import tempfile
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "--shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-cudart", "shared",
-           "-o", tmp] + sources()
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+             "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
+        flags += ["-Xptxas", "-v"]
+    work = tempfile.mkdtemp(prefix="btard_build_")
+    try:
+        def compile_one(src):
+            obj = os.path.join(work, os.path.basename(src) + ".o")
+            subprocess.run([nvcc] + flags + ["-c", "-o", obj, src], check=True)
+            return obj
+        with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+            objs = list(pool.map(compile_one, sources()))
+        tmp = LIB + ".tmp%d" % os.getpid()
+        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "--shared", "-cudart", "shared",
+                        "-o", tmp] + objs, check=True)
+        os.replace(tmp, LIB)
+    finally:
+        shutil.rmtree(work, ignore_errors=True)
     return LIB
 
 
