@@ -375,6 +375,18 @@ def test_gram_mode_eps_and_long_rows():
     assert np.array_equal(cpu(r["status"]) & 1, ref["status"] & 1)
 
 
+@pytest.mark.parametrize("n", [5, 20, 64])
+def test_gram_mode_on_very_short_rows(n):
+    """Rows shorter than one 32-column tile (the tensor-core kernel does not take them: the fp32 kernels do)."""
+    rng = np.random.default_rng(40 + n)
+    P, stride = 2, 28
+    lens = np.array([28, 5])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_MEAN, max_iters=6)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_MEAN, max_iters=6, algo=btard.ALGO_GRAM)
+    check_cclip(r, ref, lens)
+
+
 def test_gram_mode_rejects_too_many_peers():
     g = torch.zeros((1, 129, 64), device="cuda")
     with pytest.raises(btard.BtardError) as e:
