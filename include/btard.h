@@ -14,10 +14,17 @@
  *   - Every pointer marked "device" is owned by the caller and must stay valid until the work
  *     queued on `stream` has finished.  Pointers marked "host" are read before the call returns.
  *   - Calls that take device buffers are asynchronous on `stream` (a cudaStream_t passed as
- *     void*; NULL is the default stream), allocate nothing and never synchronise with the host.
- *     Scratch memory comes from `workspace`, sized by the matching *_workspace() query.
- *   - Return value: BTARD_OK, or a negative error; on error nothing was queued.  Conditions that
- *     only the device can see are reported per partition in `status` (BTARD_STATUS_* bits).
+ *     void*; NULL is the default stream).  They allocate nothing, on the device or on the host heap,
+ *     copy nothing from pageable memory and never wait for the device: the small host arrays
+ *     (part_len, tau) travel as arguments of a small kernel.  Scratch memory comes from `workspace`,
+ *     sized by the matching *_workspace() query.  What such a call does on the host besides the
+ *     launches: argument checks, a few device-attribute queries and, the first time a kernel is
+ *     used on a device, setting its shared-memory attribute.
+ *   - Return value: BTARD_OK, or a negative error.  Arguments and sizes (workspace included) are
+ *     checked before anything is queued, so on INVALID_ARG, BAD_ALIGNMENT, WORKSPACE_TOO_SMALL and
+ *     UNSUPPORTED nothing was queued.  BTARD_ERR_CUDA means a launch failed part-way: earlier
+ *     launches of the call may already be on the stream and the outputs are undefined.  Conditions
+ *     that only the device can see are reported per partition in `status` (BTARD_STATUS_* bits).
  */
 #ifndef BTARD_H_
 #define BTARD_H_
@@ -55,18 +62,10 @@ extern "C" {
 
 #define BTARD_ALGO_DIRECT 0         /* one pass over g per update, one kernel launch per update     */
 #define BTARD_ALGO_GRAM 1           /* Gram matrix pass + iteration in coefficient space + combine  */
-#define BTARD_ALGO_DIRECT_RESIDENT 2 /* as DIRECT, but partitions go through in chunks that fit the L2
-                                       cache, all updates of a chunk inside one cooperative kernel
-                                       with grid barriers; where a partition does not fit: DIRECT   */
-#define BTARD_ALGO_DIRECT_COOPERATIVE 3 /* as DIRECT, but all updates of all partitions inside one
+#define BTARD_ALGO_DIRECT_COOPERATIVE 2 /* as DIRECT, but all updates of all partitions inside one
                                        cooperative kernel: no launch per update and nothing runs
                                        after the last partition converged; where the device cannot
                                        launch it: DIRECT                                            */
-
-#define BTARD_ALGO_DIRECT_STAGED 4  /* as DIRECT, but for n_peers <= 16 and row_stride a multiple of 32
-                                       the update pass is fed by bulk asynchronous copies through a
-                                       ring of shared-memory stages instead of loads into registers;
-                                       other shapes: DIRECT                                         */
 
 /* Aggregation rule.  The paper's experiments (Sec. 4.1) compare CenteredClip with plain averaging,
    the coordinate-wise median and the geometric median; they run on the same streaming kernels. */
@@ -285,10 +284,11 @@ BTARD_API int btard_verification_checks(const btard_checks_args* args);
  * The call allocates nothing, on the device or on the host heap.
  *
  * The first call on each device looks up the array's device address (one driver query, with that
- * device current); make that first call outside any stream capture.  All calls on one GPU share the
- * array: calls that may overlap on the GPU (other streams or threads) race on it and must be
- * serialised by the caller.  Nothing needs to persist in it between calls; what must start at zero
- * is cleared on `stream` by each call.
+ * device current; the result is kept per device ordinal for the life of the process, so it is stale
+ * after a cudaDeviceReset).  Because that first call does this set-up, make it before any stream
+ * capture is begun on that device.  All calls on one GPU share the array: calls that may overlap on the GPU
+ * (other streams or threads) race on it and must be serialised by the caller.  Nothing needs to
+ * persist in it between calls; what must start at zero is cleared on `stream` by each call.
  */
 #define BTARD_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
 BTARD_API int btard_verify_projections_static(const btard_verify_args* args);
@@ -305,9 +305,11 @@ BTARD_API int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t p
 
 /*
  * The same aggregation + verification with HOST buffers: copies g to the device, runs
- * btard_centered_clip (DIRECT) and btard_verify_projections, copies the results back and waits for
+ * btard_centered_clip_verify with the algorithm in `algo`, copies the results back and waits for
  * `stream` (and for copy_stream, which only carries copies this call queued).  All device memory
- * comes from device_scratch (sized by btard_aggregate_host_scratch).
+ * comes from device_scratch (sized by btard_aggregate_host_scratch for the same n_peers, n_partitions,
+ * row_stride, n_z and algo).  With BTARD_ALGO_DIRECT in EPS mode the updates run in the cooperative
+ * kernel, so that nothing is launched after convergence.
  * Host output pointers may be NULL to skip that copy, except v.  Pinned host memory makes the
  * copies asynchronous and fast; pageable memory works too.
  */
@@ -343,6 +345,7 @@ typedef struct {
                                     on it while the kernels of the previous chunk run on `stream`; g must
                                     then be pinned host memory for the overlap to happen.  The chunks
                                     change no result: partitions are independent.                      */
+    int32_t algo;                /* BTARD_ALGO_DIRECT (0), BTARD_ALGO_GRAM or BTARD_ALGO_DIRECT_COOPERATIVE */
 } btard_host_args;
 
 BTARD_API size_t btard_aggregate_host_scratch(const btard_host_args* args);

@@ -5,7 +5,7 @@ this package is the ctypes binding.  There is no CPU fallback: importing works a
 call needs the compiled library and a CUDA device.
 """
 from .binding import (  # noqa: F401
-    INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN, ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT, ALGO_DIRECT_COOPERATIVE, ALGO_DIRECT_STAGED,
+    INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN, ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_COOPERATIVE,
     STOP_FIXED_ITERS, STOP_EPS, RULE_CENTERED_CLIP, RULE_GEOMETRIC_MEDIAN, RULE_MEAN, RULE_COORD_MEDIAN, SPLIT_PAPER, SPLIT_CEIL_PAD, STATUS_NOT_CONVERGED,
     STATUS_NONFINITE_ROW, BtardError, lib, library_path, partition_layout, centered_clip,
     centered_clip_workspace, verify_projections, verify_projections_workspace, random_vector,

@@ -10,7 +10,7 @@ import os
 import numpy as np
 
 INIT_CALLER_V0, INIT_ZERO, INIT_MEAN, INIT_COORD_MEDIAN = 0, 1, 2, 3
-ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_RESIDENT, ALGO_DIRECT_COOPERATIVE, ALGO_DIRECT_STAGED = 0, 1, 2, 3, 4
+ALGO_DIRECT, ALGO_GRAM, ALGO_DIRECT_COOPERATIVE = 0, 1, 2
 STOP_FIXED_ITERS, STOP_EPS = 0, 1
 RULE_CENTERED_CLIP, RULE_GEOMETRIC_MEDIAN, RULE_MEAN, RULE_COORD_MEDIAN = 0, 1, 2, 3
 SPLIT_PAPER, SPLIT_CEIL_PAD = 0, 1
@@ -70,7 +70,7 @@ class HostArgs(C.Structure):
                 ("s_sum", C.c_void_p), ("znorm2", C.c_void_p), ("resid_sum_norm", C.c_void_p),
                 ("status", C.c_void_p), ("device_scratch", C.c_void_p),
                 ("device_scratch_bytes", C.c_size_t), ("stream", C.c_void_p),
-                ("copy_stream", C.c_void_p)]
+                ("copy_stream", C.c_void_p), ("algo", C.c_int32)]
 
 
 class PreclipArgs(C.Structure):
@@ -516,14 +516,14 @@ def random_vector(seed, p, k, part_len, device="cuda", stream=None):
     return z[:int(part_len)]
 
 
-def aggregate_host_scratch(n, P, row_stride, K):
-    a = HostArgs(n_peers=n, n_partitions=P, row_stride=row_stride, n_z=K)
+def aggregate_host_scratch(n, P, row_stride, K, algo=ALGO_DIRECT):
+    a = HostArgs(n_peers=n, n_partitions=P, row_stride=row_stride, n_z=K, algo=algo)
     return int(lib().btard_aggregate_host_scratch(C.byref(a)))
 
 
 def aggregate_host(g_host, tau, seed, K=1, part_len=None, init_mode=INIT_COORD_MEDIAN, v_host=None,
                    stop_mode=STOP_FIXED_ITERS, max_iters=1, eps=0.0, scratch=None, out=None,
-                   device="cuda", stream=None, copy_stream=None):
+                   device="cuda", stream=None, copy_stream=None, algo=ALGO_DIRECT):
     """Whole aggregation + verification from HOST tensors (ideally pinned); blocks until done.
     `copy_stream` (a second torch.cuda.Stream) lets the host-to-device copy of the next chunk of
     partitions overlap the kernels of the current one.  Returns dict of host tensors."""
@@ -543,7 +543,7 @@ def aggregate_host(g_host, tau, seed, K=1, part_len=None, init_mode=INIT_COORD_M
         dot=host((P, n, K), torch.float64), s=host((P, n, K), torch.float64),
         s_sum=host((P, K), torch.float64), znorm2=host((P, K), torch.float64),
         resid_sum_norm=host(P, torch.float64), status=host(P, torch.int32))
-    need = aggregate_host_scratch(n, P, stride, K)
+    need = aggregate_host_scratch(n, P, stride, K, algo)
     if scratch is None:
         scratch = torch.empty(need, dtype=torch.uint8, device=device)
     a = HostArgs(n_peers=n, n_partitions=P, row_stride=stride, part_len=ln.ctypes.data,
@@ -556,7 +556,8 @@ def aggregate_host(g_host, tau, seed, K=1, part_len=None, init_mode=INIT_COORD_M
                  resid_sum_norm=o["resid_sum_norm"].data_ptr(), status=o["status"].data_ptr(),
                  device_scratch=scratch.data_ptr(), device_scratch_bytes=scratch.numel(),
                  stream=_stream_ptr(stream),
-                 copy_stream=C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None)
+                 copy_stream=C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None,
+                 algo=algo)
     with torch.cuda.device(scratch.device):
         _check(lib().btard_aggregate_host(C.byref(a)), "btard_aggregate_host")
     res = dict(o)

@@ -3,7 +3,7 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
-#include <vector>
+#include <vector>   // per-kernel timing records only (off by default)
 
 #include "btard_common.h"
 
@@ -75,6 +75,22 @@ int sm_count()
     return sms;
 }
 
+static unsigned long long device_bit()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return 0; }
+    return 1ull << dev;
+}
+bool device_needs_setup(const std::atomic<unsigned long long>& seen)
+{
+    const unsigned long long bit = device_bit();
+    return bit == 0 || !(seen.load(std::memory_order_acquire) & bit);
+}
+void mark_device_done(std::atomic<unsigned long long>& seen)
+{
+    seen.fetch_or(device_bit(), std::memory_order_release);
+}
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -95,7 +111,7 @@ int check_common(int n, int P, long long stride, const int64_t* part_len, const 
 struct CclipWorkspace {
     size_t table, slots, tot[2], flags, flags_bytes, v_lo, v_lo_bytes, total;
     size_t gslots, gram, coef;      // Gram variant only
-    size_t rslots, rflags, rflags_bytes;   // L2-resident variant
+    size_t rslots, rflags, rflags_bytes;   // cooperative variant only
 };
 
 constexpr int kMaxGramPeers = 128;
@@ -110,8 +126,7 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, in
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
     const bool gram = (algo == BTARD_ALGO_GRAM);
     const bool comp = (stop_mode == BTARD_STOP_EPS && !gram);
-    const StagedGeometry sg = cclip_staged_geometry(n, P, stride, comp);
-    const int cpp = (sg.ok && sg.g.cpp > geo.cpp) ? sg.g.cpp : geo.cpp;
+    const int cpp = geo.cpp;
     w.slots = off; off = align_up(off + sizeof(double) * (size_t)P * cpp * (n + 1), 256);
     w.tot[0] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
     w.tot[1] = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
@@ -125,11 +140,11 @@ CclipWorkspace cclip_ws_layout(int n, int P, long long stride, int stop_mode, in
         w.gram = off; off = align_up(off + sizeof(double) * (size_t)P * gg.entries, 256);
         w.coef = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
     }
-    size_t ritems = (size_t)P * geo.cpp;
-    if (ritems < (size_t)kResidentMaxGrid) ritems = kResidentMaxGrid;
-    w.rslots = off; off = align_up(off + sizeof(double) * 2 * ritems * (n + 1), 256);
-    w.rflags_bytes = sizeof(unsigned long long) * ((size_t)P + 1);   // a barrier word per chunk, error flag
-    w.rflags = off; off = align_up(off + w.rflags_bytes, 256);
+    if (algo == BTARD_ALGO_DIRECT_COOPERATIVE) {
+        w.rslots = off; off = align_up(off + sizeof(double) * 2 * (size_t)P * geo.cpp * (n + 1), 256);
+        w.rflags_bytes = sizeof(unsigned long long) * 2;             // barrier word, error flag
+        w.rflags = off; off = align_up(off + w.rflags_bytes, 256);
+    }
     w.total = off;
     return w;
 }
@@ -152,16 +167,53 @@ VerifyWorkspace verify_ws_layout(int n, int P, const VerifyGeometry& vg, const G
     return w;
 }
 
-int upload_table(PartEntry* dev, int P, const int64_t* part_len, const double* tau, cudaStream_t st)
+// Small host tables (two 64-bit words per partition) reach the device as kernel arguments, a batch
+// per launch: nothing is staged through pageable memory, nothing is allocated, and the launches are
+// ordinary stream work.
+constexpr int kPairBatch = 128;
+struct PairBatch {
+    unsigned long long w[2 * kPairBatch];
+    int count;
+};
+__global__ void fill_pairs_kernel(unsigned long long* dst, const PairBatch b)
 {
-    std::vector<PartEntry> host((size_t)P);
-    for (int p = 0; p < P; ++p) { host[p].len = part_len[p]; host[p].tau = tau[p]; }
-    // The source is pageable: the runtime stages it before returning, so `host` may go away.
-    BTARD_CUDA_TRY(cudaMemcpyAsync(dev, host.data(), sizeof(PartEntry) * P, cudaMemcpyHostToDevice, st));
+    const int i = threadIdx.x;
+    if (i < 2 * b.count) dst[i] = b.w[i];
+}
+
+__global__ void or_status_kernel(uint32_t* dst, const uint32_t* other, int P)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < P) dst[p] |= other[p];
+}
+
+template <class Fill>   // fill(p, &w0, &w1)
+int upload_pairs(void* dev, int P, cudaStream_t st, Fill fill)
+{
+    PairBatch b;
+    for (int p0 = 0; p0 < P; p0 += kPairBatch) {
+        b.count = (P - p0 < kPairBatch) ? P - p0 : kPairBatch;
+        for (int q = 0; q < b.count; ++q) fill(p0 + q, &b.w[2 * q], &b.w[2 * q + 1]);
+        fill_pairs_kernel<<<1, 2 * kPairBatch, 0, st>>>((unsigned long long*)dev + 2 * (size_t)p0, b);
+        BTARD_CUDA_TRY(cudaGetLastError());
+        count_launch();
+    }
     return BTARD_OK;
 }
 
 }  // namespace
+
+int upload_table(PartEntry* dev, int P, const int64_t* part_len, const double* tau, cudaStream_t st)
+{
+    static_assert(sizeof(PartEntry) == 16, "two 64-bit words per partition");
+    return upload_pairs(dev, P, st, [&](int p, unsigned long long* w0, unsigned long long* w1) {
+        const long long len = part_len[p];
+        const double t = tau ? tau[p] : 0.0;
+        std::memcpy(w0, &len, 8);
+        std::memcpy(w1, &t, 8);
+    });
+}
+
 }  // namespace btard
 
 using namespace btard;
@@ -253,9 +305,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
         return BTARD_ERR_INVALID_ARG;
     if (a->stop_mode != BTARD_STOP_FIXED_ITERS && a->stop_mode != BTARD_STOP_EPS)
         return BTARD_ERR_INVALID_ARG;
-    if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM &&
-        a->algo != BTARD_ALGO_DIRECT_RESIDENT && a->algo != BTARD_ALGO_DIRECT_COOPERATIVE &&
-        a->algo != BTARD_ALGO_DIRECT_STAGED)
+    if (a->algo != BTARD_ALGO_DIRECT && a->algo != BTARD_ALGO_GRAM && a->algo != BTARD_ALGO_DIRECT_COOPERATIVE)
         return BTARD_ERR_INVALID_ARG;
     if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (a->rule < BTARD_RULE_CENTERED_CLIP || a->rule > BTARD_RULE_COORD_MEDIAN) return BTARD_ERR_INVALID_ARG;
@@ -310,13 +360,10 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
         return launch_cclip_finalize(L, geo, st);
     }
 
-    // How the updates are driven: one cooperative kernel over everything (whole), one per L2-sized
-    // chunk of partitions (chunk >= 1), or one launch per update.
-    const int fit = resident_chunk_partitions(n, a->row_stride);         // partitions per L2 budget
-    const int chunk = (a->algo == BTARD_ALGO_DIRECT_RESIDENT) ? fit : 0;
+    // How the updates are driven: one cooperative kernel over everything, or one launch per update.
     const bool whole = (a->algo == BTARD_ALGO_DIRECT_COOPERATIVE) && cooperative_launch_supported();
     L.init_mode = a->init_mode;
-    if (a->init_mode == BTARD_INIT_COORD_MEDIAN && chunk < 1) {
+    if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
         rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
         if (rc != BTARD_OK) return rc;
         L.init_mode = BTARD_INIT_CALLER_V0;
@@ -351,60 +398,22 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     }
     if (whole) {
         BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.rflags, 0, ws.rflags_bytes, st));
-        unsigned long long* bars = (unsigned long long*)(base + ws.rflags);
-        unsigned int* err = (unsigned int*)(bars + P);
-        rc = launch_cclip_resident(L, geo, geo.cpp, fit >= P ? 0 : 1, (double*)(base + ws.rslots), bars, err, st);
+        unsigned long long* bar = (unsigned long long*)(base + ws.rflags);
+        unsigned int* err = (unsigned int*)(bar + 1);
+        // rows + v (fp32 and bf16) of all partitions against three quarters of the L2
+        const bool fits = (double)P * (double)a->row_stride * (4.0 * n + 6.0) <= 0.75 * (double)l2_bytes();
+        rc = launch_cclip_cooperative(L, geo, fits ? 0 : 1, (double*)(base + ws.rslots), bar, err, st);
         if (rc == BTARD_OK) return BTARD_OK;
         // the cooperative launch was refused: nothing ran, take the launch-per-update path
-    }
-
-    // Start pass and every update of a chunk in one resident kernel.
-    if (chunk >= 1) {
-        BTARD_CUDA_TRY(cudaMemsetAsync(base + ws.rflags, 0, ws.rflags_bytes, st));
-        unsigned long long* bars = (unsigned long long*)(base + ws.rflags);
-        unsigned int* err = (unsigned int*)(bars + P);
-        bool ok = true;
-        int ci = 0;
-        for (int c0 = 0; c0 < P && ok; c0 += chunk, ++ci) {
-            const int Pc = (P - c0 < chunk) ? P - c0 : chunk;
-            CclipLaunch C = L;
-            C.g = a->g + (size_t)c0 * n * a->row_stride;
-            C.v = a->v + (size_t)c0 * a->row_stride;
-            if (L.v_lo) C.v_lo = L.v_lo + (size_t)c0 * a->row_stride;
-            C.table = L.table + c0;
-            C.done = L.done + c0;
-            C.iters = a->iters + c0; C.last_step = a->last_step_norm + c0;
-            C.resid_norm = a->resid_norm + (size_t)c0 * n; C.status = a->status + c0;
-            C.P = Pc;
-            C.init_mode = a->init_mode;
-            if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
-                rc = launch_median_init(C.g, C.v, C.table, a->row_stride, n, Pc, st);
-                if (rc != BTARD_OK) return rc;
-                C.init_mode = BTARD_INIT_CALLER_V0;
-            }
-            rc = launch_cclip_resident(C, geo, 0, 0, (double*)(base + ws.rslots), bars + ci, err, st);
-            if (rc != BTARD_OK) {
-                if (c0 == 0) ok = false;      // nothing done yet: take the streaming path instead
-                else return rc;
-            }
-        }
-        if (ok) return BTARD_OK;
-        if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {          // streaming path after all
-            rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
-            if (rc != BTARD_OK) return rc;
-            L.init_mode = BTARD_INIT_CALLER_V0;
-        }
     }
 
     rc = launch_cclip_pass(L, geo, PASS_INIT, st);
     if (rc != BTARD_OK) return rc;
 
     // Update l reads the totals in buffer l % 2 and writes buffer (l + 1) % 2.
-    StagedGeometry sg = cclip_staged_geometry(n, P, a->row_stride, L.v_lo != nullptr);
-    if (a->algo != BTARD_ALGO_DIRECT_STAGED) sg.ok = 0;
     for (int l = 0; l < a->max_iters; ++l) {
         L.l = l; L.tot_in = tot[l & 1]; L.tot_out = tot[(l + 1) & 1];
-        rc = sg.ok ? launch_cclip_staged(L, sg, st) : launch_cclip_pass(L, geo, PASS_ITER, st);
+        rc = launch_cclip_pass(L, geo, PASS_ITER, st);
         if (rc != BTARD_OK) return rc;
     }
     L.tot_in = tot[a->max_iters & 1];
@@ -549,14 +558,13 @@ int upload_pack_table(void* table, int P, int64_t d, int64_t stride, const int64
                       cudaStream_t st)
 {
     if (P < 1 || P > 65535 || !off || !len || !table || d < 0 || stride < 1) return BTARD_ERR_INVALID_ARG;
-    std::vector<long long> host(2 * (size_t)P);
-    for (int p = 0; p < P; ++p) {
+    for (int p = 0; p < P; ++p)
         if (off[p] < 0 || len[p] < 0 || len[p] > stride || off[p] + len[p] > d) return BTARD_ERR_INVALID_ARG;
-        host[2 * p] = off[p];
-        host[2 * p + 1] = len[p];
-    }
-    BTARD_CUDA_TRY(cudaMemcpyAsync(table, host.data(), sizeof(long long) * 2 * P, cudaMemcpyHostToDevice, st));
-    return BTARD_OK;
+    return upload_pairs(table, P, st, [&](int p, unsigned long long* w0, unsigned long long* w1) {
+        const long long o = off[p], l = len[p];
+        std::memcpy(w0, &o, 8);
+        std::memcpy(w1, &l, 8);
+    });
 }
 }  // namespace
 
@@ -594,11 +602,10 @@ int btard_hash_partitions(int32_t P, int32_t rows_per_part, int64_t stride, cons
     if ((long long)P * rows_per_part > 0x7fffffffLL / 2) return BTARD_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return BTARD_ERR_BAD_ALIGNMENT;
     if (workspace_bytes < btard_hash_partitions_workspace(P, rows_per_part, stride)) return BTARD_ERR_WORKSPACE_TOO_SMALL;
-    std::vector<double> zeros((size_t)P, 0.0);
     for (int p = 0; p < P; ++p)
         if (part_len[p] < 0 || part_len[p] > stride) return BTARD_ERR_INVALID_ARG;
     char* base = (char*)workspace;
-    int rc = upload_table((PartEntry*)base, P, part_len, zeros.data(), (cudaStream_t)stream);
+    int rc = upload_table((PartEntry*)base, P, part_len, nullptr, (cudaStream_t)stream);
     if (rc != BTARD_OK) return rc;
     uint32_t* leaves = (uint32_t*)(base + align_up(sizeof(PartEntry) * (size_t)P, 256));
     return launch_hash_rows(x, (const PartEntry*)base, leaves, digests, stride, rows_per_part,
@@ -656,11 +663,35 @@ int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t part_len, f
 
 // ---- host-buffer path ---------------------------------------------------------------------------
 namespace {
+// With a second stream the partitions go through in up to kMaxHostChunks chunks: the copy of the
+// next chunk's rows runs on copy_stream while the kernels of the current chunk run on stream, so
+// the call takes about the longer of (copy of everything) and (all kernels) plus one chunk of the other.
+// Every chunk pays the fixed cost of its updates (a launch or a grid barrier each) again: measured on
+// 16 partitions of 16 x 698 400 with 100 updates, 4 chunks take 19.6 ms and 8 chunks 23.1 ms.
+constexpr size_t kMaxHostChunks = 4;
+
 struct HostScratch {
     size_t g, v, iters, last_step, resid_norm, status_c, status_v, norm, weight, dot, s, s_sum,
         znorm2, rsn, ws_c, ws_v, total;
     size_t ws_c_bytes, ws_v_bytes;
 };
+
+bool host_piped(const btard_host_args* a)
+{
+    return a->copy_stream != nullptr && a->copy_stream != a->stream && a->n_partitions > 1;
+}
+size_t host_chunks(const btard_host_args* a)
+{
+    const size_t P = (size_t)a->n_partitions;
+    return host_piped(a) ? (P < kMaxHostChunks ? P : kMaxHostChunks) : 1;
+}
+// The algorithm a chunk runs: in eps mode the launch-per-update path would keep launching after the
+// chunk has converged, so DIRECT becomes the cooperative kernel there.
+int host_algo(const btard_host_args* a)
+{
+    if (a->algo == BTARD_ALGO_DIRECT && a->stop_mode == BTARD_STOP_EPS) return BTARD_ALGO_DIRECT_COOPERATIVE;
+    return a->algo;
+}
 
 HostScratch host_layout(const btard_host_args* a)
 {
@@ -682,15 +713,24 @@ HostScratch host_layout(const btard_host_args* a)
     h.s_sum = take(sizeof(double) * P * K);
     h.znorm2 = take(sizeof(double) * P * K);
     h.rsn = take(sizeof(double) * P);
+    // The workspaces serve every chunk in turn.  Their layouts are not monotone in the number of
+    // partitions (fewer partitions get more CTAs each), so the size is the largest need over every
+    // chunk size this call may use, with or without a copy stream.
     btard_cclip_args ca{};
-    ca.n_peers = a->n_peers; ca.n_partitions = a->n_partitions; ca.row_stride = a->row_stride;
+    ca.n_peers = a->n_peers; ca.row_stride = a->row_stride;
     ca.stop_mode = BTARD_STOP_EPS;   // the larger of the two layouts
-    ca.algo = BTARD_ALGO_DIRECT_COOPERATIVE;
-    h.ws_c_bytes = btard_centered_clip_workspace(&ca);
+    ca.algo = (a->algo == BTARD_ALGO_GRAM) ? BTARD_ALGO_GRAM : BTARD_ALGO_DIRECT_COOPERATIVE;
     btard_verify_args va{};
-    va.n_peers = a->n_peers; va.n_partitions = a->n_partitions; va.row_stride = a->row_stride;
-    va.n_z = a->n_z;
-    h.ws_v_bytes = btard_verify_projections_workspace(&va);
+    va.n_peers = a->n_peers; va.row_stride = a->row_stride; va.n_z = a->n_z;
+    auto cover = [&](size_t parts) {
+        ca.n_partitions = va.n_partitions = (int32_t)parts;
+        const size_t c = btard_centered_clip_workspace(&ca), v = btard_verify_projections_workspace(&va);
+        if (c > h.ws_c_bytes) h.ws_c_bytes = c;
+        if (v > h.ws_v_bytes) h.ws_v_bytes = v;
+    };
+    cover(P);
+    const size_t nchunks = P < kMaxHostChunks ? P : kMaxHostChunks;
+    for (size_t c = 0; c < nchunks; ++c) cover(P * (c + 1) / nchunks - P * c / nchunks);
     h.ws_c = take(h.ws_c_bytes);
     h.ws_v = take(h.ws_v_bytes);
     h.total = off;
@@ -700,8 +740,19 @@ HostScratch host_layout(const btard_host_args* a)
 bool host_sizes_ok(const btard_host_args* a)
 {
     return a && a->n_peers >= 1 && a->n_peers <= BTARD_MAX_PEERS && a->n_partitions >= 1 &&
-           a->row_stride >= 4 && a->n_z >= 1 && a->n_z <= BTARD_MAX_Z;
+           a->row_stride >= 4 && a->n_z >= 1 && a->n_z <= BTARD_MAX_Z &&
+           (a->algo == BTARD_ALGO_DIRECT || a->algo == BTARD_ALGO_GRAM || a->algo == BTARD_ALGO_DIRECT_COOPERATIVE);
 }
+
+// Events of one call; destroyed on every way out.
+struct ChunkEvents {
+    cudaEvent_t ready[kMaxHostChunks] = {};
+    ~ChunkEvents()
+    {
+        for (size_t c = 0; c < kMaxHostChunks; ++c)
+            if (ready[c]) cudaEventDestroy(ready[c]);
+    }
+};
 }  // namespace
 
 size_t btard_aggregate_host_scratch(const btard_host_args* a)
@@ -715,6 +766,7 @@ int btard_aggregate_host(const btard_host_args* a)
     if (!host_sizes_ok(a) || !a->g || !a->v || !a->device_scratch) return BTARD_ERR_INVALID_ARG;
     int rc = check_common(a->n_peers, a->n_partitions, a->row_stride, a->part_len, a->tau);
     if (rc != BTARD_OK) return rc;
+    if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(a->device_scratch) & 255u) return BTARD_ERR_BAD_ALIGNMENT;
     const HostScratch h = host_layout(a);
     if (a->device_scratch_bytes < h.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
@@ -722,31 +774,20 @@ int btard_aggregate_host(const btard_host_args* a)
     char* base = (char*)a->device_scratch;
     const size_t n = a->n_peers, P = a->n_partitions, S = (size_t)a->row_stride, K = a->n_z;
 
-    // With a second stream the partitions go through in up to kMaxHostChunks chunks: the copy of the
-    // next chunk's rows runs on copy_stream while the kernels of the current chunk run on stream, so
-    // the call takes about the longer of (copy of everything) and (all kernels) plus one chunk of the other.
-    // Every chunk pays the fixed cost of its updates (a launch or a grid barrier each) again: measured on
-    // 16 partitions of 16 x 698 400 with 100 updates, 4 chunks take 19.6 ms and 8 chunks 23.1 ms.
-    constexpr size_t kMaxHostChunks = 4;
     cudaStream_t cs = (cudaStream_t)a->copy_stream;
-    const bool piped = a->copy_stream != nullptr && a->copy_stream != a->stream && P > 1;
-    const size_t nchunks = piped ? (P < kMaxHostChunks ? P : kMaxHostChunks) : 1;
-    cudaEvent_t ready[kMaxHostChunks] = {};
-    auto drop_events = [&]() {
-        for (size_t c = 0; c < kMaxHostChunks; ++c)
-            if (ready[c]) { cudaEventDestroy(ready[c]); ready[c] = nullptr; }
-    };
+    const bool piped = host_piped(a);
+    const size_t nchunks = host_chunks(a);
+    const int algo = host_algo(a);
+    ChunkEvents ev;
     if (a->init_mode == BTARD_INIT_CALLER_V0)
         BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.v, a->v, sizeof(float) * P * S, cudaMemcpyHostToDevice, st));
     if (piped) {
         for (size_t c = 0; c < nchunks; ++c) {
             const size_t p0 = P * c / nchunks, p1 = P * (c + 1) / nchunks;
-            cudaError_t e = cudaEventCreateWithFlags(&ready[c], cudaEventDisableTiming);
-            if (e == cudaSuccess)
-                e = cudaMemcpyAsync(base + h.g + sizeof(float) * p0 * n * S, a->g + p0 * n * S,
-                                    sizeof(float) * (p1 - p0) * n * S, cudaMemcpyHostToDevice, cs);
-            if (e == cudaSuccess) e = cudaEventRecord(ready[c], cs);
-            if (e != cudaSuccess) { set_cuda_error(e); drop_events(); return BTARD_ERR_CUDA; }
+            BTARD_CUDA_TRY(cudaEventCreateWithFlags(&ev.ready[c], cudaEventDisableTiming));
+            BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.g + sizeof(float) * p0 * n * S, a->g + p0 * n * S,
+                                           sizeof(float) * (p1 - p0) * n * S, cudaMemcpyHostToDevice, cs));
+            BTARD_CUDA_TRY(cudaEventRecord(ev.ready[c], cs));
         }
     } else {
         BTARD_CUDA_TRY(cudaMemcpyAsync(base + h.g, a->g, sizeof(float) * P * n * S, cudaMemcpyHostToDevice, st));
@@ -754,41 +795,40 @@ int btard_aggregate_host(const btard_host_args* a)
 
     for (size_t c = 0; c < nchunks; ++c) {
         const size_t p0 = P * c / nchunks, p1 = P * (c + 1) / nchunks;
-        if (piped) {
-            cudaError_t e = cudaStreamWaitEvent(st, ready[c], 0);
-            if (e != cudaSuccess) { set_cuda_error(e); drop_events(); return BTARD_ERR_CUDA; }
-        }
+        if (piped) BTARD_CUDA_TRY(cudaStreamWaitEvent(st, ev.ready[c], 0));
         btard_cclip_args ca{};
         ca.n_peers = a->n_peers; ca.n_partitions = (int32_t)(p1 - p0); ca.row_stride = a->row_stride;
         ca.part_len = a->part_len + p0; ca.g = (const float*)(base + h.g) + p0 * n * S; ca.tau = a->tau + p0;
-        // eps mode: nothing should be launched after convergence, chunk by chunk
-        ca.init_mode = a->init_mode; ca.stop_mode = a->stop_mode;
-        ca.algo = (a->stop_mode == BTARD_STOP_EPS) ? BTARD_ALGO_DIRECT_COOPERATIVE : BTARD_ALGO_DIRECT;
+        ca.init_mode = a->init_mode; ca.stop_mode = a->stop_mode; ca.algo = algo;
         ca.max_iters = a->max_iters; ca.eps = a->eps; ca.v = (float*)(base + h.v) + p0 * S;
         ca.iters = (int32_t*)(base + h.iters) + p0; ca.last_step_norm = (double*)(base + h.last_step) + p0;
         ca.resid_norm = (double*)(base + h.resid_norm) + p0 * n; ca.status = (uint32_t*)(base + h.status_c) + p0;
         ca.workspace = base + h.ws_c; ca.workspace_bytes = h.ws_c_bytes; ca.stream = a->stream;
-        rc = btard_centered_clip(&ca);
-        if (rc != BTARD_OK) { drop_events(); return rc; }
 
         btard_verify_args va{};
         va.n_peers = a->n_peers; va.n_partitions = ca.n_partitions; va.row_stride = a->row_stride;
-        va.part_len = ca.part_len; va.g = ca.g; va.v = ca.v; va.tau = ca.tau; va.seed = a->seed;
-        va.n_z = a->n_z; va.partition_base = (int32_t)p0; va.resid_norm_in = ca.resid_norm;
+        va.seed = a->seed; va.n_z = a->n_z; va.partition_base = (int32_t)p0;
         va.norm = (double*)(base + h.norm) + p0 * n; va.weight = (double*)(base + h.weight) + p0 * n;
         va.dot = (double*)(base + h.dot) + p0 * n * K; va.s = (double*)(base + h.s) + p0 * n * K;
         va.s_sum = (double*)(base + h.s_sum) + p0 * K; va.znorm2 = (double*)(base + h.znorm2) + p0 * K;
         va.resid_sum_norm = (double*)(base + h.rsn) + p0; va.resid_sum = nullptr;
         va.status = (uint32_t*)(base + h.status_v) + p0;
-        va.workspace = base + h.ws_v; va.workspace_bytes = h.ws_v_bytes; va.stream = a->stream;
-        rc = btard_verify_projections(&va);
-        if (rc != BTARD_OK) { drop_events(); return rc; }
+        va.workspace = base + h.ws_v; va.workspace_bytes = h.ws_v_bytes;
+        // one call: with the Gram variant the combine pass and the verification pass are one read of g
+        rc = btard_centered_clip_verify(&ca, &va);
+        if (rc != BTARD_OK) return rc;
     }
 
     auto back = [&](void* dst, size_t off, size_t bytes) -> cudaError_t {
         if (!dst) return cudaSuccess;
         return cudaMemcpyAsync(dst, base + off, bytes, cudaMemcpyDeviceToHost, st);
     };
+    if (a->status) {
+        or_status_kernel<<<(unsigned)((P + 127) / 128), 128, 0, st>>>((uint32_t*)(base + h.status_c),
+                                                                      (const uint32_t*)(base + h.status_v), (int)P);
+        BTARD_CUDA_TRY(cudaGetLastError());
+        count_launch();
+    }
     BTARD_CUDA_TRY(back(a->v, h.v, sizeof(float) * P * S));
     BTARD_CUDA_TRY(back(a->iters, h.iters, sizeof(int32_t) * P));
     BTARD_CUDA_TRY(back(a->last_step_norm, h.last_step, sizeof(double) * P));
@@ -799,17 +839,8 @@ int btard_aggregate_host(const btard_host_args* a)
     BTARD_CUDA_TRY(back(a->s_sum, h.s_sum, sizeof(double) * P * K));
     BTARD_CUDA_TRY(back(a->znorm2, h.znorm2, sizeof(double) * P * K));
     BTARD_CUDA_TRY(back(a->resid_sum_norm, h.rsn, sizeof(double) * P));
-    std::vector<uint32_t> sc, sv;
-    if (a->status) {
-        sc.resize(P); sv.resize(P);
-        BTARD_CUDA_TRY(cudaMemcpyAsync(sc.data(), base + h.status_c, sizeof(uint32_t) * P, cudaMemcpyDeviceToHost, st));
-        BTARD_CUDA_TRY(cudaMemcpyAsync(sv.data(), base + h.status_v, sizeof(uint32_t) * P, cudaMemcpyDeviceToHost, st));
-    }
-    const cudaError_t sync_err = cudaStreamSynchronize(st);
-    drop_events();
-    BTARD_CUDA_TRY(sync_err);
-    if (a->status)
-        for (size_t p = 0; p < P; ++p) a->status[p] = sc[p] | sv[p];
+    BTARD_CUDA_TRY(back(a->status, h.status_c, sizeof(uint32_t) * P));
+    BTARD_CUDA_TRY(cudaStreamSynchronize(st));
     return BTARD_OK;
 }
 

@@ -91,7 +91,7 @@ __device__ void row_weights(const double* sh_sum, float* sh_w, int n, double tau
 
 struct KernelArgs {
     CclipLaunch a;
-    int RG, CL, tiles, cpp;
+    int RG, CL, cpp;
 };
 
 // Records the end state of a partition (called by one CTA of it).
@@ -539,360 +539,19 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
 }
 
 // =================================================================================================
-// Staged iteration pass for n <= 16 (all rows of a column in one thread).  Same update as
-// cclip_pass_kernel<R, PASS_ITER, COMP>, but the rows reach the SM through bulk asynchronous copies
-// (one per row and tile, plus v and its low-order part) into a ring of shared-memory stages.  Per
-// stage an mbarrier counts the bytes that landed and a counter the warps that have moved their part
-// of the tile into registers; the warp that arrives last refills the stage with the tile S steps
-// ahead.  No CTA-wide barrier sits inside the loop, and the bytes in flight do not depend on the
-// registers of the threads.  Every wait is bounded; a wait that runs out sets
-// BTARD_STATUS_WAIT_EXPIRED, all loops end, and the CTA goes on to its epilogue.
+// Cooperative variant: the start pass and every update of all partitions inside ONE kernel.
 //
-// A consumer thread owns 2 columns and works on (column, column + 1) pairs with the packed fp32
-// instructions of sm_100 (add/sub/mul/fma .f32x2: the same IEEE results as two scalar operations).
-// Per element: d = x - v_hi; s += w d; r = d - e with e = v_lo + (move of v); |r|^2.  The low-order
-// part of v enters the column sum once, as -v_lo * sum_i w_i.
+// The work items are the column ranges the launch-per-update path gives to its CTAs, dealt
+// round-robin to one wave of resident CTAs that meet at a grid-wide barrier between updates: no
+// launch per update, and nothing runs once the last partition has converged.  The kernel is launched
+// cooperatively (the runtime refuses the launch if the CTAs cannot all be resident), every wait on
+// the barrier is bounded, and a wait that expires sets an error flag and status bit and makes every
+// CTA leave.
 // =================================================================================================
-constexpr int kMaxStages = 4;
-constexpr unsigned kStageWaitLimit = 1u << 22;
-constexpr int kStagedConsumerWarps = 8;
-constexpr int kStagedThreads = 32 * kStagedConsumerWarps;
-constexpr int kStagedMaxTilesPerCta = 128;        // a thread's fp32 running sums get one term per tile
-constexpr int kStagedTileQuads = 16 * kStagedConsumerWarps;      // 2 columns per consumer thread: 128 quads
-
-struct StagedArgs {
+struct CoopArgs {
     CclipLaunch a;
-    int cpp, stages;
-    unsigned stage_bytes;           // multiple of 128
-};
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
-{
-    uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// false: the wait ran out (or another warp's did: give_up, when given, points at a non-zero flag)
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity, const volatile int* give_up)
-{
-    for (unsigned spins = 0; spins < kStageWaitLimit; ++spins) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spins & 1023u) == 1023u && give_up && *give_up) return false;
-    }
-    return false;
-}
-__device__ __forceinline__ void bulk_load_hint(void* dst, const void* src, unsigned bytes, uint64_t* bar, uint64_t policy)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy) : "memory");
-}
-
-template <int R, bool COMP>
-__global__ void __launch_bounds__(kStagedThreads, 2) cclip_iter_staged_kernel(const StagedArgs k)
-{
-    extern __shared__ __align__(128) unsigned char sh_raw[];   // the stages
-    __shared__ double sh_sum[BTARD_MAX_PEERS + 1];             // totals in; slot sums of the last CTA out
-    __shared__ float sh_w[BTARD_MAX_PEERS + 16];
-    __shared__ __align__(8) float2 sh_w2[16];                  // (w_i, w_i)
-    __shared__ double sh_red[16][17];
-    __shared__ __align__(8) uint64_t sh_full[kMaxStages];
-    __shared__ int sh_taken[kMaxStages];                       // warps that hold their part of the stage's tile
-    __shared__ int sh_flag, sh_expired, sh_issued;
-    __shared__ float sh_wsum;
-
-    const CclipLaunch& a = k.a;
-    constexpr int CL = kStagedTileQuads;
-    const int n = a.n, cpp = k.cpp, S = k.stages;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool rev = (a.l & 1) == 0;
-    const int bid = rev ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
-    const int p = bid / cpp, j = bid % cpp;
-    const long long stride = a.stride;
-
-    if (a.done[p]) return;
-
-    const float* gp = a.g + (size_t)p * n * stride;
-    float* vp = a.v + (size_t)p * stride;
-    unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
-    const float inv_n = 1.0f / (float)n;
-
-    const long long Q = stride >> 2;
-    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
-    if (j > 0) q0 &= ~7LL;
-    if (j + 1 < cpp) q1 &= ~7LL;
-    const int ntiles = (int)((q1 - q0 + CL - 1) / CL);
-    constexpr unsigned row_bytes = (unsigned)CL * 16u;    // one row of a full tile
-    const uint64_t pol = policy_evict_first();
-    // v is read and written by every pass: its loads ask L2 to keep the lines, its stores are marked
-    // streaming (measured: 7 us per pass faster than default or evict-last stores of the same lines).
-    const uint64_t keep = policy_evict_last();
-    const volatile int* give_up = &sh_expired;
-
-    // One warp fills stage (t % S) with tile t of the sweep: n rows, v and (COMP) the bf16 part.
-    auto issue = [&](int t) {
-        const long long qb = q0 + (long long)(rev ? ntiles - 1 - t : t) * CL;
-        const long long rest = q1 - qb;
-        const unsigned nq = (unsigned)(rest < CL ? rest : CL);
-        unsigned char* st = sh_raw + (size_t)(t % S) * k.stage_bytes;
-        uint64_t* bar = &sh_full[t % S];
-        if (lane == 0) {
-            const unsigned total = nq * 16u * (unsigned)(n + 1) + (COMP ? nq * 8u : 0u);
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(total) : "memory");
-        }
-        __syncwarp();
-        if (lane < n) bulk_load_hint(st + (size_t)lane * row_bytes, gp + (size_t)lane * stride + qb * 4, nq * 16u, bar, pol);
-        else if (lane == n) bulk_load_hint(st + (size_t)n * row_bytes, vp + qb * 4, nq * 16u, bar, keep);
-        else if (COMP && lane == n + 1) bulk_load_hint(st + (size_t)(n + 1) * row_bytes, lop + qb * 4, nq * 8u, bar, keep);
-        __syncwarp();
-    };
-
-    // The first copies leave before anything else is read, so that the totals, the stop test and the
-    // clip weights below overlap with their flight.
-    if (warp == 0) {
-        if (lane == 0) {
-            sh_flag = 0; sh_expired = 0;
-            for (int s = 0; s < S; ++s) {
-                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&sh_full[s])));
-                sh_taken[s] = 0;
-            }
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
-        __syncwarp();
-        int issued = 0;
-        for (; issued < S && issued < ntiles; ++issued) issue(issued);
-        if (lane == 0) sh_issued = issued;
-    }
-    {
-        const double* src = a.tot_in + (size_t)p * (n + 1);
-        for (int i = tid; i <= n; i += blockDim.x) sh_sum[i] = __ldcg(src + i);
-        __syncthreads();
-        const bool converged = (a.stop_mode == BTARD_STOP_EPS) && a.l >= 1 && (sh_sum[n] <= a.eps2);
-        if (converged) {                              // same decision in every CTA of the partition
-            // the copies already issued must have landed before the CTA gives its shared memory back
-            if (tid < S && tid < ntiles) (void)mbar_wait_bounded(&sh_full[tid], 0u, nullptr);
-            __syncthreads();
-            if (j == 0) finish_partition(a, p, sh_sum, a.l, true);
-            return;
-        }
-    }
-    const long long len = a.table[p].len;
-    const double tau = a.table[p].tau;
-    const long long full_quads = len >> 2;
-
-    // Clip weights of this update (the first copies are already on their way).
-    row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, &sh_red[0][0]);
-    if (tid < 16) sh_w2[tid] = make_float2(sh_w[tid], sh_w[tid]);
-    if (tid == 0) {
-        float w = 0.0f;
-        for (int i = 0; i < n; ++i) w += sh_w[i];
-        sh_wsum = w;
-        if (j == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
-    }
-    __syncthreads();
-    const bool skip_rows = sh_flag != 0;              // some row has a non-finite norm: leave it out
-    const float wsum = sh_wsum;
-
-    uint64_t acc2[R];                                 // per row: squared residuals of the two columns
-#pragma unroll
-    for (int r = 0; r < R; ++r) acc2[r] = 0ull;
-    float step_acc = 0.0f;
-
-    {
-        const int ct = tid;                           // consumer thread: columns 2 ct, 2 ct + 1 of the tile
-        for (int t = 0; t < ntiles; ++t) {
-            const int s = t % S;
-            const long long qb = q0 + (long long)(rev ? ntiles - 1 - t : t) * CL;
-            const unsigned char* st = sh_raw + (size_t)s * k.stage_bytes;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&sh_full[s], (unsigned)((t / S) & 1), give_up));
-            if (!ok) { if (lane == 0) sh_expired = 1; break; }
-            const long long col = qb * 4 + 2 * ct;
-            const bool fast = !skip_rows && (qb + CL <= q1) && (qb + CL <= full_quads);
-            uint64_t x2[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                x2[r] = (r < n) ? reinterpret_cast<const uint64_t*>(st + (size_t)r * row_bytes)[ct] : 0ull;
-            const uint64_t v2 = reinterpret_cast<const uint64_t*>(st + (size_t)n * row_bytes)[ct];
-            uint32_t lob = 0;
-            if (COMP) lob = reinterpret_cast<const uint32_t*>(st + (size_t)(n + 1) * row_bytes)[ct];
-            // This warp's part of the tile is in registers.  The last warp to say so refills the stage.
-            __syncwarp();
-            int before = 0;
-            if (lane == 0) {
-                __threadfence_block();
-                before = atomicAdd(&sh_taken[s], 1);
-            }
-            before = __shfl_sync(0xffffffffu, before, 0);
-            if (before == kStagedConsumerWarps - 1 && t + S < ntiles) {
-                if (lane == 0) {
-                    sh_taken[s] = 0;
-                    atomicMax(&sh_issued, t + S + 1);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                }
-                issue(t + S);
-            }
-
-            float vx, vy;
-            unpack2(v2, vx, vy);
-            const float lx = bf16_value(lob & 0xFFFFu), ly = bf16_value(lob >> 16);
-            if (fast) {
-                uint64_t s2 = 0ull, t2 = 0ull;         // even and odd rows: two shorter dependency chains
-#pragma unroll
-                for (int r = 0; r < R; r += 2) {
-                    x2[r] = sub2(x2[r], v2);
-                    x2[r + 1] = sub2(x2[r + 1], v2);
-                    s2 = fma2(*reinterpret_cast<const uint64_t*>(&sh_w2[r]), x2[r], s2);
-                    t2 = fma2(*reinterpret_cast<const uint64_t*>(&sh_w2[r + 1]), x2[r + 1], t2);
-                }
-                float ux, uy, tx, ty;
-                unpack2(s2, ux, uy);
-                unpack2(t2, tx, ty);
-                ux += tx; uy += ty;
-                if (COMP) { ux = fmaf(-wsum, lx, ux); uy = fmaf(-wsum, ly, uy); }
-                ux *= inv_n; uy *= inv_n;
-                float nx, ny, ex, ey;
-                if (COMP) {
-                    uint32_t b0, b1;
-                    float l0, l1;
-                    two_sum_bf16(vx, lx + ux, nx, l0, b0);
-                    two_sum_bf16(vy, ly + uy, ny, l1, b1);
-                    ex = (nx - vx) + l0; ey = (ny - vy) + l1;
-                    __stcs(reinterpret_cast<uint32_t*>(lop + col), b0 | (b1 << 16));
-                } else {
-                    nx = vx + ux; ny = vy + uy;
-                    ex = nx - vx; ey = ny - vy;
-                }
-                step_acc += ux * ux + uy * uy;
-                __stcs(reinterpret_cast<float2*>(vp + col), make_float2(nx, ny));
-                const uint64_t e2 = pack2(ex, ey);
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const uint64_t d2 = sub2(x2[r], e2);
-                    acc2[r] = fma2(d2, d2, acc2[r]);
-                }
-            } else {
-                // ragged tile, or rows to leave out: scalar, with masks
-                const bool valid = (qb + (ct >> 1) < q1);
-                const bool m0 = valid && col < len, m1 = valid && col + 1 < len;
-                float sx = 0.f, sy = 0.f;
-                float dx[R], dy[R];
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float ax, ay;
-                    unpack2(x2[r], ax, ay);
-                    dx[r] = (valid && r < n) ? ax - vx : 0.f;
-                    dy[r] = (valid && r < n) ? ay - vy : 0.f;
-                    const float wr = sh_w[r];
-                    if (wr != 0.0f) { sx = fmaf(wr, dx[r], sx); sy = fmaf(wr, dy[r], sy); }
-                }
-                float ux = sx, uy = sy;
-                if (COMP) { ux = fmaf(-wsum, lx, ux); uy = fmaf(-wsum, ly, uy); }
-                ux *= inv_n; uy *= inv_n;
-                float nx, ny, ex, ey;
-                if (COMP) {
-                    uint32_t b0, b1;
-                    float l0, l1;
-                    two_sum_bf16(vx, lx + ux, nx, l0, b0);
-                    two_sum_bf16(vy, ly + uy, ny, l1, b1);
-                    ex = (nx - vx) + l0; ey = (ny - vy) + l1;
-                    if (!m0) b0 = 0;
-                    if (!m1) b1 = 0;
-                    if (valid) __stcs(reinterpret_cast<uint32_t*>(lop + col), b0 | (b1 << 16));
-                } else {
-                    nx = vx + ux; ny = vy + uy;
-                    ex = nx - vx; ey = ny - vy;
-                }
-                step_acc += (m0 ? ux * ux : 0.f) + (m1 ? uy * uy : 0.f);
-                if (!m0) nx = 0.f;
-                if (!m1) ny = 0.f;
-                if (valid) __stcs(reinterpret_cast<float2*>(vp + col), make_float2(nx, ny));
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float rx = m0 ? dx[r] - ex : 0.f, ry = m1 ? dy[r] - ey : 0.f;
-                    const uint64_t d2 = pack2(rx, ry);
-                    acc2[r] = fma2(d2, d2, acc2[r]);
-                }
-            }
-        }
-    }
-    __syncthreads();
-    if (sh_expired) {
-        // Copies of tiles nobody consumed may still be landing: one more bounded wait per stage
-        // before the CTA ends.
-        const int last = sh_issued - 1;
-        if (tid < S && last >= tid) {
-            const int ts = last - ((last - tid) % S);
-            (void)mbar_wait_bounded(&sh_full[tid], (unsigned)((ts / S) & 1), nullptr);
-        }
-        if (tid == 0) atomicOr(&a.status[p], BTARD_STATUS_WAIT_EXPIRED);
-        __syncthreads();
-    }
-
-    // CTA reduction, slots, and the last CTA of the partition adds the slots up: as in the
-    // register-fed pass.
-    {
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float a0, a1;
-            unpack2(acc2[r], a0, a1);
-            const double s = warp_sum((double)a0 + (double)a1);
-            if (lane == 0) sh_red[warp][r] = s;
-        }
-        const double s = warp_sum((double)step_acc);
-        if (lane == 0) sh_red[warp][16] = s;
-    }
-    __syncthreads();
-    double* slots = a.slots + (size_t)p * cpp * (n + 1);
-    double* dst = slots + (size_t)j * (n + 1);
-    for (int i = tid; i <= n; i += blockDim.x) {
-        double s = 0.0;
-        const int c = (i < n) ? i : 16;
-        for (int q = 0; q < kStagedConsumerWarps; ++q) s += sh_red[q][c];
-        dst[i] = s;
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) sh_flag = (atomicAdd(&a.ticket[p], 1u) == (unsigned)(cpp - 1));
-    __syncthreads();
-    if (!sh_flag) return;
-    __threadfence();
-    const int per = n + 1;
-    double* sh_part = sh_sum;                          // the totals read at the start are dead by now
-    int groups = blockDim.x / per;
-    if (groups > cpp) groups = cpp;
-    if (groups * per > BTARD_MAX_PEERS + 1) groups = (BTARD_MAX_PEERS + 1) / per;
-    for (int e = tid; e < groups * per; e += blockDim.x) {
-        const int cg = e / per, i = e - cg * per;
-        double s = 0.0;
-        for (int c = cg; c < cpp; c += groups) s += __ldcg(slots + (size_t)c * per + i);
-        sh_part[e] = s;
-    }
-    __syncthreads();
-    double* tot = a.tot_out + (size_t)p * per;
-    for (int i = tid; i < per; i += blockDim.x) {
-        double s = 0.0;
-        for (int cg = 0; cg < groups; ++cg) s += sh_part[cg * per + i];
-        tot[i] = s;
-    }
-    if (tid == 0) a.ticket[p] = 0;
-}
-
-// =================================================================================================
-// L2-resident variant: all updates of a chunk of partitions inside ONE cooperative kernel.
-//
-// B200 has 126 MB of L2; a chunk of partitions whose rows fit in it is read from HBM once (by the
-// start pass) and then every CenteredClip update streams it from L2 (measured 17-19 TB/s against
-// 6.5-7 TB/s from HBM).  That needs all updates of the chunk back to back with nothing else
-// flushing L2, i.e. one kernel whose CTAs all stay resident and meet at a grid-wide barrier between
-// updates.  The kernel is launched cooperatively (the runtime refuses the launch if the CTAs cannot
-// all be resident), every wait on the barrier is bounded, and a wait that expires sets an error
-// flag and status bit and makes every CTA leave.
-// =================================================================================================
-struct ResidentArgs {
-    CclipLaunch a;                  // chunk-relative pointers; a.P = partitions in the chunk
-    int RG, CL, cppc;               // cppc work items (column ranges) per partition of the chunk
-    int streaming;                  // 1: the chunk is larger than L2 (evict-first loads, alternating sweeps)
+    int RG, CL, cppc;               // cppc work items (column ranges) per partition
+    int streaming;                  // 1: the tensor is larger than L2 (evict-first loads, alternating sweeps)
     double* rslots;                 // [2][P][cppc][n+1]
     unsigned long long* barrier;    // low word: arrivals (monotonic), high word: finished partitions
     unsigned int* error;            // set when a bounded wait expired
@@ -907,10 +566,10 @@ __device__ __forceinline__ unsigned long long ld_volatile_u64(const unsigned lon
     return v;
 }
 
-// Grid-wide barrier.  Returns true when every partition of the chunk has finished (or a wait ran
+// Grid-wide barrier.  Returns true when every partition has finished (or a wait ran
 // out): the caller then leaves the kernel; CTAs still on their way see the same word and leave too,
 // so nobody is left waiting for an arrival that will not come.
-__device__ bool grid_barrier(const ResidentArgs& k, unsigned& generation, unsigned add_finished, int* sh_flag)
+__device__ bool grid_barrier(const CoopArgs& k, unsigned& generation, unsigned add_finished, int* sh_flag)
 {
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -940,7 +599,7 @@ __device__ bool grid_barrier(const ResidentArgs& k, unsigned& generation, unsign
 }
 
 template <int R, bool COMP>
-__global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs k)
+__global__ void __launch_bounds__(512) cclip_cooperative_kernel(const CoopArgs k)
 {
     extern __shared__ float4 sh_x[];                  // [2][RG][CL]
     __shared__ double sh_sum[BTARD_MAX_PEERS + 1];
@@ -950,7 +609,7 @@ __global__ void __launch_bounds__(512) cclip_resident_kernel(const ResidentArgs 
     __shared__ int sh_flag, sh_bar;
 
     const CclipLaunch& a = k.a;
-    const int n = a.n, RG = k.RG, CL = k.CL, cppc = k.cppc, Pc = a.P;
+    const int n = a.n, RG = k.RG, CL = k.CL, cppc = k.cppc, Pc = a.P;   // Pc: partitions of this launch
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
     const int items = Pc * cppc;                       // CTA b owns items b, b + gridDim.x, ...
     const long long stride = a.stride;
@@ -1390,69 +1049,6 @@ static int iter_ctas_per_sm(int R, int threads, size_t smem)
     return nb;
 }
 
-// Staged iteration kernel (n <= 16): stages of n rows + v (+ bf16 part) of 128 quads each, two CTAs
-// per SM, as many stages as their share of the shared memory holds (2 to 4).
-StagedGeometry cclip_staged_geometry(int n, int P, long long stride, bool comp)
-{
-    StagedGeometry sg{};
-    sg.ok = 0;
-    if (n > 16 || (stride & 31) != 0) return sg;
-    Geometry& g = sg.g;
-    g.R = (n <= 4) ? 4 : (n <= 8) ? 8 : 16;
-    g.RG = 1;
-    g.CL = kStagedTileQuads;
-    g.threads = kStagedThreads;
-    g.tiles = 0;
-    const size_t row_bytes = (size_t)g.CL * 16;
-    sg.stage_bytes = (unsigned)align_up((size_t)(n + 1) * row_bytes + (comp ? row_bytes / 2 : 0), 128);
-    int dev = 0, smem_sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess) {
-        (void)cudaGetLastError();
-        smem_sm = 233472;                              // sm_100 figure, for sizing without a device
-    }
-    const long long room = (long long)smem_sm / 2 - 6144 - 1024;   // static arrays, per-CTA reserve
-    int stages = (int)(room / (long long)sg.stage_bytes);
-    if (stages < 2) return sg;
-    if (stages > kMaxStages) stages = kMaxStages;
-    sg.stages = stages;
-    sg.smem = (size_t)stages * sg.stage_bytes;
-    g.slots = sm_count() * 2;
-    g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, g.slots, kStagedMaxTilesPerCta);
-    sg.ok = 1;
-    return sg;
-}
-
-template <int R>
-static int launch_staged_r(const StagedArgs& sa, size_t smem, int grid, cudaStream_t st)
-{
-    const bool comp = sa.a.v_lo != nullptr;
-    if (sa.a.l == 0) {                                 // first update of an aggregation
-        const int most = 113 * 1024;
-        cudaError_t e = comp ? cudaFuncSetAttribute(cclip_iter_staged_kernel<R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most)
-                             : cudaFuncSetAttribute(cclip_iter_staged_kernel<R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-        if (e != cudaSuccess) { set_cuda_error(e); return BTARD_ERR_CUDA; }
-    }
-    prof_begin(KIND_ITER, st);
-    if (comp) cclip_iter_staged_kernel<R, true><<<grid, kStagedThreads, smem, st>>>(sa);
-    else cclip_iter_staged_kernel<R, false><<<grid, kStagedThreads, smem, st>>>(sa);
-    prof_end(KIND_ITER, st);
-    BTARD_CUDA_TRY(cudaGetLastError());
-    count_launch();
-    return BTARD_OK;
-}
-
-int launch_cclip_staged(const CclipLaunch& a, const StagedGeometry& sg, cudaStream_t st)
-{
-    StagedArgs sa{a, sg.g.cpp, sg.stages, sg.stage_bytes};
-    const int grid = a.P * sg.g.cpp;
-    switch (sg.g.R) {
-        case 4: return launch_staged_r<4>(sa, sg.smem, grid, st);
-        case 8: return launch_staged_r<8>(sa, sg.smem, grid, st);
-        default: return launch_staged_r<16>(sa, sg.smem, grid, st);
-    }
-}
-
 // CTAs per partition.  Every CTA pays a fixed cost (its prologue, the first loads, the reduction at
 // the end) worth about one and a half tiles of streaming, and a wave of resident CTAs takes as long
 // as its longest member, so the estimate to minimise is waves x (tiles per CTA + 1.5), over the counts
@@ -1487,7 +1083,6 @@ Geometry cclip_geometry(int n, int P, long long stride)
     g.RG = (n + g.R - 1) / g.R;
     g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 8) ? 64 : 32;
     g.threads = g.RG * g.CL;
-    g.tiles = 0;
     const size_t smem = (g.RG > 1) ? sizeof(float4) * 2 * g.RG * g.CL : 0;
     const int slots = sm_count() * iter_ctas_per_sm(g.R, g.threads, smem);
     g.slots = slots;
@@ -1497,7 +1092,7 @@ Geometry cclip_geometry(int n, int P, long long stride)
 
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st)
 {
-    KernelArgs ka{a, geo.RG, geo.CL, geo.tiles, geo.cpp};
+    KernelArgs ka{a, geo.RG, geo.CL, geo.cpp};
     const size_t smem = (geo.RG > 1) ? sizeof(float4) * 2 * geo.RG * geo.CL : 0;
     const int grid = a.P * geo.cpp;
     switch (geo.R) {
@@ -1509,7 +1104,7 @@ int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaS
 
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st)
 {
-    KernelArgs ka{a, geo.RG, geo.CL, geo.tiles, geo.cpp};
+    KernelArgs ka{a, geo.RG, geo.CL, geo.cpp};
     cclip_finalize_kernel<<<a.P, 128, 0, st>>>(ka);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
@@ -1524,62 +1119,42 @@ int launch_totals_to_norms(const double* tot, double* norm, int n, int P, cudaSt
     return BTARD_OK;
 }
 
-// Resident CTAs per SM of the resident kernel (2 when no device can be asked).
-static int resident_ctas_per_sm(int R, bool comp, int threads, size_t smem)
+// CTAs per SM of the cooperative kernel (0 when no device can be asked).
+static int cooperative_ctas_per_sm(int R, bool comp, int threads, size_t smem)
 {
     int nb = 0;
     cudaError_t e;
-    if (R == 4) e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<4, true>, threads, smem)
-                         : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<4, false>, threads, smem);
-    else if (R == 8) e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<8, true>, threads, smem)
-                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<8, false>, threads, smem);
-    else e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<16, true>, threads, smem)
-                  : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_resident_kernel<16, false>, threads, smem);
+    if (R == 4) e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_cooperative_kernel<4, true>, threads, smem)
+                         : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_cooperative_kernel<4, false>, threads, smem);
+    else if (R == 8) e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_cooperative_kernel<8, true>, threads, smem)
+                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_cooperative_kernel<8, false>, threads, smem);
+    else e = comp ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_cooperative_kernel<16, true>, threads, smem)
+                  : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cclip_cooperative_kernel<16, false>, threads, smem);
     if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 0; }
     return nb;
 }
 
-int resident_chunk_partitions(int n, long long stride)
+int launch_cclip_cooperative(const CclipLaunch& a, const Geometry& geo, int streaming, double* rslots,
+                             unsigned long long* barrier, unsigned int* error, cudaStream_t st)
 {
-    int dev = 0, l2 = 0, coop = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return 0;
-    }
-    if (!coop || l2 <= 0) return 0;
-    // rows + v (fp32 and bf16) of one partition against three quarters of the L2
-    const double part_bytes = (double)stride * (4.0 * n + 6.0);
-    return (int)(0.75 * (double)l2 / part_bytes);
-}
-
-int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, int items_per_partition,
-                          int streaming, double* rslots, unsigned long long* barrier,
-                          unsigned int* error, cudaStream_t st)
-{
-    ResidentArgs ra{a, geo.RG, geo.CL, 0, streaming, rslots, barrier, error};
+    CoopArgs ra{a, geo.RG, geo.CL, 0, streaming, rslots, barrier, error};
     const bool comp = a.v_lo != nullptr;
     const size_t smem = (geo.RG > 1) ? sizeof(float4) * 2 * geo.RG * geo.CL : 0;
-    const int occ = resident_ctas_per_sm(geo.R, comp, geo.threads, smem);
+    const int occ = cooperative_ctas_per_sm(geo.R, comp, geo.threads, smem);
     if (occ < 1) return BTARD_ERR_UNSUPPORTED;
     int grid = sm_count() * occ;
-    if (grid > kResidentMaxGrid) grid = kResidentMaxGrid;
-    long long cppc = items_per_partition;
-    if (cppc < 1) {                                    // one item per resident CTA
-        if (grid < a.P) return BTARD_ERR_UNSUPPORTED;
-        cppc = grid / a.P;
-    }
+    if (grid > kCoopMaxGrid) grid = kCoopMaxGrid;
+    long long cppc = geo.cpp;                          // the work items of the launch-per-update path
     const long long most = ((a.stride >> 2) + 7) / 8;          // at least one 128-byte line per item
     if (cppc > most) cppc = most < 1 ? 1 : most;
-    if ((long long)a.P * cppc > kResidentMaxItems) return BTARD_ERR_UNSUPPORTED;
+    if ((long long)a.P * cppc > kCoopMaxItems) return BTARD_ERR_UNSUPPORTED;
     ra.cppc = (int)cppc;
     if ((long long)grid > (long long)a.P * cppc) grid = (int)((long long)a.P * cppc);
     void* args[] = {(void*)&ra};
     const void* fn;
-    if (geo.R == 4) fn = comp ? (const void*)cclip_resident_kernel<4, true> : (const void*)cclip_resident_kernel<4, false>;
-    else if (geo.R == 8) fn = comp ? (const void*)cclip_resident_kernel<8, true> : (const void*)cclip_resident_kernel<8, false>;
-    else fn = comp ? (const void*)cclip_resident_kernel<16, true> : (const void*)cclip_resident_kernel<16, false>;
+    if (geo.R == 4) fn = comp ? (const void*)cclip_cooperative_kernel<4, true> : (const void*)cclip_cooperative_kernel<4, false>;
+    else if (geo.R == 8) fn = comp ? (const void*)cclip_cooperative_kernel<8, true> : (const void*)cclip_cooperative_kernel<8, false>;
+    else fn = comp ? (const void*)cclip_cooperative_kernel<16, true> : (const void*)cclip_cooperative_kernel<16, false>;
     prof_begin(KIND_ITER, st);
     cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(geo.threads), args, smem, st);
     prof_end(KIND_ITER, st);

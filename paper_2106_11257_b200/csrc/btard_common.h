@@ -1,6 +1,7 @@
 // Shared declarations of the library's translation units (not part of the public ABI).
 #pragma once
 #include <cuda_runtime.h>
+#include <atomic>
 #include <cstddef>
 #include <cstdint>
 
@@ -21,7 +22,6 @@ struct Geometry {
     int RG;       // row groups = ceil(n / R)
     int CL;       // column lanes (multiple of 32)
     int threads;  // RG * CL
-    int tiles;    // unused
     int cpp;      // CTAs per partition
     int slots;    // CTAs resident on the whole GPU at once
 };
@@ -43,6 +43,13 @@ enum KernelKind { KIND_MEDIAN = 0, KIND_INIT = 1, KIND_ITER = 2, KIND_VERIFY = 3
 void prof_begin(int kind, cudaStream_t st);
 void prof_end(int kind, cudaStream_t st);
 int sm_count();
+// One bit per device ordinal: true until mark_device_done() has been called for the current device.
+// Used to set kernel attributes once per device instead of on every call (setting them twice is
+// harmless, so two threads racing here only repeat the work).
+bool device_needs_setup(const std::atomic<unsigned long long>& seen);
+void mark_device_done(std::atomic<unsigned long long>& seen);
+// Writes {part_len[p], tau[p]} (tau == nullptr: 0) for p < P to a device table, as kernel arguments.
+int upload_table(PartEntry* dev, int P, const int64_t* part_len, const double* tau, cudaStream_t st);
 
 #define BTARD_CUDA_TRY(expr)                         \
     do {                                             \
@@ -85,27 +92,14 @@ Geometry cclip_geometry(int n, int P, long long stride);
 int choose_ctas_per_partition(int P, long long quads, int CL, int slots, int max_tiles = kMaxTilesPerCta);
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
-// Iteration pass fed by bulk asynchronous copies through shared-memory stages (ok = 0: this shape
-// takes the register-fed pass instead).
-struct StagedGeometry {
-    Geometry g;
-    int ok, stages;
-    unsigned stage_bytes;
-    size_t smem;
-};
-StagedGeometry cclip_staged_geometry(int n, int P, long long stride, bool comp);
-int launch_cclip_staged(const CclipLaunch& a, const StagedGeometry& sg, cudaStream_t st);
-// L2-resident variant: how many partitions fit one chunk (0: not available on this device), and the
-// cooperative launch that runs the start pass and every update of one chunk.
-constexpr int kResidentMaxGrid = 148 * 8;
-constexpr long long kResidentMaxItems = 1LL << 20;
-int resident_chunk_partitions(int n, long long stride);
+// One cooperative launch that runs the start pass and every update of all partitions (work items =
+// the CTAs of launch_cclip_pass, dealt round-robin to one wave of resident CTAs).  streaming != 0:
+// the tensor does not fit L2 (evict-first loads, alternating sweep direction).
+constexpr int kCoopMaxGrid = 148 * 8;
+constexpr long long kCoopMaxItems = 1LL << 20;
 int cooperative_launch_supported();
-// items_per_partition < 1: one work item per resident CTA.  streaming != 0: the chunk does not fit
-// L2 (evict-first loads, alternating sweep direction).
-int launch_cclip_resident(const CclipLaunch& a, const Geometry& geo, int items_per_partition,
-                          int streaming, double* rslots, unsigned long long* barrier,
-                          unsigned int* error, cudaStream_t st);
+int launch_cclip_cooperative(const CclipLaunch& a, const Geometry& geo, int streaming, double* rslots,
+                             unsigned long long* barrier, unsigned int* error, cudaStream_t st);
 int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
                        int P, cudaStream_t st);
 // squared-norm totals -> norms, used when verification is asked to compute the norms itself.

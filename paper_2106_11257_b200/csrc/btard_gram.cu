@@ -955,20 +955,32 @@ GramGeometry gram_geometry(int n, int P, long long stride)
 int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
 {
     GArgs ga{a, geo};
-    if (geo.smem > 48 * 1024)
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.smem));
-    if (a.n <= 16) {
+    // shared-memory opt-in of every Gram kernel: once per device
+    static std::atomic<unsigned long long> attrs_set{0};
+    if (device_needs_setup(attrs_set)) {
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
-    }
-    CUtensorMap map;
-    if (geo.umma) {
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
-        if (!encode_rows_map(&map, a.g, a.n, a.P, a.stride)) { set_cuda_error(cudaErrorInvalidValue); return BTARD_ERR_CUDA; }
+        mark_device_done(attrs_set);
     }
+    if (geo.smem > 96 * 1024) return BTARD_ERR_UNSUPPORTED;
+    // The tensor map of the rows is a function of (g, n, P, stride): the last one is kept per thread.
+    struct MapCache { const float* g; int n, P, dev; long long stride; CUtensorMap map; bool valid; };
+    static thread_local MapCache cache{};
+    if (geo.umma) {
+        int dev = -1;
+        (void)cudaGetDevice(&dev);
+        if (!(cache.valid && cache.g == a.g && cache.n == a.n && cache.P == a.P && cache.stride == a.stride && cache.dev == dev)) {
+            cache.valid = false;
+            if (!encode_rows_map(&cache.map, a.g, a.n, a.P, a.stride)) { set_cuda_error(cudaErrorInvalidValue); return BTARD_ERR_CUDA; }
+            cache.g = a.g; cache.n = a.n; cache.P = a.P; cache.stride = a.stride; cache.dev = dev; cache.valid = true;
+        }
+    }
+    const CUtensorMap& map = cache.map;
     prof_begin(KIND_GRAM, st);
     if (a.n <= 16) {
         const int grid = a.P * geo.cpp;
@@ -992,8 +1004,11 @@ int launch_gram_iterate(const GramLaunch& a, const GramGeometry& geo, cudaStream
 {
     GArgs ga{a, geo};
     const size_t smem = sizeof(double) * ((size_t)a.n * a.n + a.n);
-    if (smem > 48 * 1024)
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_iterate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    static std::atomic<unsigned long long> attrs_set{0};
+    if (device_needs_setup(attrs_set)) {      // n <= 128: at most 129 KB
+        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_iterate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 132 * 1024));
+        mark_device_done(attrs_set);
+    }
     prof_begin(KIND_COEF, st);
     if (a.n <= 16) gram_iterate_warp_kernel<16><<<a.P, 32, 0, st>>>(ga);
     else if (a.n <= 32) gram_iterate_warp_kernel<32><<<a.P, 32, 0, st>>>(ga);

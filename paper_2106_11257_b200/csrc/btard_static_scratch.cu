@@ -25,7 +25,7 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[BTARD_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-constexpr int kMaxStaticPartitions = 1024;     // bounds the on-stack copy of the partition table
+constexpr int kMaxStaticPartitions = 1024;     // more partitions than this never fit the array
 std::mutex g_addr_mu;
 void* g_scratch_addr[kMaxDevices] = {};
 
@@ -69,13 +69,9 @@ extern "C" int btard_verify_projections_static(const btard_verify_args* a)
         return BTARD_ERR_BAD_ALIGNMENT;
     // Beyond this many partitions the problem does not fit the built-in scratch anyway.
     if (P > kMaxStaticPartitions) return BTARD_ERR_WORKSPACE_TOO_SMALL;
-    PartEntry table_host[kMaxStaticPartitions];
-    for (int p = 0; p < P; ++p) {
+    for (int p = 0; p < P; ++p)
         if (a->part_len[p] < 0 || a->part_len[p] > stride || !(a->tau[p] >= 0.0))
             return BTARD_ERR_INVALID_ARG;
-        table_host[p].len = a->part_len[p];
-        table_host[p].tau = a->tau[p];
-    }
 
     // Carve the fixed array; refuse problems that need more than it holds.
     const VerifyGeometry vg = verify_geometry(n, P, stride, K);
@@ -97,9 +93,8 @@ extern "C" int btard_verify_projections_static(const btard_verify_args* a)
     cudaStream_t st = (cudaStream_t)a->stream;
 
     PartEntry* table = (PartEntry*)(base + o_table);
-    // Pageable source: staged by the runtime before the call returns, so the stack copy may go away.
-    BTARD_CUDA_TRY(cudaMemcpyAsync(table, table_host, sizeof(PartEntry) * (size_t)P,
-                                   cudaMemcpyHostToDevice, st));
+    rc = upload_table(table, P, a->part_len, a->tau, st);     // as kernel arguments: no host-memory copy
+    if (rc != BTARD_OK) return rc;
 
     const double* norms = a->resid_norm_in;
     if (!norms) {   // one more pass over g: residual norms at v

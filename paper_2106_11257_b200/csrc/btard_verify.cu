@@ -22,7 +22,7 @@ __device__ __forceinline__ double warp_sum(double x)
 
 struct VArgs {
     VerifyLaunch a;
-    int RG, CL, tiles, cpp, slots;
+    int RG, CL, cpp, slots;
 };
 
 // slot layout per CTA: [n*KT] dots (row-major i, k), [KT] znorm2, [1] squared norm of resid_sum
@@ -673,8 +673,32 @@ int occ_r(int KT, int threads, size_t smem, int* nb)
     return (int)e;
 }
 
+// Dynamic shared memory of the shared-z kernel: z block [2][KT][CL], column sums [2][RG][CL] and, with
+// the combine pass fused in, the moves of v [2][RG][CL], as float4.  At most 80 KB (KT = 8, CL = 256),
+// which is above the 48 KB a kernel gets without opting in: every instantiation opts in once per device.
+constexpr int kVerifyMaxSmem = 96 * 1024;
+
+template <int R, int KT>
+void verify_opt_in()
+{
+    (void)cudaFuncSetAttribute(verify_kernel<R, KT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifyMaxSmem);
+    (void)cudaFuncSetAttribute(verify_kernel<R, KT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifyMaxSmem);
+}
+
+void ensure_verify_attrs()
+{
+    static std::atomic<unsigned long long> attrs_set{0};
+    if (!device_needs_setup(attrs_set)) return;
+    verify_opt_in<4, 1>(); verify_opt_in<4, 2>(); verify_opt_in<4, 4>(); verify_opt_in<4, 8>();
+    verify_opt_in<8, 1>(); verify_opt_in<8, 2>(); verify_opt_in<8, 4>(); verify_opt_in<8, 8>();
+    verify_opt_in<16, 1>(); verify_opt_in<16, 2>();
+    (void)cudaGetLastError();                          // no device: the sizing falls back to fixed figures
+    mark_device_done(attrs_set);
+}
+
 int verify_ctas_per_sm(int R, int KT, int threads, size_t smem)
 {
+    ensure_verify_attrs();                             // the occupancy answer depends on the opt-in
     int nb = 0, e;
     if (R == 4) e = occ_r<4>(KT, threads, smem, &nb);
     else if (R == 8) e = occ_r<8>(KT, threads, smem, &nb);
@@ -726,7 +750,6 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
         g.RG = 1;
         g.CL = 256;
         g.threads = 256;
-        g.tiles = 0;
         vg.KT = K;
         g.slots = sm_count() * rows_ctas_per_sm(g.R, K);
         g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, g.slots);
@@ -756,7 +779,6 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     while (kt < K && kt < 8) kt <<= 1;
     if (g.R == 16 && kt > 2) kt = 2;          // 16 rows per thread: keep the accumulators in registers
     vg.KT = kt;
-    g.tiles = 0;
     const size_t smem = sizeof(float4) * (2 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
     const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, g.threads, smem);
     g.slots = slots;
@@ -768,9 +790,11 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
 int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t st)
 {
     const Geometry& g = vg.g;
-    VArgs va{a, g.RG, g.CL, g.tiles, g.cpp, vg.slots};
+    VArgs va{a, g.RG, g.CL, g.cpp, vg.slots};
     const size_t smem = sizeof(float4) * (2 * (size_t)vg.KT * g.CL + (a.combine ? 4 : 2) * (size_t)g.RG * g.CL);
     const int grid = a.P * g.cpp;
+    if (smem > (size_t)kVerifyMaxSmem) return BTARD_ERR_UNSUPPORTED;
+    ensure_verify_attrs();
     int rc;
     if (vg.own_z) {
         switch (g.R) {

@@ -36,24 +36,32 @@ def run_gpu_cclip(g_np, tau, lens, **kw):
     return g, r
 
 
-def check_cclip(r, ref, lens, eps_mode=False):
+def check_cclip(r, ref, lens, eps_mode=False, g=None, tau=None, init=None, v0=None, rule=0):
+    """Compares one aggregation with the oracle's.  In eps mode the update counts may differ by one
+    (the stop test sits on a rounding edge); the GPU result is then compared with the oracle run for
+    exactly the GPU's number of updates, which needs the inputs (g, tau, init)."""
     P = ref["v"].shape[0]
     v = cpu(r["v"])
     it = cpu(r["iters"])
     for p in range(P):
         L = int(lens[p])
+        refp = {k: ref[k][p] for k in ("v", "resid_norm", "last_step_norm", "iters")}
         if eps_mode:
             assert abs(int(it[p]) - int(ref["iters"][p])) <= 1, (p, it[p], ref["iters"][p])
             if it[p] != ref["iters"][p]:
-                continue
+                if g is None:
+                    continue
+                again = oracle.centered_clip(g[p], float(np.broadcast_to(tau, (P,))[p]), lens[p:p + 1], init_mode=init,
+                                             v0=None if v0 is None else v0[p], max_iters=int(it[p]), rule=rule)
+                refp = {k: again[k][0] for k in ("v", "resid_norm", "last_step_norm", "iters")}
         else:
             assert it[p] == ref["iters"][p]
-        assert rel_l2(v[p, :L], ref["v"][p, :L]) <= RTOL, ("v", p)
+        assert rel_l2(v[p, :L], refp["v"][:L]) <= RTOL, ("v", p)
         assert np.all(v[p, L:] == 0)
-        assert rel_l2(cpu(r["resid_norm"])[p], ref["resid_norm"][p]) <= RTOL
-        ls, lr = cpu(r["last_step_norm"])[p], ref["last_step_norm"][p]
+        assert rel_l2(cpu(r["resid_norm"])[p], refp["resid_norm"]) <= RTOL
+        ls, lr = cpu(r["last_step_norm"])[p], refp["last_step_norm"]
         # the last step is a difference of nearly equal vectors: absolute floor from fp32 v
-        assert abs(ls - lr) <= 1e-4 * lr + 3e-7 * (1 + np.linalg.norm(ref["v"][p, :L])), (p, ls, lr)
+        assert abs(ls - lr) <= 1e-4 * lr + 3e-7 * (1 + np.linalg.norm(refp["v"][:L])), (p, ls, lr)
 
 
 # ----------------------------------------------------------------------------- z and layout
@@ -85,7 +93,7 @@ def make_case(rng, P, n, stride, lens, far_rows=0, scale=0.02):
     return g
 
 
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED, btard.ALGO_DIRECT_COOPERATIVE])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
 @pytest.mark.parametrize("n", [1, 3, 4, 7, 8, 16, 23, 64, 100, 256])
 @pytest.mark.parametrize("init", [btard.INIT_ZERO, btard.INIT_MEAN, btard.INIT_COORD_MEDIAN,
                                   btard.INIT_CALLER_V0])
@@ -104,7 +112,7 @@ def test_fixed_iterations_match_oracle(n, init, algo):
     assert not (cpu(r["status"]) & 4).any()
 
 
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
 @pytest.mark.parametrize("stop", [btard.STOP_FIXED_ITERS, btard.STOP_EPS])
 def test_many_tiles_per_cta_and_many_ctas(algo, stop):
     """One long partition: several CTAs, each with many tiles, plus a ragged last tile."""
@@ -114,7 +122,7 @@ def test_many_tiles_per_cta_and_many_ctas(algo, stop):
     g = make_case(rng, P, n, stride, lens, far_rows=5, scale=0.001)
     ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4, stop_mode=stop, eps=1e-9)
     _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=4, algo=algo, stop_mode=stop, eps=1e-9)
-    check_cclip(r, ref, lens, eps_mode=(stop == btard.STOP_EPS))
+    check_cclip(r, ref, lens, eps_mode=(stop == btard.STOP_EPS), g=g, tau=1.0, init=oracle.INIT_COORD_MEDIAN)
 
 
 def test_config1_fixed_and_eps():
@@ -127,11 +135,11 @@ def test_config1_fixed_and_eps():
                                stop_mode=oracle.STOP_EPS, max_iters=100, eps=1e-6)
     _, r = run_gpu_cclip(g, w.tau, w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
                          stop_mode=btard.STOP_EPS, max_iters=100, eps=1e-6)
-    check_cclip(r, ref, w.part_len, eps_mode=True)
+    check_cclip(r, ref, w.part_len, eps_mode=True, g=g, tau=w.tau, init=oracle.INIT_COORD_MEDIAN)
     assert cpu(r["status"])[0] == ref["status"][0] == 0
 
 
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED, btard.ALGO_DIRECT_COOPERATIVE])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
 def test_eps_mode_counts_and_cap_flag(algo):
     rng = np.random.default_rng(6)
     P, n, stride = 4, 8, 2048
@@ -142,7 +150,7 @@ def test_eps_mode_counts_and_cap_flag(algo):
                                    max_iters=cap, eps=eps)
         _, r = run_gpu_cclip(g, 0.7, lens, init_mode=btard.INIT_MEAN, stop_mode=btard.STOP_EPS,
                              max_iters=cap, eps=eps, algo=algo)
-        check_cclip(r, ref, lens, eps_mode=True)
+        check_cclip(r, ref, lens, eps_mode=True, g=g, tau=0.7, init=oracle.INIT_MEAN)
         same = cpu(r["iters"]) == ref["iters"]
         assert np.array_equal(cpu(r["status"])[same] & 1, ref["status"][same] & 1)
     assert len(set(ref["iters"])) >= 1
@@ -162,7 +170,7 @@ def test_special_radii():
     assert np.all(v[1] == 0)                                               # tau = 0: never moves
 
 
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
 @pytest.mark.parametrize("stride", [1024, 40_000])
 def test_non_finite_rows_take_weight_zero(algo, stride):
     rng = np.random.default_rng(8)
@@ -184,6 +192,47 @@ def test_non_finite_rows_take_weight_zero(algo, stride):
     assert np.array_equal(np.isfinite(rn), np.isfinite(ref["resid_norm"]))
 
 
+@pytest.mark.parametrize("n", [5, 16, 40])
+def test_non_finite_rows_with_a_median_start(n):
+    """A Byzantine row holding NaN / inf together with the coordinate-median start (the start every
+    benchmark uses): the median orders NaNs at the ends, the row takes weight 0 in every update; direct,
+    Gram and one-call paths."""
+    rng = np.random.default_rng(80 + n)
+    P, stride = 2, 4096
+    lens = np.array([4096, 4001])
+    g = make_case(rng, P, n, stride, lens)
+    g[0, 2, 17] = np.nan
+    g[0, 2, 18] = -np.nan
+    g[1, n - 1, 900] = np.inf
+    g[1, n - 1, 3] = -np.inf
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=5)
+    assert np.all(np.isfinite(ref["v"])) and (ref["status"] & oracle.STATUS_NONFINITE_ROW).all()
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM, btard.ALGO_DIRECT_COOPERATIVE):
+        _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=5, algo=algo)
+        v = cpu(r["v"])
+        assert np.all(np.isfinite(v))
+        for p in range(P):
+            assert rel_l2(v[p], ref["v"][p]) <= RTOL, (algo, p)
+            assert cpu(r["status"])[p] & btard.STATUS_NONFINITE_ROW
+        rn = cpu(r["resid_norm"])
+        fin = np.isfinite(ref["resid_norm"])
+        assert np.array_equal(np.isfinite(rn), fin) and rel_l2(rn[fin], ref["resid_norm"][fin]) <= RTOL
+    rc, rv = btard.centered_clip_verify(torch.from_numpy(g).cuda(), 1.0, 5, K=2, part_len=lens,
+                                        init_mode=btard.INIT_COORD_MEDIAN, max_iters=5, algo=btard.ALGO_GRAM)
+    torch.cuda.synchronize()
+    v = cpu(rc["v"])
+    refv = oracle.verify(g, v, 1.0, 5, K=2, part_len=lens)
+    for p in range(P):
+        assert rel_l2(v[p], ref["v"][p]) <= RTOL
+        assert cpu(rc["status"])[p] & btard.STATUS_NONFINITE_ROW and cpu(rv["status"])[p] & btard.STATUS_NONFINITE_ROW
+        fin = np.isfinite(refv["norm"][p])
+        assert np.array_equal(np.isfinite(cpu(rv["norm"])[p]), fin)
+        assert np.array_equal(cpu(rv["weight"])[p] == 0.0, ~fin)
+        assert rel_l2(cpu(rv["s"])[p][fin], refv["s"][p][fin]) <= RTOL
+        scale = np.abs(refv["s"][p]).sum(0) + 1e-300
+        assert np.all(np.abs(cpu(rv["s_sum"])[p] - refv["s_sum"][p]) <= RTOL * scale)
+
+
 def test_peer_and_partition_indexing():
     """Row i / slab p of every output belongs to peer i / partition p: distinct magnitudes."""
     P, n, stride = 4, 5, 256
@@ -198,27 +247,10 @@ def test_peer_and_partition_indexing():
     assert np.allclose(cpu(r["v"]), ref["v"], rtol=1e-6)
 
 
-# ----------------------------------------------------------------------------- L2-resident variant
-@pytest.mark.parametrize("n", [1, 4, 16, 23, 64, 256])
-@pytest.mark.parametrize("init", [btard.INIT_ZERO, btard.INIT_MEAN, btard.INIT_COORD_MEDIAN,
-                                  btard.INIT_CALLER_V0])
-def test_resident_variant_matches_oracle(n, init):
-    """All updates of a chunk inside one cooperative kernel with grid barriers: same numbers."""
-    rng = np.random.default_rng(400 + n)
-    P, stride = 3, 5024
-    lens = np.array([5024, 4097, 0 if n % 2 else 13])
-    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
-    tau = np.array([0.5, 1.0, 2.0])
-    v0 = rng.standard_normal((P, stride)).astype(np.float32) if init == btard.INIT_CALLER_V0 else None
-    ref = oracle.centered_clip(g, tau, lens, init_mode=init, v0=v0, max_iters=6)
-    _, r = run_gpu_cclip(g, tau, lens, init_mode=init, v0=v0, max_iters=6, algo=btard.ALGO_DIRECT_RESIDENT)
-    check_cclip(r, ref, lens)
-    assert not (cpu(r["status"]) & 4).any()
-
-
-def test_resident_variant_eps_mode_and_chunks():
-    """Rows long enough that the partitions go through in several L2-sized chunks; eps stop with
-    partitions finishing at different updates."""
+# ----------------------------------------------------------------------------- cooperative variant
+def test_cooperative_variant_eps_mode_many_items_per_cta():
+    """All updates inside one cooperative kernel with grid barriers; rows long enough that every
+    resident CTA holds several work items, eps stop with partitions finishing at different updates."""
     rng = np.random.default_rng(12)
     P, n, stride = 5, 16, 600_000
     lens = np.array([600_000, 599_999, 123_457, 600_000, 31])
@@ -227,14 +259,14 @@ def test_resident_variant_eps_mode_and_chunks():
     ref = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN,
                                stop_mode=oracle.STOP_EPS, max_iters=60, eps=1e-5)
     _, r = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_COORD_MEDIAN, stop_mode=btard.STOP_EPS,
-                         max_iters=60, eps=1e-5, algo=btard.ALGO_DIRECT_RESIDENT)
-    check_cclip(r, ref, lens, eps_mode=True)
+                         max_iters=60, eps=1e-5, algo=btard.ALGO_DIRECT_COOPERATIVE)
+    check_cclip(r, ref, lens, eps_mode=True, g=g, tau=tau, init=oracle.INIT_COORD_MEDIAN)
     assert len(set(ref["iters"].tolist())) > 1
+    assert not (cpu(r["status"]) & 4).any()
 
 
 # ----------------------------------------------------------------------------- baseline aggregators
-@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_STAGED, btard.ALGO_DIRECT_COOPERATIVE,
-                                  btard.ALGO_DIRECT_RESIDENT])
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE])
 @pytest.mark.parametrize("n", [3, 16, 64])
 def test_geometric_median_rule_matches_oracle(n, algo):
     rng = np.random.default_rng(500 + n)
@@ -247,7 +279,8 @@ def test_geometric_median_rule_matches_oracle(n, algo):
                                    max_iters=iters, eps=eps, rule=oracle.RULE_GEOMETRIC_MEDIAN)
         _, r = run_gpu_cclip(g, floor, lens, init_mode=btard.INIT_MEAN, stop_mode=stop, max_iters=iters,
                              eps=eps, algo=algo, rule=btard.RULE_GEOMETRIC_MEDIAN)
-        check_cclip(r, ref, lens, eps_mode=(stop == btard.STOP_EPS))
+        check_cclip(r, ref, lens, eps_mode=(stop == btard.STOP_EPS), g=g, tau=floor, init=oracle.INIT_MEAN,
+                    rule=oracle.RULE_GEOMETRIC_MEDIAN)
 
 
 @pytest.mark.parametrize("n", [1, 4, 16, 23, 64, 100])
@@ -371,7 +404,7 @@ def test_gram_mode_eps_and_long_rows():
                                stop_mode=oracle.STOP_EPS, max_iters=300, eps=1e-6)
     _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, stop_mode=btard.STOP_EPS,
                          max_iters=300, eps=1e-6, algo=btard.ALGO_GRAM)
-    check_cclip(r, ref, lens, eps_mode=True)
+    check_cclip(r, ref, lens, eps_mode=True, g=g, tau=1.0, init=oracle.INIT_COORD_MEDIAN)
     assert np.array_equal(cpu(r["status"]) & 1, ref["status"] & 1)
 
 
@@ -408,7 +441,8 @@ def check_verify(out, ref, K):
 
 
 @pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (4, 2), (5, 3), (8, 2), (13, 2), (16, 8), (16, 1), (16, 2),
-                                 (23, 4), (64, 4), (64, 8), (64, 11), (100, 2), (200, 5)])
+                                 (23, 4), (64, 4), (64, 8), (64, 11), (100, 2), (200, 5),
+                                 (1, 8), (4, 8), (4, 64)])       # one row group, 8 directions: the largest z block
 def test_verify_matches_oracle(n, K):
     rng = np.random.default_rng(200 + n + K)
     P, stride = 3, 5024
@@ -441,7 +475,8 @@ def test_verify_matches_oracle(n, K):
 
 @pytest.mark.parametrize("algo", [btard.ALGO_GRAM, btard.ALGO_DIRECT])
 @pytest.mark.parametrize("n,K", [(1, 1), (4, 1), (7, 2), (16, 1), (16, 2), (16, 3), (16, 8), (23, 1), (64, 2),
-                                 (64, 4), (64, 11), (100, 2)])
+                                 (64, 4), (64, 11), (100, 2),
+                                 (4, 3), (4, 8), (7, 8)])         # fused pass with more than 48 KB of shared memory
 def test_one_call_aggregation_and_verification(n, K, algo):
     """btard_centered_clip_verify against the oracle's aggregation followed by its verification.  With the
     Gram variant the combine and verification passes are one kernel (all rows of a column in one thread
@@ -610,12 +645,53 @@ def test_aggregate_host_matches_device_path():
         assert rel_l2(h2[key].numpy(), h[key].numpy()) <= 1e-6, key
 
 
+def test_aggregate_host_gram_path_and_uneven_chunks():
+    """The host-buffer call with the Gram variant, and a partition count whose chunks of P/4 need more
+    workspace than the whole batch would (fewer partitions get more CTAs each): 38 partitions, K = 8."""
+    rng = np.random.default_rng(21)
+    P, n, stride, K = 38, 16, 8192, 8
+    lens = np.full(P, stride)
+    lens[-1] = 4097
+    g = make_case(rng, P, n, stride, lens, far_rows=4)
+    gh = torch.from_numpy(g).pin_memory()
+    refc = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=7)
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
+        for cs in (None, torch.cuda.Stream()):
+            h = btard.aggregate_host(gh, 1.0, 77, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                     max_iters=7, copy_stream=cs, algo=algo)
+            hc = dict(v=h["v"].cuda(), iters=h["iters"], resid_norm=h["norm"], last_step_norm=h["last_step_norm"])
+            check_cclip(hc, refc, lens)
+            refv = oracle.verify(g, h["v"].numpy(), 1.0, 77, K=K, part_len=lens, norm_in=h["norm"].numpy())
+            check_verify(h, refv, K)
+            assert not h["status"].numpy().any()
+    # eps mode through the host call: the cooperative kernel per chunk, and the Gram variant
+    refe = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, stop_mode=oracle.STOP_EPS,
+                                max_iters=40, eps=1e-4)
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
+        h = btard.aggregate_host(gh, 1.0, 77, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                 stop_mode=btard.STOP_EPS, max_iters=40, eps=1e-4,
+                                 copy_stream=torch.cuda.Stream(), algo=algo)
+        hc = dict(v=h["v"].cuda(), iters=h["iters"], resid_norm=h["norm"], last_step_norm=h["last_step_norm"])
+        check_cclip(hc, refe, lens, eps_mode=True, g=g, tau=1.0, init=oracle.INIT_COORD_MEDIAN)
+
+
 # ----------------------------------------------------------------------------- full-size configs
+_WORKLOADS = {}
+_ORACLE_MEMO = {}
+
+
+def _workload(cfg):
+    """Full-size configurations 2-4 on the GPU, generated once per test session (5.6 GB in all)."""
+    if cfg not in _WORKLOADS:
+        _WORKLOADS[cfg] = workloads.make_workload(cfg, device="cuda")
+    return _WORKLOADS[cfg]
+
+
 def _full_config(cfg, sample, max_iters=None, stop=None, algo=None, one_call=False):
-    """Runs configuration `cfg` at full size on the GPU in the benchmark's launch configuration and
-    compares the sampled partitions with the oracle.  one_call: through btard_centered_clip_verify, as
-    the benchmark does for the Gram variant."""
-    w = workloads.make_workload(cfg, device="cuda")
+    """Runs configuration `cfg` (a number, or a workload already on the GPU) at full size in the
+    benchmark's launch configuration and compares the sampled partitions with the oracle.  one_call:
+    through btard_centered_clip_verify, as the benchmark does for the Gram variant."""
+    w = _workload(cfg) if isinstance(cfg, int) else cfg
     stop_mode = w.stop_mode if stop is None else stop
     iters = w.max_iters if max_iters is None else max_iters
     if one_call:
@@ -629,81 +705,66 @@ def _full_config(cfg, sample, max_iters=None, stop=None, algo=None, one_call=Fal
         o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
                                      resid_norm_in=r["resid_norm"])
     torch.cuda.synchronize()
-    for p in sample:
-        gp = cpu(w.g[p:p + 1])
-        lens = w.part_len[p:p + 1]
-        ref = oracle.centered_clip(gp, w.tau[p], lens, init_mode=oracle.INIT_COORD_MEDIAN,
-                                   stop_mode=stop_mode, max_iters=iters, eps=w.eps)
-        sub = {k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}
-        check_cclip(sub, ref, lens, eps_mode=(stop_mode == btard.STOP_EPS))
-        vp = cpu(r["v"][p:p + 1])
-        nin = cpu(r["resid_norm"][p:p + 1])
-        refv = oracle.verify(gp, vp, w.tau[p], w.zseed, K=w.K, part_len=lens, norm_in=nin,
-                             first_partition=p)
+    sample = list(sample)
+    idx = torch.tensor(sample, device=w.g.device)
+    gs = cpu(w.g.index_select(0, idx))                       # the oracle runs the sampled partitions in parallel
+    lens, taus = w.part_len[sample], w.tau[sample]
+    key = (id(w), tuple(sample), stop_mode, iters)           # the same reference serves every algorithm
+    if key not in _ORACLE_MEMO:
+        _ORACLE_MEMO.clear()
+        _ORACLE_MEMO[key] = oracle.centered_clip(gs, taus, lens, init_mode=oracle.INIT_COORD_MEDIAN,
+                                                 stop_mode=stop_mode, max_iters=iters, eps=w.eps)
+    ref = _ORACLE_MEMO[key]
+    sub = {k: r[k].index_select(0, idx) for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}
+    check_cclip(sub, ref, lens, eps_mode=(stop_mode == btard.STOP_EPS), g=gs, tau=taus,
+                init=oracle.INIT_COORD_MEDIAN)
+    for s, p in enumerate(sample):                           # z is keyed by the partition's true index
+        refv = oracle.verify(gs[s:s + 1], cpu(sub["v"][s:s + 1]), taus[s], w.zseed, K=w.K, part_len=lens[s:s + 1],
+                             norm_in=cpu(sub["resid_norm"][s:s + 1]), first_partition=p)
         subo = {k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2",
                                           "resid_sum_norm")}
         check_verify(subo, refv, w.K)
     return w, r, o
 
 
-def test_config2_full_size_sampled():
-    w, r, o = _full_config(2, sample=[0, 15])
+def test_config2_full_size_all_partitions():
+    _full_config(2, sample=range(16))
     # fixed-iteration parity at full size as well (eps mode may differ by one update)
-    _full_config(2, sample=[7], max_iters=10, stop=btard.STOP_FIXED_ITERS)
+    _full_config(2, sample=range(16), max_iters=10, stop=btard.STOP_FIXED_ITERS)
 
 
-def test_config3_full_size_sampled():
-    _full_config(3, sample=[3, 15], max_iters=10, stop=btard.STOP_FIXED_ITERS)
-    _full_config(3, sample=[9])
+def test_config3_full_size_all_partitions():
+    _full_config(3, sample=range(16), max_iters=10, stop=btard.STOP_FIXED_ITERS)
+    _full_config(3, sample=range(16))
 
 
-def test_config4_full_size_sampled():
-    _full_config(4, sample=[0, 63])
-    _full_config(4, sample=[31], max_iters=5, stop=btard.STOP_FIXED_ITERS)
+def test_config4_full_size_all_partitions():
+    _full_config(4, sample=range(0, 64, 2))
+    _full_config(4, sample=range(1, 64, 2), max_iters=5, stop=btard.STOP_FIXED_ITERS)
 
 
-def test_config2_and_4_gram_mode_full_size_sampled():
-    _full_config(2, sample=[5], max_iters=20, stop=btard.STOP_FIXED_ITERS, algo=btard.ALGO_GRAM)
-    _full_config(4, sample=[17], algo=btard.ALGO_GRAM)
+def test_config2_and_4_gram_mode_full_size():
+    _full_config(2, sample=range(16), max_iters=20, stop=btard.STOP_FIXED_ITERS, algo=btard.ALGO_GRAM)
+    _full_config(4, sample=range(0, 64, 4), algo=btard.ALGO_GRAM)
 
 
-def test_gram_one_call_full_size_sampled():
+def test_gram_one_call_full_size():
     """The Gram variant through the one-call entry point (fused combine-and-verify pass) at full size."""
-    _full_config(2, sample=[11], max_iters=20, stop=btard.STOP_FIXED_ITERS, algo=btard.ALGO_GRAM, one_call=True)
-    _full_config(3, sample=[6], algo=btard.ALGO_GRAM, one_call=True)
-    _full_config(4, sample=[40], algo=btard.ALGO_GRAM, one_call=True)
+    _full_config(2, sample=range(16), max_iters=20, stop=btard.STOP_FIXED_ITERS, algo=btard.ALGO_GRAM, one_call=True)
+    _full_config(3, sample=range(16), algo=btard.ALGO_GRAM, one_call=True)
+    _full_config(4, sample=range(2, 64, 4), algo=btard.ALGO_GRAM, one_call=True)
 
 
 def test_config5_full_size_sampled():
-    """Config 5 at full size (64 GiB of rows): fixed 20 iterations and the Gram variant side by side,
-    one 1 GiB partition checked against the oracle, then the verification pass (K = 4) on it."""
+    """Config 5 at full size (64 GiB of rows): fixed 20 iterations and the Gram variant side by side
+    (separate calls and the one-call entry point), four 1 GiB partitions checked against the oracle
+    together with the verification pass (K = 4)."""
+    _WORKLOADS.clear()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     d = 1 << 28 if free > 90 * (1 << 30) else 1 << 26              # smaller boards: a quarter of the length
     w = workloads.make_workload(5, device="cuda", d=d)
-    p = 41
-    gp = cpu(w.g[p:p + 1])
-    lens = w.part_len[p:p + 1]
-    ref = oracle.centered_clip(gp, w.tau[p], lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=20)
-    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
-        r = btard.centered_clip(w.g, w.tau, part_len=w.part_len, init_mode=btard.INIT_COORD_MEDIAN,
-                                stop_mode=btard.STOP_FIXED_ITERS, max_iters=20, algo=algo)
-        torch.cuda.synchronize()
-        sub = {k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}
-        check_cclip(sub, ref, lens)
-    o = btard.verify_projections(w.g, r["v"], w.tau, w.zseed, K=w.K, part_len=w.part_len,
-                                 resid_norm_in=r["resid_norm"])
-    torch.cuda.synchronize()
-    refv = oracle.verify(gp, cpu(r["v"][p:p + 1]), w.tau[p], w.zseed, K=w.K, part_len=lens,
-                         norm_in=cpu(r["resid_norm"][p:p + 1]), first_partition=p)
-    subo = {k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm")}
-    check_verify(subo, refv, w.K)
-    # and the Gram variant through the one-call entry point (combine and verification in one pass)
-    r, o = btard.centered_clip_verify(w.g, w.tau, w.zseed, K=w.K, part_len=w.part_len,
-                                      init_mode=btard.INIT_COORD_MEDIAN, stop_mode=btard.STOP_FIXED_ITERS,
-                                      max_iters=20, algo=btard.ALGO_GRAM)
-    torch.cuda.synchronize()
-    check_cclip({k: r[k][p:p + 1] for k in ("v", "iters", "resid_norm", "last_step_norm", "status")}, ref, lens)
-    refv = oracle.verify(gp, cpu(r["v"][p:p + 1]), w.tau[p], w.zseed, K=w.K, part_len=lens,
-                         norm_in=cpu(r["resid_norm"][p:p + 1]), first_partition=p)
-    check_verify({k: o[k][p:p + 1] for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2", "resid_sum_norm")},
-                 refv, w.K)
+    sample = [3, 22, 41, 60]
+    _full_config(w, sample, algo=btard.ALGO_DIRECT)
+    _full_config(w, sample, algo=btard.ALGO_GRAM)
+    _full_config(w, sample, algo=btard.ALGO_GRAM, one_call=True)

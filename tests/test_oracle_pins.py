@@ -286,6 +286,46 @@ def test_coordinate_median_start_is_the_sorted_middle():
         assert np.array_equal(r["v"][0], np.median(x.astype(np.float64), axis=0))
 
 
+def test_coordinate_median_orders_nans_at_the_ends():
+    """IEEE 754 totalOrder puts -NaN below -inf and +NaN above +inf, so NaNs planted in a column never
+    land in the middle while they are a minority: hand-worked columns of 5 and 4 rows."""
+    pnan = np.float32(np.nan)
+    nnan = np.frombuffer(np.uint32(0xFFC00000).tobytes(), dtype=np.float32)[0]
+    assert not np.signbit(pnan) and np.signbit(nnan)
+    cols = [([1.0, pnan, 3.0, nnan, 2.0], 2.0),            # -NaN 1 2 3 +NaN: middle is 2
+            ([pnan, pnan, 1.0, 2.0, 3.0], 3.0),            # 1 2 3 +NaN +NaN: middle is 3
+            ([nnan, 5.0, nnan, 4.0, 6.0], 4.0),            # -NaN -NaN 4 5 6: middle is 4
+            ([nnan, -np.inf, 7.0, np.inf, pnan], 7.0),     # -NaN -inf 7 +inf +NaN
+            ([nnan, 1.0, 2.0, pnan], 1.5),                 # even count: mean of the two middle values
+            ([pnan, 1.0, 2.0, 4.0], 3.0)]                  # 1 2 4 +NaN: (2 + 4) / 2
+    for col, want in cols:
+        x = np.zeros((len(col), 8), dtype=np.float32)
+        x[:, 3] = np.array(col, dtype=np.float32)
+        r = oracle.centered_clip(x, 0.0, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=1)
+        assert r["v"][0, 3] == want, (col, r["v"][0, 3])
+
+
+def test_a_nan_row_with_a_median_start_takes_weight_zero():
+    """Reading of the non-finite rule together with the median start: the row that holds a NaN is left
+    out of every update, so the result equals the aggregation of the other rows from the same start."""
+    rng = np.random.default_rng(81)
+    x = rand_rows(rng, 5, 40)
+    bad = x.copy()
+    bad[2, 7] = np.nan
+    v0 = oracle.centered_clip(bad, 0.0, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=1)["v"][0].astype(np.float32)
+    a = oracle.centered_clip(bad, 0.5, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4)
+    # restated with numpy on the other four rows; the divisor stays the full peer count n = 5
+    keep = np.delete(x, 2, axis=0)
+    v = v0.astype(np.float64)
+    for _ in range(4):
+        r = keep.astype(np.float64) - v
+        rho = np.sqrt((r * r).sum(1))
+        w = np.where(rho <= 0.5, 1.0, 0.5 / rho)
+        v = v + (w[:, None] * r).sum(0) / 5.0
+    assert np.allclose(a["v"][0], v, rtol=0, atol=1e-14)
+    assert a["status"][0] & oracle.STATUS_NONFINITE_ROW and np.isnan(a["resid_norm"][0, 2])
+
+
 def test_padding_does_not_change_the_result():
     """Zero columns past part_len are ignored: a padded run equals the unpadded run."""
     rng = np.random.default_rng(9)

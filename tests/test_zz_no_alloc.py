@@ -5,12 +5,14 @@ component living in a process whose framework already reserved the whole GPU for
 loop that must never call cudaMalloc because the call can stall the device.  It uses an array built
 into the library instead of a caller workspace, and every call on a GPU shares that array.  The test
 therefore calls it twice in a row on different inputs (the second call finds the first call's leftovers
-in the array) and checks both results, through the C ABI, against btard_verify_projections.
+in the array) and checks both results, through the C ABI, against btard_verify_projections and against
+the float64 oracle.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2106_11257_b200 as btard
 
 pytestmark = pytest.mark.gpu
@@ -52,6 +54,15 @@ def test_static_scratch_matches_workspace_entry_twice_in_a_row():
                                               want_resid_sum=True)
         torch.cuda.synchronize()
         _same(got, ref, KEYS + ("resid_sum",))
+        # and against the float64 oracle, on the same terms as the workspace entry point's own test
+        exp = oracle.verify(g.cpu().numpy(), v.cpu().numpy(), c["tau"], 1234, K=c["K"], part_len=c["lens"])
+        for k in ("norm", "weight", "dot", "s"):
+            x = got[k].cpu().numpy()
+            for p in range(c["P"]):
+                den = np.linalg.norm(exp[k][p].ravel())
+                assert np.linalg.norm((x[p] - exp[k][p]).ravel()) <= RTOL * den + 1e-300, (k, p)
+        assert np.allclose(got["znorm2"].cpu().numpy(), exp["znorm2"], rtol=1e-6)
+        assert np.all(np.abs(got["s_sum"].cpu().numpy() - exp["s_sum"]) <= RTOL * (np.abs(exp["s"]).sum(1) + 1e-300))
         # norms handed over by the caller: the other branch of the entry point
         got2 = btard.verify_projections_static(g, v, c["tau"], 1234, K=c["K"], part_len=c["lens"],
                                                resid_norm_in=ref["norm"])
