@@ -7,6 +7,8 @@
 // multiplies its R rows x 4 columns of residuals against it.  Per-thread accumulators are fp32 over
 // at most kMaxTilesPerCta tiles; everything that crosses threads is fp64, written to per-CTA slots
 // and summed in a fixed order by the finalize kernel.
+#include <type_traits>
+
 #include "btard_common.h"
 #include "btard_philox.cuh"
 
@@ -20,23 +22,38 @@ __device__ __forceinline__ double warp_sum(double x)
     return x;
 }
 
+// Streaming 128-bit load of a row's quad as two (column, column + 1) pairs.
+__device__ __forceinline__ void ld_stream_pairs(const float* p, uint64_t& lo, uint64_t& hi)
+{
+    asm volatile("ld.global.cs.v2.b64 {%0, %1}, [%2];" : "=l"(lo), "=l"(hi) : "l"(p));
+}
+
 struct VArgs {
     VerifyLaunch a;
     int RG, CL, cpp, slots;
 };
 
 // slot layout per CTA: [n*KT] dots (row-major i, k), [KT] znorm2, [1] squared norm of resid_sum
+//
+// A CTA is RG row groups x CL column lanes; a thread owns R rows x 4 columns of every tile, held as
+// (column, column + 1) pairs so that residuals, projections, weighted sums and squared norms run on the
+// packed fp32 instructions of sm_100 (two IEEE results per instruction).  The z block of tile t + 1
+// is generated during tile t, while the thread's own loads of tile t are in flight, into the third of
+// three buffers, so the one CTA barrier per tile hands over what was written a whole tile earlier and
+// never waits for the generator.
 // COMBINE: as in verify_rows_kernel, the pass first forms v = v0 + sum_j a_j (x_j - v0) from the
 // coefficients of the Gram variant.  The row groups' partial moves of v are exchanged through shared
-// memory before the CTA barrier that the z block needs anyway, so the tile loop keeps one barrier.
-template <int R, int KT, bool COMBINE>
-__global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
+// memory before the same barrier, so the tile loop keeps one barrier.
+// Interior tiles (inside the CTA's range and the data, no row to leave out) take a path without any
+// predicate; ragged tiles and CTAs with a weight-0 row take the guarded one.
+template <int R, int KT, bool COMBINE, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
 {
-    extern __shared__ float4 sh_dyn[];   // z: [2][KT][CL], column sums: [2][RG][CL], (COMBINE) moves of v: [2][RG][CL]
-    __shared__ float sh_w[BTARD_MAX_PEERS];
-    __shared__ float sh_c[COMBINE ? BTARD_MAX_PEERS : 1];          // coefficients a_j
-    __shared__ double sh_ga[COMBINE ? BTARD_MAX_PEERS + 1 : 1];    // (G a)_i, then a^T G a
-    __shared__ double sh_red[16][R * KT + KT + 1 + (COMBINE ? R : 0)];
+    extern __shared__ float4 sh_dyn[];   // z: [3][KT][CL], column sums: [2][RG][CL], (COMBINE) moves of v: [2][RG][CL]
+    __shared__ __align__(8) float2 sh_w2[BTARD_MAX_PEERS + 16];               // (w_i, w_i), zero beyond row n - 1
+    __shared__ __align__(8) float2 sh_c2[COMBINE ? BTARD_MAX_PEERS + 16 : 1]; // coefficients (a_j, a_j)
+    __shared__ double sh_ga[COMBINE ? BTARD_MAX_PEERS + 1 : 1];               // (G a)_i, then a^T G a
+    __shared__ double sh_red[MAXT / 32][R * KT + KT + 1 + (COMBINE ? R : 0)];
 
     const VerifyLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
@@ -46,9 +63,15 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     const long long stride = a.stride, len = a.table[p].len;
     const double tau = a.table[p].tau;
     float4* sh_z = sh_dyn;
-    float4* sh_s = sh_dyn + 2 * KT * CL;
+    float4* sh_s = sh_dyn + 3 * KT * CL;
     float4* sh_u = sh_s + 2 * RG * CL;
 
+    for (int i = tid; i < BTARD_MAX_PEERS + 16; i += nthr) {
+        sh_w2[i] = make_float2(0.f, 0.f);
+        if (COMBINE) sh_c2[i] = make_float2(0.f, 0.f);
+    }
+    __syncthreads();
+    int skip = 0;                                      // some row of this partition must be left out
     if (COMBINE) {
         // clip weights from the Gram matrix: rho_i^2 = G_ii - 2 (G a)_i + a^T G a (rows with a_j = 0 are skipped)
         const double* G = a.gram + (size_t)p * a.gram_entries;
@@ -60,7 +83,9 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
                 if (cq != 0.0) ga += G[gram_entry_index(a.gram_nb, i, q)] * cq;
             }
             sh_ga[i] = ga;
-            sh_c[i] = (float)cf[i];
+            const float c = (float)cf[i];
+            sh_c2[i] = make_float2(c, c);
+            if (c == 0.0f) skip = 1;
         }
         __syncthreads();
         if (tid == 0) {
@@ -76,35 +101,43 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
             const double rho = sqrt(rho2);
             float w = 0.0f;
             if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
-            sh_w[i] = w;
+            sh_w2[i] = make_float2(w, w);
+            if (w == 0.0f) skip = 1;
         }
     } else {
         for (int i = tid; i < n; i += nthr) {
             const double rho = a.norm_in[(size_t)p * n + i];
             float w = 0.0f;
             if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
-            sh_w[i] = w;
+            sh_w2[i] = make_float2(w, w);
+            if (w == 0.0f) skip = 1;
         }
     }
-    __syncthreads();
-    float w[R];
-    float cw[COMBINE ? R : 1];                         // this thread's coefficients
-    float nacc[COMBINE ? R : 1];                       // squared residual norms at the new v
+    const bool any_skip = __syncthreads_or(skip) != 0;
+    const uint64_t* w2 = reinterpret_cast<const uint64_t*>(sh_w2) + rg * R;     // this thread's rows
+    const uint64_t* c2 = reinterpret_cast<const uint64_t*>(sh_c2) + (COMBINE ? rg * R : 0);
+    unsigned wmask = 0, cmask = 0;                     // rows that enter the weighted sums
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const int i = rg * R + r;
-        w[r] = (i < n) ? sh_w[i] : 0.0f;
-        if (COMBINE) { cw[r] = (i < n) ? sh_c[i] : 0.0f; nacc[r] = 0.0f; }
+        if (sh_w2[rg * R + r].x != 0.0f) wmask |= 1u << r;
+        if (COMBINE && sh_c2[rg * R + r].x != 0.0f) cmask |= 1u << r;
     }
 
-    float acc[R][KT];
+    // Projections: with few enough of them the sums are kept per (column pair); otherwise one sum
+    // per (row, direction) and the two halves of a pair are added on the way in.
+    constexpr bool PACC = (2 * R * KT + 4 * R + (COMBINE ? 2 * R : 0) <= ((65536 / (MAXT * MINB) >= 160) ? 140 : 72));
+    uint64_t acc2[PACC ? R * KT : 1];
+    float acc1[PACC ? 1 : R * KT];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+    for (int e = 0; e < (PACC ? R * KT : 1); ++e) acc2[e] = 0ull;
 #pragma unroll
-        for (int q = 0; q < KT; ++q) acc[r][q] = 0.0f;
-    float zz[KT];
+    for (int e = 0; e < (PACC ? 1 : R * KT); ++e) acc1[e] = 0.0f;
+    uint64_t nacc2[COMBINE ? R : 1];                   // squared residual norms at the new v
 #pragma unroll
-    for (int q = 0; q < KT; ++q) zz[q] = 0.0f;
+    for (int r = 0; r < (COMBINE ? R : 1); ++r) nacc2[r] = 0ull;
+    uint64_t zz2[KT];
+#pragma unroll
+    for (int q = 0; q < KT; ++q) zz2[q] = 0ull;
     float rs2 = 0.0f;
 
     // This CTA's share of the partition in groups of 4 columns, cut on 128-byte lines.
@@ -112,12 +145,31 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
     if (j > 0) q0 &= ~7LL;
     if (j + 1 < cpp) q1 &= ~7LL;
+    const long long full_quads = len >> 2;             // quads that lie entirely inside the data
     const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v + (size_t)p * stride;
     float* rsp = a.resid_sum ? a.resid_sum + (size_t)p * stride : nullptr;
     const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
     const uint32_t pg = (uint32_t)(a.p_base + p);
 
+    // The block of z of the tile that starts at quad qb, into buffer `zbuf` (0..2).
+    auto gen_z = [&](long long qb, int zbuf) {
+        float4* zb = sh_z + (size_t)zbuf * KT * CL;
+        for (int idx = tid; idx < KT * CL; idx += nthr) {
+            const int kq = idx >> cl_shift, cq = idx & (CL - 1);
+            const long long col = (qb + cq) * 4;
+            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (kq < a.kc && qb + cq < q1 && col < len) {
+                z = z_quad((uint32_t)(qb + cq), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
+                if (col + 3 >= len) {                  // only the last quad of a ragged partition
+                    if (col + 1 >= len) z.y = 0.f;
+                    if (col + 2 >= len) z.z = 0.f;
+                    z.w = 0.f;
+                }
+            }
+            zb[kq * CL + cq] = z;
+        }
+    };
     // Adds up the row groups' column sums of the tile at quad qb (written one tile earlier).
     auto consume_sums = [&](long long qb, int par) {
         if (rg != 0) return;
@@ -133,136 +185,133 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
         if (rsp) *reinterpret_cast<float4*>(rsp + col) = s4;
     };
 
-    int par = 0;
-    for (long long qb = q0; qb < q1; qb += CL, par ^= 1) {
-        // 0. this thread's rows and columns are requested first, so that they are in flight while the
-        //    block of z is generated
+    // One tile.  GUARD = false: every lane's quad lies inside the CTA's range and the data, and no row
+    // has to be left out, so nothing is predicated.
+    auto tile = [&](auto guard_tag, long long qb, int par, int zcur) {
+        constexpr bool GUARD = decltype(guard_tag)::value;
         const long long col = (qb + cl) * 4;
-        const bool valid = qb + cl < q1;
-        const bool m0 = valid && col < len, m1 = valid && col + 1 < len;
-        const bool m2 = valid && col + 2 < len, m3 = valid && col + 3 < len;
-        float4 x[R];
-        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        const bool valid = !GUARD || (qb + cl < q1);
+        uint64_t xa[R], xb[R];                         // columns (0, 1) and (2, 3) of the thread's rows
+        uint64_t va = 0ull, vb = 0ull;
         if (valid) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const int i = rg * R + r;
-                x[r] = (i < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)i * stride + col))
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i < n) ld_stream_pairs(gp + (size_t)i * stride + col, xa[r], xb[r]);
+                else { xa[r] = 0ull; xb[r] = 0ull; }
             }
-            v4 = *reinterpret_cast<const float4*>(vp + col);
+            const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
+            va = pk2(v4.x, v4.y);
+            vb = pk2(v4.z, v4.w);
+            if (GUARD && col + 3 >= len) {             // what lies beyond the data counts as 0, in the rows and in v
+                const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len;
+                va = pk2(m0 ? v4.x : 0.f, m1 ? v4.y : 0.f);
+                vb = pk2(m2 ? v4.z : 0.f, 0.f);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float x0, x1, x2, x3;
+                    upk2(xa[r], x0, x1);
+                    upk2(xb[r], x2, x3);
+                    xa[r] = pk2(m0 ? x0 : 0.f, m1 ? x1 : 0.f);
+                    xb[r] = pk2(m2 ? x2 : 0.f, 0.f);
+                }
+            }
         } else {
 #pragma unroll
-            for (int r = 0; r < R; ++r) x[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r = 0; r < R; ++r) { xa[r] = 0ull; xb[r] = 0ull; }
         }
-        // 1. this tile's block of z
-        float4* zb = sh_z + (size_t)par * KT * CL;
-        for (int idx = tid; idx < KT * CL; idx += nthr) {
-            const int kq = idx >> cl_shift, cq = idx & (CL - 1);
-            const long long col = (qb + cq) * 4;
-            float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kq < a.kc && qb + cq < q1 && col < len) {
-                z = z_quad((uint32_t)(qb + cq), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
-                if (col + 3 >= len) {                  // only the last quad of a ragged partition
-                    if (col + 1 >= len) z.y = 0.f;
-                    if (col + 2 >= len) z.z = 0.f;
-                    z.w = 0.f;
-                }
-            }
-            zb[kq * CL + cq] = z;
-        }
+        // the next tile's z, while the rows of this one are on their way; read after the next barrier
+        if (qb + CL < q1) gen_z(qb + CL, zcur == 2 ? 0 : zcur + 1);
         if (COMBINE) {
             // residuals at v0 and this row group's share of the move of v, published before the barrier
-            if (m3) {                                  // whole quad inside the data: no predicates
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
-                }
-            } else {
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    x[r].x = m0 ? x[r].x - v4.x : 0.f; x[r].y = m1 ? x[r].y - v4.y : 0.f;
-                    x[r].z = m2 ? x[r].z - v4.z : 0.f; x[r].w = 0.f;
-                }
-            }
-            float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+            uint64_t ua = 0ull, ub = 0ull;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                if (cw[r] != 0.0f) {                   // coefficient 0: the row is left out, not multiplied
-                    u.x = fmaf(cw[r], x[r].x, u.x); u.y = fmaf(cw[r], x[r].y, u.y);
-                    u.z = fmaf(cw[r], x[r].z, u.z); u.w = fmaf(cw[r], x[r].w, u.w);
+                xa[r] = pk_sub(xa[r], va);
+                xb[r] = pk_sub(xb[r], vb);
+                if (!GUARD || ((cmask >> r) & 1u)) {   // coefficient 0: the row is left out, not multiplied
+                    const uint64_t c = c2[r];
+                    ua = pk_fma(c, xa[r], ua);
+                    ub = pk_fma(c, xb[r], ub);
                 }
             }
+            float4 u;
+            upk2(ua, u.x, u.y);
+            upk2(ub, u.z, u.w);
             sh_u[(size_t)par * RG * CL + rg * CL + cl] = u;
         }
         __syncthreads();
         if (first_chunk && qb > q0) consume_sums(qb - CL, par ^ 1);
 
-        // 2. residuals of this thread's rows and columns
         if (COMBINE) {
-            const float4* ub = sh_u + (size_t)par * RG * CL;
-            float4 u = ub[cl];
+            const float4* ubuf = sh_u + (size_t)par * RG * CL;
+            float4 u = ubuf[cl];
             for (int q = 1; q < RG; ++q) {
-                const float4 o = ub[q * CL + cl];
+                const float4 o = ubuf[q * CL + cl];
                 u.x += o.x; u.y += o.y; u.z += o.z; u.w += o.w;
             }
-            const float4 vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
-            const float4 dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);   // what v really moved by
-            if (rg == 0 && valid)
-                *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) =
-                    make_float4(m0 ? vn.x : 0.f, m1 ? vn.y : 0.f, m2 ? vn.z : 0.f, m3 ? vn.w : 0.f);
-            if (m3) {
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    x[r].x -= dv.x; x[r].y -= dv.y; x[r].z -= dv.z; x[r].w -= dv.w;
-                }
-            } else {
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    x[r].x = m0 ? x[r].x - dv.x : 0.f; x[r].y = m1 ? x[r].y - dv.y : 0.f;
-                    x[r].z = m2 ? x[r].z - dv.z : 0.f; x[r].w = 0.f;
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                nacc[r] += fmaf(x[r].x, x[r].x, fmaf(x[r].y, x[r].y, fmaf(x[r].z, x[r].z, x[r].w * x[r].w)));
-        } else if (m3) {                               // whole quad inside the data: no predicates
+            float v0x, v0y, v0z, v0w;
+            upk2(va, v0x, v0y);
+            upk2(vb, v0z, v0w);
+            const float4 vn = make_float4(v0x + u.x, v0y + u.y, v0z + u.z, v0w + u.w);
+            // what v really moved by (the rounded difference)
+            const uint64_t da = pk2(vn.x - v0x, vn.y - v0y), db = pk2(vn.z - v0z, vn.w - v0w);
+            if (rg == 0 && valid) *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) = vn;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
+                xa[r] = pk_sub(xa[r], da);
+                xb[r] = pk_sub(xb[r], db);
+                nacc2[r] = pk_fma(xb[r], xb[r], pk_fma(xa[r], xa[r], nacc2[r]));
             }
         } else {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                x[r].x = m0 ? x[r].x - v4.x : 0.f;
-                x[r].y = m1 ? x[r].y - v4.y : 0.f;
-                x[r].z = m2 ? x[r].z - v4.z : 0.f;
-                x[r].w = 0.f;
+                xa[r] = pk_sub(xa[r], va);
+                xb[r] = pk_sub(xb[r], vb);
             }
         }
-        // 3. projections
+        // projections
+        const float4* zb = sh_z + (size_t)zcur * KT * CL;
 #pragma unroll
         for (int q = 0; q < KT; ++q) {
             const float4 z = zb[q * CL + cl];
-            if (rg == 0) zz[q] += fmaf(z.x, z.x, fmaf(z.y, z.y, fmaf(z.z, z.z, z.w * z.w)));
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                acc[r][q] += fmaf(x[r].x, z.x, fmaf(x[r].y, z.y, fmaf(x[r].z, z.z, x[r].w * z.w)));
-        }
-        // 4. clipped-residual column sums of this row group
-        if (first_chunk) {
-            float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            const uint64_t za = pk2(z.x, z.y), zc = pk2(z.z, z.w);
+            if (rg == 0) zz2[q] = pk_fma(zc, zc, pk_fma(za, za, zz2[q]));
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                if (w[r] != 0.0f) {
-                    s4.x = fmaf(w[r], x[r].x, s4.x);
-                    s4.y = fmaf(w[r], x[r].y, s4.y);
-                    s4.z = fmaf(w[r], x[r].z, s4.z);
-                    s4.w = fmaf(w[r], x[r].w, s4.w);
+                if (PACC) {
+                    acc2[r * KT + q] = pk_fma(xb[r], zc, pk_fma(xa[r], za, acc2[r * KT + q]));
+                } else {
+                    float lo, hi;
+                    upk2(pk_fma(xb[r], zc, pk_mul(xa[r], za)), lo, hi);
+                    acc1[r * KT + q] += lo + hi;
                 }
             }
+        }
+        // clipped-residual column sums of this row group
+        if (first_chunk) {
+            uint64_t sa = 0ull, sb = 0ull;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                if (!GUARD || ((wmask >> r) & 1u)) {   // weight 0: the row is left out, not multiplied
+                    const uint64_t w = w2[r];
+                    sa = pk_fma(w, xa[r], sa);
+                    sb = pk_fma(w, xb[r], sb);
+                }
+            }
+            float4 s4;
+            upk2(sa, s4.x, s4.y);
+            upk2(sb, s4.z, s4.w);
             sh_s[(size_t)par * RG * CL + rg * CL + cl] = s4;
         }
+    };
+
+    if (q0 < q1) gen_z(q0, 0);                         // made visible by the first tile's barrier
+    int par = 0, zcur = 0;
+    for (long long qb = q0; qb < q1; qb += CL, par ^= 1, zcur = (zcur == 2 ? 0 : zcur + 1)) {
+        const bool inner = !any_skip && qb + CL <= q1 && qb + CL <= full_quads;
+        if (inner) tile(std::false_type{}, qb, par, zcur);
+        else tile(std::true_type{}, qb, par, zcur);
     }
     __syncthreads();
     if (first_chunk && q1 > q0) consume_sums(q0 + (q1 - q0 - 1) / CL * CL, par ^ 1);
@@ -273,12 +322,22 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int q = 0; q < KT; ++q) {
-            const double s = warp_sum((double)acc[r][q]);
+            float d;
+            if (PACC) {
+                float lo, hi;
+                upk2(acc2[r * KT + q], lo, hi);
+                d = lo + hi;
+            } else {
+                d = acc1[r * KT + q];
+            }
+            const double s = warp_sum((double)d);
             if (lane == 0) sh_red[warp][r * KT + q] = s;
         }
 #pragma unroll
     for (int q = 0; q < KT; ++q) {
-        const double s = warp_sum((double)zz[q]);
+        float lo, hi;
+        upk2(zz2[q], lo, hi);
+        const double s = warp_sum((double)lo + (double)hi);
         if (lane == 0) sh_red[warp][R * KT + q] = s;
     }
     {
@@ -288,7 +347,9 @@ __global__ void __launch_bounds__(512) verify_kernel(const VArgs k)
     if (COMBINE) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const double s = warp_sum((double)nacc[r]);
+            float lo, hi;
+            upk2(nacc2[r], lo, hi);
+            const double s = warp_sum((double)lo + (double)hi);
             if (lane == 0) sh_red[warp][R * KT + KT + 1 + r] = s;
         }
     }
@@ -636,74 +697,64 @@ __global__ void random_vector_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_
     *reinterpret_cast<float4*>(z + 4 * q) = v;
 }
 
-template <int R, int KT>
-int launch_rk(const VArgs& va, int threads, size_t smem, int grid, cudaStream_t st)
+// Register budgets: up to 192 threads (16 rows per thread, n <= 64) two CTAs share an SM with 170
+// registers per thread; the 256-thread shapes get 128; shapes of more than 256 threads (n > 64) one CTA.
+template <int R, int KT, int MAXT, int MINB>
+const void* verify_fn_of(bool combine)
 {
-    prof_begin(KIND_VERIFY, st);
-    if (va.a.combine) verify_kernel<R, KT, true><<<grid, threads, smem, st>>>(va);
-    else verify_kernel<R, KT, false><<<grid, threads, smem, st>>>(va);
-    prof_end(KIND_VERIFY, st);
-    BTARD_CUDA_TRY(cudaGetLastError());
-    count_launch();
-    return BTARD_OK;
+    return combine ? (const void*)verify_kernel<R, KT, true, MAXT, MINB> : (const void*)verify_kernel<R, KT, false, MAXT, MINB>;
 }
 
-template <int R>
-int launch_r(const VArgs& va, int KT, int threads, size_t smem, int grid, cudaStream_t st)
+const void* verify_fn(int R, int KT, bool combine, int threads)
 {
-    if (KT == 1) return launch_rk<R, 1>(va, threads, smem, grid, st);
-    if (KT == 2) return launch_rk<R, 2>(va, threads, smem, grid, st);
-    if constexpr (R <= 8) {                 // 16 rows per thread never run more than 2 vectors
-        if (KT == 4) return launch_rk<R, 4>(va, threads, smem, grid, st);
-        if (KT == 8) return launch_rk<R, 8>(va, threads, smem, grid, st);
+    if (R == 4) {
+        if (KT == 1) return verify_fn_of<4, 1, 256, 2>(combine);
+        if (KT == 2) return verify_fn_of<4, 2, 256, 2>(combine);
+        if (KT == 4) return verify_fn_of<4, 4, 256, 2>(combine);
+        if (KT == 8) return verify_fn_of<4, 8, 256, 2>(combine);
+    } else if (R == 8) {
+        if (KT == 1) return verify_fn_of<8, 1, 256, 2>(combine);
+        if (KT == 2) return verify_fn_of<8, 2, 256, 2>(combine);
+        if (KT == 4) return verify_fn_of<8, 4, 256, 2>(combine);
+        if (KT == 8) return verify_fn_of<8, 8, 256, 2>(combine);
+    } else if (R == 16 && threads <= 192) {
+        if (KT == 1) return verify_fn_of<16, 1, 192, 2>(combine);
+        if (KT == 2) return verify_fn_of<16, 2, 192, 2>(combine);
+    } else if (R == 16) {
+        if (KT == 1) return verify_fn_of<16, 1, 512, 1>(combine);
+        if (KT == 2) return verify_fn_of<16, 2, 512, 1>(combine);
     }
-    return BTARD_ERR_UNSUPPORTED;
+    return nullptr;
 }
 
-template <int R>
-int occ_r(int KT, int threads, size_t smem, int* nb)
-{
-    cudaError_t e = cudaErrorInvalidValue;
-    if (KT == 1) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 1, false>, threads, smem);
-    else if (KT == 2) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 2, false>, threads, smem);
-    if constexpr (R <= 8) {
-        if (KT == 4) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 4, false>, threads, smem);
-        else if (KT == 8) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(nb, verify_kernel<R, 8, false>, threads, smem);
-    }
-    return (int)e;
-}
-
-// Dynamic shared memory of the shared-z kernel: z block [2][KT][CL], column sums [2][RG][CL] and, with
-// the combine pass fused in, the moves of v [2][RG][CL], as float4.  At most 80 KB (KT = 8, CL = 256),
+// Dynamic shared memory of the shared-z kernel: z block [3][KT][CL], column sums [2][RG][CL] and, with
+// the combine pass fused in, the moves of v [2][RG][CL], as float4.  At most 112 KB (KT = 8, CL = 256),
 // which is above the 48 KB a kernel gets without opting in: every instantiation opts in once per device.
-constexpr int kVerifyMaxSmem = 96 * 1024;
-
-template <int R, int KT>
-void verify_opt_in()
-{
-    (void)cudaFuncSetAttribute(verify_kernel<R, KT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifyMaxSmem);
-    (void)cudaFuncSetAttribute(verify_kernel<R, KT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifyMaxSmem);
-}
+constexpr int kVerifyMaxSmem = 128 * 1024;
 
 void ensure_verify_attrs()
 {
     static std::atomic<unsigned long long> attrs_set{0};
     if (!device_needs_setup(attrs_set)) return;
-    verify_opt_in<4, 1>(); verify_opt_in<4, 2>(); verify_opt_in<4, 4>(); verify_opt_in<4, 8>();
-    verify_opt_in<8, 1>(); verify_opt_in<8, 2>(); verify_opt_in<8, 4>(); verify_opt_in<8, 8>();
-    verify_opt_in<16, 1>(); verify_opt_in<16, 2>();
+    const int shapes[][3] = {{4, 1, 256}, {4, 2, 256}, {4, 4, 256}, {4, 8, 256}, {8, 1, 256}, {8, 2, 256}, {8, 4, 256},
+                             {8, 8, 256}, {16, 1, 128}, {16, 2, 128}, {16, 1, 512}, {16, 2, 512}};
+    for (const auto& sh : shapes)
+        for (int combine = 0; combine < 2; ++combine)
+            (void)cudaFuncSetAttribute(verify_fn(sh[0], sh[1], combine != 0, sh[2]),
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, kVerifyMaxSmem);
     (void)cudaGetLastError();                          // no device: the sizing falls back to fixed figures
     mark_device_done(attrs_set);
 }
 
-int verify_ctas_per_sm(int R, int KT, int threads, size_t smem)
+int verify_ctas_per_sm(int R, int KT, bool combine, int threads, size_t smem)
 {
     ensure_verify_attrs();                             // the occupancy answer depends on the opt-in
-    int nb = 0, e;
-    if (R == 4) e = occ_r<4>(KT, threads, smem, &nb);
-    else if (R == 8) e = occ_r<8>(KT, threads, smem, &nb);
-    else e = occ_r<16>(KT, threads, smem, &nb);
-    if (e != 0 || nb < 1) { (void)cudaGetLastError(); return 2; }
+    int nb = 0;
+    const void* fn = verify_fn(R, KT, combine, threads);
+    if (!fn || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, threads, smem) != cudaSuccess || nb < 1) {
+        (void)cudaGetLastError();
+        return 2;
+    }
     return nb;
 }
 
@@ -759,8 +810,8 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     g.R = (n <= 16) ? 4 : 8;
     g.RG = (n + g.R - 1) / g.R;
     g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 4) ? 64 : 32;
-    g.threads = g.RG * g.CL;      // n <= 256 with R = 8 gives at most 32 x 32 = 1024
-    if (g.threads > 512) {        // keep CTAs at 512 threads: more rows per thread would be needed
+    g.threads = g.RG * g.CL;
+    if (g.threads > 256) {        // n > 64: 16 rows per thread, one warp-wide column lane per row group
         g.R = 16;
         g.RG = (n + 15) / 16;
         g.CL = 32;
@@ -779,8 +830,8 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     while (kt < K && kt < 8) kt <<= 1;
     if (g.R == 16 && kt > 2) kt = 2;          // 16 rows per thread: keep the accumulators in registers
     vg.KT = kt;
-    const size_t smem = sizeof(float4) * (2 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
-    const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, g.threads, smem);
+    const size_t smem = sizeof(float4) * (3 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
+    const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, false, g.threads, smem);
     g.slots = slots;
     g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, slots);
     vg.slots = n * kt + kt + 1 + n;             // room for the squared norms of the fused combine pass
@@ -791,7 +842,7 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
 {
     const Geometry& g = vg.g;
     VArgs va{a, g.RG, g.CL, g.cpp, vg.slots};
-    const size_t smem = sizeof(float4) * (2 * (size_t)vg.KT * g.CL + (a.combine ? 4 : 2) * (size_t)g.RG * g.CL);
+    const size_t smem = sizeof(float4) * (3 * (size_t)vg.KT * g.CL + (a.combine ? 4 : 2) * (size_t)g.RG * g.CL);
     const int grid = a.P * g.cpp;
     if (smem > (size_t)kVerifyMaxSmem) return BTARD_ERR_UNSUPPORTED;
     ensure_verify_attrs();
@@ -802,11 +853,16 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
             case 8: rc = launch_rows_r<8>(va, vg.KT, grid, st); break;
             default: rc = launch_rows_r<16>(va, vg.KT, grid, st); break;
         }
-    } else
-    switch (g.R) {
-        case 4: rc = launch_r<4>(va, vg.KT, g.threads, smem, grid, st); break;
-        case 8: rc = launch_r<8>(va, vg.KT, g.threads, smem, grid, st); break;
-        default: rc = launch_r<16>(va, vg.KT, g.threads, smem, grid, st); break;
+    } else {
+        const void* fn = verify_fn(g.R, vg.KT, a.combine != 0, g.threads);
+        if (!fn) return BTARD_ERR_UNSUPPORTED;
+        void* args[] = {(void*)&va};
+        prof_begin(KIND_VERIFY, st);
+        const cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)grid), dim3((unsigned)g.threads), args, smem, st);
+        prof_end(KIND_VERIFY, st);
+        BTARD_CUDA_TRY(e);
+        count_launch();
+        rc = BTARD_OK;
     }
     if (rc != BTARD_OK) return rc;
     verify_finalize_kernel<<<a.P, 128, sizeof(double) * vg.slots, st>>>(va, vg.KT);
