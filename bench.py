@@ -322,7 +322,7 @@ def run_ours(args):
     if dist:
         dist.barrier()
 
-    w = workloads.make_workload(cfg, device="cuda")
+    w = workloads.make_workload(cfg, device="cuda", d=args.d)
     if args.max_iters:
         w.max_iters = args.max_iters
     if args.stop:
@@ -569,6 +569,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--algo", default="direct", choices=["direct", "gram", "cooperative"])
     ap.add_argument("--max-iters", type=int, default=None, help="override the configuration's iteration cap")
+    ap.add_argument("--d", type=int, default=None,
+                    help="override the configuration's vector length (smaller cases for profiler captures)")
     ap.add_argument("--stop", default=None, choices=["fixed", "eps"], help="override the configuration's stop rule")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="skip the event-bracketed run that gives the per-kernel breakdown")

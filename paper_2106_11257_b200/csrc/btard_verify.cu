@@ -58,7 +58,6 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     const VerifyLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL, nthr = blockDim.x;
-    const int cl_shift = 31 - __clz(CL);              // CL is a power of two
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
     const long long stride = a.stride, len = a.table[p].len;
     const double tau = a.table[p].tau;
@@ -125,7 +124,7 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
 
     // Projections: with few enough of them the sums are kept per (column pair); otherwise one sum
     // per (row, direction) and the two halves of a pair are added on the way in.
-    constexpr bool PACC = (2 * R * KT + 4 * R + (COMBINE ? 2 * R : 0) <= ((65536 / (MAXT * MINB) >= 160) ? 140 : 72));
+    constexpr bool PACC = (2 * R * KT + 4 * R + (COMBINE ? 2 * R : 0) <= ((65536 / (MAXT * MINB) >= 250) ? 200 : (65536 / (MAXT * MINB) >= 160) ? 140 : 72));
     uint64_t acc2[PACC ? R * KT : 1];
     float acc1[PACC ? 1 : R * KT];
 #pragma unroll
@@ -146,28 +145,32 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     if (j > 0) q0 &= ~7LL;
     if (j + 1 < cpp) q1 &= ~7LL;
     const long long full_quads = len >> 2;             // quads that lie entirely inside the data
-    const float* gp = a.g + (size_t)p * n * stride;
+    const float* xrow0 = a.g + ((size_t)p * n + (size_t)rg * R) * stride;   // this thread's first row
+    const long long stride_bytes = stride * 4;
+    const int nrows = (n - rg * R < R) ? n - rg * R : R;                    // rows of this group that exist
     const float* vp = a.v + (size_t)p * stride;
     float* rsp = a.resid_sum ? a.resid_sum + (size_t)p * stride : nullptr;
     const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
     const uint32_t pg = (uint32_t)(a.p_base + p);
 
-    // The block of z of the tile that starts at quad qb, into buffer `zbuf` (0..2).
+    // The block of z of the tile that starts at quad qb, into buffer `zbuf` (0..2).  A thread draws
+    // the quads of its own column lane: directions rg, rg + RG, ... (the column tests are made once).
     auto gen_z = [&](long long qb, int zbuf) {
-        float4* zb = sh_z + (size_t)zbuf * KT * CL;
-        for (int idx = tid; idx < KT * CL; idx += nthr) {
-            const int kq = idx >> cl_shift, cq = idx & (CL - 1);
-            const long long col = (qb + cq) * 4;
+        float4* zb = sh_z + (size_t)zbuf * KT * CL + cl;
+        const long long quad = qb + cl, col = quad * 4;
+        const bool inside = quad < q1 && col < len;
+        const bool ragged = col + 3 >= len;            // only the last quad of a ragged partition
+        for (int kq = rg; kq < KT; kq += RG) {
             float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kq < a.kc && qb + cq < q1 && col < len) {
-                z = z_quad((uint32_t)(qb + cq), pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
-                if (col + 3 >= len) {                  // only the last quad of a ragged partition
+            if (inside && kq < a.kc) {
+                z = z_quad((uint32_t)quad, pg, (uint32_t)(a.k0 + kq), a.seed_lo, a.seed_hi);
+                if (ragged) {
                     if (col + 1 >= len) z.y = 0.f;
                     if (col + 2 >= len) z.z = 0.f;
                     z.w = 0.f;
                 }
             }
-            zb[kq * CL + cq] = z;
+            zb[kq * CL] = z;
         }
     };
     // Adds up the row groups' column sums of the tile at quad qb (written one tile earlier).
@@ -195,10 +198,15 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
         uint64_t va = 0ull, vb = 0ull;
         if (valid) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int i = rg * R + r;
-                if (i < n) ld_stream_pairs(gp + (size_t)i * stride + col, xa[r], xb[r]);
-                else { xa[r] = 0ull; xb[r] = 0ull; }
+            for (int r = 0; r < R; ++r) { xa[r] = 0ull; xb[r] = 0ull; }
+            const char* xr = reinterpret_cast<const char*>(xrow0 + col);      // row rg R, then one stride per row
+            if (nrows == R) {
+#pragma unroll
+                for (int r = 0; r < R; ++r, xr += stride_bytes) ld_stream_pairs(reinterpret_cast<const float*>(xr), xa[r], xb[r]);
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r, xr += stride_bytes)
+                    if (r < nrows) ld_stream_pairs(reinterpret_cast<const float*>(xr), xa[r], xb[r]);
             }
             const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
             va = pk2(v4.x, v4.y);
@@ -307,12 +315,13 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     };
 
     if (q0 < q1) gen_z(q0, 0);                         // made visible by the first tile's barrier
+    // interior tiles come first: a run without predicates, then the guarded rest
+    long long inner_end = (q1 < full_quads) ? q1 : full_quads;
+    if (any_skip) inner_end = q0;
     int par = 0, zcur = 0;
-    for (long long qb = q0; qb < q1; qb += CL, par ^= 1, zcur = (zcur == 2 ? 0 : zcur + 1)) {
-        const bool inner = !any_skip && qb + CL <= q1 && qb + CL <= full_quads;
-        if (inner) tile(std::false_type{}, qb, par, zcur);
-        else tile(std::true_type{}, qb, par, zcur);
-    }
+    long long qb = q0;
+    for (; qb + CL <= inner_end; qb += CL, par ^= 1, zcur = (zcur == 2 ? 0 : zcur + 1)) tile(std::false_type{}, qb, par, zcur);
+    for (; qb < q1; qb += CL, par ^= 1, zcur = (zcur == 2 ? 0 : zcur + 1)) tile(std::true_type{}, qb, par, zcur);
     __syncthreads();
     if (first_chunk && q1 > q0) consume_sums(q0 + (q1 - q0 - 1) / CL * CL, par ^ 1);
 
@@ -697,8 +706,11 @@ __global__ void random_vector_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_
     *reinterpret_cast<float4*>(z + 4 * q) = v;
 }
 
-// Register budgets: up to 192 threads (16 rows per thread, n <= 64) two CTAs share an SM with 170
-// registers per thread; the 256-thread shapes get 128; shapes of more than 256 threads (n > 64) one CTA.
+// Shapes and register budgets.  Up to 16 peers: 4 rows per thread in CTAs of at most 128 threads, three
+// to an SM (170 registers).  17 to 64 peers: 16 rows per thread in CTAs of 128 or 192 threads; with one
+// or two directions two or three CTAs share an SM (168 registers), with four the accumulators need the
+// whole file (255 registers, two CTAs of 128 threads).  More peers: one warp-wide lane per row group,
+// up to 512 threads.
 template <int R, int KT, int MAXT, int MINB>
 const void* verify_fn_of(bool combine)
 {
@@ -708,18 +720,16 @@ const void* verify_fn_of(bool combine)
 const void* verify_fn(int R, int KT, bool combine, int threads)
 {
     if (R == 4) {
-        if (KT == 1) return verify_fn_of<4, 1, 256, 2>(combine);
-        if (KT == 2) return verify_fn_of<4, 2, 256, 2>(combine);
-        if (KT == 4) return verify_fn_of<4, 4, 256, 2>(combine);
-        if (KT == 8) return verify_fn_of<4, 8, 256, 2>(combine);
-    } else if (R == 8) {
-        if (KT == 1) return verify_fn_of<8, 1, 256, 2>(combine);
-        if (KT == 2) return verify_fn_of<8, 2, 256, 2>(combine);
-        if (KT == 4) return verify_fn_of<8, 4, 256, 2>(combine);
-        if (KT == 8) return verify_fn_of<8, 8, 256, 2>(combine);
+        if (KT == 1) return verify_fn_of<4, 1, 128, 3>(combine);
+        if (KT == 2) return verify_fn_of<4, 2, 128, 3>(combine);
+        if (KT == 4) return verify_fn_of<4, 4, 128, 3>(combine);
+        if (KT == 8) return verify_fn_of<4, 8, 128, 3>(combine);
     } else if (R == 16 && threads <= 192) {
         if (KT == 1) return verify_fn_of<16, 1, 192, 2>(combine);
         if (KT == 2) return verify_fn_of<16, 2, 192, 2>(combine);
+        // four directions: 168 registers hold the plain pass (three CTAs of 128 threads per SM); fused with
+        // the combine pass it needs the whole file (measured: 17.1 ms against 18.0 ms with spills, n = 64, d = 2^28)
+        if (KT == 4) return combine ? (const void*)verify_kernel<16, 4, true, 192, 1> : (const void*)verify_kernel<16, 4, false, 192, 2>;
     } else if (R == 16) {
         if (KT == 1) return verify_fn_of<16, 1, 512, 1>(combine);
         if (KT == 2) return verify_fn_of<16, 2, 512, 1>(combine);
@@ -736,8 +746,8 @@ void ensure_verify_attrs()
 {
     static std::atomic<unsigned long long> attrs_set{0};
     if (!device_needs_setup(attrs_set)) return;
-    const int shapes[][3] = {{4, 1, 256}, {4, 2, 256}, {4, 4, 256}, {4, 8, 256}, {8, 1, 256}, {8, 2, 256}, {8, 4, 256},
-                             {8, 8, 256}, {16, 1, 128}, {16, 2, 128}, {16, 1, 512}, {16, 2, 512}};
+    const int shapes[][3] = {{4, 1, 128}, {4, 2, 128}, {4, 4, 128}, {4, 8, 128}, {16, 1, 128}, {16, 2, 128},
+                             {16, 4, 128}, {16, 1, 512}, {16, 2, 512}};
     for (const auto& sh : shapes)
         for (int combine = 0; combine < 2; ++combine)
             (void)cudaFuncSetAttribute(verify_fn(sh[0], sh[1], combine != 0, sh[2]),
@@ -807,28 +817,22 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
         vg.slots = n * K + K + 1 + n;      // room for the squared norms of the fused combine pass
         return vg;
     }
-    g.R = (n <= 16) ? 4 : 8;
-    g.RG = (n + g.R - 1) / g.R;
-    g.CL = (g.RG == 1) ? 256 : (g.RG == 2) ? 128 : (g.RG <= 4) ? 64 : 32;
-    g.threads = g.RG * g.CL;
-    if (g.threads > 256) {        // n > 64: 16 rows per thread, one warp-wide column lane per row group
-        g.R = 16;
-        g.RG = (n + 15) / 16;
-        g.CL = 32;
-        g.threads = g.RG * g.CL;
-    }
-    if (n > 16 && n <= 64 && K <= 2) {
-        // few directions: the accumulators of 16 rows per thread fit in registers, and fewer row groups
-        // exchange column sums (measured at n = 64, K = 1: 0.725 ms against 0.761 ms with 8 rows per
-        // thread; fused with the combine pass 1.10 ms against 1.23 ms)
-        g.R = 16;
-        g.RG = (n + 15) / 16;
-        g.CL = (g.RG >= 4) ? 32 : 64;
-        g.threads = g.RG * g.CL;
-    }
     int kt = 1;
     while (kt < K && kt < 8) kt <<= 1;
-    if (g.R == 16 && kt > 2) kt = 2;          // 16 rows per thread: keep the accumulators in registers
+    if (n <= 16) {                // more than two directions: 4 rows per thread, CTAs of about 128 threads
+        g.R = 4;
+        g.RG = (n + 3) / 4;
+        g.CL = (g.RG == 1) ? 128 : (g.RG == 2) ? 64 : 32;
+    } else {
+        // 16 rows per thread: few row groups exchange column sums, and the per-tile bookkeeping of a thread
+        // is spread over 64 elements (measured at n = 64: 8 rows per thread ran 2.5 times the instructions)
+        g.R = 16;
+        g.RG = (n + 15) / 16;
+        g.CL = (g.RG == 2 || g.RG == 3) ? 64 : 32;
+        if (kt > 4) kt = 4;                   // the accumulators of 4 directions are all the registers hold
+        if (g.RG > 4 && kt > 2) kt = 2;       // more than 256 threads: 128 registers per thread
+    }
+    g.threads = g.RG * g.CL;
     vg.KT = kt;
     const size_t smem = sizeof(float4) * (3 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
     const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, false, g.threads, smem);
