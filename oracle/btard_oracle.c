@@ -173,24 +173,33 @@ void btard_oracle_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t par
 /* order of their bit patterns (-NaN < -inf < ... < -0 < +0 < ... < +inf <     */
 /* +NaN); for even n the result is the mean of the two middle values.          */
 /* ------------------------------------------------------------------------- */
-static uint32_t order_key(float f)
+static uint64_t order_key64(double d)
 {
-    uint32_t u = f32_as_u32(f);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    uint64_t u; memcpy(&u, &d, 8);
+    return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
 }
-static int cmp_key(const void *a, const void *b)
+static int cmp_key64(const void *a, const void *b)
 {
-    uint32_t x = order_key(*(const float *)a), y = order_key(*(const float *)b);
+    uint64_t x = order_key64(*(const double *)a), y = order_key64(*(const double *)b);
     return (x > y) - (x < y);
 }
-static void coord_median(const float *g, int32_t n, int64_t stride, int64_t len, double *v)
+/* Row i as the aggregation sees it: f_i g_i when per-row factors are given (the per-part clipping of
+   BTARD-Clipped-SGD, Alg. 9, applied on the fly), g_i otherwise.  A factor of exactly 0 drops the row
+   (it reads as zeros whatever it holds); a factor of 1 changes nothing, bit for bit. */
+static double row_value(const float *x, int64_t c, double f)
 {
-    float *col = (float *)malloc(sizeof(float) * (size_t)n);
+    return (f == 0.0) ? 0.0 : f * (double)x[c];
+}
+static double factor_of(const double *row_scale, int32_t i) { return row_scale ? row_scale[i] : 1.0; }
+
+static void coord_median(const float *g, int32_t n, int64_t stride, int64_t len, const double *row_scale, double *v)
+{
+    double *col = (double *)malloc(sizeof(double) * (size_t)n);
     for (int64_t c = 0; c < len; ++c) {
-        for (int32_t i = 0; i < n; ++i) col[i] = g[(int64_t)i * stride + c];
-        qsort(col, (size_t)n, sizeof(float), cmp_key);
-        if (n & 1) v[c] = (double)col[n / 2];
-        else v[c] = ((double)col[n / 2 - 1] + (double)col[n / 2]) / 2.0;
+        for (int32_t i = 0; i < n; ++i) col[i] = row_value(g + (int64_t)i * stride, c, factor_of(row_scale, i));
+        qsort(col, (size_t)n, sizeof(double), cmp_key64);
+        if (n & 1) v[c] = col[n / 2];
+        else v[c] = (col[n / 2 - 1] + col[n / 2]) / 2.0;
     }
     free(col);
 }
@@ -209,11 +218,11 @@ static double clip_weight(double rho, double tau, uint32_t *status)
     return tau / rho;
 }
 
-static double residual_norm(const float *x, const double *v, int64_t len)
+static double residual_norm(const float *x, double f, const double *v, int64_t len)
 {
     double acc = 0.0;
     for (int64_t c = 0; c < len; ++c) {
-        double r = (double)x[c] - v[c];
+        double r = row_value(x, c, f) - v[c];
         acc += r * r;
     }
     return sqrt(acc);
@@ -229,6 +238,12 @@ int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t 
                                int32_t stop_mode, int32_t max_iters, double eps,
                                double *v, double *resid_norm, int32_t *iters,
                                double *last_step_norm, uint32_t *status);
+int btard_oracle_aggregate_one_ex(int32_t rule, const float *g, int32_t n, int64_t stride, int64_t len,
+                                  double tau, const double *tau_sched, const double *row_scale,
+                                  int32_t init_mode, const float *v0,
+                                  int32_t stop_mode, int32_t max_iters, double eps,
+                                  double *v, double *resid_norm, int32_t *iters,
+                                  double *last_step_norm, uint32_t *status);
 
 int btard_oracle_centered_clip_one(const float *g, int32_t n, int64_t stride, int64_t len,
                                    double tau, int32_t init_mode, const float *v0,
@@ -247,12 +262,28 @@ int btard_oracle_centered_clip_one(const float *g, int32_t n, int64_t stride, in
  *   GEOMETRIC_MEDIAN: Weiszfeld, v <- sum_i x_i / rho_i / sum_i 1 / rho_i with rho_i floored at tau,
  *                     written as v += sum_i (1/rho_i) r_i / sum_i (1/rho_i); same stop rules.
  *   MEAN / COORD_MEDIAN: v is the mean / coordinate-wise median of the rows; no update, iters = 0.
+ * Two optional inputs:
+ *   tau_sched [max_iters]: update l uses the radius tau_sched[l] (the schedule tau_l of App. D.2) instead of
+ *     the constant tau;
+ *   row_scale [n]: row i enters as row_scale[i] g_i, the per-part clipped gradient of BTARD-Clipped-SGD
+ *     (Alg. 9: g~_i(l) = min{1, lambda / ||g_i(l)||} g_i(l)) without rewriting g.
  */
 int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t stride, int64_t len,
                                double tau, int32_t init_mode, const float *v0,
                                int32_t stop_mode, int32_t max_iters, double eps,
                                double *v, double *resid_norm, int32_t *iters,
                                double *last_step_norm, uint32_t *status)
+{
+    return btard_oracle_aggregate_one_ex(rule, g, n, stride, len, tau, NULL, NULL, init_mode, v0, stop_mode,
+                                         max_iters, eps, v, resid_norm, iters, last_step_norm, status);
+}
+
+int btard_oracle_aggregate_one_ex(int32_t rule, const float *g, int32_t n, int64_t stride, int64_t len,
+                                  double tau, const double *tau_sched, const double *row_scale,
+                                  int32_t init_mode, const float *v0,
+                                  int32_t stop_mode, int32_t max_iters, double eps,
+                                  double *v, double *resid_norm, int32_t *iters,
+                                  double *last_step_norm, uint32_t *status)
 {
     if (n < 1 || len < 0 || stride < len || max_iters < 1) return -1;
     if (!(tau >= 0.0)) return -1;
@@ -268,11 +299,11 @@ int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t 
     } else if (init_mode == ORACLE_INIT_MEAN) {
         for (int64_t c = 0; c < len; ++c) {
             double acc = 0.0;
-            for (int32_t i = 0; i < n; ++i) acc += (double)g[(int64_t)i * stride + c];
+            for (int32_t i = 0; i < n; ++i) acc += row_value(g + (int64_t)i * stride, c, factor_of(row_scale, i));
             v[c] = acc / n;
         }
     } else if (init_mode == ORACLE_INIT_COORD_MEDIAN) {
-        coord_median(g, n, stride, len, v);
+        coord_median(g, n, stride, len, row_scale, v);
     } else {
         return -1;
     }
@@ -282,10 +313,14 @@ int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t 
     double step = 0.0;
     int32_t done = 0;
     for (int32_t l = 0; l < max_iters; ++l) {
+        if (tau_sched) {                                /* tau_l of App. D.2 */
+            tau = tau_sched[l];
+            if (!(tau >= 0.0)) { free(w); free(u); return -1; }
+        }
         if (rule == ORACLE_RULE_GEOMETRIC_MEDIAN) {
             double total = 0.0;
             for (int32_t i = 0; i < n; ++i) {
-                double rho = residual_norm(g + (int64_t)i * stride, v, len);
+                double rho = residual_norm(g + (int64_t)i * stride, factor_of(row_scale, i), v, len);
                 if (!isfinite(rho)) { st |= ORACLE_STATUS_NONFINITE_ROW; w[i] = 0.0; }
                 else w[i] = 1.0 / (rho > tau ? rho : tau);
                 total += w[i];
@@ -294,13 +329,14 @@ int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t 
             for (int32_t i = 0; i < n; ++i) w[i] = total > 0.0 ? n * w[i] / total : 0.0;
         } else {
             for (int32_t i = 0; i < n; ++i)
-                w[i] = clip_weight(residual_norm(g + (int64_t)i * stride, v, len), tau, &st);
+                w[i] = clip_weight(residual_norm(g + (int64_t)i * stride, factor_of(row_scale, i), v, len), tau, &st);
         }
         for (int64_t c = 0; c < len; ++c) u[c] = 0.0;
         for (int32_t i = 0; i < n; ++i) {
             if (w[i] == 0.0) continue;                  /* weight 0: the row is left out */
             const float *x = g + (int64_t)i * stride;
-            for (int64_t c = 0; c < len; ++c) u[c] += w[i] * ((double)x[c] - v[c]);
+            const double f = factor_of(row_scale, i);
+            for (int64_t c = 0; c < len; ++c) u[c] += w[i] * (row_value(x, c, f) - v[c]);
         }
         double s2 = 0.0;
         for (int64_t c = 0; c < len; ++c) {
@@ -314,7 +350,7 @@ int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t 
     }
     if (stop_mode == ORACLE_STOP_EPS && !(step <= eps)) st |= ORACLE_STATUS_NOT_CONVERGED;
     for (int32_t i = 0; i < n; ++i) {
-        double rho = residual_norm(g + (int64_t)i * stride, v, len);
+        double rho = residual_norm(g + (int64_t)i * stride, factor_of(row_scale, i), v, len);
         if (!isfinite(rho)) st |= ORACLE_STATUS_NONFINITE_ROW;
         resid_norm[i] = rho;
     }
@@ -334,11 +370,29 @@ int btard_oracle_aggregate_one(int32_t rule, const float *g, int32_t n, int64_t 
 /* v is the fp32 vector a peer would have received.  If norm_in is not NULL    */
 /* the weights are taken from those norms (as reported by the aggregation).    */
 /* ------------------------------------------------------------------------- */
+int btard_oracle_verify_one_ex(const float *g, int32_t n, int64_t stride, int64_t len,
+                               const float *v, double tau, const double *row_scale, uint64_t seed, int32_t p, int32_t K,
+                               const double *norm_in, double *norm, double *weight, double *dot,
+                               double *s, double *s_sum, double *znorm2, double *resid_sum_norm,
+                               double *resid_sum /* [len] or NULL */, uint32_t *status);
+
 int btard_oracle_verify_one(const float *g, int32_t n, int64_t stride, int64_t len,
                             const float *v, double tau, uint64_t seed, int32_t p, int32_t K,
                             const double *norm_in, double *norm, double *weight, double *dot,
                             double *s, double *s_sum, double *znorm2, double *resid_sum_norm,
                             double *resid_sum /* [len] or NULL */, uint32_t *status)
+{
+    return btard_oracle_verify_one_ex(g, n, stride, len, v, tau, NULL, seed, p, K, norm_in, norm, weight, dot, s,
+                                      s_sum, znorm2, resid_sum_norm, resid_sum, status);
+}
+
+/* row_scale [n] or NULL: row i enters as row_scale[i] g_i (the clipped gradients of Alg. 9), as in the
+   aggregation. */
+int btard_oracle_verify_one_ex(const float *g, int32_t n, int64_t stride, int64_t len,
+                               const float *v, double tau, const double *row_scale, uint64_t seed, int32_t p, int32_t K,
+                               const double *norm_in, double *norm, double *weight, double *dot,
+                               double *s, double *s_sum, double *znorm2, double *resid_sum_norm,
+                               double *resid_sum /* [len] or NULL */, uint32_t *status)
 {
     if (n < 1 || len < 0 || stride < len || K < 1 || !(tau >= 0.0)) return -1;
     uint32_t st = 0;
@@ -348,7 +402,7 @@ int btard_oracle_verify_one(const float *g, int32_t n, int64_t stride, int64_t l
     for (int64_t c = 0; c < len; ++c) vd[c] = (double)v[c];
 
     for (int32_t i = 0; i < n; ++i) {
-        norm[i] = norm_in ? norm_in[i] : residual_norm(g + (int64_t)i * stride, vd, len);
+        norm[i] = norm_in ? norm_in[i] : residual_norm(g + (int64_t)i * stride, factor_of(row_scale, i), vd, len);
         weight[i] = clip_weight(norm[i], tau, &st);
     }
     for (int32_t k = 0; k < K; ++k) {
@@ -359,8 +413,9 @@ int btard_oracle_verify_one(const float *g, int32_t n, int64_t stride, int64_t l
         s_sum[k] = 0.0;
         for (int32_t i = 0; i < n; ++i) {
             const float *x = g + (int64_t)i * stride;
+            const double f = factor_of(row_scale, i);
             double acc = 0.0;
-            for (int64_t c = 0; c < len; ++c) acc += ((double)x[c] - vd[c]) * (double)z[c];
+            for (int64_t c = 0; c < len; ++c) acc += (row_value(x, c, f) - vd[c]) * (double)z[c];
             dot[(int64_t)i * K + k] = acc;
             /* an empty partition has no coordinates: the inner product is the empty sum, 0 */
             double sik = (weight[i] == 0.0 || zz == 0.0) ? 0.0 : weight[i] * acc / sqrt(zz);
@@ -371,7 +426,8 @@ int btard_oracle_verify_one(const float *g, int32_t n, int64_t stride, int64_t l
     for (int32_t i = 0; i < n; ++i) {
         if (weight[i] == 0.0) continue;
         const float *x = g + (int64_t)i * stride;
-        for (int64_t c = 0; c < len; ++c) rs[c] += weight[i] * ((double)x[c] - vd[c]);
+        const double f = factor_of(row_scale, i);
+        for (int64_t c = 0; c < len; ++c) rs[c] += weight[i] * (row_value(x, c, f) - vd[c]);
     }
     double acc = 0.0;
     for (int64_t c = 0; c < len; ++c) {
@@ -406,6 +462,31 @@ int btard_oracle_aggregate(int32_t rule, const float *g, int32_t n, int32_t P, i
         int rc = btard_oracle_aggregate_one(
             rule, g + (int64_t)p * n * stride, n, stride, part_len[p], tau[p], init_mode,
             v0 ? v0 + (int64_t)p * stride : NULL, stop_mode, max_iters, eps, vp,
+            resid_norm + (int64_t)p * n, iters + p, last_step_norm + p, status + p);
+        if (rc) {
+#pragma omp atomic write
+            rc_all = rc;
+        }
+    }
+    return rc_all;
+}
+
+/* The same with the two optional inputs: tau_sched [P][max_iters] and row_scale [P][n] (either may be NULL). */
+int btard_oracle_aggregate_ex(int32_t rule, const float *g, int32_t n, int32_t P, int64_t stride,
+                              const int64_t *part_len, const double *tau, const double *tau_sched,
+                              const double *row_scale, int32_t init_mode, const float *v0, int32_t stop_mode,
+                              int32_t max_iters, double eps, double *v, double *resid_norm, int32_t *iters,
+                              double *last_step_norm, uint32_t *status)
+{
+    int rc_all = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t p = 0; p < P; ++p) {
+        double *vp = v + (int64_t)p * stride;
+        for (int64_t c = 0; c < stride; ++c) vp[c] = 0.0;
+        int rc = btard_oracle_aggregate_one_ex(
+            rule, g + (int64_t)p * n * stride, n, stride, part_len[p], tau[p],
+            tau_sched ? tau_sched + (int64_t)p * max_iters : NULL, row_scale ? row_scale + (int64_t)p * n : NULL,
+            init_mode, v0 ? v0 + (int64_t)p * stride : NULL, stop_mode, max_iters, eps, vp,
             resid_norm + (int64_t)p * n, iters + p, last_step_norm + p, status + p);
         if (rc) {
 #pragma omp atomic write

@@ -95,9 +95,11 @@ def _per_part(x, P, dtype):
 
 
 def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v0=None, stop_mode=STOP_FIXED,
-                  max_iters=1, eps=0.0, rule=RULE_CENTERED_CLIP):
+                  max_iters=1, eps=0.0, rule=RULE_CENTERED_CLIP, tau_schedule=None, row_scale=None):
     """Batched CenteredClip.  g: [P][n][stride] fp32 (or [n][stride]).
 
+    tau_schedule [P][max_iters]: the radius of update l (tau_l of App. D.2) instead of the constant tau.
+    row_scale [P][n]: row i enters as row_scale[p][i] * g[p][i] (the clipped gradients of Alg. 9).
     Returns dict(v [P][stride] f64, resid_norm [P][n], iters [P], last_step_norm [P], status [P]).
     """
     g = _as_g(g)
@@ -106,14 +108,19 @@ def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v0=None, stop_mode
     tau = _per_part(tau, P, np.float64)
     if v0 is not None:
         v0 = np.ascontiguousarray(v0, dtype=np.float32).reshape(P, stride)
+    if tau_schedule is not None:
+        tau_schedule = np.ascontiguousarray(np.broadcast_to(np.asarray(tau_schedule, np.float64), (P, max_iters)))
+    if row_scale is not None:
+        row_scale = np.ascontiguousarray(np.asarray(row_scale, np.float64).reshape(P, n))
     v = np.zeros((P, stride), dtype=np.float64)
     rn = np.zeros((P, n), dtype=np.float64)
     it = np.zeros(P, dtype=np.int32)
     ls = np.zeros(P, dtype=np.float64)
     st = np.zeros(P, dtype=np.uint32)
-    rc = _load().btard_oracle_aggregate(
+    rc = _load().btard_oracle_aggregate_ex(
         C.c_int32(rule), _p(g, C.c_float), C.c_int32(n), C.c_int32(P), C.c_int64(stride), _p(ln, C.c_int64),
-        _p(tau, C.c_double), C.c_int32(init_mode), _p(v0, C.c_float), C.c_int32(stop_mode),
+        _p(tau, C.c_double), _p(tau_schedule, C.c_double), _p(row_scale, C.c_double),
+        C.c_int32(init_mode), _p(v0, C.c_float), C.c_int32(stop_mode),
         C.c_int32(max_iters), C.c_double(eps), _p(v, C.c_double), _p(rn, C.c_double),
         _p(it, C.c_int32), _p(ls, C.c_double), _p(st, C.c_uint32))
     if rc:
@@ -122,7 +129,7 @@ def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v0=None, stop_mode
 
 
 def verify(g, v, tau, seed, K=1, part_len=None, norm_in=None, want_resid_sum=False,
-           first_partition=0):
+           first_partition=0, row_scale=None):
     """Batched verification metadata.  v: [P][stride] fp32 (the vector a peer received).
 
     ``first_partition`` shifts the partition index that keys the z stream, so that a
@@ -140,7 +147,9 @@ def verify(g, v, tau, seed, K=1, part_len=None, norm_in=None, want_resid_sum=Fal
                resid_sum_norm=np.zeros(P), status=np.zeros(P, dtype=np.uint32))
     rs = np.zeros((P, stride)) if want_resid_sum else None
     lib = _load()
-    if first_partition == 0:
+    if row_scale is not None:
+        row_scale = np.ascontiguousarray(np.asarray(row_scale, np.float64).reshape(P, n))
+    if first_partition == 0 and row_scale is None:
         rc = lib.btard_oracle_verify(
             _p(g, C.c_float), C.c_int32(n), C.c_int32(P), C.c_int64(stride), _p(ln, C.c_int64),
             _p(v, C.c_float), _p(tau, C.c_double), C.c_uint64(int(seed)), C.c_int32(K),
@@ -154,9 +163,10 @@ def verify(g, v, tau, seed, K=1, part_len=None, norm_in=None, want_resid_sum=Fal
         for p in range(P):
             rsn = C.c_double(0.0)
             stt = C.c_uint32(0)
-            rc = lib.btard_oracle_verify_one(
+            rc = lib.btard_oracle_verify_one_ex(
                 _p(g[p], C.c_float), C.c_int32(n), C.c_int64(stride), C.c_int64(int(ln[p])),
-                _p(v[p], C.c_float), C.c_double(float(tau[p])), C.c_uint64(int(seed)),
+                _p(v[p], C.c_float), C.c_double(float(tau[p])),
+                _p(row_scale[p], C.c_double) if row_scale is not None else None, C.c_uint64(int(seed)),
                 C.c_int32(first_partition + p), C.c_int32(K),
                 _p(norm_in[p], C.c_double) if norm_in is not None else None,
                 _p(out["norm"][p], C.c_double), _p(out["weight"][p], C.c_double),

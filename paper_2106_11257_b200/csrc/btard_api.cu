@@ -153,12 +153,16 @@ struct VerifyWorkspace {
     size_t table, part, norms, cslots, ctot, cticket, total;
 };
 
-VerifyWorkspace verify_ws_layout(int n, int P, const VerifyGeometry& vg, const Geometry& cg)
+// One layout serves the plain pass and the pass fused with the combine step: their CTA counts may
+// differ, so the per-CTA slots are sized for the larger of the two.
+VerifyWorkspace verify_ws_layout(int n, int P, long long stride, int K, const Geometry& cg)
 {
+    const VerifyGeometry plain = verify_geometry(n, P, stride, K, false), fused = verify_geometry(n, P, stride, K, true);
+    const size_t ctas = (size_t)(plain.g.cpp > fused.g.cpp ? plain.g.cpp : fused.g.cpp);
     VerifyWorkspace w;
     size_t off = 0;
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
-    w.part = off; off = align_up(off + sizeof(double) * (size_t)P * vg.g.cpp * vg.slots, 256);
+    w.part = off; off = align_up(off + sizeof(double) * (size_t)P * ctas * plain.slots, 256);
     w.norms = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
     w.cslots = off; off = align_up(off + sizeof(double) * (size_t)P * cg.cpp * (n + 1), 256);
     w.ctot = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);
@@ -427,9 +431,8 @@ size_t btard_verify_projections_workspace(const btard_verify_args* a)
     if (!a || a->n_peers < 1 || a->n_peers > BTARD_MAX_PEERS || a->n_partitions < 1 ||
         a->row_stride < 4 || a->n_z < 1)
         return 0;
-    const VerifyGeometry vg = verify_geometry(a->n_peers, a->n_partitions, a->row_stride, a->n_z);
     const Geometry cg = cclip_geometry(a->n_peers, a->n_partitions, a->row_stride);
-    return verify_ws_layout(a->n_peers, a->n_partitions, vg, cg).total;
+    return verify_ws_layout(a->n_peers, a->n_partitions, a->row_stride, a->n_z, cg).total;
 }
 
 static int check_verify_args(const btard_verify_args* a)
@@ -453,9 +456,9 @@ static int launch_fused_verify(const btard_cclip_args* c, const btard_verify_arg
                                const unsigned int* gram_error, cudaStream_t st)
 {
     const int n = c->n_peers, P = c->n_partitions, K = a->n_z;
-    const VerifyGeometry vg = verify_geometry(n, P, c->row_stride, K);
+    const VerifyGeometry vg = verify_geometry(n, P, c->row_stride, K, true);
     const Geometry cg = cclip_geometry(n, P, c->row_stride);
-    const VerifyWorkspace ws = verify_ws_layout(n, P, vg, cg);
+    const VerifyWorkspace ws = verify_ws_layout(n, P, c->row_stride, K, cg);
     if (a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
     char* base = (char*)a->workspace;
     VerifyLaunch V{};
@@ -493,9 +496,8 @@ int btard_centered_clip_verify(const btard_cclip_args* c, const btard_verify_arg
     int rc = check_verify_args(&vv);
     if (rc != BTARD_OK) return rc;
     if (fusable(c, &vv)) {
-        const VerifyGeometry vg = verify_geometry(c->n_peers, c->n_partitions, c->row_stride, vv.n_z);
         const Geometry cg = cclip_geometry(c->n_peers, c->n_partitions, c->row_stride);
-        if (vv.workspace_bytes < verify_ws_layout(c->n_peers, c->n_partitions, vg, cg).total)
+        if (vv.workspace_bytes < verify_ws_layout(c->n_peers, c->n_partitions, c->row_stride, vv.n_z, cg).total)
             return BTARD_ERR_WORKSPACE_TOO_SMALL;   // before anything is queued
         return cclip_run(c, &vv);
     }
@@ -512,7 +514,7 @@ int btard_verify_projections(const btard_verify_args* a)
     const int n = a->n_peers, P = a->n_partitions, K = a->n_z;
     const VerifyGeometry vg = verify_geometry(n, P, a->row_stride, K);
     const Geometry cg = cclip_geometry(n, P, a->row_stride);
-    const VerifyWorkspace ws = verify_ws_layout(n, P, vg, cg);
+    const VerifyWorkspace ws = verify_ws_layout(n, P, a->row_stride, K, cg);
     if (a->workspace_bytes < ws.total) return BTARD_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)a->stream;
     char* base = (char*)a->workspace;

@@ -200,7 +200,8 @@ struct VerifyGeometry {
     int own_z;   // n <= 16 and K <= 2: each thread draws the z of its own columns (verify_rows_kernel)
 };
 
-VerifyGeometry verify_geometry(int n, int P, long long stride, int K);
+// fused: the pass also carries the combine step of the Gram variant (its kernel may hold fewer CTAs per SM)
+VerifyGeometry verify_geometry(int n, int P, long long stride, int K, bool fused = false);
 int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t st);
 int launch_checks(const btard_checks_args& a, cudaStream_t st);
 int launch_random_vector(uint64_t seed, int p, int k, long long len, float* z, cudaStream_t st);

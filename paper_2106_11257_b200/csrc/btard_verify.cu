@@ -801,7 +801,7 @@ int rows_ctas_per_sm(int R, int KT)
 
 }  // namespace
 
-VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
+VerifyGeometry verify_geometry(int n, int P, long long stride, int K, bool fused)
 {
     VerifyGeometry vg;
     Geometry& g = vg.g;
@@ -835,7 +835,8 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K)
     g.threads = g.RG * g.CL;
     vg.KT = kt;
     const size_t smem = sizeof(float4) * (3 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
-    const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, false, g.threads, smem);
+    const size_t smem_fused = smem + sizeof(float4) * 2 * (size_t)g.RG * g.CL;
+    const int slots = sm_count() * verify_ctas_per_sm(g.R, kt, fused, g.threads, fused ? smem_fused : smem);
     g.slots = slots;
     g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, slots);
     vg.slots = n * kt + kt + 1 + n;             // room for the squared norms of the fused combine pass

@@ -630,3 +630,89 @@ def test_commitment_is_the_stated_tree_of_sha256():
     z = x.copy(); z[1, 2, 1023:] = 7.0
     assert not np.array_equal(oracle.commitment(y, lens)[1, 2], out[1, 2])
     assert np.array_equal(oracle.commitment(z, lens), out)
+
+
+# ----------------------------------------------------------------------------- tau_l schedule, clipped rows
+def test_constant_schedule_and_unit_factors_change_nothing():
+    """A schedule that repeats tau and factors of 1 must reproduce the plain call bit for bit."""
+    rng = np.random.default_rng(31)
+    x = np.stack([rand_rows(rng, 7, 50), rand_rows(rng, 7, 50, 4.0)])
+    x[0, 1, 3] = np.inf
+    tau = np.array([0.7, 2.0])
+    for init in (oracle.INIT_ZERO, oracle.INIT_MEAN, oracle.INIT_COORD_MEDIAN):
+        a = oracle.centered_clip(x, tau, init_mode=init, max_iters=6)
+        b = oracle.centered_clip(x, tau, init_mode=init, max_iters=6, tau_schedule=np.repeat(tau[:, None], 6, 1),
+                                 row_scale=np.ones((2, 7)))
+        for k in ("v", "resid_norm", "last_step_norm", "iters", "status"):
+            assert np.array_equal(a[k], b[k], equal_nan=True), k
+    v32 = a["v"].astype(np.float32)
+    p = oracle.verify(x[1:], v32[1:], 2.0, 5, K=2)
+    q = oracle.verify(x[1:], v32[1:], 2.0, 5, K=2, row_scale=np.ones((1, 7)))
+    for k in ("norm", "weight", "dot", "s", "s_sum", "resid_sum_norm"):
+        assert np.array_equal(p[k], q[k]), k
+
+
+def test_schedule_walks_a_single_row_by_tau_l():
+    """n = 1, row at distance 10: while it is farther than tau_l, update l moves v by exactly tau_l toward it
+    (App. D.2 with the schedule tau_l)."""
+    x = np.zeros((1, 4), dtype=np.float32)
+    x[0, 2] = 10.0
+    sched = np.array([1.0, 2.5, 0.25, 3.0])
+    for iters in range(1, 5):
+        r = oracle.centered_clip(x, 99.0, init_mode=oracle.INIT_ZERO, max_iters=iters, tau_schedule=sched[:iters])
+        assert abs(r["v"][0, 2] - sched[:iters].sum()) < 1e-13
+        assert abs(r["last_step_norm"][0] - sched[iters - 1]) < 1e-13
+    # and a radius that covers the rest lands on the row
+    r = oracle.centered_clip(x, 0.0, init_mode=oracle.INIT_ZERO, max_iters=3, tau_schedule=[1.0, 2.0, 50.0])
+    assert r["v"][0, 2] == 10.0
+
+
+def test_two_value_schedule_by_hand():
+    """Three collinear points and two updates with different radii, worked out by hand:
+    x = -1, 0, 5 on a line, v0 = 0.  Update 0 with tau = 2: residuals -1, 0, 5 -> weights 1, 1, 2/5 -> step
+    (-1 + 0 + 2)/3 = 1/3.  Update 1 with tau = 1/2: residuals -4/3, -1/3, 14/3 -> clipped to -1/2, -1/3, 1/2
+    -> step (-1/3)/3 = -1/9.  v = 1/3 - 1/9 = 2/9."""
+    x = np.zeros((3, 2), dtype=np.float32)
+    x[:, 0] = [-1.0, 0.0, 5.0]
+    r = oracle.centered_clip(x, 7.0, init_mode=oracle.INIT_ZERO, max_iters=2, tau_schedule=[2.0, 0.5])
+    assert abs(r["v"][0, 0] - 2.0 / 9.0) < 1e-15 and r["v"][0, 1] == 0.0
+
+
+def test_row_factors_equal_rescaled_rows():
+    """Factors that are powers of two rescale fp32 rows exactly, so aggregating (f_i, g_i) must equal
+    aggregating the rows f_i g_i written out, bit for bit; a factor of 0 reads the row as zeros even if it
+    holds an inf."""
+    rng = np.random.default_rng(32)
+    x = rand_rows(rng, 6, 41, 3.0)
+    f = np.array([1.0, 0.5, 0.25, 2.0, 0.0, 1.0])
+    y = (x.astype(np.float64) * f[:, None]).astype(np.float32)
+    x[4, 7] = np.inf                                               # dropped by its factor of 0
+    for init in (oracle.INIT_MEAN, oracle.INIT_COORD_MEDIAN):
+        a = oracle.centered_clip(x, 0.8, init_mode=init, max_iters=5, row_scale=f)
+        b = oracle.centered_clip(y, 0.8, init_mode=init, max_iters=5)
+        for k in ("v", "resid_norm", "last_step_norm", "status"):
+            assert np.array_equal(a[k], b[k]), k
+    v32 = a["v"].astype(np.float32)
+    p = oracle.verify(x, v32, 0.8, 11, K=3, row_scale=f, want_resid_sum=True)
+    q = oracle.verify(y, v32, 0.8, 11, K=3, want_resid_sum=True)
+    for k in ("norm", "weight", "dot", "s", "s_sum", "resid_sum", "resid_sum_norm"):
+        assert np.array_equal(p[k], q[k]), k
+
+
+def test_clipped_sgd_aggregation_is_clip_then_aggregate():
+    """Alg. 9: peers clip their parts to lambda, then ButterflyClip aggregates them.  One update from v = 0,
+    restated with numpy on the clipped rows, against the oracle fed with the clip factors."""
+    rng = np.random.default_rng(33)
+    x = rand_rows(rng, 8, 60, 0.2)
+    x[::3] *= 40.0
+    lam, tau = 1.5, 0.9
+    pc = oracle.preclip(x, lam)
+    assert (pc["factor"] < 1).any() and (pc["factor"] == 1).any()
+    gt = pc["g"][0]                                                # clipped rows, float64
+    assert np.all(np.linalg.norm(gt, axis=1) <= lam * (1 + 1e-12))
+    rho = np.linalg.norm(gt, axis=1)
+    w = np.where(rho <= tau, 1.0, tau / rho)
+    v1 = (w[:, None] * gt).sum(0) / 8
+    r = oracle.centered_clip(x, tau, init_mode=oracle.INIT_ZERO, max_iters=1, row_scale=pc["factor"])
+    assert np.allclose(r["v"][0], v1, rtol=0, atol=1e-15)
+    assert np.allclose(r["resid_norm"][0], np.linalg.norm(gt - v1, axis=1), rtol=1e-13)
