@@ -149,6 +149,13 @@ typedef struct {
     size_t workspace_bytes;
     void* stream;                /* cudaStream_t                                                    */
     int32_t rule;                /* BTARD_RULE_*; 0 = CenteredClip                                  */
+    const double* tau_schedule;  /* device [P][max_iters] or NULL: update l of partition p uses the radius
+                                    tau_schedule[p][l] (the schedule tau_l of App. D.2) instead of tau[p];
+                                    entries must be >= 0 (not checked: they live on the device)         */
+    const double* row_scale;     /* device [P][n] or NULL: row i of slab p enters as row_scale[p][i] g[p][i][:],
+                                    e.g. the factors of btard_preclip_factors (Alg. 9) - the clipped
+                                    gradients are aggregated without rewriting g.  A factor of exactly 0
+                                    makes the row read as zeros.  DIRECT and GRAM algorithms              */
 } btard_cclip_args;
 
 /* Bytes of workspace btard_centered_clip needs for these arguments (0 on invalid arguments).
@@ -189,6 +196,7 @@ typedef struct {
     void* workspace;
     size_t workspace_bytes;
     void* stream;
+    const double* row_scale;     /* device [P][n] or NULL: as in btard_cclip_args                   */
 } btard_verify_args;
 
 BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* args);
@@ -198,7 +206,7 @@ BTARD_API int btard_verify_projections(const btard_verify_args* args);
  * Aggregation and verification of Alg. 2 line 5 and Alg. 6 lines 6-14 in one call: the same results as
  * btard_centered_clip(clip) followed by btard_verify_projections(verify) on the aggregate it returned.
  * `verify` supplies the seed, n_z, partition_base, its outputs and its own workspace; its g, v, part_len,
- * tau, resid_norm_in and stream are taken from `clip` (what it holds there is ignored), and its n_peers,
+ * tau, row_scale, resid_norm_in and stream are taken from `clip` (what it holds there is ignored), and its n_peers,
  * n_partitions and row_stride must equal clip's.  Both workspaces are sized by the two *_workspace()
  * queries as for the separate calls.
  * What the one call buys: with BTARD_ALGO_GRAM the pass that forms v from the coefficients and the
@@ -211,11 +219,14 @@ BTARD_API int btard_centered_clip_verify(const btard_cclip_args* clip, const bta
 /*
  * Per-part gradient clipping of BTARD-Clipped-SGD (Alg. 9 and the paragraph after it):
  *     g~_i(l) = min{1, lambda / ||g_i(l)||_2} g_i(l)
- * applied IN PLACE to g [P][n][row_stride] (row i of slab l is g_i(l)) before it is aggregated.
+ * Two forms.  btard_preclip_factors reads g once and returns row_norm [P][n] = ||g_i(l)||_2 and
+ * factor [P][n] = the multiplier min{1, lambda / ||g_i(l)||} (1 for a row inside the radius; 0 for a row
+ * with a non-finite norm, flagged in status); g is not modified.  Handing `factor` to btard_centered_clip /
+ * btard_verify_projections as `row_scale` aggregates the clipped gradients: one extra pass over g for a
+ * Clipped-SGD aggregation.  btard_preclip does the same and then rescales the clipped rows IN PLACE (a row
+ * with a non-finite norm is set to zero): a second pass, for callers that want g~ itself.
  * lambda: host [P] (the paper uses one lambda_k per step; per-part values are allowed), >= 0, +inf = no
- * clipping.  Outputs: row_norm [P][n] = ||g_i(l)||_2 before clipping, factor [P][n] = the multiplier
- * applied (1 when the row is left untouched; 0 for a row with a non-finite norm, which is set to zero
- * and flagged in status).  Two passes over g (norms, then rescaling of the clipped rows only).
+ * clipping.
  */
 typedef struct {
     int32_t n_peers, n_partitions;
@@ -232,6 +243,7 @@ typedef struct {
 } btard_preclip_args;
 BTARD_API size_t btard_preclip_workspace(const btard_preclip_args* args);
 BTARD_API int btard_preclip(const btard_preclip_args* args);
+BTARD_API int btard_preclip_factors(const btard_preclip_args* args);   /* same arguments and workspace; g is read only */
 
 /*
  * The predicates of Verifications 1-3 (Alg. 6 lines 17-38) on the scalars peers broadcast.  For

@@ -24,6 +24,7 @@ EXPORTS = [
     "btard_verify_projections_static", "btard_verification_checks", "btard_preclip_workspace",
     "btard_preclip", "btard_split_gradients", "btard_merge_partitions",
     "btard_hash_partitions_workspace", "btard_hash_partitions", "btard_centered_clip_verify",
+    "btard_preclip_factors",
 ]
 
 _ERRORS = {-1: "invalid argument", -2: "bad alignment", -3: "workspace too small",
@@ -46,7 +47,8 @@ class CclipArgs(C.Structure):
                 ("max_iters", C.c_int32), ("eps", C.c_double), ("v", C.c_void_p),
                 ("iters", C.c_void_p), ("last_step_norm", C.c_void_p), ("resid_norm", C.c_void_p),
                 ("status", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("stream", C.c_void_p), ("rule", C.c_int32)]
+                ("stream", C.c_void_p), ("rule", C.c_int32), ("tau_schedule", C.c_void_p),
+                ("row_scale", C.c_void_p)]
 
 
 class VerifyArgs(C.Structure):
@@ -57,7 +59,7 @@ class VerifyArgs(C.Structure):
                 ("dot", C.c_void_p), ("s", C.c_void_p), ("s_sum", C.c_void_p),
                 ("znorm2", C.c_void_p), ("resid_sum_norm", C.c_void_p), ("resid_sum", C.c_void_p),
                 ("status", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("stream", C.c_void_p)]
+                ("stream", C.c_void_p), ("row_scale", C.c_void_p)]
 
 
 class HostArgs(C.Structure):
@@ -124,6 +126,8 @@ def lib():
         L.btard_preclip_workspace.argtypes = [C.POINTER(PreclipArgs)]
         L.btard_preclip.restype = C.c_int
         L.btard_preclip.argtypes = [C.POINTER(PreclipArgs)]
+        L.btard_preclip_factors.restype = C.c_int
+        L.btard_preclip_factors.argtypes = [C.POINTER(PreclipArgs)]
         L.btard_verification_checks.restype = C.c_int
         L.btard_verification_checks.argtypes = [C.POINTER(ChecksArgs)]
         L.btard_random_vector.restype = C.c_int
@@ -198,6 +202,15 @@ def _host_arr(x, P, dtype):
     return np.ascontiguousarray(np.broadcast_to(np.asarray(x, dtype=dtype), (P,)))
 
 
+def _dev_f64(t, shape):
+    """Optional device float64 tensor of the given shape -> pointer (None stays None)."""
+    if t is None:
+        return None
+    torch = _torch()
+    assert t.is_cuda and t.dtype == torch.float64 and t.is_contiguous() and tuple(t.shape) == tuple(shape), shape
+    return t.data_ptr()
+
+
 def centered_clip_workspace(n, P, row_stride, stop_mode=STOP_EPS, algo=ALGO_DIRECT):
     a = CclipArgs(n_peers=n, n_partitions=P, row_stride=row_stride, stop_mode=stop_mode, algo=algo)
     return int(lib().btard_centered_clip_workspace(C.byref(a)))
@@ -205,9 +218,10 @@ def centered_clip_workspace(n, P, row_stride, stop_mode=STOP_EPS, algo=ALGO_DIRE
 
 def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v=None, stop_mode=STOP_FIXED_ITERS,
                   max_iters=1, eps=0.0, algo=ALGO_DIRECT, workspace=None, out=None, stream=None,
-                  rule=RULE_CENTERED_CLIP):
+                  rule=RULE_CENTERED_CLIP, tau_schedule=None, row_scale=None):
     """g: CUDA float32 [P][n][row_stride].  Returns dict of CUDA tensors
-    (v, iters, last_step_norm, resid_norm, status).  Asynchronous on the current stream."""
+    (v, iters, last_step_norm, resid_norm, status).  Asynchronous on the current stream.
+    tau_schedule: CUDA float64 [P][max_iters] or None; row_scale: CUDA float64 [P][n] or None."""
     torch = _torch()
     assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
     P, n, stride = g.shape
@@ -232,7 +246,8 @@ def centered_clip(g, tau, part_len=None, init_mode=INIT_ZERO, v=None, stop_mode=
                   iters=o["iters"].data_ptr(), last_step_norm=o["last_step_norm"].data_ptr(),
                   resid_norm=o["resid_norm"].data_ptr(), status=o["status"].data_ptr(),
                   workspace=workspace.data_ptr(), workspace_bytes=workspace.numel(),
-                  stream=_stream_ptr(stream), rule=rule)
+                  stream=_stream_ptr(stream), rule=rule,
+                  tau_schedule=_dev_f64(tau_schedule, (P, max_iters)), row_scale=_dev_f64(row_scale, (P, n)))
     with torch.cuda.device(dev):
         _check(lib().btard_centered_clip(C.byref(a)), "btard_centered_clip")
     res = dict(o)
@@ -247,7 +262,7 @@ def verify_projections_workspace(n, P, row_stride, K):
 
 
 def verify_projections(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None, partition_base=0,
-                       want_resid_sum=False, workspace=None, out=None, stream=None):
+                       want_resid_sum=False, workspace=None, out=None, stream=None, row_scale=None):
     """Returns dict of CUDA tensors: norm, weight [P][n]; dot, s [P][n][K]; s_sum, znorm2 [P][K];
     resid_sum_norm [P]; status [P]; resid_sum [P][row_stride] if asked."""
     torch = _torch()
@@ -282,7 +297,7 @@ def verify_projections(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None, 
                    resid_sum_norm=o["resid_sum_norm"].data_ptr(),
                    resid_sum=rs.data_ptr() if rs is not None else None, status=o["status"].data_ptr(),
                    workspace=workspace.data_ptr(), workspace_bytes=workspace.numel(),
-                   stream=_stream_ptr(stream))
+                   stream=_stream_ptr(stream), row_scale=_dev_f64(row_scale, (P, n)))
     with torch.cuda.device(dev):
         _check(lib().btard_verify_projections(C.byref(a)), "btard_verify_projections")
     res = dict(o)
@@ -294,7 +309,8 @@ def verify_projections(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None, 
 
 def centered_clip_verify(g, tau, seed, K=1, part_len=None, init_mode=INIT_ZERO, v=None,
                          stop_mode=STOP_FIXED_ITERS, max_iters=1, eps=0.0, algo=ALGO_DIRECT, partition_base=0,
-                         want_resid_sum=False, workspaces=None, out=None, stream=None):
+                         want_resid_sum=False, workspaces=None, out=None, stream=None, tau_schedule=None,
+                         row_scale=None):
     """btard_centered_clip_verify: aggregation and verification in one call.  Returns (clip, verify), the
     dicts that centered_clip and verify_projections return.  workspaces / out: optional pairs to reuse."""
     torch = _torch()
@@ -333,7 +349,8 @@ def centered_clip_verify(g, tau, seed, K=1, part_len=None, init_mode=INIT_ZERO, 
                    iters=oc["iters"].data_ptr(), last_step_norm=oc["last_step_norm"].data_ptr(),
                    resid_norm=oc["resid_norm"].data_ptr(), status=oc["status"].data_ptr(),
                    workspace=wc.data_ptr(), workspace_bytes=wc.numel(), stream=_stream_ptr(stream),
-                   rule=RULE_CENTERED_CLIP)
+                   rule=RULE_CENTERED_CLIP, tau_schedule=_dev_f64(tau_schedule, (P, max_iters)),
+                   row_scale=_dev_f64(row_scale, (P, n)))
     va = VerifyArgs(n_peers=n, n_partitions=P, row_stride=stride, seed=int(seed), n_z=K,
                     partition_base=partition_base,
                     norm=ov["norm"].data_ptr(), weight=ov["weight"].data_ptr(), dot=ov["dot"].data_ptr(),
@@ -353,7 +370,7 @@ def centered_clip_verify(g, tau, seed, K=1, part_len=None, init_mode=INIT_ZERO, 
 
 
 def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in=None,
-                              partition_base=0, want_resid_sum=False, out=None, stream=None):
+                              partition_base=0, want_resid_sum=False, out=None, stream=None, row_scale=None):
     """verify_projections for callers that cannot allocate device memory: the library's built-in
     scratch array is used instead of a workspace.  Pass `out` (pre-made output tensors, same keys as
     verify_projections returns) to keep this wrapper from allocating too; calls on one GPU must not
@@ -382,7 +399,8 @@ def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in
                    s=o["s"].data_ptr(), s_sum=o["s_sum"].data_ptr(), znorm2=o["znorm2"].data_ptr(),
                    resid_sum_norm=o["resid_sum_norm"].data_ptr(),
                    resid_sum=rs.data_ptr() if rs is not None else None, status=o["status"].data_ptr(),
-                   workspace=None, workspace_bytes=0, stream=_stream_ptr(stream))
+                   workspace=None, workspace_bytes=0, stream=_stream_ptr(stream),
+                   row_scale=_dev_f64(row_scale, (P, n)))
     with torch.cuda.device(dev):
         _check(lib().btard_verify_projections_static(C.byref(a)), "btard_verify_projections_static")
     res = dict(o)
@@ -453,9 +471,11 @@ def hash_partitions(x, part_len=None, stream=None):
     return out
 
 
-def preclip(g, lam, part_len=None, stream=None):
-    """In-place per-part clipping g_i(l) <- min{1, lam/||g_i(l)||} g_i(l) of a CUDA float32 tensor
-    [P][n][row_stride].  Returns dict(row_norm, factor [P][n] float64, status [P])."""
+def preclip(g, lam, part_len=None, stream=None, in_place=True):
+    """Per-part clipping g_i(l) <- min{1, lam/||g_i(l)||} g_i(l) of a CUDA float32 tensor
+    [P][n][row_stride]: in place, or (in_place=False, btard_preclip_factors) only the norms and the
+    factors, to be handed to centered_clip / verify_projections as row_scale.
+    Returns dict(row_norm, factor [P][n] float64, status [P])."""
     torch = _torch()
     assert g.is_cuda and g.dtype == torch.float32 and g.dim() == 3 and g.is_contiguous()
     P, n, stride = g.shape
@@ -473,7 +493,10 @@ def preclip(g, lam, part_len=None, stream=None):
     a.workspace = ws.data_ptr()
     a.workspace_bytes = ws.numel()
     with torch.cuda.device(dev):
-        _check(lib().btard_preclip(C.byref(a)), "btard_preclip")
+        if in_place:
+            _check(lib().btard_preclip(C.byref(a)), "btard_preclip")
+        else:
+            _check(lib().btard_preclip_factors(C.byref(a)), "btard_preclip_factors")
     o["workspace"] = ws
     return o
 

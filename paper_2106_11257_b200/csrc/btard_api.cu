@@ -314,6 +314,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     if (a->algo == BTARD_ALGO_GRAM && a->n_peers > kMaxGramPeers) return BTARD_ERR_UNSUPPORTED;
     if (a->rule < BTARD_RULE_CENTERED_CLIP || a->rule > BTARD_RULE_COORD_MEDIAN) return BTARD_ERR_INVALID_ARG;
     if (a->rule != BTARD_RULE_CENTERED_CLIP && a->algo == BTARD_ALGO_GRAM) return BTARD_ERR_UNSUPPORTED;
+    if (a->row_scale && a->algo == BTARD_ALGO_DIRECT_COOPERATIVE) return BTARD_ERR_UNSUPPORTED;
     if (a->rule == BTARD_RULE_GEOMETRIC_MEDIAN)
         for (int p = 0; p < a->n_partitions; ++p)
             if (!(a->tau[p] > 0.0) || std::isinf(a->tau[p])) return BTARD_ERR_INVALID_ARG;
@@ -338,6 +339,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     L.stride = a->row_stride; L.n = n; L.P = P;
     L.stop_mode = a->stop_mode; L.max_iters = a->max_iters; L.eps2 = a->eps * a->eps;
     L.rule = a->rule;
+    L.tau_sched = a->tau_schedule; L.row_scale = a->row_scale;
     double* tot[2] = {(double*)(base + ws.tot[0]), (double*)(base + ws.tot[1])};
 
     rc = upload_table((PartEntry*)(base + ws.table), P, a->part_len, a->tau, st);
@@ -353,7 +355,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     if (a->rule == BTARD_RULE_MEAN || a->rule == BTARD_RULE_COORD_MEDIAN) {
         L.init_mode = BTARD_INIT_MEAN;
         if (a->rule == BTARD_RULE_COORD_MEDIAN) {
-            rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
+            rc = launch_median_init(a->g, a->v, L.table, a->row_scale, a->row_stride, n, P, st);
             if (rc != BTARD_OK) return rc;
             L.init_mode = BTARD_INIT_CALLER_V0;
         }
@@ -368,7 +370,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     const bool whole = (a->algo == BTARD_ALGO_DIRECT_COOPERATIVE) && cooperative_launch_supported();
     L.init_mode = a->init_mode;
     if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
-        rc = launch_median_init(a->g, a->v, L.table, a->row_stride, n, P, st);
+        rc = launch_median_init(a->g, a->v, L.table, a->row_scale, a->row_stride, n, P, st);
         if (rc != BTARD_OK) return rc;
         L.init_mode = BTARD_INIT_CALLER_V0;
     }
@@ -390,6 +392,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
         G.iters = a->iters; G.last_step = a->last_step_norm; G.status = a->status;
         G.stride = a->row_stride; G.n = n; G.P = P;
         G.stop_mode = a->stop_mode; G.max_iters = a->max_iters; G.eps2 = a->eps * a->eps;
+        G.tau_sched = a->tau_schedule; G.row_scale = a->row_scale;
         rc = launch_gram(G, gg, st);
         if (rc != BTARD_OK) return rc;
         rc = launch_gram_iterate(G, gg, st);
@@ -471,6 +474,7 @@ static int launch_fused_verify(const btard_cclip_args* c, const btard_verify_arg
     V.seed_lo = (uint32_t)a->seed; V.seed_hi = (uint32_t)(a->seed >> 32);
     V.coef = coef; V.gram = gram; V.gram_entries = gg.entries; V.gram_nb = gg.NB;
     V.resid_norm_out = c->resid_norm; V.cclip_status = c->status; V.gram_error = gram_error;
+    V.row_scale = c->row_scale;
     // The first group of directions carries the combine; further groups (K beyond what one launch
     // holds) are plain verification launches on the v and the norms the first one left.
     for (int k0 = 0; k0 < K; k0 += vg.KT) {
@@ -491,7 +495,7 @@ int btard_centered_clip_verify(const btard_cclip_args* c, const btard_verify_arg
         return BTARD_ERR_INVALID_ARG;
     // the verification reads what the aggregation produced, on the same stream
     btard_verify_args vv = *v;
-    vv.g = c->g; vv.v = c->v; vv.part_len = c->part_len; vv.tau = c->tau;
+    vv.g = c->g; vv.v = c->v; vv.part_len = c->part_len; vv.tau = c->tau; vv.row_scale = c->row_scale;
     vv.resid_norm_in = c->resid_norm; vv.stream = c->stream;
     int rc = check_verify_args(&vv);
     if (rc != BTARD_OK) return rc;
@@ -530,7 +534,7 @@ int btard_verify_projections(const btard_verify_args* a)
         L.tot_out = (double*)(base + ws.ctot);
         L.ticket = (unsigned int*)(base + ws.cticket);
         BTARD_CUDA_TRY(cudaMemsetAsync(L.ticket, 0, sizeof(unsigned int) * (size_t)P, st));
-        L.stride = a->row_stride; L.n = n; L.P = P;
+        L.stride = a->row_stride; L.n = n; L.P = P; L.row_scale = a->row_scale;
         rc = launch_cclip_pass(L, cg, PASS_NORMS, st);
         if (rc != BTARD_OK) return rc;
         rc = launch_totals_to_norms(L.tot_out, (double*)(base + ws.norms), n, P, st);
@@ -546,6 +550,7 @@ int btard_verify_projections(const btard_verify_args* a)
     V.znorm2 = a->znorm2; V.resid_sum_norm = a->resid_sum_norm; V.status = a->status;
     V.stride = a->row_stride; V.n = n; V.P = P; V.K = K; V.p_base = a->partition_base;
     V.seed_lo = (uint32_t)a->seed; V.seed_hi = (uint32_t)(a->seed >> 32);
+    V.row_scale = a->row_scale;
     for (int k0 = 0; k0 < K; k0 += vg.KT) {
         V.k0 = k0;
         V.kc = (K - k0 < vg.KT) ? K - k0 : vg.KT;
@@ -623,7 +628,7 @@ size_t btard_preclip_workspace(const btard_preclip_args* a)
            align_up(sizeof(double) * (size_t)a->n_peers * a->n_partitions * chunks, 256);
 }
 
-int btard_preclip(const btard_preclip_args* a)
+static int preclip_run(const btard_preclip_args* a, bool rewrite)
 {
     if (!a) return BTARD_ERR_INVALID_ARG;
     int rc = check_common(a->n_peers, a->n_partitions, a->row_stride, a->part_len, a->lambda);
@@ -639,8 +644,11 @@ int btard_preclip(const btard_preclip_args* a)
     double* slots = (double*)(base + align_up(sizeof(PartEntry) * (size_t)a->n_partitions, 256));
     const int chunks = preclip_chunks(a->n_peers, a->n_partitions, a->row_stride);
     return launch_preclip(a->g, table, slots, a->row_norm, a->factor, a->status, a->row_stride,
-                          a->n_peers, a->n_partitions, chunks, st);
+                          a->n_peers, a->n_partitions, chunks, rewrite, st);
 }
+
+int btard_preclip(const btard_preclip_args* a) { return preclip_run(a, true); }
+int btard_preclip_factors(const btard_preclip_args* a) { return preclip_run(a, false); }
 
 int btard_verification_checks(const btard_checks_args* a)
 {

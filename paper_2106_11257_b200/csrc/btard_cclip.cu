@@ -179,9 +179,11 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     __shared__ int sh_flag;
     __shared__ float sh_wsum;                         // sum of the clip weights (PASS_ITER)
     __shared__ __align__(8) float2 sh_w2[(MODE == PASS_ITER) ? BTARD_MAX_PEERS + 16 : 1];   // (w_i, w_i)
+    __shared__ float sh_f[BTARD_MAX_PEERS + 16];      // row factors (with row_scale)
 
     const CclipLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
+    const bool scaled = a.row_scale != nullptr;       // rows enter as f_i x_i: the guarded tile path applies f
     const int tid = threadIdx.x, cl = tid % CL, rg = tid / CL;
     // Consecutive passes sweep the tensor in opposite directions, so that a pass starts on the
     // lines the previous one touched last and finds part of them still in L2.
@@ -227,6 +229,10 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
 
+    if (scaled) {                                     // row_scale is an input: nothing in the chain of passes writes it
+        for (int i = threadIdx.x; i < BTARD_MAX_PEERS + 16; i += blockDim.x)
+            sh_f[i] = (i < n) ? (float)a.row_scale[(size_t)p * n + i] : 0.0f;
+    }
     if (MODE == PASS_ITER) {
         if (a.done[p]) return;
         // Totals the previous pass left behind: squared norms at the current v, and its squared step.
@@ -240,7 +246,9 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         }
         if (tid == 0) sh_flag = 0;
         __syncthreads();
-        row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, sh_part);
+        // the radius of this update: the schedule's tau_l when one is given
+        const double tau_l = a.tau_sched ? a.tau_sched[(size_t)p * a.max_iters + a.l] : tau;
+        row_weights(sh_sum, sh_w, n, tau_l, a.rule, &sh_flag, sh_part);
         if (tid == 0) {
             float w = 0.0f;
             for (int i = 0; i < n; ++i) w += sh_w[i];
@@ -264,6 +272,8 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         skip_rows = sh_flag != 0;
         __syncthreads();
     }
+
+    if (scaled) __syncthreads();                      // the row factors are in shared memory
 
     float acc[R];
 #pragma unroll
@@ -291,6 +301,10 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
             for (int r = 0; r < R; ++r) {
                 const int i = rg * R + r;
                 x[r] = (i < n) ? ld_policy(gp + (size_t)i * stride + col, policy) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (scaled) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) x[r] = scale_row(x[r], sh_f[rg * R + r]);
             }
             if (MODE != PASS_INIT || a.init_mode == BTARD_INIT_CALLER_V0) {
                 if (KEEPV) asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;" : "=f"(v4.x), "=f"(v4.y), "=f"(v4.z), "=f"(v4.w) : "l"(vp + col), "l"(keep));
@@ -477,7 +491,7 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         const long long qb = q0 + (rev ? ntiles - 1 - t : t) * CL;
         const bool inner = (qb + CL <= q1 && qb + CL <= full_quads);
         if (MODE == PASS_ITER) {
-            if (inner && !skip_rows) fast_tile(qb, (int)(t & 1), pol);
+            if (inner && !skip_rows && !scaled) fast_tile(qb, (int)(t & 1), pol);
             else tile(std::true_type{}, qb, (int)(t & 1), pol);
         } else {
             if (inner) tile(std::false_type{}, qb, (int)(t & 1), pol);
@@ -844,7 +858,8 @@ __global__ void __launch_bounds__(512) cclip_cooperative_kernel(const CoopArgs k
                     add_finished += 1;
                 }
             } else {
-                row_weights(sh_sum, sh_w, n, tau, a.rule, &sh_flag, sh_part);
+                const double tau_l = a.tau_sched ? a.tau_sched[(size_t)p * a.max_iters + l] : tau;
+                row_weights(sh_sum, sh_w, n, tau_l, a.rule, &sh_flag, sh_part);
                 if (j == 0 && tid == 0 && sh_flag) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
                 sweep(std::false_type{}, (l + 1) & 1, backwards);
             }
@@ -943,8 +958,8 @@ __device__ __forceinline__ float signed_key_value(int k)
 // the column is padded to N2 inputs with the largest key and the middle is picked at run time.
 template <int N2, bool EXACT>
 __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float* v,
-                                                          const PartEntry* table, long long stride,
-                                                          int n)
+                                                          const PartEntry* table, const double* row_scale,
+                                                          long long stride, int n)
 {
     const int p = blockIdx.y;
     const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -954,9 +969,22 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
     if (c < len) {
         const float* gp = g + (size_t)p * n * stride + c;
         int key[N2];
+        if (row_scale) {                               // rows enter as f_i x_i (a factor of 0 reads as zeros)
+            const double* fp = row_scale + (size_t)p * n;
 #pragma unroll
-        for (int i = 0; i < N2; ++i)
-            key[i] = (EXACT || i < n) ? signed_key(__ldcs(gp + (size_t)i * stride)) : 0x7fffffff;
+            for (int i = 0; i < N2; ++i) {
+                float x = 0.0f;
+                if (EXACT || i < n) {
+                    const float f = (float)fp[i];
+                    x = (f == 0.0f) ? 0.0f : f * __ldcs(gp + (size_t)i * stride);
+                }
+                key[i] = (EXACT || i < n) ? signed_key(x) : 0x7fffffff;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < N2; ++i)
+                key[i] = (EXACT || i < n) ? signed_key(__ldcs(gp + (size_t)i * stride)) : 0x7fffffff;
+        }
         OddEvenNetwork<N2>::template sort<0, N2>(key);
         int ka = 0, kb = 0;
         if (EXACT) {
@@ -977,7 +1005,7 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
 }
 
 // Any n: rank every value by counting (O(n^2) compares per column), pick the two middle ranks.
-__global__ void median_rank_kernel(const float* g, float* v, const PartEntry* table,
+__global__ void median_rank_kernel(const float* g, float* v, const PartEntry* table, const double* row_scale,
                                    long long stride, int n)
 {
     const int p = blockIdx.y;
@@ -989,11 +1017,18 @@ __global__ void median_rank_kernel(const float* g, float* v, const PartEntry* ta
         const float* gp = g + (size_t)p * n * stride + c;
         const int ia = (n - 1) >> 1, ib = n >> 1;
         uint32_t ka = 0, kb = 0;
+        const double* fp = row_scale ? row_scale + (size_t)p * n : nullptr;
+        auto value = [&](int i) {                      // row i as it enters: f_i x_i (a factor of 0 reads as zeros)
+            const float x = gp[(size_t)i * stride];
+            if (!fp) return x;
+            const float f = (float)fp[i];
+            return (f == 0.0f) ? 0.0f : f * x;
+        };
         for (int i = 0; i < n; ++i) {
-            const uint32_t ki = order_key(gp[(size_t)i * stride]);
+            const uint32_t ki = order_key(value(i));
             int rank = 0;
             for (int q = 0; q < n; ++q) {
-                const uint32_t kq = order_key(gp[(size_t)q * stride]);
+                const uint32_t kq = order_key(value(q));
                 rank += (kq < ki) || (kq == ki && q < i);
             }
             if (rank == ia) ka = ki;
@@ -1175,25 +1210,25 @@ int cooperative_launch_supported()
     return coop;
 }
 
-int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
-                       int P, cudaStream_t st)
+int launch_median_init(const float* g, float* v, const PartEntry* table, const double* row_scale,
+                       long long stride, int n, int P, cudaStream_t st)
 {
     const int threads = 128;
     dim3 grid((unsigned)((stride + threads - 1) / threads), (unsigned)P);
     prof_begin(KIND_MEDIAN, st);
-    if (n == 1) median_sort_kernel<1, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n == 2) median_sort_kernel<2, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n == 4) median_sort_kernel<4, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n == 8) median_sort_kernel<8, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n == 16) median_sort_kernel<16, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n == 32) median_sort_kernel<32, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n == 64) median_sort_kernel<64, true><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n < 4) median_sort_kernel<4, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n < 8) median_sort_kernel<8, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n < 16) median_sort_kernel<16, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n < 32) median_sort_kernel<32, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else if (n < 64) median_sort_kernel<64, false><<<grid, threads, 0, st>>>(g, v, table, stride, n);
-    else median_rank_kernel<<<grid, threads, 0, st>>>(g, v, table, stride, n);
+    if (n == 1) median_sort_kernel<1, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n == 2) median_sort_kernel<2, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n == 4) median_sort_kernel<4, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n == 8) median_sort_kernel<8, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n == 16) median_sort_kernel<16, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n == 32) median_sort_kernel<32, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n == 64) median_sort_kernel<64, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n < 4) median_sort_kernel<4, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n < 8) median_sort_kernel<8, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n < 16) median_sort_kernel<16, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n < 32) median_sort_kernel<32, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else if (n < 64) median_sort_kernel<64, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    else median_rank_kernel<<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
     prof_end(KIND_MEDIAN, st);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();

@@ -86,7 +86,16 @@ struct CclipLaunch {
     int init_mode;            // PASS_INIT
     int rule;                 // BTARD_RULE_*: how the row weights follow from the norms
     int v_fits_l2;            // v (and its bf16 part) of all partitions takes at most 60 % of the L2
+    const double* tau_sched;  // device [P][max_iters] radius of update l, or nullptr (the table's tau)
+    const double* row_scale;  // device [P][n] factor applied to row i on load, or nullptr
 };
+
+// x scaled by a row factor; a factor of exactly 0 drops the row whatever it holds.
+__device__ __forceinline__ float4 scale_row(float4 x, float f)
+{
+    if (f == 0.0f) return make_float4(0.f, 0.f, 0.f, 0.f);
+    return make_float4(x.x * f, x.y * f, x.z * f, x.w * f);
+}
 
 Geometry cclip_geometry(int n, int P, long long stride);
 int choose_ctas_per_partition(int P, long long quads, int CL, int slots, int max_tiles = kMaxTilesPerCta);
@@ -100,8 +109,8 @@ constexpr long long kCoopMaxItems = 1LL << 20;
 int cooperative_launch_supported();
 int launch_cclip_cooperative(const CclipLaunch& a, const Geometry& geo, int streaming, double* rslots,
                              unsigned long long* barrier, unsigned int* error, cudaStream_t st);
-int launch_median_init(const float* g, float* v, const PartEntry* table, long long stride, int n,
-                       int P, cudaStream_t st);
+int launch_median_init(const float* g, float* v, const PartEntry* table, const double* row_scale,
+                       long long stride, int n, int P, cudaStream_t st);
 // squared-norm totals -> norms, used when verification is asked to compute the norms itself.
 int launch_totals_to_norms(const double* tot, double* norm, int n, int P, cudaStream_t st);
 
@@ -133,6 +142,8 @@ struct GramLaunch {
     int n, P;
     int stop_mode, max_iters;
     double eps2;
+    const double* tau_sched;    // device [P][max_iters] or nullptr
+    const double* row_scale;    // device [P][n] or nullptr
 };
 GramGeometry gram_geometry(int n, int P, long long stride);
 int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st);
@@ -143,8 +154,9 @@ int launch_gram_finalize(const double* tot, double* resid_norm, uint32_t* status
 
 // ---- per-part gradient clipping (btard_preclip.cu) ----------------------------------------------
 int preclip_chunks(int n, int P, long long stride);
+// rewrite = false: norms and factors only, g untouched
 int launch_preclip(float* g, const PartEntry* table, double* slots, double* row_norm, double* factor,
-                   uint32_t* status, long long stride, int n, int P, int chunks, cudaStream_t st);
+                   uint32_t* status, long long stride, int n, int P, int chunks, bool rewrite, cudaStream_t st);
 
 // ---- Split / Merge copies (btard_pack.cu); table_dev: device {offset, len}[P] as two int64 each ---
 int launch_split(const float* grads, float* g, const void* table_dev, long long d, long long stride,
@@ -180,6 +192,7 @@ struct VerifyLaunch {
     double* resid_norm_out;       // device [P][n]: the aggregation's resid_norm output
     uint32_t* cclip_status;       // device [P]: the aggregation's status word (bits are OR-ed in)
     const unsigned int* gram_error;   // device: a bounded wait of the Gram kernel expired
+    const double* row_scale;          // device [P][n] factor applied to row i on load, or nullptr
 };
 
 // Where entry (i, j) of a partition's Gram matrix sits: upper-triangular 8 x 8 blocks, NB = ceil(n / 8)

@@ -79,7 +79,8 @@ __global__ void __launch_bounds__(kGramThreads) gram_kernel(const GArgs k)
                 const int row = e / q4, c4 = e - row * q4;
                 const long long col = cb + 4 * c4;
                 if (col < c1) {
-                    const float4 x = __ldcs(reinterpret_cast<const float4*>(gp + (size_t)row * stride + col));
+                    float4 x = __ldcs(reinterpret_cast<const float4*>(gp + (size_t)row * stride + col));
+                    if (a.row_scale) x = scale_row(x, (float)a.row_scale[(size_t)p * n + row]);
                     const float4 v = *reinterpret_cast<const float4*>(vp + col);
                     r.x = (col < len) ? x.x - v.x : 0.f;
                     r.y = (col + 1 < len) ? x.y - v.y : 0.f;
@@ -212,10 +213,16 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
     constexpr int STAGE = rows_stage_bytes<R>();
     extern __shared__ __align__(16) unsigned char sh_stage[];          // [kRowsStages][R + 1][kRowsTile] floats
     __shared__ double sh_acc[kRowsThreads / 32][NP];
+    __shared__ float sh_f[R];                          // row factors (with row_scale)
     __shared__ int sh_last;
     const GramLaunch& a = k.a;
     const int n = a.n, cpp = k.g.cpp, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const bool scaled = a.row_scale != nullptr;        // rows enter as f_i x_i
+    if (scaled) {
+        if (tid < R) sh_f[tid] = (tid < n) ? (float)a.row_scale[(size_t)p * n + tid] : 0.0f;
+        __syncthreads();
+    }
     const long long stride = a.stride, len = a.table[p].len;
     const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v0 + (size_t)p * stride;
@@ -272,6 +279,14 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
 #pragma unroll
         for (int r = 0; r < R; ++r)
             asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x[r].x), "=f"(x[r].y) : "r"(src + (uint32_t)r * (kRowsTile * 4)) : "memory");
+        if (scaled) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float f = sh_f[r];
+                x[r].x = (f == 0.0f) ? 0.0f : f * x[r].x;
+                x[r].y = (f == 0.0f) ? 0.0f : f * x[r].y;
+            }
+        }
         // residuals; what was never copied (rows >= n, columns beyond the CTA's range or the data) reads as 0
         if (FULL && c0 + (long long)(t + 1) * kRowsTile <= (len < c1 ? len : c1)) {       // whole tile inside
 #pragma unroll
@@ -423,9 +438,12 @@ __global__ void __launch_bounds__(kWsThreads, 2) gram_umma_ws_kernel(const GArgs
     __shared__ uint32_t sh_tmem;
     __shared__ int sh_last;
     __shared__ int sh_fail;
+    __shared__ float sh_f[64];                         // row factors (with row_scale)
     const GramLaunch& a = k.a;
     const int n = a.n, cpp = k.g.cpp, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const bool scaled = a.row_scale != nullptr;        // rows enter as f_i x_i
+    if (scaled && tid < 64) sh_f[tid] = (tid < n) ? (float)a.row_scale[(size_t)p * n + tid] : 0.0f;   // before the CTA barrier below
     const long long stride = a.stride, len = a.table[p].len;
     const float* vp = a.v0 + (size_t)p * stride;
     // The CTAs of a partition take its 32-column tiles round-robin (tile j, j + cpp, ...): resident
@@ -536,6 +554,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) gram_umma_ws_kernel(const GArgs
                 for (int i = 0; i < 8; ++i) {
                     const int m = 8 * half + i;
                     if (ROWS_FULL || q + 4 * m < n) {
+                        if (scaled) x[i] = scale_row(x[i], sh_f[q + 4 * m]);
                         float r0 = x[i].x - v4.x, r1 = x[i].y - v4.y, r2 = x[i].z - v4.z, r3 = x[i].w - v4.w;
                         if (!inside) {                 // ragged end: what lies beyond len (stale bytes included) is 0
                             r0 = m0 ? r0 : 0.f; r1 = m1 ? r1 : 0.f; r2 = m2 ? r2 : 0.f; r3 = 0.f;
@@ -729,12 +748,13 @@ __global__ void __launch_bounds__(kGramThreads) gram_iterate_kernel(const GArgs 
     int iters = 0;
     for (int l = 0; l < a.max_iters; ++l) {
         const double aGa = block_sum((row && !bad) ? ai * Gai : 0.0, red);
+        const double tau_l = a.tau_sched ? a.tau_sched[(size_t)p * a.max_iters + l] : tau;   // tau_l of App. D.2
         double w = 0.0;
         if (row && !bad) {
             double rho2 = gii - 2.0 * Gai + aGa;
             if (rho2 < 0.0) rho2 = 0.0;
             const double rho = sqrt(rho2);
-            if (isfinite(rho)) w = (rho <= tau) ? 1.0 : tau / rho;
+            if (isfinite(rho)) w = (rho <= tau_l) ? 1.0 : tau_l / rho;
         }
         const double W = block_sum(w, red);
         const double d = (row && !bad) ? (w - W * ai) / (double)n : 0.0;
@@ -811,12 +831,14 @@ __global__ void __launch_bounds__(32) gram_iterate_warp_kernel(const GArgs k)
     double ai = 0.0, Gai = 0.0, step2 = 0.0;
     double aGa = 0.0;              // a^T G a, carried along: (a + d)^T G (a + d) = a^T G a + 2 d^T G a + d^T G d
     int iters = 0;
+    const double* sched = a.tau_sched ? a.tau_sched + (size_t)p * a.max_iters : nullptr;   // tau_l of App. D.2
     for (int l = 0; l < a.max_iters; ++l) {
+        const double tau_l = sched ? sched[l] : tau, tau_l2 = sched ? tau_l * tau_l : tau2;
         double w = 0.0;
         if (live) {
             double rho2 = gii - 2.0 * Gai + aGa;
             if (rho2 < 0.0) rho2 = 0.0;
-            if (isfinite(rho2)) w = (rho2 <= tau2) ? 1.0 : tau * rsqrt(rho2);
+            if (isfinite(rho2)) w = (rho2 <= tau_l2) ? 1.0 : tau_l * rsqrt(rho2);
         }
         const double W = warp_allsum(w);
         const double d = live ? (w - W * ai) * inv_n : 0.0;

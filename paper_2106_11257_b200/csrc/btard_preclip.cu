@@ -30,6 +30,7 @@ struct PreArgs {
     uint32_t* status;           // [P] out
     long long stride;
     int n, P, chunks;
+    int rewrite;                // 1: rescale the clipped rows in place; -1: norms and factors only (one CTA per row)
 };
 
 __device__ __forceinline__ void chunk_range(long long quads, int c, int chunks, long long& q0, long long& q1)
@@ -70,8 +71,9 @@ __global__ void __launch_bounds__(kPreThreads) preclip_norm_kernel(const PreArgs
 __global__ void __launch_bounds__(kPreThreads) preclip_scale_kernel(const PreArgs a)
 {
     __shared__ double sh_norm2;
-    const long long row = blockIdx.x / a.chunks;
-    const int c = blockIdx.x % a.chunks, p = (int)(row / a.n);
+    // rewrite < 0: one CTA per row, norms and factors only
+    const long long row = (a.rewrite < 0) ? blockIdx.x : blockIdx.x / a.chunks;
+    const int c = (a.rewrite < 0) ? 0 : blockIdx.x % a.chunks, p = (int)(row / a.n);
     const long long len = a.table[p].len;
     const double lambda = a.table[p].tau;
     if (threadIdx.x == 0) {
@@ -89,7 +91,7 @@ __global__ void __launch_bounds__(kPreThreads) preclip_scale_kernel(const PreArg
         a.factor[row] = f;
         if (!isfinite(norm)) atomicOr(&a.status[p], BTARD_STATUS_NONFINITE_ROW);
     }
-    if (f == 1.0) return;                             // untouched rows cost no write traffic
+    if (f == 1.0 || a.rewrite <= 0) return;               // untouched rows cost no write traffic
     float* x = a.g + (size_t)row * a.stride;
     long long q0, q1;
     chunk_range(a.stride >> 2, c, a.chunks, q0, q1);
@@ -123,14 +125,16 @@ int preclip_chunks(int n, int P, long long stride)
 }
 
 int launch_preclip(float* g, const PartEntry* table, double* slots, double* row_norm, double* factor,
-                   uint32_t* status, long long stride, int n, int P, int chunks, cudaStream_t st)
+                   uint32_t* status, long long stride, int n, int P, int chunks, bool rewrite, cudaStream_t st)
 {
-    PreArgs a{g, table, slots, row_norm, factor, status, stride, n, P, chunks};
+    PreArgs a{g, table, slots, row_norm, factor, status, stride, n, P, chunks, rewrite ? 1 : 0};
     const long long grid = (long long)n * P * chunks;
     if (grid > 0x7fffffffLL) return BTARD_ERR_UNSUPPORTED;
     preclip_reset_kernel<<<(P + 127) / 128, 128, 0, st>>>(status, P);
     preclip_norm_kernel<<<(unsigned)grid, kPreThreads, 0, st>>>(a);
-    preclip_scale_kernel<<<(unsigned)grid, kPreThreads, 0, st>>>(a);
+    // without the rewrite one CTA per row is enough: it adds up the slots and writes norm and factor
+    if (rewrite) preclip_scale_kernel<<<(unsigned)grid, kPreThreads, 0, st>>>(a);
+    else preclip_scale_kernel<<<(unsigned)((long long)n * P), 32, 0, st>>>(PreArgs{g, table, slots, row_norm, factor, status, stride, n, P, chunks, -1});
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch(3);
     return BTARD_OK;

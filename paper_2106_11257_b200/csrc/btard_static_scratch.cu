@@ -105,7 +105,7 @@ extern "C" int btard_verify_projections_static(const btard_verify_args* a)
         L.ticket = (unsigned int*)(base + o_ticket);
         // The array keeps whatever the previous call left: the finish counters must start at zero.
         BTARD_CUDA_TRY(cudaMemsetAsync(L.ticket, 0, sizeof(unsigned int) * (size_t)P, st));
-        L.stride = stride; L.n = n; L.P = P;
+        L.stride = stride; L.n = n; L.P = P; L.row_scale = a->row_scale;
         rc = launch_cclip_pass(L, cg, PASS_NORMS, st);
         if (rc != BTARD_OK) return rc;
         rc = launch_totals_to_norms(L.tot_out, (double*)(base + o_norms), n, P, st);
@@ -121,6 +121,7 @@ extern "C" int btard_verify_projections_static(const btard_verify_args* a)
     V.znorm2 = a->znorm2; V.resid_sum_norm = a->resid_sum_norm; V.status = a->status;
     V.stride = stride; V.n = n; V.P = P; V.K = K; V.p_base = a->partition_base;
     V.seed_lo = (uint32_t)a->seed; V.seed_hi = (uint32_t)(a->seed >> 32);
+    V.row_scale = a->row_scale;
     for (int k0 = 0; k0 < K; k0 += vg.KT) {
         V.k0 = k0;
         V.kc = (K - k0 < vg.KT) ? K - k0 : vg.KT;

@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     __shared__ __align__(8) float2 sh_c2[COMBINE ? BTARD_MAX_PEERS + 16 : 1]; // coefficients (a_j, a_j)
     __shared__ double sh_ga[COMBINE ? BTARD_MAX_PEERS + 1 : 1];               // (G a)_i, then a^T G a
     __shared__ double sh_red[MAXT / 32][R * KT + KT + 1 + (COMBINE ? R : 0)];
+    __shared__ float sh_f[BTARD_MAX_PEERS + 16];      // row factors (with row_scale)
 
     const VerifyLaunch& a = k.a;
     const int n = a.n, RG = k.RG, CL = k.CL, cpp = k.cpp;
@@ -65,9 +66,11 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     float4* sh_s = sh_dyn + 3 * KT * CL;
     float4* sh_u = sh_s + 2 * RG * CL;
 
+    const bool scaled = a.row_scale != nullptr;       // rows enter as f_i x_i: applied in the guarded tile path
     for (int i = tid; i < BTARD_MAX_PEERS + 16; i += nthr) {
         sh_w2[i] = make_float2(0.f, 0.f);
         if (COMBINE) sh_c2[i] = make_float2(0.f, 0.f);
+        if (scaled) sh_f[i] = (i < n) ? (float)a.row_scale[(size_t)p * n + i] : 0.0f;
     }
     __syncthreads();
     int skip = 0;                                      // some row of this partition must be left out
@@ -208,6 +211,17 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
                 for (int r = 0; r < R; ++r, xr += stride_bytes)
                     if (r < nrows) ld_stream_pairs(reinterpret_cast<const float*>(xr), xa[r], xb[r]);
             }
+            if (GUARD && scaled) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float x0, x1, x2, x3;
+                    upk2(xa[r], x0, x1);
+                    upk2(xb[r], x2, x3);
+                    const float4 y = scale_row(make_float4(x0, x1, x2, x3), sh_f[rg * R + r]);
+                    xa[r] = pk2(y.x, y.y);
+                    xb[r] = pk2(y.z, y.w);
+                }
+            }
             const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
             va = pk2(v4.x, v4.y);
             vb = pk2(v4.z, v4.w);
@@ -317,7 +331,7 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     if (q0 < q1) gen_z(q0, 0);                         // made visible by the first tile's barrier
     // interior tiles come first: a run without predicates, then the guarded rest
     long long inner_end = (q1 < full_quads) ? q1 : full_quads;
-    if (any_skip) inner_end = q0;
+    if (any_skip || scaled) inner_end = q0;
     int par = 0, zcur = 0;
     long long qb = q0;
     for (; qb + CL <= inner_end; qb += CL, par ^= 1, zcur = (zcur == 2 ? 0 : zcur + 1)) tile(std::false_type{}, qb, par, zcur);
@@ -400,12 +414,15 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
     __shared__ float sh_c[16];                      // COMBINE: coefficients a_j
     __shared__ double sh_ga[17];                    // COMBINE: (G a)_i, then a^T G a
     __shared__ double sh_red[8][R * KT + KT + 1 + (COMBINE ? R : 0)];
+    __shared__ float sh_f[16];                      // row factors (with row_scale)
 
     const VerifyLaunch& a = k.a;
     const int n = a.n, cpp = k.cpp;
     constexpr int CL = 256;
     const int tid = threadIdx.x;
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const bool scaled = a.row_scale != nullptr;     // rows enter as f_i x_i
+    if (scaled && tid < 16) sh_f[tid] = (tid < n) ? (float)a.row_scale[(size_t)p * n + tid] : 0.0f;   // before the barriers below
     const long long stride = a.stride, len = a.table[p].len;
     const double tau = a.table[p].tau;
 
@@ -481,6 +498,10 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
         for (int r = 0; r < R; ++r)
             x[r] = (r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
                            : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (scaled) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] = scale_row(x[r], sh_f[r]);
+        }
         const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
         // this thread's quads of z, drawn while the rows are on their way
         float4 z[KT];

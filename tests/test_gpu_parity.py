@@ -376,6 +376,68 @@ def test_preclip_matches_oracle(n, stride):
     assert cpu(out["status"])[1] & btard.STATUS_NONFINITE_ROW and np.all(got[1, 1, :lens[1]] == 0)
 
 
+# ----------------------------------------------------------------------------- tau_l schedule, Clipped-SGD factors
+@pytest.mark.parametrize("algo", [btard.ALGO_DIRECT, btard.ALGO_GRAM, btard.ALGO_DIRECT_COOPERATIVE])
+@pytest.mark.parametrize("n", [3, 16, 23, 64, 100])
+def test_tau_schedule_matches_oracle(n, algo):
+    """Update l uses the radius tau_l (App. D.2): every algorithm against the oracle's scheduled run."""
+    rng = np.random.default_rng(1300 + n)
+    P, stride, iters = 3, 5024, 7
+    lens = np.array([5024, 4097, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    sched = np.abs(rng.standard_normal((P, iters))) + 0.2
+    sched[1, 2] = np.inf
+    sched[2, 4] = 0.0
+    ref = oracle.centered_clip(g, 1.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=iters, tau_schedule=sched)
+    _, r = run_gpu_cclip(g, 1.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=iters, algo=algo,
+                         tau_schedule=torch.from_numpy(sched).cuda())
+    check_cclip(r, ref, lens)
+
+
+@pytest.mark.parametrize("n,K", [(4, 1), (16, 2), (16, 5), (23, 1), (64, 1), (64, 4), (100, 2)])
+def test_clipped_sgd_factors_applied_on_load(n, K):
+    """BTARD-Clipped-SGD (Alg. 9) without rewriting g: btard_preclip_factors, then aggregation and
+    verification with row_scale, against the oracle's clip factors and its scaled aggregation; direct and
+    Gram algorithms, separate calls and the one-call entry point.  One row holds an inf (factor 0)."""
+    rng = np.random.default_rng(1400 + 3 * n + K)
+    P, stride = 3, 20_032
+    lens = np.array([20_032, 17_001, 13])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    g[1, n - 1, 5] = np.inf
+    lam = np.array([200.0, 150.0, 5.0])
+    tau = np.array([0.5, 1.0, 2.0])
+    pc = oracle.preclip(g, lam, part_len=lens)
+    assert (pc["factor"] < 1).any() and (pc["factor"] == 1).any() and pc["factor"][1, n - 1] == 0
+    gd = torch.from_numpy(g).cuda()
+    keep = gd.clone()
+    out = btard.preclip(gd, lam, part_len=lens, in_place=False)
+    torch.cuda.synchronize()
+    assert torch.equal(gd, keep)                                  # g untouched
+    fin = np.isfinite(pc["row_norm"])
+    assert rel_l2(cpu(out["row_norm"])[fin], pc["row_norm"][fin]) <= 1e-6
+    assert rel_l2(cpu(out["factor"]), pc["factor"]) <= 1e-6 and cpu(out["factor"])[1, n - 1] == 0
+    assert cpu(out["status"])[1] & btard.STATUS_NONFINITE_ROW
+    f = out["factor"]
+    refc = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=6, row_scale=pc["factor"])
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
+        if algo == btard.ALGO_GRAM and n > 128:
+            continue
+        r = btard.centered_clip(gd, tau, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=6, algo=algo,
+                                row_scale=f)
+        torch.cuda.synchronize()
+        check_cclip(r, refc, lens)
+        v32 = cpu(r["v"])
+        refv = oracle.verify(g, v32, tau, 21, K=K, part_len=lens, row_scale=pc["factor"], want_resid_sum=True)
+        o = btard.verify_projections(gd, r["v"], tau, 21, K=K, part_len=lens, row_scale=f, want_resid_sum=True)
+        torch.cuda.synchronize()
+        check_verify(o, refv, K)
+        rc, rv = btard.centered_clip_verify(gd, tau, 21, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                            max_iters=6, algo=algo, row_scale=f)
+        torch.cuda.synchronize()
+        check_cclip(rc, refc, lens)
+        check_verify(rv, oracle.verify(g, cpu(rc["v"]), tau, 21, K=K, part_len=lens, row_scale=pc["factor"]), K)
+
+
 # ----------------------------------------------------------------------------- Gram variant
 @pytest.mark.parametrize("n", [1, 3, 8, 16, 23, 64, 100, 128])
 @pytest.mark.parametrize("init", [btard.INIT_MEAN, btard.INIT_COORD_MEDIAN, btard.INIT_CALLER_V0])
