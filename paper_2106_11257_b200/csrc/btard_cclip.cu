@@ -961,7 +961,12 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
                                                           const PartEntry* table, const double* row_scale,
                                                           long long stride, int n)
 {
+    __shared__ float sh_f[N2];                         // row factors (with row_scale)
     const int p = blockIdx.y;
+    if (row_scale) {
+        if (threadIdx.x < N2) sh_f[threadIdx.x] = ((int)threadIdx.x < n) ? (float)row_scale[(size_t)p * n + threadIdx.x] : 0.0f;
+        __syncthreads();
+    }
     const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= stride) return;
     const long long len = table[p].len;
@@ -970,12 +975,11 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
         const float* gp = g + (size_t)p * n * stride + c;
         int key[N2];
         if (row_scale) {                               // rows enter as f_i x_i (a factor of 0 reads as zeros)
-            const double* fp = row_scale + (size_t)p * n;
 #pragma unroll
             for (int i = 0; i < N2; ++i) {
                 float x = 0.0f;
                 if (EXACT || i < n) {
-                    const float f = (float)fp[i];
+                    const float f = sh_f[i];
                     x = (f == 0.0f) ? 0.0f : f * __ldcs(gp + (size_t)i * stride);
                 }
                 key[i] = (EXACT || i < n) ? signed_key(x) : 0x7fffffff;
