@@ -196,6 +196,9 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     const double tau = a.table[p].tau;
 
     const float* gp = a.g + (size_t)p * n * stride;
+    const float* xrow0 = gp + (size_t)(rg * R) * stride;   // this thread's first row; one stride per further row
+    const long long stride_bytes = stride * 4;
+    const int nrows = (n - rg * R < R) ? n - rg * R : R;   // rows of this group that exist
     float* vp = a.v + (size_t)p * stride;
     unsigned short* lop = COMP ? a.v_lo + (size_t)p * stride : nullptr;
     const float inv_n = 1.0f / (float)n;
@@ -297,11 +300,10 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
         float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f);      // low-order part of v (COMP)
         if (valid) {
+            const char* xr = reinterpret_cast<const char*>(xrow0 + col);
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int i = rg * R + r;
-                x[r] = (i < n) ? ld_policy(gp + (size_t)i * stride + col, policy) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int r = 0; r < R; ++r, xr += stride_bytes)
+                x[r] = (r < nrows) ? ld_policy(reinterpret_cast<const float*>(xr), policy) : make_float4(0.f, 0.f, 0.f, 0.f);
             if (scaled) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) x[r] = scale_row(x[r], sh_f[rg * R + r]);
@@ -412,11 +414,16 @@ __global__ void __launch_bounds__(512) cclip_pass_kernel(const KernelArgs k)
     auto fast_tile = [&](long long qb, int parity, uint64_t policy) {
         const long long col = (qb + cl) * 4;
         uint64_t xa[R], xb[R];
+        const char* xr = reinterpret_cast<const char*>(xrow0 + col);
+        if (nrows == R) {                              // the usual case: no row test, no zero fill
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int i = rg * R + r;
-            if (i < n) ld_row_pairs(gp + (size_t)i * stride + col, policy, xa[r], xb[r]);
-            else { xa[r] = 0ull; xb[r] = 0ull; }
+            for (int r = 0; r < R; ++r, xr += stride_bytes) ld_row_pairs(reinterpret_cast<const float*>(xr), policy, xa[r], xb[r]);
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r, xr += stride_bytes) {
+                if (r < nrows) ld_row_pairs(reinterpret_cast<const float*>(xr), policy, xa[r], xb[r]);
+                else { xa[r] = 0ull; xb[r] = 0ull; }
+            }
         }
         float4 v4;
         asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
