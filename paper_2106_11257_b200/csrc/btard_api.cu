@@ -369,7 +369,9 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     // How the updates are driven: one cooperative kernel over everything, or one launch per update.
     const bool whole = (a->algo == BTARD_ALGO_DIRECT_COOPERATIVE) && cooperative_launch_supported();
     L.init_mode = a->init_mode;
-    if (a->init_mode == BTARD_INIT_COORD_MEDIAN) {
+    // up to 16 peers the Gram pass takes the median start itself (every row of a column sits in one thread)
+    const bool gram_takes_median = (a->algo == BTARD_ALGO_GRAM && a->init_mode == BTARD_INIT_COORD_MEDIAN && n <= 16);
+    if (a->init_mode == BTARD_INIT_COORD_MEDIAN && !gram_takes_median) {
         rc = launch_median_init(a->g, a->v, L.table, a->row_scale, a->row_stride, n, P, st);
         if (rc != BTARD_OK) return rc;
         L.init_mode = BTARD_INIT_CALLER_V0;
@@ -384,7 +386,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
         }
         const GramGeometry gg = gram_geometry(n, P, a->row_stride);
         GramLaunch G{};
-        G.g = a->g; G.v0 = a->v; G.table = L.table;
+        G.g = a->g; G.v0 = a->v; G.v0_out = a->v; G.fuse_median = gram_takes_median ? 1 : 0; G.table = L.table;
         G.slots = (double*)(base + ws.gslots); G.gram = (double*)(base + ws.gram);
         G.ticket = (unsigned int*)(base + ws.flags) + 2 * P;
         G.error = (unsigned int*)(base + ws.flags) + 3 * P;

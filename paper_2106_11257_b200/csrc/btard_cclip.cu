@@ -16,6 +16,7 @@
 #include <type_traits>
 
 #include "btard_common.h"
+#include "btard_median.cuh"
 
 namespace btard {
 namespace {
@@ -914,52 +915,6 @@ __device__ __forceinline__ float key_value(uint32_t key)
     return __uint_as_float((key & 0x80000000u) ? (key & 0x7FFFFFFFu) : ~key);
 }
 
-// Batcher's odd-even merge sort as a comparator network on registers (N a power of two).  All
-// indices are compile-time constants, so when only the middle outputs are used the compiler drops
-// every comparator that does not feed them.
-template <int N>
-struct OddEvenNetwork {
-    template <int LO, int CNT, int R>
-    static __device__ __forceinline__ void merge(int (&k)[N])
-    {
-        constexpr int STEP = R * 2;
-        if constexpr (STEP < CNT) {
-            merge<LO, CNT, STEP>(k);
-            merge<LO + R, CNT, STEP>(k);
-#pragma unroll
-            for (int i = LO + R; i + R < LO + CNT; i += STEP) {
-                const int lo = min(k[i], k[i + R]), hi = max(k[i], k[i + R]);
-                k[i] = lo;
-                k[i + R] = hi;
-            }
-        } else {
-            const int lo = min(k[LO], k[LO + R]), hi = max(k[LO], k[LO + R]);
-            k[LO] = lo;
-            k[LO + R] = hi;
-        }
-    }
-    template <int LO, int CNT>
-    static __device__ __forceinline__ void sort(int (&k)[N])
-    {
-        if constexpr (CNT > 1) {
-            sort<LO, CNT / 2>(k);
-            sort<LO + CNT / 2, CNT / 2>(k);
-            merge<LO, CNT, 1>(k);
-        }
-    }
-};
-
-// Signed-integer image of a float whose integer order is the IEEE total order of the floats.
-__device__ __forceinline__ int signed_key(float f)
-{
-    const int b = __float_as_int(f);
-    return b ^ ((b >> 31) & 0x7fffffff);
-}
-__device__ __forceinline__ float signed_key_value(int k)
-{
-    return __int_as_float(k ^ ((k >> 31) & 0x7fffffff));
-}
-
 // One thread takes the median of the n values of one column.  EXACT: n == N2 is known at compile
 // time (the two middle outputs are fixed registers and the network is pruned to them); otherwise
 // the column is padded to N2 inputs with the largest key and the middle is picked at run time.
@@ -996,21 +951,7 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
             for (int i = 0; i < N2; ++i)
                 key[i] = (EXACT || i < n) ? signed_key(__ldcs(gp + (size_t)i * stride)) : 0x7fffffff;
         }
-        OddEvenNetwork<N2>::template sort<0, N2>(key);
-        int ka = 0, kb = 0;
-        if (EXACT) {
-            ka = key[(N2 - 1) / 2];
-            kb = key[N2 / 2];
-        } else {
-            // n is a run-time value: pick the two middle keys without dynamic register indexing.
-            const int ia = (n - 1) >> 1, ib = n >> 1;
-#pragma unroll
-            for (int i = 0; i < N2; ++i) {
-                if (i == ia) ka = key[i];
-                if (i == ib) kb = key[i];
-            }
-        }
-        out = (float)(((double)signed_key_value(ka) + (double)signed_key_value(kb)) * 0.5);
+        out = median_of_keys<N2, EXACT>(key, n);
     }
     v[(size_t)p * stride + c] = out;
 }

@@ -129,6 +129,8 @@ struct GramGeometry {
 struct GramLaunch {
     const float* g;
     const float* v0;            // device [P][stride] centre of the Gram matrix
+    float* v0_out;              // fuse_median: the same buffer, written by the Gram pass
+    int fuse_median;            // n <= 16: the Gram pass takes the coordinate-wise median itself (v0 is an output)
     const PartEntry* table;
     double* slots;              // device [P][cpp][entries]
     double* gram;               // device [P][entries] summed blocks

@@ -17,6 +17,7 @@
 #include <cuda.h>
 
 #include "btard_common.h"
+#include "btard_median.cuh"
 
 namespace btard {
 namespace {
@@ -206,7 +207,9 @@ template <int R>
 __host__ __device__ constexpr int rows_stage_bytes() { return (R + 1) * kRowsTile * 4; }   // R rows and v0
 
 // FULL: n == R, no row predicate anywhere.
-template <int R, bool FULL>
+// MEDIAN: the centre v0 is the coordinate-wise median of the rows, taken here (the thread holds every row of
+// its two columns) and written out, instead of being read: the median start costs no pass of its own.
+template <int R, bool FULL, bool MEDIAN>
 __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs k)
 {
     constexpr int NP = R * (R + 1) / 2;
@@ -226,6 +229,7 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
     const long long stride = a.stride, len = a.table[p].len;
     const float* gp = a.g + (size_t)p * n * stride;
     const float* vp = a.v0 + (size_t)p * stride;
+    float* vout = MEDIAN ? a.v0_out + (size_t)p * stride : nullptr;
     // columns of this CTA, cut on 128-byte lines
     long long c0 = stride * j / cpp, c1 = stride * (j + 1) / cpp;
     if (j > 0) c0 &= ~31LL;
@@ -249,8 +253,9 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
                 if (FULL || r < n)
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)r * (kRowsTile * 4)),
                                  "l"(gp + (size_t)r * stride + col) : "memory");
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)R * (kRowsTile * 4)),
-                         "l"(vp + col) : "memory");
+            if (!MEDIAN)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst + (uint32_t)R * (kRowsTile * 4)),
+                             "l"(vp + col) : "memory");
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -274,8 +279,9 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
         const long long col = c0 + (long long)t * kRowsTile + 2 * tid;
         const bool m0 = col < len && col < c1, m1 = col + 1 < len && col < c1;
         const uint32_t src = my_base + (uint32_t)(t % kRowsStages) * STAGE;
-        float2 x[R], v2;
-        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v2.x), "=f"(v2.y) : "r"(src + (uint32_t)R * (kRowsTile * 4)) : "memory");
+        float2 x[R], v2 = make_float2(0.f, 0.f);
+        if (!MEDIAN)
+            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v2.x), "=f"(v2.y) : "r"(src + (uint32_t)R * (kRowsTile * 4)) : "memory");
 #pragma unroll
         for (int r = 0; r < R; ++r)
             asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(x[r].x), "=f"(x[r].y) : "r"(src + (uint32_t)r * (kRowsTile * 4)) : "memory");
@@ -285,6 +291,20 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
                 const float f = sh_f[r];
                 x[r].x = (f == 0.0f) ? 0.0f : f * x[r].x;
                 x[r].y = (f == 0.0f) ? 0.0f : f * x[r].y;
+            }
+        }
+        if (MEDIAN) {
+            // the centre of these two columns: median of the rows as they enter, one column at a time (the
+            // comparator network runs on the integer pipe, next to the products below on the other one)
+            if (col < c1) {                            // row_stride is a multiple of 4: the pair is in or out whole
+                int key[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) key[r] = (FULL || r < n) ? signed_key(x[r].x) : 0x7fffffff;
+                v2.x = m0 ? median_of_keys<R, FULL>(key, n) : 0.0f;
+#pragma unroll
+                for (int r = 0; r < R; ++r) key[r] = (FULL || r < n) ? signed_key(x[r].y) : 0x7fffffff;
+                v2.y = m1 ? median_of_keys<R, FULL>(key, n) : 0.0f;
+                *reinterpret_cast<float2*>(vout + col) = v2;   // 0 beyond the data
             }
         }
         // residuals; what was never copied (rows >= n, columns beyond the CTA's range or the data) reads as 0
@@ -924,6 +944,17 @@ bool encode_rows_map(CUtensorMap* map, const float* g, int n, int P, long long s
 
 }  // namespace
 
+// The n <= 16 Gram kernel for R rows per thread (4, 8 or 16), with or without row predicates and median.
+static const void* rows_fn(int R, bool full, bool median)
+{
+    if (R == 4) return full ? (median ? (const void*)gram_rows_kernel<4, true, true> : (const void*)gram_rows_kernel<4, true, false>)
+                            : (median ? (const void*)gram_rows_kernel<4, false, true> : (const void*)gram_rows_kernel<4, false, false>);
+    if (R == 8) return full ? (median ? (const void*)gram_rows_kernel<8, true, true> : (const void*)gram_rows_kernel<8, true, false>)
+                            : (median ? (const void*)gram_rows_kernel<8, false, true> : (const void*)gram_rows_kernel<8, false, false>);
+    return full ? (median ? (const void*)gram_rows_kernel<16, true, true> : (const void*)gram_rows_kernel<16, true, false>)
+                : (median ? (const void*)gram_rows_kernel<16, false, true> : (const void*)gram_rows_kernel<16, false, false>);
+}
+
 GramGeometry gram_geometry(int n, int P, long long stride)
 {
     GramGeometry g;
@@ -981,10 +1012,11 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     static std::atomic<unsigned long long> attrs_set{0};
     if (device_needs_setup(attrs_set)) {
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<8>()));
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
-        BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_rows_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowsStages * rows_stage_bytes<16>()));
+        for (int r = 4; r <= 16; r *= 2)
+            for (int full = 0; full < 2; ++full)
+                for (int med = 0; med < 2; ++med)
+                    BTARD_CUDA_TRY(cudaFuncSetAttribute(rows_fn(r, full != 0, med != 0), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                        kRowsStages * rows_stage_bytes<16>()));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
         BTARD_CUDA_TRY(cudaFuncSetAttribute(gram_umma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWsSmem));
         mark_device_done(attrs_set);
@@ -1006,12 +1038,11 @@ int launch_gram(const GramLaunch& a, const GramGeometry& geo, cudaStream_t st)
     prof_begin(KIND_GRAM, st);
     if (a.n <= 16) {
         const int grid = a.P * geo.cpp;
-        if (a.n == 16) gram_rows_kernel<16, true><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<16>(), st>>>(ga);
-        else if (a.n > 8) gram_rows_kernel<16, false><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<16>(), st>>>(ga);
-        else if (a.n == 8) gram_rows_kernel<8, true><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<8>(), st>>>(ga);
-        else if (a.n > 4) gram_rows_kernel<8, false><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<8>(), st>>>(ga);
-        else if (a.n == 4) gram_rows_kernel<4, true><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<4>(), st>>>(ga);
-        else gram_rows_kernel<4, false><<<grid, kRowsThreads, kRowsStages * rows_stage_bytes<4>(), st>>>(ga);
+        const int R = (a.n <= 4) ? 4 : (a.n <= 8) ? 8 : 16;
+        const size_t smem = (size_t)kRowsStages * (R == 4 ? rows_stage_bytes<4>() : R == 8 ? rows_stage_bytes<8>() : rows_stage_bytes<16>());
+        void* args[] = {(void*)&ga};
+        const cudaError_t e = cudaLaunchKernel(rows_fn(R, a.n == R, a.fuse_median != 0), dim3((unsigned)grid), dim3(kRowsThreads), args, smem, st);
+        if (e != cudaSuccess) { set_cuda_error(e); prof_end(KIND_GRAM, st); return BTARD_ERR_CUDA; }
     }
     else if (geo.umma && a.n == 64) gram_umma_ws_kernel<true><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
     else if (geo.umma) gram_umma_ws_kernel<false><<<a.P * geo.cpp, kWsThreads, kWsSmem, st>>>(ga, a.error, map);
