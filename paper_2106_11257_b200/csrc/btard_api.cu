@@ -159,10 +159,11 @@ VerifyWorkspace verify_ws_layout(int n, int P, long long stride, int K, const Ge
 {
     const VerifyGeometry plain = verify_geometry(n, P, stride, K, false), fused = verify_geometry(n, P, stride, K, true);
     const size_t ctas = (size_t)(plain.g.cpp > fused.g.cpp ? plain.g.cpp : fused.g.cpp);
+    const size_t slots = (size_t)(plain.slots > fused.slots ? plain.slots : fused.slots);
     VerifyWorkspace w;
     size_t off = 0;
     w.table = off; off = align_up(off + sizeof(PartEntry) * P, 256);
-    w.part = off; off = align_up(off + sizeof(double) * (size_t)P * ctas * plain.slots, 256);
+    w.part = off; off = align_up(off + sizeof(double) * (size_t)P * ctas * slots, 256);
     w.norms = off; off = align_up(off + sizeof(double) * (size_t)P * n, 256);
     w.cslots = off; off = align_up(off + sizeof(double) * (size_t)P * cg.cpp * (n + 1), 256);
     w.ctot = off; off = align_up(off + sizeof(double) * (size_t)P * (n + 1), 256);

@@ -184,7 +184,7 @@ struct VerifyLaunch {
     int n, P, K, k0, kc;      // this launch covers z indices k0 .. k0+kc-1
     int p_base;
     uint32_t seed_lo, seed_hi;
-    // Fused with the combine pass of the Gram variant (n <= 16, K <= 2 only): v holds v0 on entry and
+    // Fused with the combine pass of the Gram variant: v holds v0 on entry and
     // receives v = v0 + sum_j coef_j (x_j - v0); the norms come out of this pass (norm_in is not read).
     int combine;
     float* v_out;                 // == v
@@ -212,7 +212,7 @@ struct VerifyGeometry {
     Geometry g;
     int KT;      // z vectors per launch (compile-time choice)
     int slots;   // doubles per CTA in part_out
-    int own_z;   // n <= 16 and K <= 2: each thread draws the z of its own columns (verify_rows_kernel)
+    int own_z;   // n <= 16: each thread draws the z of its own columns (verify_rows_kernel)
 };
 
 // fused: the pass also carries the combine step of the Gram variant (its kernel may hold fewer CTAs per SM)

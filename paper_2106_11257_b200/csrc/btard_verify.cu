@@ -2,11 +2,13 @@
 // [P][n][row_stride] tensor produces, per partition, the projections <g_i - v, z_k> on K random
 // directions, ||z_k||^2, and the clipped-residual sum sum_i w_i (g_i - v) with its norm.
 //
-// z is generated on the fly: the CTA's threads share the Philox/Box-Muller work of a
-// [K][tile columns] block of z, stage it in shared memory (double buffered), and every thread then
-// multiplies its R rows x 4 columns of residuals against it.  Per-thread accumulators are fp32 over
-// at most kMaxTilesPerCta tiles; everything that crosses threads is fp64, written to per-CTA slots
-// and summed in a fixed order by the finalize kernel.
+// z is generated on the fly, each quad once per launch.  Up to 16 peers a thread holds every row of
+// its 4 columns and draws their z itself (verify_rows_kernel); with more peers the CTA's threads
+// share the Philox/Box-Muller work of a [K][tile columns] block of z, stage it in shared memory
+// (three buffers), and every thread multiplies its R rows x 4 columns of residuals against it
+// (verify_kernel).  Per-thread accumulators are fp32 over at most kMaxTilesPerCta tiles; everything
+// that crosses threads is fp64, written to per-CTA slots and summed in a fixed order by the finalize
+// kernel.
 #include <type_traits>
 
 #include "btard_common.h"
@@ -398,27 +400,34 @@ __global__ void __launch_bounds__(MAXT, MINB) verify_kernel(const VArgs k)
     }
 }
 
-// n <= 16 and at most two directions per launch: one thread holds every row of its 4 columns (R >= n
+// n <= 16, up to eight directions per launch: one thread holds every row of its 4 columns (R >= n
 // rows x 4 columns in registers, as in the CenteredClip passes), so it draws the z quads of those
-// columns itself.  Each quad of z is still generated exactly once per launch, nothing is staged in
+// columns itself (measured against the shared-z kernel with 4 rows per thread, n = 16, d/P = 698 400,
+// P = 16: 0.32 against 0.36 ms at K = 4, 0.50 against 0.52 ms at K = 8; n = 4, K = 8: 0.23 against 0.28).  Each quad of z is still generated exactly once per launch, nothing is staged in
 // shared memory and the tile loop has no barrier.  Same per-CTA slot layout as verify_kernel.
 // COMBINE: the pass also forms v = v0 + sum_j a_j (x_j - v0) from the coefficients of the Gram variant
 // (the combine pass and the verification pass in one read of the rows): v holds v0 on entry, every
 // thread rewrites its own 4 columns, and the squared residual norms at the new v are one more set of
 // per-row sums (slot entries behind the others).  The clip weights that the clipped-residual sum needs
 // before the norms of this pass exist come from the Gram matrix: rho_i^2 = G_ii - 2 (G a)_i + a^T G a.
-template <int R, int KT, bool COMBINE>
-__global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
+// CTAs per SM by shape: the sums of 16 rows x 4 or 8 directions need the 255 registers of two CTAs of
+// 128 threads; smaller shapes run faster with three or four (measured, K = 4 and 8 at n = 4, 8, 16).
+constexpr int rows_min_ctas(int R, int KT)
+{
+    return (KT <= 2 || R == 16) ? 2 : (R == 8 && KT == 8) ? 3 : 4;
+}
+
+template <int R, int KT, bool COMBINE, int CL>
+__global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(const VArgs k)
 {
     __shared__ float sh_w[16];
     __shared__ float sh_c[16];                      // COMBINE: coefficients a_j
     __shared__ double sh_ga[17];                    // COMBINE: (G a)_i, then a^T G a
-    __shared__ double sh_red[8][R * KT + KT + 1 + (COMBINE ? R : 0)];
+    __shared__ double sh_red[CL / 32][R * KT + KT + 1 + (COMBINE ? R : 0)];
     __shared__ float sh_f[16];                      // row factors (with row_scale)
 
     const VerifyLaunch& a = k.a;
     const int n = a.n, cpp = k.cpp;
-    constexpr int CL = 256;
     const int tid = threadIdx.x;
     const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
     const bool scaled = a.row_scale != nullptr;     // rows enter as f_i x_i
@@ -503,20 +512,25 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
             for (int r = 0; r < R; ++r) x[r] = scale_row(x[r], sh_f[r]);
         }
         const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
-        // this thread's quads of z, drawn while the rows are on their way
-        float4 z[KT];
-#pragma unroll
-        for (int q = 0; q < KT; ++q) {
-            z[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        // this thread's quads of z: up to two are drawn while the rows are on their way, further ones
+        // one at a time between the sums below (registers)
+        constexpr int ZE = (KT <= 2) ? KT : 1;
+        const bool tail_quad = col + 3 >= len;         // only the last quad of a ragged partition
+        auto draw = [&](int q) {
+            float4 zq = make_float4(0.f, 0.f, 0.f, 0.f);
             if (q < a.kc && col < len) {
-                z[q] = z_quad((uint32_t)qb, pg, (uint32_t)(a.k0 + q), a.seed_lo, a.seed_hi);
-                if (col + 3 >= len) {                  // only the last quad of a ragged partition
-                    if (col + 1 >= len) z[q].y = 0.f;
-                    if (col + 2 >= len) z[q].z = 0.f;
-                    z[q].w = 0.f;
+                zq = z_quad((uint32_t)qb, pg, (uint32_t)(a.k0 + q), a.seed_lo, a.seed_hi);
+                if (tail_quad) {
+                    if (col + 1 >= len) zq.y = 0.f;
+                    if (col + 2 >= len) zq.z = 0.f;
+                    zq.w = 0.f;
                 }
             }
-        }
+            return zq;
+        };
+        float4 z[ZE];
+#pragma unroll
+        for (int q = 0; q < ZE; ++q) z[q] = draw(q);
         if (col + 3 < len) {                           // whole quad inside the data: no predicates
 #pragma unroll
             for (int r = 0; r < R; ++r) {
@@ -558,10 +572,11 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
         }
 #pragma unroll
         for (int q = 0; q < KT; ++q) {
-            zz[q] += fmaf(z[q].x, z[q].x, fmaf(z[q].y, z[q].y, fmaf(z[q].z, z[q].z, z[q].w * z[q].w)));
+            const float4 zq = (q < ZE) ? z[q] : draw(q);
+            zz[q] += fmaf(zq.x, zq.x, fmaf(zq.y, zq.y, fmaf(zq.z, zq.z, zq.w * zq.w)));
 #pragma unroll
             for (int r = 0; r < R; ++r)
-                acc[r][q] += fmaf(x[r].x, z[q].x, fmaf(x[r].y, z[q].y, fmaf(x[r].z, z[q].z, x[r].w * z[q].w)));
+                acc[r][q] = fmaf(x[r].x, zq.x, fmaf(x[r].y, zq.y, fmaf(x[r].z, zq.z, fmaf(x[r].w, zq.w, acc[r][q]))));
         }
         if (first_chunk) {                             // clipped-residual sum of these 4 columns
             float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -612,7 +627,7 @@ __global__ void __launch_bounds__(256, 2) verify_rows_kernel(const VArgs k)
     for (int e = tid; e < total; e += CL) {
         const int col = (e < n * KT) ? e : R * KT + (e - n * KT);
         double s = 0.0;
-        for (int u = 0; u < 8; ++u) s += sh_red[u][col];
+        for (int u = 0; u < CL / 32; ++u) s += sh_red[u][col];
         dst[e] = s;
     }
 }
@@ -727,11 +742,10 @@ __global__ void random_vector_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_
     *reinterpret_cast<float4*>(z + 4 * q) = v;
 }
 
-// Shapes and register budgets.  Up to 16 peers: 4 rows per thread in CTAs of at most 128 threads, three
-// to an SM (170 registers).  17 to 64 peers: 16 rows per thread in CTAs of 128 or 192 threads; with one
-// or two directions two or three CTAs share an SM (168 registers), with four the accumulators need the
-// whole file (255 registers, two CTAs of 128 threads).  More peers: one warp-wide lane per row group,
-// up to 512 threads.
+// Shapes and register budgets of the shared-z kernel.  17 to 64 peers: 16 rows per thread in CTAs of
+// 128 or 192 threads; with one or two directions two or three CTAs share an SM (168 registers), with
+// four the accumulators need the whole file (255 registers, two CTAs of 128 threads).  More peers: one
+// warp-wide lane per row group, up to 512 threads.
 template <int R, int KT, int MAXT, int MINB>
 const void* verify_fn_of(bool combine)
 {
@@ -740,12 +754,7 @@ const void* verify_fn_of(bool combine)
 
 const void* verify_fn(int R, int KT, bool combine, int threads)
 {
-    if (R == 4) {
-        if (KT == 1) return verify_fn_of<4, 1, 128, 3>(combine);
-        if (KT == 2) return verify_fn_of<4, 2, 128, 3>(combine);
-        if (KT == 4) return verify_fn_of<4, 4, 128, 3>(combine);
-        if (KT == 8) return verify_fn_of<4, 8, 128, 3>(combine);
-    } else if (R == 16 && threads <= 192) {
+    if (R == 16 && threads <= 192) {
         if (KT == 1) return verify_fn_of<16, 1, 192, 2>(combine);
         if (KT == 2) return verify_fn_of<16, 2, 192, 2>(combine);
         // four directions: 168 registers hold the plain pass (three CTAs of 128 threads per SM); fused with
@@ -767,8 +776,7 @@ void ensure_verify_attrs()
 {
     static std::atomic<unsigned long long> attrs_set{0};
     if (!device_needs_setup(attrs_set)) return;
-    const int shapes[][3] = {{4, 1, 128}, {4, 2, 128}, {4, 4, 128}, {4, 8, 128}, {16, 1, 128}, {16, 2, 128},
-                             {16, 4, 128}, {16, 1, 512}, {16, 2, 512}};
+    const int shapes[][3] = {{16, 1, 128}, {16, 2, 128}, {16, 4, 128}, {16, 1, 512}, {16, 2, 512}};
     for (const auto& sh : shapes)
         for (int combine = 0; combine < 2; ++combine)
             (void)cudaFuncSetAttribute(verify_fn(sh[0], sh[1], combine != 0, sh[2]),
@@ -789,34 +797,42 @@ int verify_ctas_per_sm(int R, int KT, bool combine, int threads, size_t smem)
     return nb;
 }
 
-template <int R>
-int launch_rows_r(const VArgs& va, int KT, int grid, cudaStream_t st)
+// One thread per 4 columns with every row: 256 threads for one or two directions (128 registers), 128
+// threads for four or eight, whose sums need most of the register file.
+inline int rows_threads(int KT) { return KT <= 2 ? 256 : 128; }
+
+template <int R, int KT>
+const void* rows_fn_of(bool combine)
 {
-    prof_begin(KIND_VERIFY, st);
-    if (va.a.combine) {
-        if (KT == 1) verify_rows_kernel<R, 1, true><<<grid, 256, 0, st>>>(va);
-        else verify_rows_kernel<R, 2, true><<<grid, 256, 0, st>>>(va);
-    } else {
-        if (KT == 1) verify_rows_kernel<R, 1, false><<<grid, 256, 0, st>>>(va);
-        else verify_rows_kernel<R, 2, false><<<grid, 256, 0, st>>>(va);
-    }
-    prof_end(KIND_VERIFY, st);
-    BTARD_CUDA_TRY(cudaGetLastError());
-    count_launch();
-    return BTARD_OK;
+    constexpr int CL = (KT <= 2) ? 256 : 128;
+    return combine ? (const void*)verify_rows_kernel<R, KT, true, CL> : (const void*)verify_rows_kernel<R, KT, false, CL>;
 }
 
-int rows_ctas_per_sm(int R, int KT)
+template <int R>
+const void* rows_fn_r(int KT, bool combine)
+{
+    switch (KT) {
+        case 1: return rows_fn_of<R, 1>(combine);
+        case 2: return rows_fn_of<R, 2>(combine);
+        case 4: return rows_fn_of<R, 4>(combine);
+        case 8: return rows_fn_of<R, 8>(combine);
+        default: return nullptr;
+    }
+}
+
+const void* rows_fn(int R, int KT, bool combine)
+{
+    return (R == 4) ? rows_fn_r<4>(KT, combine) : (R == 8) ? rows_fn_r<8>(KT, combine) : rows_fn_r<16>(KT, combine);
+}
+
+int rows_ctas_per_sm(int R, int KT, bool combine)
 {
     int nb = 0;
-    cudaError_t e;
-    if (R == 4) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 1, false>, 256, 0)
-                              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<4, 2, false>, 256, 0);
-    else if (R == 8) e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 1, false>, 256, 0)
-                                   : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<8, 2, false>, 256, 0);
-    else e = (KT == 1) ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 1, false>, 256, 0)
-                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_rows_kernel<16, 2, false>, 256, 0);
-    if (e != cudaSuccess || nb < 1) { (void)cudaGetLastError(); return 2; }
+    const void* fn = rows_fn(R, KT, combine);
+    if (!fn || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, rows_threads(KT), 0) != cudaSuccess || nb < 1) {
+        (void)cudaGetLastError();
+        return 2;
+    }
     return nb;
 }
 
@@ -826,34 +842,29 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K, bool fused
 {
     VerifyGeometry vg;
     Geometry& g = vg.g;
-    vg.own_z = (n <= 16 && K <= 2) ? 1 : 0;
-    if (vg.own_z) {                  // every row of a column in one thread: z drawn in registers
-        g.R = (n <= 4) ? 4 : (n <= 8) ? 8 : 16;
-        g.RG = 1;
-        g.CL = 256;
-        g.threads = 256;
-        vg.KT = K;
-        g.slots = sm_count() * rows_ctas_per_sm(g.R, K);
-        g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, g.slots);
-        vg.slots = n * K + K + 1 + n;      // room for the squared norms of the fused combine pass
-        return vg;
-    }
     int kt = 1;
     while (kt < K && kt < 8) kt <<= 1;
-    if (n <= 16) {                // more than two directions: 4 rows per thread, CTAs of about 128 threads
-        g.R = 4;
-        g.RG = (n + 3) / 4;
-        g.CL = (g.RG == 1) ? 128 : (g.RG == 2) ? 64 : 32;
-    } else {
-        // 16 rows per thread: few row groups exchange column sums, and the per-tile bookkeeping of a thread
-        // is spread over 64 elements (measured at n = 64, K = 4: 14.5 thread instructions per element against
-        // 23.5 with 8 rows per thread)
-        g.R = 16;
-        g.RG = (n + 15) / 16;
-        g.CL = (g.RG == 2 || g.RG == 3) ? 64 : 32;
-        if (kt > 4) kt = 4;                   // the accumulators of 4 directions are all the registers hold
-        if (g.RG > 4 && kt > 2) kt = 2;       // more than 256 threads: 128 registers per thread
+    vg.own_z = (n <= 16) ? 1 : 0;
+    if (vg.own_z) {                  // every row of a column in one thread: z drawn in registers
+        g.R = (n <= 4) ? 4 : (n <= 8) ? 8 : 16;
+        if (g.R == 16 && fused && kt > 4) kt = 4;      // 16 rows x 8 directions + the combine pass: 2 KB of spills
+        g.RG = 1;
+        g.CL = rows_threads(kt);
+        g.threads = g.CL;
+        vg.KT = kt;
+        g.slots = sm_count() * rows_ctas_per_sm(g.R, kt, fused);
+        g.cpp = choose_ctas_per_partition(P, stride >> 2, g.CL, g.slots);
+        vg.slots = n * kt + kt + 1 + n;    // room for the squared norms of the fused combine pass
+        return vg;
     }
+    // 16 rows per thread: few row groups exchange column sums, and the per-tile bookkeeping of a thread
+    // is spread over 64 elements (measured at n = 64, K = 4: 14.5 thread instructions per element against
+    // 23.5 with 8 rows per thread)
+    g.R = 16;
+    g.RG = (n + 15) / 16;
+    g.CL = (g.RG == 2 || g.RG == 3) ? 64 : 32;
+    if (kt > 4) kt = 4;                   // the accumulators of 4 directions are all the registers hold
+    if (g.RG > 4 && kt > 2) kt = 2;       // more than 256 threads: 128 registers per thread
     g.threads = g.RG * g.CL;
     vg.KT = kt;
     const size_t smem = sizeof(float4) * (3 * (size_t)kt * g.CL + 2 * (size_t)g.RG * g.CL);
@@ -874,18 +885,13 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
     if (smem > (size_t)kVerifyMaxSmem) return BTARD_ERR_UNSUPPORTED;
     ensure_verify_attrs();
     int rc;
-    if (vg.own_z) {
-        switch (g.R) {
-            case 4: rc = launch_rows_r<4>(va, vg.KT, grid, st); break;
-            case 8: rc = launch_rows_r<8>(va, vg.KT, grid, st); break;
-            default: rc = launch_rows_r<16>(va, vg.KT, grid, st); break;
-        }
-    } else {
-        const void* fn = verify_fn(g.R, vg.KT, a.combine != 0, g.threads);
+    {
+        const void* fn = vg.own_z ? rows_fn(g.R, vg.KT, a.combine != 0) : verify_fn(g.R, vg.KT, a.combine != 0, g.threads);
         if (!fn) return BTARD_ERR_UNSUPPORTED;
         void* args[] = {(void*)&va};
         prof_begin(KIND_VERIFY, st);
-        const cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)grid), dim3((unsigned)g.threads), args, smem, st);
+        const cudaError_t e = cudaLaunchKernel(fn, dim3((unsigned)grid), dim3((unsigned)g.threads), args,
+                                               vg.own_z ? 0 : smem, st);
         prof_end(KIND_VERIFY, st);
         BTARD_CUDA_TRY(e);
         count_launch();
