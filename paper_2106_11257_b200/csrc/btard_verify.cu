@@ -500,7 +500,13 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
     const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
     const uint32_t pg = (uint32_t)(a.p_base + p);
 
-    for (long long qb = q0 + tid; qb < q1; qb += CL) {
+    // a row with weight 0 or coefficient 0 (a non-finite row) is left out of the sums, not multiplied
+    bool any_skip = false;
+    for (int r = 0; r < n; ++r) any_skip |= (sh_w[r] == 0.0f) || (COMBINE && sh_c[r] == 0.0f);
+
+    // GUARD: the quad reaches past the partition's length, or some row has to be left out
+    auto tile = [&](auto guard_tag, long long qb) {
+        constexpr bool GUARD = decltype(guard_tag)::value;
         const long long col = qb * 4;
         float4 x[R];
 #pragma unroll
@@ -515,14 +521,15 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
         // this thread's quads of z: up to two are drawn while the rows are on their way, further ones
         // one at a time between the sums below (registers)
         constexpr int ZE = (KT <= 2) ? KT : 1;
-        const bool tail_quad = col + 3 >= len;         // only the last quad of a ragged partition
+        const bool m0 = !GUARD || col < len, m1 = !GUARD || col + 1 < len, m2 = !GUARD || col + 2 < len,
+                   m3 = !GUARD || col + 3 < len;
         auto draw = [&](int q) {
             float4 zq = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (q < a.kc && col < len) {
+            if (q < a.kc && m0) {
                 zq = z_quad((uint32_t)qb, pg, (uint32_t)(a.k0 + q), a.seed_lo, a.seed_hi);
-                if (tail_quad) {
-                    if (col + 1 >= len) zq.y = 0.f;
-                    if (col + 2 >= len) zq.z = 0.f;
+                if (GUARD && !m3) {                    // only the last quad of a ragged partition
+                    if (!m1) zq.y = 0.f;
+                    if (!m2) zq.z = 0.f;
                     zq.w = 0.f;
                 }
             }
@@ -531,20 +538,12 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
         float4 z[ZE];
 #pragma unroll
         for (int q = 0; q < ZE; ++q) z[q] = draw(q);
-        if (col + 3 < len) {                           // whole quad inside the data: no predicates
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                x[r].x -= v4.x; x[r].y -= v4.y; x[r].z -= v4.z; x[r].w -= v4.w;
-            }
-        } else {
-            const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                x[r].x = m0 ? x[r].x - v4.x : 0.f;
-                x[r].y = m1 ? x[r].y - v4.y : 0.f;
-                x[r].z = m2 ? x[r].z - v4.z : 0.f;
-                x[r].w = 0.f;
-            }
+        for (int r = 0; r < R; ++r) {
+            x[r].x = m0 ? x[r].x - v4.x : 0.f;
+            x[r].y = m1 ? x[r].y - v4.y : 0.f;
+            x[r].z = m2 ? x[r].z - v4.z : 0.f;
+            x[r].w = m3 ? x[r].w - v4.w : 0.f;
         }
         if (COMBINE) {
             // x holds the residuals at v0: move v by u = sum_j a_j (x_j - v0), then the residuals by what v
@@ -553,14 +552,13 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const float cr = sh_c[r];
-                if (cr != 0.0f) {                      // coefficient 0: the row is left out, not multiplied
+                if (!GUARD || cr != 0.0f) {
                     u.x = fmaf(cr, x[r].x, u.x); u.y = fmaf(cr, x[r].y, u.y);
                     u.z = fmaf(cr, x[r].z, u.z); u.w = fmaf(cr, x[r].w, u.w);
                 }
             }
             const float4 vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
             const float4 dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
-            const bool m0 = col < len, m1 = col + 1 < len, m2 = col + 2 < len, m3 = col + 3 < len;
             *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) =
                 make_float4(m0 ? vn.x : 0.f, m1 ? vn.y : 0.f, m2 ? vn.z : 0.f, m3 ? vn.w : 0.f);
 #pragma unroll
@@ -583,7 +581,7 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const float wr = sh_w[r];
-                if (wr != 0.0f) {                      // weight 0: the row is left out, not multiplied
+                if (!GUARD || wr != 0.0f) {
                     s4.x = fmaf(wr, x[r].x, s4.x);
                     s4.y = fmaf(wr, x[r].y, s4.y);
                     s4.z = fmaf(wr, x[r].z, s4.z);
@@ -593,6 +591,10 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
             rs2 += fmaf(s4.x, s4.x, fmaf(s4.y, s4.y, fmaf(s4.z, s4.z, s4.w * s4.w)));
             if (rsp) *reinterpret_cast<float4*>(rsp + col) = s4;
         }
+    };
+    for (long long qb = q0 + tid; qb < q1; qb += CL) {
+        if (!any_skip && qb * 4 + 3 < len) tile(std::false_type{}, qb);
+        else tile(std::true_type{}, qb);
     }
 
     // CTA reduction
@@ -805,7 +807,11 @@ template <int R, int KT>
 const void* rows_fn_of(bool combine)
 {
     constexpr int CL = (KT <= 2) ? 256 : 128;
-    return combine ? (const void*)verify_rows_kernel<R, KT, true, CL> : (const void*)verify_rows_kernel<R, KT, false, CL>;
+    if constexpr (R == 16 && KT == 8) {                // fused with the combine pass this shape spills 2 KB: not built
+        return combine ? nullptr : (const void*)verify_rows_kernel<R, KT, false, CL>;
+    } else {
+        return combine ? (const void*)verify_rows_kernel<R, KT, true, CL> : (const void*)verify_rows_kernel<R, KT, false, CL>;
+    }
 }
 
 template <int R>
