@@ -919,8 +919,12 @@ __device__ __forceinline__ float key_value(uint32_t key)
 
 // One thread takes the median of the n values of one column.  EXACT: n == N2 is known at compile
 // time (the two middle outputs are fixed registers and the network is pruned to them); otherwise
-// the column is padded to N2 inputs with the largest key and the middle is picked at run time.
-template <int N2, bool EXACT>
+// the column is padded to N2 inputs with the largest value and the middle is picked at run time.
+// The kernel is bound by the pipe that executes minimum and maximum, so everything else is kept off
+// it: a column whose sum is not NaN holds no NaN and is sorted as floats (no key per input; the sum is
+// 64 additions on the other pipe), and with NARROW (row pitch x rows below 4 GiB) the address of row i
+// is one wide multiply-add, base + i * pitch, on the multiplier instead of 64-bit additions.
+template <int N2, bool EXACT, bool NARROW>
 __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float* v,
                                                           const PartEntry* table, const double* row_scale,
                                                           long long stride, int n)
@@ -937,23 +941,49 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
     float out = 0.0f;
     if (c < len) {
         const float* gp = g + (size_t)p * n * stride + c;
-        int key[N2];
-        if (row_scale) {                               // rows enter as f_i x_i (a factor of 0 reads as zeros)
+        const uint32_t pitch = (uint32_t)(stride * 4);     // bytes between rows (NARROW only)
+        auto row = [&](int i) {
+            if (NARROW) {
+                uint64_t at;
+                asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(at) : "r"((uint32_t)i), "r"(pitch), "l"(gp));
+                return __ldcs(reinterpret_cast<const float*>(at));
+            }
+            return __ldcs(gp + (size_t)i * stride);
+        };
+        float x[N2];
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+        const float inf = __int_as_float(0x7f800000);      // unused inputs: +infinity
+        if (row_scale) {                                   // rows enter as f_i x_i (a factor of 0 reads as zeros)
 #pragma unroll
             for (int i = 0; i < N2; ++i) {
-                float x = 0.0f;
+                float xi = inf;
                 if (EXACT || i < n) {
                     const float f = sh_f[i];
-                    x = (f == 0.0f) ? 0.0f : f * __ldcs(gp + (size_t)i * stride);
+                    xi = (f == 0.0f) ? 0.0f : f * row(i);
+                    sum[i & 3] += xi;
                 }
-                key[i] = (EXACT || i < n) ? signed_key(x) : 0x7fffffff;
+                x[i] = xi;
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < N2; ++i)
-                key[i] = (EXACT || i < n) ? signed_key(__ldcs(gp + (size_t)i * stride)) : 0x7fffffff;
+            for (int i = 0; i < N2; ++i) {
+                float xi = inf;
+                if (EXACT || i < n) {
+                    xi = row(i);
+                    sum[i & 3] += xi;
+                }
+                x[i] = xi;
+            }
         }
-        out = median_of_keys<N2, EXACT>(key, n);
+        const float total = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        if (total == total) {                              // no NaN in the column (nor +inf beside -inf)
+            out = median_of_values<N2, EXACT>(x, n);
+        } else {
+            int key[N2];
+#pragma unroll
+            for (int i = 0; i < N2; ++i) key[i] = (EXACT || i < n) ? signed_key(x[i]) : 0x7fffffff;
+            out = median_of_keys<N2, EXACT>(key, n);
+        }
     }
     v[(size_t)p * stride + c] = out;
 }
@@ -1170,19 +1200,26 @@ int launch_median_init(const float* g, float* v, const PartEntry* table, const d
     const int threads = 128;
     dim3 grid((unsigned)((stride + threads - 1) / threads), (unsigned)P);
     prof_begin(KIND_MEDIAN, st);
-    if (n == 1) median_sort_kernel<1, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n == 2) median_sort_kernel<2, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n == 4) median_sort_kernel<4, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n == 8) median_sort_kernel<8, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n == 16) median_sort_kernel<16, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n == 32) median_sort_kernel<32, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n == 64) median_sort_kernel<64, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n < 4) median_sort_kernel<4, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n < 8) median_sort_kernel<8, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n < 16) median_sort_kernel<16, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n < 32) median_sort_kernel<32, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
-    else if (n < 64) median_sort_kernel<64, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+    const bool narrow = stride * 4 * (long long)(n > 1 ? n : 1) < (1LL << 32);
+#define BTARD_MEDIAN(N2, EX)                                                                              \
+    do {                                                                                                  \
+        if (narrow) median_sort_kernel<N2, EX, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);  \
+        else median_sort_kernel<N2, EX, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);        \
+    } while (0)
+    if (n == 1) BTARD_MEDIAN(1, true);
+    else if (n == 2) BTARD_MEDIAN(2, true);
+    else if (n == 4) BTARD_MEDIAN(4, true);
+    else if (n == 8) BTARD_MEDIAN(8, true);
+    else if (n == 16) BTARD_MEDIAN(16, true);
+    else if (n == 32) BTARD_MEDIAN(32, true);
+    else if (n == 64) BTARD_MEDIAN(64, true);
+    else if (n < 4) BTARD_MEDIAN(4, false);
+    else if (n < 8) BTARD_MEDIAN(8, false);
+    else if (n < 16) BTARD_MEDIAN(16, false);
+    else if (n < 32) BTARD_MEDIAN(32, false);
+    else if (n < 64) BTARD_MEDIAN(64, false);
     else median_rank_kernel<<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);
+#undef BTARD_MEDIAN
     prof_end(KIND_MEDIAN, st);
     BTARD_CUDA_TRY(cudaGetLastError());
     count_launch();
