@@ -923,11 +923,13 @@ __device__ __forceinline__ float key_value(uint32_t key)
 // The kernel is bound by the pipe that executes minimum and maximum, so everything else is kept off
 // it: a column whose sum is not NaN holds no NaN and is sorted as floats (no key per input; the sum is
 // 64 additions on the other pipe), and with NARROW (row pitch x rows below 4 GiB) the address of row i
-// is one wide multiply-add, base + i * pitch, on the multiplier instead of 64-bit additions.
-template <int N2, bool EXACT, bool NARROW>
-__global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float* v,
-                                                          const PartEntry* table, const double* row_scale,
-                                                          long long stride, int n)
+// is one wide multiply-add, base + i * pitch, on the multiplier instead of 64-bit additions.  CW = 2
+// (exactly 32 or 64 rows): a thread loads two neighbouring columns per row with one address and sorts
+// them one after the other.
+template <int N2, bool EXACT, bool NARROW, int CW>
+__global__ void __launch_bounds__(128, CW == 2 ? 3 : 1) median_sort_kernel(const float* g, float* v,
+                                                                           const PartEntry* table, const double* row_scale,
+                                                                           long long stride, int n)
 {
     __shared__ float sh_f[N2];                         // row factors (with row_scale)
     const int p = blockIdx.y;
@@ -935,57 +937,75 @@ __global__ void __launch_bounds__(128) median_sort_kernel(const float* g, float*
         if (threadIdx.x < N2) sh_f[threadIdx.x] = ((int)threadIdx.x < n) ? (float)row_scale[(size_t)p * n + threadIdx.x] : 0.0f;
         __syncthreads();
     }
-    const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long c = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * CW;
     if (c >= stride) return;
     const long long len = table[p].len;
-    float out = 0.0f;
+    float out[CW];
+#pragma unroll
+    for (int w = 0; w < CW; ++w) out[w] = 0.0f;
     if (c < len) {
         const float* gp = g + (size_t)p * n * stride + c;
         const uint32_t pitch = (uint32_t)(stride * 4);     // bytes between rows (NARROW only)
-        auto row = [&](int i) {
+        auto row = [&](int i, float (&o)[CW]) {
+            const float* at = gp + (size_t)i * stride;
             if (NARROW) {
-                uint64_t at;
-                asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(at) : "r"((uint32_t)i), "r"(pitch), "l"(gp));
-                return __ldcs(reinterpret_cast<const float*>(at));
+                uint64_t a64;
+                asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(a64) : "r"((uint32_t)i), "r"(pitch), "l"(gp));
+                at = reinterpret_cast<const float*>(a64);
             }
-            return __ldcs(gp + (size_t)i * stride);
+            if constexpr (CW == 2) {
+                const float2 t = __ldcs(reinterpret_cast<const float2*>(at));
+                o[0] = t.x; o[1] = t.y;
+            } else {
+                o[0] = __ldcs(at);
+            }
         };
-        float x[N2];
-        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+        float x[CW][N2];
+        float sum[CW][2];
+#pragma unroll
+        for (int w = 0; w < CW; ++w) sum[w][0] = sum[w][1] = 0.f;
         const float inf = __int_as_float(0x7f800000);      // unused inputs: +infinity
+#pragma unroll
+        for (int i = 0; i < N2; ++i) {
+            float xi[CW];
+#pragma unroll
+            for (int w = 0; w < CW; ++w) xi[w] = inf;
+            if (EXACT || i < n) row(i, xi);
+#pragma unroll
+            for (int w = 0; w < CW; ++w) x[w][i] = xi[w];
+        }
         if (row_scale) {                                   // rows enter as f_i x_i (a factor of 0 reads as zeros)
 #pragma unroll
             for (int i = 0; i < N2; ++i) {
-                float xi = inf;
                 if (EXACT || i < n) {
                     const float f = sh_f[i];
-                    xi = (f == 0.0f) ? 0.0f : f * row(i);
-                    sum[i & 3] += xi;
-                }
-                x[i] = xi;
-            }
-        } else {
 #pragma unroll
-            for (int i = 0; i < N2; ++i) {
-                float xi = inf;
-                if (EXACT || i < n) {
-                    xi = row(i);
-                    sum[i & 3] += xi;
+                    for (int w = 0; w < CW; ++w) x[w][i] = (f == 0.0f) ? 0.0f : f * x[w][i];
                 }
-                x[i] = xi;
             }
         }
-        const float total = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-        if (total == total) {                              // no NaN in the column (nor +inf beside -inf)
-            out = median_of_values<N2, EXACT>(x, n);
-        } else {
-            int key[N2];
 #pragma unroll
-            for (int i = 0; i < N2; ++i) key[i] = (EXACT || i < n) ? signed_key(x[i]) : 0x7fffffff;
-            out = median_of_keys<N2, EXACT>(key, n);
+        for (int i = 0; i < N2; ++i)
+            if (EXACT || i < n) {
+#pragma unroll
+                for (int w = 0; w < CW; ++w) sum[w][i & 1] += x[w][i];
+            }
+#pragma unroll
+        for (int w = 0; w < CW; ++w) {
+            if (w > 0 && c + w >= len) break;
+            const float total = sum[w][0] + sum[w][1];
+            if (total == total) {                          // no NaN in the column (nor +inf beside -inf)
+                out[w] = median_of_values<N2, EXACT>(x[w], n);
+            } else {
+                int key[N2];
+#pragma unroll
+                for (int i = 0; i < N2; ++i) key[i] = (EXACT || i < n) ? signed_key(x[w][i]) : 0x7fffffff;
+                out[w] = median_of_keys<N2, EXACT>(key, n);
+            }
         }
     }
-    v[(size_t)p * stride + c] = out;
+    if constexpr (CW == 2) *reinterpret_cast<float2*>(v + (size_t)p * stride + c) = make_float2(out[0], out[1]);
+    else v[(size_t)p * stride + c] = out[0];
 }
 
 // Any n: rank every value by counting (O(n^2) compares per column), pick the two middle ranks.
@@ -1198,13 +1218,15 @@ int launch_median_init(const float* g, float* v, const PartEntry* table, const d
                        long long stride, int n, int P, cudaStream_t st)
 {
     const int threads = 128;
-    dim3 grid((unsigned)((stride + threads - 1) / threads), (unsigned)P);
+    const int cw = (n == 32 || n == 64) ? 2 : 1;       // two columns per thread: one address per row and pair
+    dim3 grid((unsigned)((stride / cw + threads - 1) / threads), (unsigned)P);
     prof_begin(KIND_MEDIAN, st);
     const bool narrow = stride * 4 * (long long)(n > 1 ? n : 1) < (1LL << 32);
 #define BTARD_MEDIAN(N2, EX)                                                                              \
     do {                                                                                                  \
-        if (narrow) median_sort_kernel<N2, EX, true><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);  \
-        else median_sort_kernel<N2, EX, false><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);        \
+        constexpr int CW = (N2 > 16 && EX) ? 2 : 1;                                                           \
+        if (narrow) median_sort_kernel<N2, EX, true, CW><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);  \
+        else median_sort_kernel<N2, EX, false, CW><<<grid, threads, 0, st>>>(g, v, table, row_scale, stride, n);        \
     } while (0)
     if (n == 1) BTARD_MEDIAN(1, true);
     else if (n == 2) BTARD_MEDIAN(2, true);
