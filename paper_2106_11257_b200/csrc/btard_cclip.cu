@@ -907,9 +907,8 @@ __global__ void totals_to_norms_kernel(const double* tot, double* norm, int n)
 
 // ---- coordinate-wise median start ---------------------------------------------------------------
 // Order-preserving map of float bit patterns to unsigned integers (IEEE total order).
-__device__ __forceinline__ uint32_t order_key(float f)
+__device__ __forceinline__ uint32_t order_key_bits(uint32_t u)
 {
-    const uint32_t u = __float_as_uint(f);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 __device__ __forceinline__ float key_value(uint32_t key)
@@ -980,7 +979,10 @@ __global__ void __launch_bounds__(128, CW == 2 ? 3 : 1) median_sort_kernel(const
                 if (EXACT || i < n) {
                     const float f = sh_f[i];
 #pragma unroll
-                    for (int w = 0; w < CW; ++w) x[w][i] = (f == 0.0f) ? 0.0f : f * x[w][i];
+                    for (int w = 0; w < CW; ++w) {     // a NaN keeps its own bits (its sign places it in the order)
+                        const float xi = x[w][i];
+                        x[w][i] = (f == 0.0f) ? 0.0f : (xi == xi) ? f * xi : xi;
+                    }
                 }
             }
         }
@@ -1018,21 +1020,26 @@ __global__ void median_rank_kernel(const float* g, float* v, const PartEntry* ta
     const long long len = table[p].len;
     float out = 0.0f;
     if (c < len) {
-        const float* gp = g + (size_t)p * n * stride + c;
+        // The rows are read as bit patterns: the key of a NaN depends on its sign bit, which a floating-point
+        // move or product need not keep (with float loads here the key of a positive NaN came out as that of -0).
+        const uint32_t* gp = reinterpret_cast<const uint32_t*>(g) + (size_t)p * n * stride + c;
         const int ia = (n - 1) >> 1, ib = n >> 1;
         uint32_t ka = 0, kb = 0;
         const double* fp = row_scale ? row_scale + (size_t)p * n : nullptr;
-        auto value = [&](int i) {                      // row i as it enters: f_i x_i (a factor of 0 reads as zeros)
-            const float x = gp[(size_t)i * stride];
-            if (!fp) return x;
-            const float f = (float)fp[i];
-            return (f == 0.0f) ? 0.0f : f * x;
+        auto key_of = [&](int i) {                     // row i as it enters: f_i x_i (a factor of 0 reads as zeros)
+            const uint32_t bits = gp[(size_t)i * stride];
+            if (fp) {
+                const float f = (float)fp[i], x = __uint_as_float(bits);
+                if (f == 0.0f) return order_key_bits(0u);
+                if (x == x) return order_key_bits(__float_as_uint(f * x));   // a NaN keeps its own bits
+            }
+            return order_key_bits(bits);
         };
         for (int i = 0; i < n; ++i) {
-            const uint32_t ki = order_key(value(i));
+            const uint32_t ki = key_of(i);
             int rank = 0;
             for (int q = 0; q < n; ++q) {
-                const uint32_t kq = order_key(value(q));
+                const uint32_t kq = key_of(q);
                 rank += (kq < ki) || (kq == ki && q < i);
             }
             if (rank == ia) ka = ki;

@@ -90,11 +90,13 @@ struct CclipLaunch {
     const double* row_scale;  // device [P][n] factor applied to row i on load, or nullptr
 };
 
-// x scaled by a row factor; a factor of exactly 0 drops the row whatever it holds.
+// x scaled by a row factor; a factor of exactly 0 drops the row whatever it holds.  A NaN keeps its own
+// bits: its sign decides at which end of a column's order it sits (coordinate median).
+__device__ __forceinline__ float scale_value(float x, float f) { return (x == x) ? x * f : x; }
 __device__ __forceinline__ float4 scale_row(float4 x, float f)
 {
     if (f == 0.0f) return make_float4(0.f, 0.f, 0.f, 0.f);
-    return make_float4(x.x * f, x.y * f, x.z * f, x.w * f);
+    return make_float4(scale_value(x.x, f), scale_value(x.y, f), scale_value(x.z, f), scale_value(x.w, f));
 }
 
 Geometry cclip_geometry(int n, int P, long long stride);

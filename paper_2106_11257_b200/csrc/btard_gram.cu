@@ -289,8 +289,8 @@ __global__ void __launch_bounds__(kRowsThreads, 1) gram_rows_kernel(const GArgs 
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const float f = sh_f[r];
-                x[r].x = (f == 0.0f) ? 0.0f : f * x[r].x;
-                x[r].y = (f == 0.0f) ? 0.0f : f * x[r].y;
+                x[r].x = (f == 0.0f) ? 0.0f : scale_value(x[r].x, f);
+                x[r].y = (f == 0.0f) ? 0.0f : scale_value(x[r].y, f);
             }
         }
         if (MEDIAN) {

@@ -296,6 +296,48 @@ def test_mean_and_coordinate_median_rules_match_oracle(n):
         assert (cpu(r["iters"]) == 0).all()
 
 
+@pytest.mark.parametrize("n", [2, 5, 16, 32, 33, 64, 100])
+def test_coordinate_median_with_special_values_is_exact(n):
+    """The median kernel sorts a column as floats when its sum is not NaN and on integer keys otherwise:
+    columns with infinities of one or both signs, NaNs of both signs, zeros of both signs and ties must
+    come out as the oracle's, value for value (the sign of a zero aside)."""
+    rng = np.random.default_rng(900 + n)
+    P, stride = 2, 2048
+    lens = np.array([2048, 1999])
+    g = (rng.standard_normal((P, n, stride)) * 1e-2).astype(np.float32)
+    for p in range(P):
+        g[p, :, lens[p]:] = 0.0
+    rows = rng.integers(0, n, size=(P, 64))
+    for p in range(P):
+        for t in range(64):
+            c, r = 16 * t, rows[p, t]
+            kind = t % 8
+            if kind == 0: g[p, r, c] = np.inf
+            elif kind == 1: g[p, r, c] = -np.inf
+            elif kind == 2: g[p, r, c] = np.inf; g[p, (r + 1) % n, c] = -np.inf
+            elif kind == 3: g[p, r, c] = np.nan
+            elif kind == 4: g[p, r, c] = -np.nan; g[p, (r + 1) % n, c] = np.nan
+            elif kind == 5: g[p, :, c] = 0.0; g[p, r, c] = -0.0
+            elif kind == 6: g[p, :, c] = g[p, 0, c]
+            else: g[p, : (n + 1) // 2, c] = np.inf
+    scale = rng.uniform(0.5, 1.0, size=(P, n))
+    scale[0, n - 1] = 0.0                                # a dropped row
+    scale[1, 0] = 1.0
+    for rs in (None, scale):
+        ref = oracle.centered_clip(g, 1.0, lens, rule=oracle.RULE_COORD_MEDIAN, row_scale=rs)
+        _, r = run_gpu_cclip(g, 1.0, lens, rule=btard.RULE_COORD_MEDIAN,
+                             row_scale=None if rs is None else torch.from_numpy(rs).cuda())
+        v = cpu(r["v"])
+        for p in range(P):
+            a, b = v[p, : lens[p]] + np.float32(0.0), ref["v"][p, : lens[p]].astype(np.float32) + np.float32(0.0)
+            if rs is None:
+                assert np.array_equal(a, b, equal_nan=True), (p, np.nonzero(~((a == b) | (np.isnan(a) & np.isnan(b))))[0][:8])
+            else:                                        # the products f x are rounded to fp32 on the GPU only
+                fin = np.isfinite(b)
+                assert np.array_equal(np.isnan(a), np.isnan(b)) and np.array_equal(a[~fin & ~np.isnan(b)], b[~fin & ~np.isnan(b)])
+                assert np.all(np.abs(a[fin] - b[fin]) <= 2e-7 * np.abs(b[fin]) + 5e-9), p   # values are O(1e-2): one rounding of f x
+
+
 def test_geometric_median_rule_rejects_a_zero_floor_and_gram():
     g = torch.zeros((1, 4, 64), device="cuda")
     with pytest.raises(btard.BtardError):
