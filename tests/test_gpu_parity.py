@@ -192,7 +192,7 @@ def test_non_finite_rows_take_weight_zero(algo, stride):
     assert np.array_equal(np.isfinite(rn), np.isfinite(ref["resid_norm"]))
 
 
-@pytest.mark.parametrize("n", [5, 16, 40])
+@pytest.mark.parametrize("n", [5, 16, 40, 64, 100])
 def test_non_finite_rows_with_a_median_start(n):
     """A Byzantine row holding NaN / inf together with the coordinate-median start (the start every
     benchmark uses): the median orders NaNs at the ends, the row takes weight 0 in every update; direct,
