@@ -610,6 +610,50 @@ def test_one_call_aggregation_and_verification(n, K, algo):
     assert np.array_equal(cpu(rc["status"]), np.zeros(P, dtype=np.int32))
 
 
+@pytest.mark.parametrize("n,K", [(4, 1), (16, 2), (16, 8), (40, 4), (64, 1), (100, 2)])
+def test_nan_beyond_the_partition_length_is_never_data(n, K):
+    """Columns at and beyond part_len[p] are masked whatever they hold: here they hold NaN (also in the
+    caller's v0 and under row factors), the lengths end inside a quad of columns, and every path must give
+    the oracle's finite results: direct, cooperative, Gram, the verification and the one-call entry."""
+    rng = np.random.default_rng(700 + 3 * n + K)
+    P, stride = 3, 12_320
+    lens = np.array([12_317, 9_002, 5])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    for p in range(P):
+        g[p, :, lens[p]:] = np.nan
+    tau = np.array([0.5, 1.0, 2.0])
+    seed = 0xABCD00 + n
+    ref = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=6)
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE, btard.ALGO_GRAM):
+        _, r = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=6, algo=algo)
+        assert np.all(np.isfinite(cpu(r["v"]))), algo
+        check_cclip(r, ref, lens)
+        assert not cpu(r["status"]).any()
+    v0 = rng.standard_normal((P, stride)).astype(np.float32)
+    for p in range(P):
+        v0[p, lens[p]:] = np.nan
+    ref0 = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_CALLER, v0=v0, max_iters=3)
+    _, r0 = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_CALLER_V0, v0=v0, max_iters=3)
+    check_cclip(r0, ref0, lens)
+    gd = torch.from_numpy(g).cuda()
+    for algo in (btard.ALGO_GRAM, btard.ALGO_DIRECT):
+        rc, rv = btard.centered_clip_verify(gd, tau, seed, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                            max_iters=6, algo=algo, want_resid_sum=True)
+        torch.cuda.synchronize()
+        check_cclip(rc, ref, lens)
+        v32 = cpu(rc["v"])
+        assert np.all(np.isfinite(v32))
+        refv = oracle.verify(g, v32, tau, seed, K=K, part_len=lens, want_resid_sum=True)
+        check_verify(rv, refv, K)
+        assert np.all(np.isfinite(cpu(rv["resid_sum"]))) and not cpu(rv["status"]).any()
+    scale = rng.uniform(0.5, 1.0, size=(P, n))
+    refs = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4, row_scale=scale)
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_GRAM):
+        _, r = run_gpu_cclip(g, tau, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=4, algo=algo,
+                             row_scale=torch.from_numpy(scale).cuda())
+        check_cclip(r, refs, lens)
+
+
 @pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
 def test_empty_partition_in_every_path(n, K):
     """A partition without coordinates (possible when d < P): v stays 0, norms and projections are
