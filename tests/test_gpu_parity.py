@@ -654,6 +654,39 @@ def test_nan_beyond_the_partition_length_is_never_data(n, K):
         check_cclip(r, refs, lens)
 
 
+@pytest.mark.parametrize("n,K", [(16, 1), (16, 8), (64, 4)])
+def test_all_work_is_ordered_on_the_callers_stream(n, K):
+    """The inputs become valid only late on a side stream (behind ~50 ms of other work there) and the
+    outputs are read after that stream alone is synchronised: anything the library queued on another
+    stream would read the zeros the buffers held before, or be read too early."""
+    rng = np.random.default_rng(1300 + n + K)
+    P, stride = 2, 20_000
+    lens = np.array([20_000, 17_003])
+    g = make_case(rng, P, n, stride, lens, far_rows=n // 3)
+    tau = np.array([0.7, 1.5])
+    seed = 99
+    ref = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=5)
+    staged = torch.from_numpy(g).cuda()
+    busy = torch.randn((4096, 4096), device="cuda")
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE, btard.ALGO_GRAM):
+        gd = torch.zeros_like(staged)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            acc = busy
+            for _ in range(40):
+                acc = acc @ busy * 1e-3
+            gd.copy_(staged, non_blocking=True)
+            rc, rv = btard.centered_clip_verify(gd, tau, seed, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                                max_iters=5, algo=algo, stream=side)
+        side.synchronize()
+        check_cclip(rc, ref, lens)
+        refv = oracle.verify(g, cpu(rc["v"]), tau, seed, K=K, part_len=lens)
+        check_verify(rv, refv, K)
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
 def test_empty_partition_in_every_path(n, K):
     """A partition without coordinates (possible when d < P): v stays 0, norms and projections are
