@@ -687,6 +687,36 @@ def test_all_work_is_ordered_on_the_callers_stream(n, K):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("n,K", [(16, 2), (64, 4), (100, 1)])
+def test_results_are_bitwise_reproducible(n, K):
+    """Cross-CTA sums go through per-CTA slots added in a fixed order, never through floating-point
+    atomics: the same call on the same inputs gives the same bits, whatever order the CTAs ran in and
+    whatever an earlier call left in the workspaces."""
+    rng = np.random.default_rng(1400 + n)
+    P, stride = 5, 60_000                       # several CTAs per partition
+    lens = np.array([60_000, 59_999, 31_000, 7, 0])
+    g = torch.from_numpy(make_case(rng, P, n, stride, lens, far_rows=n // 4)).cuda()
+    tau = np.array([0.5, 1.0, 2.0, 1.0, 1.0])
+    for algo, stop in ((btard.ALGO_DIRECT, btard.STOP_EPS), (btard.ALGO_DIRECT_COOPERATIVE, btard.STOP_EPS),
+                       (btard.ALGO_GRAM, btard.STOP_FIXED_ITERS)):
+        runs = []
+        ws = None
+        for rep in range(3):
+            rc, rv = btard.centered_clip_verify(g, tau, 4242, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                                stop_mode=stop, max_iters=12, eps=1e-4, algo=algo,
+                                                want_resid_sum=True, workspaces=ws)
+            torch.cuda.synchronize()
+            ws = (rc["workspace"], rv["workspace"])
+            runs.append({**{"c_" + k: cpu(rc[k]).copy() for k in ("v", "iters", "last_step_norm", "resid_norm", "status")},
+                         **{"v_" + k: cpu(rv[k]).copy() for k in ("norm", "weight", "dot", "s", "s_sum", "znorm2",
+                                                                   "resid_sum_norm", "resid_sum", "status")}})
+            ws[0].fill_(0xA5)                       # leftovers of another kind for the next call
+            ws[1].fill_(0x5A)
+        for k in runs[0]:
+            for other in runs[1:]:
+                assert runs[0][k].tobytes() == other[k].tobytes(), (algo, k)
+
+
 @pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
 def test_empty_partition_in_every_path(n, K):
     """A partition without coordinates (possible when d < P): v stays 0, norms and projections are
