@@ -717,6 +717,28 @@ def test_results_are_bitwise_reproducible(n, K):
                 assert runs[0][k].tobytes() == other[k].tobytes(), (algo, k)
 
 
+@pytest.mark.parametrize("n,K", [(4, 1), (16, 3), (40, 2), (100, 1)])
+def test_many_small_partitions(n, K):
+    """More partitions than the per-launch batch of the partition table (128), than CTAs that fit the GPU at
+    once and than SMs: P = 700 short partitions of every length from 0 to the stride."""
+    rng = np.random.default_rng(1500 + n)
+    P, stride = 700, 96
+    lens = rng.integers(0, stride + 1, size=P)
+    lens[:3] = (0, stride, 1)
+    g = make_case(rng, P, n, stride, lens)       # no far rows: over <= 96 columns their projections are ill-conditioned
+    tau = rng.uniform(0.3, 2.0, size=P)
+    seed = 31337
+    ref = oracle.centered_clip(g, tau, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=4)
+    gd = torch.from_numpy(g).cuda()
+    for algo in (btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE, btard.ALGO_GRAM):
+        rc, rv = btard.centered_clip_verify(gd, tau, seed, K=K, part_len=lens, init_mode=btard.INIT_COORD_MEDIAN,
+                                            max_iters=4, algo=algo, partition_base=5)
+        torch.cuda.synchronize()
+        check_cclip(rc, ref, lens)
+        refv = oracle.verify(g, cpu(rc["v"]), tau, seed, K=K, part_len=lens, first_partition=5)
+        check_verify(rv, refv, K)
+
+
 @pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
 def test_empty_partition_in_every_path(n, K):
     """A partition without coordinates (possible when d < P): v stays 0, norms and projections are
