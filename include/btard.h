@@ -3,7 +3,7 @@
  *
  * The library implements the arithmetic core of Byzantine-Tolerant All-Reduce (BTARD,
  * arXiv 2106.11257): the robust aggregation that replaces averaging in ButterflyClip
- * (Alg. 2, line 5) and the metadata of Verifications 1-2 (Alg. 6).  The n peers are rows of
+ * (Alg. 2, the ButterflyClip aggregation of every part) and the metadata of Verifications 1-2 (Alg. 6).  The n peers are rows of
  * one tensor in device memory; the P butterfly partitions are slabs of that tensor.
  *
  * Conventions
@@ -94,7 +94,7 @@ BTARD_API int btard_partition_layout(int64_t d, int32_t P, int32_t mode, int32_t
                            int64_t* part_offset, int64_t* part_len, int64_t* row_stride);
 
 /*
- * Commitments of Alg. 2 lines 2 and 6 (hash(g_i[j]) and hash(g^_i), broadcast before the parts travel).
+ * Commitments of Alg. 2 (hash(g_i[j]) and hash(g^_i), broadcast before the parts travel).
  * The paper asks only for "a cryptographic hash"; this library fixes SHA-256 (FIPS 180-4) in a two-level
  * tree so that one part is hashed by many threads:
  *     H(row) = SHA256( SHA256(chunk_0) || SHA256(chunk_1) || ... || LE64(byte length) ),
@@ -111,8 +111,8 @@ BTARD_API int btard_hash_partitions(int32_t n_partitions, int32_t rows_per_part,
 /*
  * Split and Merge of App. D.1 as device copies.  btard_split_gradients turns the n gradient vectors
  * grads [n][d] into the slab tensor g [P][n][row_stride] (row i of slab p = part p of peer i, padding
- * columns zero): with all peers on one GPU this is what the all-to-all of Alg. 2 lines 3-4 delivers.
- * btard_merge_partitions concatenates the aggregated parts v [P][row_stride] into out [d] (Alg. 2 line 9).
+ * columns zero): with all peers on one GPU this is what the all-to-all of Alg. 2 (every peer sends part j to aggregator j) delivers.
+ * btard_merge_partitions concatenates the aggregated parts v [P][row_stride] into out [d] (Alg. 2, Merge).
  * part_offset / part_len: host [P] as returned by btard_partition_layout; table: device scratch of
  * 16 * P bytes.  All tensors device memory; asynchronous on `stream`.
  */
@@ -164,7 +164,7 @@ BTARD_API size_t btard_centered_clip_workspace(const btard_cclip_args* args);
 BTARD_API int btard_centered_clip(const btard_cclip_args* args);
 
 /*
- * Verification metadata, Sec. 3.1 eq. (2) and Alg. 6 lines 6-14, for all partitions:
+ * Verification metadata, Sec. 3.1 eq. (2) and Alg. 6 (norms, clip weights and projections each aggregator broadcasts), for all partitions:
  *     norm_i = ||g_i - v||_2,  w_i = min{1, tau/norm_i},
  *     dot_ik = <g_i - v, z_k>  with z_k = GetRandomVector(seed) restricted to partition p, unnormalised,
  *     s_ik   = w_i dot_ik / ||z_k||_2   (the paper's s_i^j = <z[j], Delta_i^j>),
@@ -203,7 +203,7 @@ BTARD_API size_t btard_verify_projections_workspace(const btard_verify_args* arg
 BTARD_API int btard_verify_projections(const btard_verify_args* args);
 
 /*
- * Aggregation and verification of Alg. 2 line 5 and Alg. 6 lines 6-14 in one call: the same results as
+ * Aggregation (Alg. 2) and verification metadata (Alg. 6) in one call: the same results as
  * btard_centered_clip(clip) followed by btard_verify_projections(verify) on the aggregate it returned.
  * `verify` supplies the seed, n_z, partition_base, its outputs and its own workspace; its g, v, part_len,
  * tau, row_scale, resid_norm_in and stream are taken from `clip` (what it holds there is ignored), and its n_peers,
@@ -246,7 +246,7 @@ BTARD_API int btard_preclip(const btard_preclip_args* args);
 BTARD_API int btard_preclip_factors(const btard_preclip_args* args);   /* same arguments and workspace; g is read only */
 
 /*
- * The predicates of Verifications 1-3 (Alg. 6 lines 17-38) on the scalars peers broadcast.  For
+ * The predicates of Verifications 1-3 (Alg. 6) on the scalars peers broadcast.  For
  * partition p (aggregated by peer p) and peer i:
  *   Verification 1: norm_mismatch[p][i] = reported norm_ip differs from ||g_i(p) - v(p)||;
  *   Verification 2: s_mismatch[p][i][k] = reported s_i^p differs from <z_k[p], Delta_i^p>;
@@ -306,7 +306,7 @@ BTARD_API int btard_verification_checks(const btard_checks_args* args);
 BTARD_API int btard_verify_projections_static(const btard_verify_args* args);
 
 /*
- * GetRandomVector (Alg. 6 line 5) made visible: writes the unnormalised float32 coordinates
+ * GetRandomVector (Alg. 6) made visible: writes the unnormalised float32 coordinates
  * z_k[0 .. part_len) of partition p to device memory (z_out, 16-byte aligned, room for
  * part_len rounded up to a multiple of 4).  Coordinates 4q..4q+3 are the Box-Muller images of the
  * four words of Philox4x32-10 with counter (q, p, k, 0x42544152) and key (seed low, seed high).

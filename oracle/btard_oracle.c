@@ -444,7 +444,7 @@ int btard_oracle_verify_one_ex(const float *g, int32_t n, int64_t stride, int64_
 
 /* ------------------------------------------------------------------------- */
 /* Batched drivers over the [P][n][stride] tensor: the P partitions of          */
-/* ButterflyClip (Alg. 2, line 5) are independent, so they are simply looped;  */
+/* ButterflyClip (Alg. 2, aggregation) are independent, so they are simply looped;  */
 /* OpenMP, when enabled, runs whole partitions on different cores and changes  */
 /* no arithmetic.  v is [P][stride] doubles (entries past part_len[p] are 0).  */
 /* ------------------------------------------------------------------------- */
@@ -546,7 +546,7 @@ int btard_oracle_verify(const float *g, int32_t n, int32_t P, int64_t stride,
 }
 
 /* ------------------------------------------------------------------------- */
-/* Verifications 1-3 on the broadcast scalars (Alg. 6 lines 17-38), for one     */
+/* Verifications 1-3 on the broadcast scalars (Alg. 6, Verifications), for one       */
 /* partition.  "differs" is |a - b| > rel_tol max(|a|,|b|) + abs_tol (NaN        */
 /* differs); all-zero tolerances give the paper's exact tests.                   */
 /* ------------------------------------------------------------------------- */
@@ -604,7 +604,7 @@ void btard_oracle_preclip_row(const float *x, int64_t len, double lambda, double
 }
 
 /* ------------------------------------------------------------------------- */
-/* Commitments (Alg. 2 lines 2 and 6): SHA-256 (FIPS 180-4), byte oriented, and  */
+/* Commitments (Alg. 2, hash broadcasts): SHA-256 (FIPS 180-4), byte oriented, and  */
 /* the two-level tree over 4096-byte chunks that the library defines:            */
 /*   H(row) = SHA256(SHA256(chunk_0) || ... || SHA256(chunk_m-1) || LE64(bytes)). */
 /* ------------------------------------------------------------------------- */

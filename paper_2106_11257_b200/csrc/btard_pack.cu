@@ -1,7 +1,7 @@
 // Split and Merge of App. D.1 as device copies: the n gradient vectors [n][d] become the slab tensor
-// [P][n][row_stride] that the aggregation reads (this is what the all-to-all of Alg. 2 lines 3-4
+// [P][n][row_stride] that the aggregation reads (this is what the all-to-all of Alg. 2 (every peer sends part j to aggregator j)
 // delivers when every peer is a row of one GPU), and the aggregated parts [P][row_stride] are
-// concatenated back into one vector of d coordinates (Alg. 2 line 9).  Source offsets are arbitrary,
+// concatenated back into one vector of d coordinates (Alg. 2, Merge).  Source offsets are arbitrary,
 // so the copies use coalesced 32-bit accesses; padding columns are written as zero.
 #include "btard_common.h"
 

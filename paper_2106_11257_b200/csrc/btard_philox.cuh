@@ -1,4 +1,4 @@
-// Device-side GetRandomVector (Alg. 6 line 5): Philox4x32-10 words mapped to standard normals.
+// Device-side GetRandomVector (Alg. 6): Philox4x32-10 words mapped to standard normals.
 //
 // z is never stored on the verification path; each group of four coordinates is produced in
 // registers from the counter (q, partition, k, tag) and the 64-bit seed as key.  The word -> normal

@@ -1,4 +1,4 @@
-// Verification pass (Sec. 3.1 eq. (2); Alg. 6 lines 5-14) for sm_100a: one read of the
+// Verification pass (Sec. 3.1 eq. (2); Alg. 6, from GetRandomVector to the broadcast of norms and projections) for sm_100a: one read of the
 // [P][n][row_stride] tensor produces, per partition, the projections <g_i - v, z_k> on K random
 // directions, ||z_k||^2, and the clipped-residual sum sum_i w_i (g_i - v) with its norm.
 //
@@ -690,7 +690,7 @@ __global__ void verify_finalize_kernel(const VArgs k, int KT)
     if (a.k0 == 0 && threadIdx.x == 0) a.resid_sum_norm[p] = sqrt(sh_v[n * KT + KT]);
 }
 
-// Verifications 1-3 on broadcast scalars (Alg. 6 lines 17-38): one CTA per partition.
+// Verifications 1-3 on broadcast scalars (Alg. 6, the checks each peer runs on them): one CTA per partition.
 __device__ __forceinline__ bool differs(double x, double y, double rel_tol, double abs_tol)
 {
     const double scale = fmax(fabs(x), fabs(y));
