@@ -538,9 +538,11 @@ def check_verify(out, ref, K):
         for key in ("norm", "weight", "dot", "s"):
             assert rel_l2(cpu(out[key])[p], ref[key][p]) <= RTOL, (key, p)
         assert np.allclose(cpu(out["znorm2"])[p], ref["znorm2"][p], rtol=1e-6)
-        scale = np.abs(ref["s"][p]).sum(0) + 1e-300
-        assert np.all(np.abs(cpu(out["s_sum"])[p] - ref["s_sum"][p]) <= RTOL * scale), ("s_sum", p)
         rscale = (ref["weight"][p] * ref["norm"][p]).sum() + 1e-300
+        # |s_i| <= w_i rho_i, and the fp32 error of a projection goes with rho_i, not with the projection: a
+        # direction that happens to be nearly orthogonal to every residual has sum |s_i| far below that scale
+        scale = np.maximum(np.abs(ref["s"][p]).sum(0), 1e-4 * rscale) + 1e-300
+        assert np.all(np.abs(cpu(out["s_sum"])[p] - ref["s_sum"][p]) <= RTOL * scale), ("s_sum", p)
         assert abs(cpu(out["resid_sum_norm"])[p] - ref["resid_sum_norm"][p]) <= RTOL * rscale
 
 
@@ -737,6 +739,66 @@ def test_many_small_partitions(n, K):
         check_cclip(rc, ref, lens)
         refv = oracle.verify(g, cpu(rc["v"]), tau, seed, K=K, part_len=lens, first_partition=5)
         check_verify(rv, refv, K)
+
+
+@pytest.mark.parametrize("case", range(32))
+def test_random_shapes_match_oracle(case):
+    """Seeded random draws of everything a caller chooses: peers, partitions, row stride, ragged and empty
+    lengths, radii, start, stop rule, algorithm, directions, and optionally a radius schedule and row factors."""
+    rng = np.random.default_rng(7000 + case)
+    n = int(rng.choice([1, 2, 3, 5, 8, 11, 16, 17, 24, 32, 33, 48, 63, 64, 65, 96, 128, 130, 200]))
+    P = int(rng.integers(1, 7))
+    stride = 32 * int(rng.integers(1, 260))
+    lens = rng.integers(0, stride + 1, size=P)
+    lens[rng.integers(0, P)] = stride
+    if case % 5 == 0:
+        lens[rng.integers(0, P)] = 0
+    K = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16]))
+    tau = rng.uniform(0.2, 3.0, size=P)
+    algos = [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE] + ([btard.ALGO_GRAM] if n <= 128 else [])
+    algo = algos[int(rng.integers(0, len(algos)))]
+    init_g, init_o = [(btard.INIT_ZERO, oracle.INIT_ZERO), (btard.INIT_MEAN, oracle.INIT_MEAN),
+                      (btard.INIT_COORD_MEDIAN, oracle.INIT_COORD_MEDIAN),
+                      (btard.INIT_CALLER_V0, oracle.INIT_CALLER)][int(rng.integers(0, 4))]
+    if algo == btard.ALGO_GRAM and init_g in (btard.INIT_ZERO, btard.INIT_CALLER_V0):
+        init_g, init_o = btard.INIT_COORD_MEDIAN, oracle.INIT_COORD_MEDIAN    # the Gram variant wants a robust centre
+    eps_mode = bool(rng.integers(0, 2))
+    max_iters = int(rng.integers(1, 12)) if not eps_mode else 60
+    g = make_case(rng, P, n, stride, lens, far_rows=int(rng.integers(0, n // 3 + 1)))
+    v0 = rng.standard_normal((P, stride)).astype(np.float32) if init_g == btard.INIT_CALLER_V0 else None
+    sched = rng.uniform(0.2, 3.0, size=(P, max_iters)) if (case % 3 == 0 and not eps_mode) else None
+    scale = rng.uniform(0.3, 1.0, size=(P, n)) if case % 4 == 1 else None
+    if scale is not None and algo == btard.ALGO_DIRECT_COOPERATIVE:
+        algo = btard.ALGO_DIRECT                           # the cooperative kernel takes no row factors
+    kw_o = dict(init_mode=init_o, v0=v0, max_iters=max_iters, tau_schedule=sched, row_scale=scale)
+    kw_g = dict(init_mode=init_g, max_iters=max_iters, algo=algo,
+                tau_schedule=None if sched is None else torch.from_numpy(sched).cuda(),
+                row_scale=None if scale is None else torch.from_numpy(scale).cuda())
+    if eps_mode:
+        kw_o.update(stop_mode=oracle.STOP_EPS, eps=1e-4)
+        kw_g.update(stop_mode=btard.STOP_EPS, eps=1e-4)
+    ref = oracle.centered_clip(g, tau, lens, **kw_o)
+    gd = torch.from_numpy(g).cuda()
+    vd = torch.from_numpy(v0).cuda().clone() if v0 is not None else None
+    seed = 0xC0FFEE + case
+    rc, rv = btard.centered_clip_verify(gd, tau, seed, K=K, part_len=lens, v=vd, partition_base=case,
+                                        want_resid_sum=True, **kw_g)
+    torch.cuda.synchronize()
+    if eps_mode:
+        it = cpu(rc["iters"])
+        assert np.all(np.abs(it - ref["iters"]) <= 1), (it, ref["iters"])
+        same = it == ref["iters"]
+        v = cpu(rc["v"])
+        for p in np.nonzero(same)[0]:
+            assert rel_l2(v[p, : lens[p]], ref["v"][p, : lens[p]]) <= RTOL, ("v", p)
+    else:
+        check_cclip(rc, ref, lens)
+    refv = oracle.verify(g, cpu(rc["v"]), tau, seed, K=K, part_len=lens, first_partition=case, want_resid_sum=True,
+                         row_scale=scale)
+    check_verify(rv, refv, K)
+    for p in range(P):
+        rscale = (refv["weight"][p] * refv["norm"][p]).sum() + 1e-300
+        assert np.linalg.norm(cpu(rv["resid_sum"])[p, : lens[p]] - refv["resid_sum"][p, : lens[p]]) <= RTOL * rscale
 
 
 @pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
