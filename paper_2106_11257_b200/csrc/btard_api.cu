@@ -372,7 +372,10 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
     L.init_mode = a->init_mode;
     // up to 16 peers the Gram pass takes the median start itself (every row of a column sits in one thread)
     const bool gram_takes_median = (a->algo == BTARD_ALGO_GRAM && a->init_mode == BTARD_INIT_COORD_MEDIAN && n <= 16);
-    if (a->init_mode == BTARD_INIT_COORD_MEDIAN && !gram_takes_median) {
+    // 32 or 64 peers, launch-per-update path: the median start and the start pass are one kernel
+    const bool fused_start = (a->algo == BTARD_ALGO_DIRECT && a->init_mode == BTARD_INIT_COORD_MEDIAN &&
+                              median_norms_supported(n, a->row_stride, a->row_scale));
+    if (a->init_mode == BTARD_INIT_COORD_MEDIAN && !gram_takes_median && !fused_start) {
         rc = launch_median_init(a->g, a->v, L.table, a->row_scale, a->row_stride, n, P, st);
         if (rc != BTARD_OK) return rc;
         L.init_mode = BTARD_INIT_CALLER_V0;
@@ -417,7 +420,7 @@ static int cclip_run(const btard_cclip_args* a, const btard_verify_args* fv)
         // the cooperative launch was refused: nothing ran, take the launch-per-update path
     }
 
-    rc = launch_cclip_pass(L, geo, PASS_INIT, st);
+    rc = fused_start ? launch_median_norms(L, geo, st) : launch_cclip_pass(L, geo, PASS_INIT, st);
     if (rc != BTARD_OK) return rc;
 
     // Update l reads the totals in buffer l % 2 and writes buffer (l + 1) % 2.

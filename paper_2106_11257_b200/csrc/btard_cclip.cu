@@ -1010,6 +1010,95 @@ __global__ void __launch_bounds__(128, CW == 2 ? 3 : 1) median_sort_kernel(const
     else v[(size_t)p * stride + c] = out[0];
 }
 
+// The median start and the start pass of the direct algorithm in one read of the rows (exactly 32 or 64
+// rows, no row factors): a thread takes the median of a column as above, then reads the column's rows a
+// second time (they are in L1: the first read is not marked streaming here) and adds (x_i - v0)^2 to one
+// running sum per row.  The sorted copy and the sums are all the registers hold, so the rows are not kept.
+// A thread covers at most 512 columns (256 where the slot count allows: fp32 running sums stay short); per-CTA slots and the
+// last-CTA reduction are those of the pass kernels, so the first update finds its totals where the start
+// pass would have left them.
+template <int N2>
+__global__ void __launch_bounds__(128, 3) median_norms_kernel(const float* g, float* v, const PartEntry* table,
+                                                              long long stride, double* slots_base, double* tot_out,
+                                                              unsigned int* ticket, int* done, uint32_t* status,
+                                                              long long cols_per_cta)
+{
+    __shared__ double sh_red[4][N2];
+    __shared__ double sh_part[128];
+    __shared__ int sh_flag;
+    constexpr int n = N2;
+    const int p = blockIdx.y, j = blockIdx.x, cpp = gridDim.x, tid = threadIdx.x;
+    const long long len = table[p].len;
+    if (j == 0 && tid == 0) { done[p] = 0; status[p] = 0; }
+    const long long c0 = (long long)j * cols_per_cta;
+    long long c1 = c0 + cols_per_cta;
+    if (c1 > stride) c1 = stride;
+    const float* gp = g + (size_t)p * n * stride;
+    const uint32_t pitch = (uint32_t)(stride * 4);         // bytes between rows: the host checked that n rows stay below 4 GiB
+    float acc[N2];
+#pragma unroll
+    for (int i = 0; i < N2; ++i) acc[i] = 0.0f;
+    for (long long c = c0 + tid; c < c1; c += 128) {
+        float out = 0.0f;
+        if (c < len) {
+            const float* base = gp + c;
+            auto row = [&](int i) {
+                uint64_t at;
+                asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(at) : "r"((uint32_t)i), "r"(pitch), "l"(base));
+                return __ldg(reinterpret_cast<const float*>(at));
+            };
+            float s[N2];
+            float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < N2; ++i) {
+                s[i] = row(i);
+                sum[i & 3] += s[i];
+            }
+            const float total = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+            if (total == total) {                          // no NaN in the column (nor +inf beside -inf)
+                out = median_of_values<N2, true>(s, n);
+            } else {
+                int key[N2];
+#pragma unroll
+                for (int i = 0; i < N2; ++i) key[i] = signed_key(s[i]);
+                out = median_of_keys<N2, true>(key, n);
+            }
+#pragma unroll
+            for (int i = 0; i < N2; ++i) {
+                const float d = row(i) - out;
+                acc[i] = fmaf(d, d, acc[i]);
+            }
+        }
+        v[(size_t)p * stride + c] = out;
+    }
+    // CTA reduction, per-CTA slot, last CTA of the partition adds the slots in a fixed order
+    const int warp = tid >> 5, lane = tid & 31;
+#pragma unroll
+    for (int i = 0; i < N2; ++i) {
+        double x = (double)acc[i];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
+        if (lane == 0) sh_red[warp][i] = x;
+    }
+    __syncthreads();
+    const int per = n + 1;
+    double* slots = slots_base + (size_t)p * cpp * per;
+    if (tid < per) slots[(size_t)j * per + tid] = (tid < n) ? (sh_red[0][tid] + sh_red[1][tid]) + (sh_red[2][tid] + sh_red[3][tid]) : 0.0;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sh_flag = (atomicAdd(&ticket[p], 1u) == (unsigned)(cpp - 1));
+    __syncthreads();
+    if (!sh_flag) return;
+    __threadfence();
+    if (tid < per) {
+        double t = 0.0;
+        for (int c = 0; c < cpp; ++c) t += __ldcg(slots + (size_t)c * per + tid);
+        tot_out[(size_t)p * per + tid] = t;
+    }
+    (void)sh_part;
+    if (tid == 0) ticket[p] = 0;
+}
+
 // Any n: rank every value by counting (O(n^2) compares per column), pick the two middle ranks.
 __global__ void median_rank_kernel(const float* g, float* v, const PartEntry* table, const double* row_scale,
                                    long long stride, int n)
@@ -1219,6 +1308,38 @@ int cooperative_launch_supported()
         return 0;
     }
     return coop;
+}
+
+// Whether the fused median + start kernel serves this shape.
+bool median_norms_supported(int n, long long stride, const double* row_scale)
+{
+    // 16 rows: the two separate kernels are both HBM-bound and faster (0.128 + 0.124 against 0.32 ms)
+    return (n == 32 || n == 64) && !row_scale && stride * 4 * (long long)n < (1LL << 32);
+}
+
+int launch_median_norms(const CclipLaunch& a, const Geometry& geo, cudaStream_t st)
+{
+    // 256 columns per thread where the slots allow it (the pass kernels' CTAs cover up to 65 536 columns each, so
+    // at most 512), enough CTAs for a few waves, and no more CTAs than the slots of the pass kernels hold
+    long long cpp = (a.stride + 128LL * 256 - 1) / (128LL * 256);
+    const long long want = (4LL * 3 * sm_count() + a.P - 1) / a.P;
+    if (cpp < want) cpp = want;
+    if (cpp > geo.cpp) cpp = geo.cpp;
+    if (cpp < 1) cpp = 1;
+    long long cols = (a.stride + cpp - 1) / cpp;
+    cols = (cols + 127) / 128 * 128;
+    if (cols > 128LL * 512) return BTARD_ERR_UNSUPPORTED;      // cannot happen: geo.cpp bounds the pass kernels' CTAs to 65 536 columns
+    cpp = (a.stride + cols - 1) / cols;
+    dim3 grid((unsigned)cpp, (unsigned)a.P);
+    prof_begin(KIND_MEDIAN, st);
+    if (a.n == 64)
+        median_norms_kernel<64><<<grid, 128, 0, st>>>(a.g, a.v, a.table, a.stride, a.slots, a.tot_out, a.ticket, a.done, a.status, cols);
+    else
+        median_norms_kernel<32><<<grid, 128, 0, st>>>(a.g, a.v, a.table, a.stride, a.slots, a.tot_out, a.ticket, a.done, a.status, cols);
+    prof_end(KIND_MEDIAN, st);
+    BTARD_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BTARD_OK;
 }
 
 int launch_median_init(const float* g, float* v, const PartEntry* table, const double* row_scale,

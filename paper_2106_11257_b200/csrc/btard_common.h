@@ -103,6 +103,9 @@ Geometry cclip_geometry(int n, int P, long long stride);
 int choose_ctas_per_partition(int P, long long quads, int CL, int slots, int max_tiles = kMaxTilesPerCta);
 int launch_cclip_pass(const CclipLaunch& a, const Geometry& geo, int mode, cudaStream_t st);
 int launch_cclip_finalize(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
+// Median start and the start pass of the direct algorithm in one kernel (32 or 64 rows, no row factors).
+bool median_norms_supported(int n, long long stride, const double* row_scale);
+int launch_median_norms(const CclipLaunch& a, const Geometry& geo, cudaStream_t st);
 // One cooperative launch that runs the start pass and every update of all partitions (work items =
 // the CTAs of launch_cclip_pass, dealt round-robin to one wave of resident CTAs).  streaming != 0:
 // the tensor does not fit L2 (evict-first loads, alternating sweep direction).

@@ -345,6 +345,47 @@ def test_coordinate_median_with_special_values_is_exact(n):
                 assert np.all(np.abs(a[fin] - b[fin]) <= 2e-7 * np.abs(b[fin]) + 5e-9), p   # values are O(1e-2): one rounding of f x
 
 
+@pytest.mark.parametrize("n", [32, 64])
+def test_fused_median_start_with_special_values(n):
+    """32 and 64 peers, direct algorithm: the median start and the start pass are one kernel.  With tau = 0
+    every weight is 0, so the aggregate stays at the start and must equal the oracle's median value for
+    value, on columns with an infinity, NaNs of both signs, zeros of both signs and ties; the norms at the
+    start are compared too."""
+    rng = np.random.default_rng(950 + n)
+    P, stride = 3, 33_024                      # more than 256 columns per thread of one CTA: several CTAs
+    lens = np.array([33_024, 20_001, 77])
+    g = (rng.standard_normal((P, n, stride)) * 1e-2).astype(np.float32)
+    for p in range(P):
+        g[p, :, lens[p]:] = 77.0
+    bad_rows = [set() for _ in range(P)]
+    for p in range(P):
+        for t in range(min(60, lens[p] // 16)):
+            c, r = 16 * t + 3, int(rng.integers(0, n))
+            kind = t % 6
+            if kind == 0: g[p, r, c] = np.inf; bad_rows[p].add(r)
+            elif kind == 1: g[p, r, c] = -np.inf; bad_rows[p].add(r)
+            elif kind == 2: g[p, r, c] = np.nan; bad_rows[p].add(r)
+            elif kind == 3:
+                g[p, r, c] = -np.nan; g[p, (r + 1) % n, c] = np.nan
+                bad_rows[p].update((r, (r + 1) % n))
+            elif kind == 4: g[p, :, c] = 0.0; g[p, r, c] = -0.0
+            else: g[p, :, c] = g[p, 0, c]
+    ref = oracle.centered_clip(g, 0.0, lens, init_mode=oracle.INIT_COORD_MEDIAN, max_iters=1)
+    med = oracle.centered_clip(g, 1.0, lens, rule=oracle.RULE_COORD_MEDIAN)
+    _, r = run_gpu_cclip(g, 0.0, lens, init_mode=btard.INIT_COORD_MEDIAN, max_iters=1, algo=btard.ALGO_DIRECT)
+    v, rn = cpu(r["v"]), cpu(r["resid_norm"])
+    for p in range(P):
+        L = lens[p]
+        a = v[p, :L] + np.float32(0.0)
+        assert np.array_equal(a, med["v"][p, :L].astype(np.float32) + np.float32(0.0)), p
+        assert np.array_equal(a, ref["v"][p, :L].astype(np.float32) + np.float32(0.0)), p
+        fin = np.isfinite(ref["resid_norm"][p])
+        assert set(np.nonzero(~fin)[0]) == bad_rows[p]
+        assert np.array_equal(np.isfinite(rn[p]), fin)
+        assert rel_l2(rn[p][fin], ref["resid_norm"][p][fin]) <= RTOL
+        assert cpu(r["status"])[p] & btard.STATUS_NONFINITE_ROW
+
+
 def test_geometric_median_rule_rejects_a_zero_floor_and_gram():
     g = torch.zeros((1, 4, 64), device="cuda")
     with pytest.raises(btard.BtardError):
