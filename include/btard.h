@@ -321,7 +321,8 @@ BTARD_API int btard_random_vector(uint64_t seed, int32_t p, int32_t k, int64_t p
  * `stream` (and for copy_stream, which only carries copies this call queued).  All device memory
  * comes from device_scratch (sized by btard_aggregate_host_scratch for the same n_peers, n_partitions,
  * row_stride, n_z and algo).  With BTARD_ALGO_DIRECT in EPS mode the updates run in the cooperative
- * kernel, so that nothing is launched after convergence.
+ * kernel, so that nothing is launched after convergence (except with a coordinate-median start at 32
+ * or 64 peers, where the launch-per-update path saves a pass over the rows and stays).
  * Host output pointers may be NULL to skip that copy, except v.  Pinned host memory makes the
  * copies asynchronous and fast; pageable memory works too.
  */
