@@ -113,8 +113,10 @@ BTARD_API int btard_hash_partitions(int32_t n_partitions, int32_t rows_per_part,
  * grads [n][d] into the slab tensor g [P][n][row_stride] (row i of slab p = part p of peer i, padding
  * columns zero): with all peers on one GPU this is what the all-to-all of Alg. 2 (every peer sends part j to aggregator j) delivers.
  * btard_merge_partitions concatenates the aggregated parts v [P][row_stride] into out [d] (Alg. 2, Merge).
- * part_offset / part_len: host [P] as returned by btard_partition_layout; table: device scratch of
- * 16 * P bytes.  All tensors device memory; asynchronous on `stream`.
+ * part_offset / part_len: host [P], as returned by btard_partition_layout or any P pairs with
+ * 0 <= offset, len <= row_stride, offset + len <= d (slab q then holds coordinates offset[q] .. offset[q] +
+ * len[q] - 1: a permutation of the parts gives a send buffer ordered by destination); table: device scratch
+ * of 16 * P bytes.  All tensors device memory; asynchronous on `stream`.
  */
 BTARD_API int btard_split_gradients(int64_t d, int32_t n_peers, int32_t n_partitions, int64_t row_stride,
                                     const int64_t* part_offset, const int64_t* part_len,

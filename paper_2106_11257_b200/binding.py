@@ -409,12 +409,20 @@ def verify_projections_static(g, v, tau, seed, K=1, part_len=None, resid_norm_in
     return res
 
 
-def split_gradients(grads, P, mode=SPLIT_CEIL_PAD, align_elems=32, stream=None):
-    """grads: CUDA float32 [n][d] -> (g [P][n][row_stride], part_offset, part_len)."""
+def split_gradients(grads, P, mode=SPLIT_CEIL_PAD, align_elems=32, stream=None, layout=None):
+    """grads: CUDA float32 [n][d] -> (g [P][n][row_stride], part_offset, part_len).
+    layout: optional (part_offset, part_len, row_stride) to use instead of btard_partition_layout's, one entry
+    per slab in the order the slabs are wanted (a permutation of the parts, for instance)."""
     torch = _torch()
     assert grads.is_cuda and grads.dtype == torch.float32 and grads.dim() == 2 and grads.is_contiguous()
     n, d = grads.shape
-    off, ln, stride = partition_layout(d, P, mode, align_elems)
+    if layout is None:
+        off, ln, stride = partition_layout(d, P, mode, align_elems)
+    else:
+        off = np.ascontiguousarray(layout[0], dtype=np.int64)
+        ln = np.ascontiguousarray(layout[1], dtype=np.int64)
+        stride = int(layout[2])
+        assert off.shape == (P,) and ln.shape == (P,)
     g = torch.empty((P, n, stride), dtype=torch.float32, device=grads.device)
     table = torch.empty(16 * P, dtype=torch.uint8, device=grads.device)
     L = lib()
