@@ -588,8 +588,10 @@ def check_verify(out, ref, K):
         assert np.allclose(cpu(out["znorm2"])[p], ref["znorm2"][p], rtol=1e-6)
         rscale = (ref["weight"][p] * ref["norm"][p]).sum() + 1e-300
         # |s_i| <= w_i rho_i, and the fp32 error of a projection goes with rho_i, not with the projection: a
-        # direction that happens to be nearly orthogonal to every residual has sum |s_i| far below that scale
-        scale = np.maximum(np.abs(ref["s"][p]).sum(0), 1e-4 * rscale) + 1e-300
+        # direction that happens to be nearly orthogonal to every residual has sum |s_i| far below that scale.
+        # s_i = w_i <r_i, z> / |z| evaluated in fp32 carries an error of about eps_fp32 w_i rho_i (1.2e-7; seen:
+        # up to 2.8e-8 sum_i w_i rho_i with row factors and far rows), so the floor is 1e-7 sum_i w_i rho_i
+        scale = np.maximum(np.abs(ref["s"][p]).sum(0), 1e-2 * rscale) + 1e-300
         assert np.all(np.abs(cpu(out["s_sum"])[p] - ref["s_sum"][p]) <= RTOL * scale), ("s_sum", p)
         assert abs(cpu(out["resid_sum_norm"])[p] - ref["resid_sum_norm"][p]) <= RTOL * rscale
 
