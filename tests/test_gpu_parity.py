@@ -791,8 +791,8 @@ def test_many_small_partitions(n, K):
         check_verify(rv, refv, K)
 
 
-@pytest.mark.parametrize("case", range(32))
-def test_random_shapes_match_oracle(case):
+@pytest.mark.parametrize("case", list(range(32)) + [2125])   # 2125: 3 far rows with factors, 16 directions, one of them
+def test_random_shapes_match_oracle(case):                   # nearly orthogonal to every residual (the s_sum floor)
     """Seeded random draws of everything a caller chooses: peers, partitions, row stride, ragged and empty
     lengths, radii, start, stop rule, algorithm, directions, and optionally a radius schedule and row factors."""
     rng = np.random.default_rng(7000 + case)
