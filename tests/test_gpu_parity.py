@@ -858,6 +858,44 @@ def test_random_shapes_match_oracle(case):                   # nearly orthogonal
         assert np.linalg.norm(cpu(rv["resid_sum"])[p, : lens[p]] - refv["resid_sum"][p, : lens[p]]) <= RTOL * rscale
 
 
+@pytest.mark.parametrize("case", range(10))
+def test_random_long_rows_match_oracle(case):
+    """The same kind of draw with rows of 10 000 to 190 000 columns (several tiles and CTAs per partition, ragged
+    ends inside a tile), a few fixed updates: peers, radii, start, algorithm, directions, schedule, row factors."""
+    rng = np.random.default_rng(90000 + case)
+    n = int(rng.choice([2, 5, 8, 12, 16, 17, 24, 32, 40, 48, 63, 64, 65, 100]))
+    P = int(rng.integers(1, 4))
+    stride = 32 * int(rng.integers(300, 6000))
+    lens = rng.integers(stride // 2, stride + 1, size=P)
+    lens[rng.integers(0, P)] = stride
+    K = int(rng.choice([1, 2, 4, 5, 8]))
+    tau = rng.uniform(2.0, 30.0, size=P)
+    algo = [btard.ALGO_DIRECT, btard.ALGO_DIRECT_COOPERATIVE, btard.ALGO_GRAM][int(rng.integers(0, 3))]
+    init_g, init_o = [(btard.INIT_MEAN, oracle.INIT_MEAN),
+                      (btard.INIT_COORD_MEDIAN, oracle.INIT_COORD_MEDIAN)][int(rng.integers(0, 2))]
+    max_iters = int(rng.integers(1, 6))
+    g = make_case(rng, P, n, stride, lens, far_rows=int(rng.integers(0, n // 3 + 1)))
+    sched = rng.uniform(2.0, 30.0, size=(P, max_iters)) if case % 3 == 0 else None
+    scale = rng.uniform(0.3, 1.0, size=(P, n)) if case % 4 == 1 else None
+    if scale is not None:                                  # as above: no large common mean under row factors
+        g = (g - np.float32(0.95) * g.mean(axis=1, keepdims=True)).astype(np.float32)
+        for p in range(P):
+            g[p, :, lens[p]:] = 77.0
+        if algo == btard.ALGO_DIRECT_COOPERATIVE:
+            algo = btard.ALGO_DIRECT
+    ref = oracle.centered_clip(g, tau, lens, init_mode=init_o, max_iters=max_iters, tau_schedule=sched, row_scale=scale)
+    seed = 0xBEEF + case
+    rc, rv = btard.centered_clip_verify(torch.from_numpy(g).cuda(), tau, seed, K=K, part_len=lens, partition_base=case,
+                                        want_resid_sum=True, init_mode=init_g, max_iters=max_iters, algo=algo,
+                                        tau_schedule=None if sched is None else torch.from_numpy(sched).cuda(),
+                                        row_scale=None if scale is None else torch.from_numpy(scale).cuda())
+    torch.cuda.synchronize()
+    check_cclip(rc, ref, lens, gram=(algo == btard.ALGO_GRAM))
+    refv = oracle.verify(g, cpu(rc["v"]), tau, seed, K=K, part_len=lens, first_partition=case, want_resid_sum=True,
+                         row_scale=scale)
+    check_verify(rv, refv, K)
+
+
 @pytest.mark.parametrize("n,K", [(5, 1), (16, 2), (16, 3), (40, 1)])
 def test_empty_partition_in_every_path(n, K):
     """A partition without coordinates (possible when d < P): v stays 0, norms and projections are
