@@ -644,6 +644,262 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
     }
 }
 
+// 49 .. 64 peers, the verification pass fused with the combine pass, one or two directions per launch: the four
+// lanes 4k .. 4k + 3 of a warp share 4 columns and hold 16 rows each (lane g: rows 16 g .. 16 g + 15, R x 4
+// columns in registers as in verify_rows_kernel), so what the 64 rows of a column have to add up (the move of
+// v, the clipped-residual sum) crosses lanes by two shuffle steps and the tile loop has no CTA barrier and no
+// shared-memory staging at all.  Direction q of a launch is drawn by lane q of the group and handed to the
+// others by shuffle, so every quad of z is still generated once.  Slot layout as verify_kernel.
+constexpr int kLanesThreads = 128;
+constexpr int kLanesRows = 64;
+
+// One or two directions per launch.  Measured on 64 x 64 x 276 320, K = 1: 0.91 ms with four CTAs per SM (128
+// registers, 80 bytes of spills), 0.96 with three (168 registers), 1.02 for the row-group kernel: the pass waits on
+// its loads, and more warps hide more of that; two directions spill 280 bytes at 128 registers and keep three
+// CTAs.  At four directions (64 x 64 x 4 194 304) neither four lanes of 16 rows (255 registers, two CTAs: 19.9
+// against 19.0 ms) nor eight lanes of 8 rows (26.3 ms) beats the row-group kernel, so it keeps them.
+template <int KT>
+constexpr int lanes_min_ctas() { return KT == 1 ? 4 : 3; }
+
+template <int KT, bool COMBINE>
+__global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<KT>()) verify_lanes_kernel(const VArgs k)
+{
+    constexpr int R = 16, NR = kLanesRows, CL = kLanesThreads, G = NR / R;   // G = 4 lanes share a quad
+    __shared__ float sh_w[NR];
+    __shared__ float sh_c[NR];                      // COMBINE: coefficients a_j
+    __shared__ double sh_ga[NR + 1];                // COMBINE: (G a)_i, then a^T G a
+    __shared__ double sh_red[CL / 32][NR * KT + KT + 1 + (COMBINE ? NR : 0)];
+    __shared__ float sh_f[NR];                      // row factors (with row_scale)
+
+    const VerifyLaunch& a = k.a;
+    const int n = a.n, cpp = k.cpp;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = tid & (G - 1), rb = R * g;        // lane of the group, its first row
+    const unsigned gmask = ((1u << G) - 1u) << (lane & ~(G - 1));   // the lanes that share this thread's columns
+    const int p = blockIdx.x / cpp, j = blockIdx.x % cpp;
+    const bool scaled = a.row_scale != nullptr;     // rows enter as f_i x_i
+    if (scaled && tid < NR) sh_f[tid] = (tid < n) ? (float)a.row_scale[(size_t)p * n + tid] : 0.0f;   // before the barriers below
+    const long long stride = a.stride, len = a.table[p].len;
+    const double tau = a.table[p].tau;
+
+    if (COMBINE) {
+        const double* G = a.gram + (size_t)p * a.gram_entries;
+        const double* cf = a.coef + (size_t)p * n;
+        if (tid < NR) {
+            double ga = 0.0;
+            if (tid < n)
+                for (int q = 0; q < n; ++q) {
+                    const double cq = cf[q];
+                    if (cq != 0.0) ga += G[gram_entry_index(a.gram_nb, tid, q)] * cq;   // weight-0 rows are skipped
+                }
+            sh_ga[tid] = ga;
+            sh_c[tid] = (tid < n) ? (float)cf[tid] : 0.0f;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double aga = 0.0;
+            for (int q = 0; q < n; ++q)
+                if (cf[q] != 0.0) aga += cf[q] * sh_ga[q];
+            sh_ga[NR] = aga;
+        }
+        __syncthreads();
+        if (tid < NR) {
+            float w = 0.0f;
+            if (tid < n) {
+                double rho2 = G[gram_entry_index(a.gram_nb, tid, tid)] - 2.0 * sh_ga[tid] + sh_ga[NR];
+                if (rho2 < 0.0) rho2 = 0.0;
+                const double rho = sqrt(rho2);
+                if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+            }
+            sh_w[tid] = w;
+        }
+    } else if (tid < NR) {
+        float w = 0.0f;
+        if (tid < n) {
+            const double rho = a.norm_in[(size_t)p * n + tid];
+            if (isfinite(rho)) w = (rho <= tau) ? 1.0f : (float)(tau / rho);
+        }
+        sh_w[tid] = w;
+    }
+    __syncthreads();
+
+    float nacc[COMBINE ? R : 1];                       // COMBINE: squared residual norms at the new v
+#pragma unroll
+    for (int r = 0; r < (COMBINE ? R : 1); ++r) nacc[r] = 0.0f;
+    float acc[R][KT];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int q = 0; q < KT; ++q) acc[r][q] = 0.0f;
+    float zz[KT];
+#pragma unroll
+    for (int q = 0; q < KT; ++q) zz[q] = 0.0f;
+    float rs2 = 0.0f;
+
+    // This CTA's share of the partition in groups of 4 columns, cut on 128-byte lines.
+    const long long Q = stride >> 2;
+    long long q0 = Q * j / cpp, q1 = Q * (j + 1) / cpp;
+    if (j > 0) q0 &= ~7LL;
+    if (j + 1 < cpp) q1 &= ~7LL;
+    const float* gp = a.g + ((size_t)p * n + rb) * stride;        // this lane's first row
+    const float* vp = a.v + (size_t)p * stride;
+    float* rsp = a.resid_sum ? a.resid_sum + (size_t)p * stride : nullptr;
+    const bool first_chunk = (a.k0 == 0);          // the residual sum is produced once, not per chunk
+    const uint32_t pg = (uint32_t)(a.p_base + p);
+
+    // a row with weight 0 or coefficient 0 (a non-finite row) is left out of the sums, not multiplied
+    bool any_skip = false;
+    for (int r = 0; r < n; ++r) any_skip |= (sh_w[r] == 0.0f) || (COMBINE && sh_c[r] == 0.0f);
+    const bool rows_whole = (n == NR);                 // no row of any lane is missing
+
+    auto four_sum = [&](float4& s) {                   // sum over the lanes of the group, every lane gets it
+#pragma unroll
+        for (int o = 1; o < G; o <<= 1) {
+            s.x += __shfl_xor_sync(gmask, s.x, o);
+            s.y += __shfl_xor_sync(gmask, s.y, o);
+            s.z += __shfl_xor_sync(gmask, s.z, o);
+            s.w += __shfl_xor_sync(gmask, s.w, o);
+        }
+    };
+
+    // GUARD: the quad reaches past the partition's length, or some row is missing or has to be left out
+    auto tile = [&](auto guard_tag, long long qb) {
+        constexpr bool GUARD = decltype(guard_tag)::value;
+        const long long col = qb * 4;
+        float4 x[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            x[r] = (!GUARD || rb + r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (scaled) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] = scale_row(x[r], sh_f[rb + r]);
+        }
+        const float4 v4 = *reinterpret_cast<const float4*>(vp + col);
+        const bool m0 = !GUARD || col < len, m1 = !GUARD || col + 1 < len, m2 = !GUARD || col + 2 < len,
+                   m3 = !GUARD || col + 3 < len;
+        // lane q of the group draws direction q while the rows are on their way
+        float4 zmine = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (g < KT && g < a.kc && m0) {
+            zmine = z_quad((uint32_t)qb, pg, (uint32_t)(a.k0 + g), a.seed_lo, a.seed_hi);
+            if (GUARD && !m3) {                        // only the last quad of a ragged partition
+                if (!m1) zmine.y = 0.f;
+                if (!m2) zmine.z = 0.f;
+                zmine.w = 0.f;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const bool rp = !GUARD || rb + r < n;
+            x[r].x = (m0 && rp) ? x[r].x - v4.x : 0.f;
+            x[r].y = (m1 && rp) ? x[r].y - v4.y : 0.f;
+            x[r].z = (m2 && rp) ? x[r].z - v4.z : 0.f;
+            x[r].w = (m3 && rp) ? x[r].w - v4.w : 0.f;
+        }
+        if (COMBINE) {
+            // x holds the residuals at v0: move v by u = sum_j a_j (x_j - v0) over all 64 rows, then the residuals
+            // by what v really moved (the rounded difference), and add up the squared norms at the new v
+            float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float cr = sh_c[rb + r];
+                if (!GUARD || cr != 0.0f) {
+                    u.x = fmaf(cr, x[r].x, u.x); u.y = fmaf(cr, x[r].y, u.y);
+                    u.z = fmaf(cr, x[r].z, u.z); u.w = fmaf(cr, x[r].w, u.w);
+                }
+            }
+            four_sum(u);
+            const float4 vn = make_float4(v4.x + u.x, v4.y + u.y, v4.z + u.z, v4.w + u.w);
+            const float4 dv = make_float4(vn.x - v4.x, vn.y - v4.y, vn.z - v4.z, vn.w - v4.w);
+            if (g == 0)
+                *reinterpret_cast<float4*>(a.v_out + (size_t)p * stride + col) =
+                    make_float4(m0 ? vn.x : 0.f, m1 ? vn.y : 0.f, m2 ? vn.z : 0.f, m3 ? vn.w : 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const bool rp = !GUARD || rb + r < n;
+                x[r].x = (m0 && rp) ? x[r].x - dv.x : 0.f; x[r].y = (m1 && rp) ? x[r].y - dv.y : 0.f;
+                x[r].z = (m2 && rp) ? x[r].z - dv.z : 0.f; x[r].w = (m3 && rp) ? x[r].w - dv.w : 0.f;
+                nacc[r] += fmaf(x[r].x, x[r].x, fmaf(x[r].y, x[r].y, fmaf(x[r].z, x[r].z, x[r].w * x[r].w)));
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            const int src = (lane & ~(G - 1)) | q;     // the lane of the group that drew direction q
+            float4 zq;
+            zq.x = __shfl_sync(gmask, zmine.x, src);
+            zq.y = __shfl_sync(gmask, zmine.y, src);
+            zq.z = __shfl_sync(gmask, zmine.z, src);
+            zq.w = __shfl_sync(gmask, zmine.w, src);
+            if (g == 0) zz[q] += fmaf(zq.x, zq.x, fmaf(zq.y, zq.y, fmaf(zq.z, zq.z, zq.w * zq.w)));
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                acc[r][q] = fmaf(x[r].x, zq.x, fmaf(x[r].y, zq.y, fmaf(x[r].z, zq.z, fmaf(x[r].w, zq.w, acc[r][q]))));
+        }
+        if (first_chunk) {                             // clipped-residual sum of these 4 columns
+            float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float wr = sh_w[rb + r];
+                if (!GUARD || wr != 0.0f) {
+                    s4.x = fmaf(wr, x[r].x, s4.x);
+                    s4.y = fmaf(wr, x[r].y, s4.y);
+                    s4.z = fmaf(wr, x[r].z, s4.z);
+                    s4.w = fmaf(wr, x[r].w, s4.w);
+                }
+            }
+            four_sum(s4);
+            if (g == 0) {
+                rs2 += fmaf(s4.x, s4.x, fmaf(s4.y, s4.y, fmaf(s4.z, s4.z, s4.w * s4.w)));
+                if (rsp) *reinterpret_cast<float4*>(rsp + col) = s4;
+            }
+        }
+    };
+    for (long long qb = q0 + tid / G; qb < q1; qb += CL / G) {
+        if (rows_whole && !any_skip && qb * 4 + 3 < len) tile(std::false_type{}, qb);
+        else tile(std::true_type{}, qb);
+    }
+
+    // CTA reduction: lanes with the same g hold the same rows
+    auto rows_sum = [&](double s) {
+#pragma unroll
+        for (int o = 16; o >= G; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        return s;
+    };
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int q = 0; q < KT; ++q) {
+            const double s = rows_sum((double)acc[r][q]);
+            if (lane < G) sh_red[warp][(rb + r) * KT + q] = s;
+        }
+#pragma unroll
+    for (int q = 0; q < KT; ++q) {
+        const double s = warp_sum((double)zz[q]);
+        if (lane == 0) sh_red[warp][NR * KT + q] = s;
+    }
+    {
+        const double s = warp_sum((double)rs2);
+        if (lane == 0) sh_red[warp][NR * KT + KT] = s;
+    }
+    if (COMBINE) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const double s = rows_sum((double)nacc[r]);
+            if (lane < G) sh_red[warp][NR * KT + KT + 1 + rb + r] = s;
+        }
+    }
+    __syncthreads();
+    double* dst = a.part_out + ((size_t)p * cpp + j) * k.slots;
+    // slot: [n KT] dots, [KT] znorm2, the resid-sum slot, then (COMBINE) [n] squared norms
+    const int total = n * KT + KT + 1 + (COMBINE ? n : 0);
+    for (int e = tid; e < total; e += CL) {
+        const int col = (e < n * KT) ? e : NR * KT + (e - n * KT);
+        double s = 0.0;
+        for (int u = 0; u < CL / 32; ++u) s += sh_red[u][col];
+        dst[e] = s;
+    }
+}
+
 // Sums the CTA slots of a partition in a fixed order and writes the outputs of z indices
 // k0 .. k0+kc-1 (and, with the first chunk, the per-row and per-partition values).
 __global__ void verify_finalize_kernel(const VArgs k, int KT)
@@ -843,6 +1099,26 @@ const void* rows_fn(int R, int KT, bool combine)
     return (R == 4) ? rows_fn_r<4>(KT, combine) : (R == 8) ? rows_fn_r<8>(KT, combine) : rows_fn_r<16>(KT, combine);
 }
 
+const void* lanes_fn(int KT, bool combine)
+{
+    switch (KT) {
+        case 1: return combine ? (const void*)verify_lanes_kernel<1, true> : (const void*)verify_lanes_kernel<1, false>;
+        case 2: return combine ? (const void*)verify_lanes_kernel<2, true> : (const void*)verify_lanes_kernel<2, false>;
+        default: return nullptr;
+    }
+}
+
+int lanes_ctas_per_sm(int KT, bool combine)
+{
+    int nb = 0;
+    const void* fn = lanes_fn(KT, combine);
+    if (!fn || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kLanesThreads, 0) != cudaSuccess || nb < 1) {
+        (void)cudaGetLastError();
+        return 2;
+    }
+    return nb;
+}
+
 int rows_ctas_per_sm(int R, int KT, bool combine)
 {
     int nb = 0;
@@ -875,6 +1151,19 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K, bool fused
         vg.slots = n * kt + kt + 1 + n;    // room for the squared norms of the fused combine pass
         return vg;
     }
+    if (fused && n > 48 && n <= kLanesRows && kt <= 2) {   // fused with the combine pass, 49 .. 64 peers (with fewer, lanes
+                                                           // of every four would hold no rows), one or two directions:
+        vg.own_z = 2;                                      // four lanes share the rows of a column quad
+        g.R = 16;
+        g.RG = 1;
+        g.CL = kLanesThreads;
+        g.threads = kLanesThreads;
+        vg.KT = kt;
+        g.slots = sm_count() * lanes_ctas_per_sm(kt, true);
+        g.cpp = choose_ctas_per_partition(P, stride >> 2, kLanesThreads / 4, g.slots);
+        vg.slots = n * kt + kt + 1 + n;
+        return vg;
+    }
     // 16 rows per thread: few row groups exchange column sums, and the per-tile bookkeeping of a thread
     // is spread over 64 elements (measured at n = 64, K = 4: 14.5 thread instructions per element against
     // 23.5 with 8 rows per thread)
@@ -904,7 +1193,8 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
     ensure_verify_attrs();
     int rc;
     {
-        const void* fn = vg.own_z ? rows_fn(g.R, vg.KT, a.combine != 0) : verify_fn(g.R, vg.KT, a.combine != 0, g.threads);
+        const void* fn = vg.own_z == 2 ? lanes_fn(vg.KT, a.combine != 0)
+                       : vg.own_z ? rows_fn(g.R, vg.KT, a.combine != 0) : verify_fn(g.R, vg.KT, a.combine != 0, g.threads);
         if (!fn) return BTARD_ERR_UNSUPPORTED;
         void* args[] = {(void*)&va};
         prof_begin(KIND_VERIFY, st);
