@@ -644,8 +644,8 @@ __global__ void __launch_bounds__(CL, rows_min_ctas(R, KT)) verify_rows_kernel(c
     }
 }
 
-// 49 .. 64 peers, the verification pass fused with the combine pass, one or two directions per launch: the four
-// lanes 4k .. 4k + 3 of a warp share 4 columns and hold 16 rows each (lane g: rows 16 g .. 16 g + 15, R x 4
+// 41 .. 64 peers, the verification pass fused with the combine pass, one or two directions per launch: the four
+// lanes 4k .. 4k + 3 of a warp share 4 columns and hold R = 12 or 16 rows each (lane g: rows R g .. R g + R - 1, R x 4
 // columns in registers as in verify_rows_kernel), so what the 64 rows of a column have to add up (the move of
 // v, the clipped-residual sum) crosses lanes by two shuffle steps and the tile loop has no CTA barrier and no
 // shared-memory staging at all.  Direction q of a launch is drawn by lane q of the group and handed to the
@@ -658,13 +658,16 @@ constexpr int kLanesRows = 64;
 // its loads, and more warps hide more of that; two directions spill 280 bytes at 128 registers and keep three
 // CTAs.  At four directions (64 x 64 x 4 194 304) neither four lanes of 16 rows (255 registers, two CTAs: 19.9
 // against 19.0 ms) nor eight lanes of 8 rows (26.3 ms) beats the row-group kernel, so it keeps them.
-template <int KT>
-constexpr int lanes_min_ctas() { return KT == 1 ? 4 : 3; }
+// R rows per lane: 12 (41 .. 48 peers) or 16 (49 .. 64).  Measured against the row-group kernel on 16 x n x 276 320,
+// K = 1: n = 48: 0.166 against 0.245 ms, n = 40: 0.233 against 0.235, n = 32 (8 rows per lane): 0.129 against 0.127,
+// n = 24: 0.175 against 0.116 (half of the lanes hold no rows): used above 40 peers.
+template <int R, int KT>
+constexpr int lanes_min_ctas() { return (R == 16 && KT == 2) ? 3 : 4; }
 
-template <int KT, bool COMBINE>
-__global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<KT>()) verify_lanes_kernel(const VArgs k)
+template <int R, int KT, bool COMBINE>
+__global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<R, KT>()) verify_lanes_kernel(const VArgs k)
 {
-    constexpr int R = 16, NR = kLanesRows, CL = kLanesThreads, G = NR / R;   // G = 4 lanes share a quad
+    constexpr int G = 4, NR = G * R, CL = kLanesThreads;   // four lanes share a quad
     __shared__ float sh_w[NR];
     __shared__ float sh_c[NR];                      // COMBINE: coefficients a_j
     __shared__ double sh_ga[NR + 1];                // COMBINE: (G a)_i, then a^T G a
@@ -1099,19 +1102,28 @@ const void* rows_fn(int R, int KT, bool combine)
     return (R == 4) ? rows_fn_r<4>(KT, combine) : (R == 8) ? rows_fn_r<8>(KT, combine) : rows_fn_r<16>(KT, combine);
 }
 
-const void* lanes_fn(int KT, bool combine)
+template <int R>
+const void* lanes_fn_r(int KT, bool combine)
 {
     switch (KT) {
-        case 1: return combine ? (const void*)verify_lanes_kernel<1, true> : (const void*)verify_lanes_kernel<1, false>;
-        case 2: return combine ? (const void*)verify_lanes_kernel<2, true> : (const void*)verify_lanes_kernel<2, false>;
+        case 1: return combine ? (const void*)verify_lanes_kernel<R, 1, true> : (const void*)verify_lanes_kernel<R, 1, false>;
+        case 2: return combine ? (const void*)verify_lanes_kernel<R, 2, true> : (const void*)verify_lanes_kernel<R, 2, false>;
         default: return nullptr;
     }
 }
 
-int lanes_ctas_per_sm(int KT, bool combine)
+inline int lanes_rows(int n) { return n <= 48 ? 12 : 16; }
+
+const void* lanes_fn(int n, int KT, bool combine)
+{
+    const int R = lanes_rows(n);
+    return R == 12 ? lanes_fn_r<12>(KT, combine) : lanes_fn_r<16>(KT, combine);
+}
+
+int lanes_ctas_per_sm(int n, int KT, bool combine)
 {
     int nb = 0;
-    const void* fn = lanes_fn(KT, combine);
+    const void* fn = lanes_fn(n, KT, combine);
     if (!fn || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kLanesThreads, 0) != cudaSuccess || nb < 1) {
         (void)cudaGetLastError();
         return 2;
@@ -1151,15 +1163,15 @@ VerifyGeometry verify_geometry(int n, int P, long long stride, int K, bool fused
         vg.slots = n * kt + kt + 1 + n;    // room for the squared norms of the fused combine pass
         return vg;
     }
-    if (fused && n > 48 && n <= kLanesRows && kt <= 2) {   // fused with the combine pass, 49 .. 64 peers (with fewer, lanes
-                                                           // of every four would hold no rows), one or two directions:
+    if (fused && n > 40 && n <= kLanesRows && kt <= 2) {   // fused with the combine pass, 41 .. 64 peers (with fewer, lanes
+                                                           // of every four would hold few rows or none), one or two directions:
         vg.own_z = 2;                                      // four lanes share the rows of a column quad
-        g.R = 16;
+        g.R = lanes_rows(n);
         g.RG = 1;
         g.CL = kLanesThreads;
         g.threads = kLanesThreads;
         vg.KT = kt;
-        g.slots = sm_count() * lanes_ctas_per_sm(kt, true);
+        g.slots = sm_count() * lanes_ctas_per_sm(n, kt, true);
         g.cpp = choose_ctas_per_partition(P, stride >> 2, kLanesThreads / 4, g.slots);
         vg.slots = n * kt + kt + 1 + n;
         return vg;
@@ -1193,7 +1205,7 @@ int launch_verify(const VerifyLaunch& a, const VerifyGeometry& vg, cudaStream_t 
     ensure_verify_attrs();
     int rc;
     {
-        const void* fn = vg.own_z == 2 ? lanes_fn(vg.KT, a.combine != 0)
+        const void* fn = vg.own_z == 2 ? lanes_fn(a.n, vg.KT, a.combine != 0)
                        : vg.own_z ? rows_fn(g.R, vg.KT, a.combine != 0) : verify_fn(g.R, vg.KT, a.combine != 0, g.threads);
         if (!fn) return BTARD_ERR_UNSUPPORTED;
         void* args[] = {(void*)&va};
