@@ -664,7 +664,9 @@ constexpr int kLanesRows = 64;
 template <int R, int KT>
 constexpr int lanes_min_ctas() { return (R == 16 && KT == 2) ? 3 : 4; }
 
-template <int R, int KT, bool COMBINE>
+// WHOLE: n == 4 R, every lane has all of its rows (a kernel of its own: the row clamp of the other form costs the
+// 64-peer shape 5 % through its registers).
+template <int R, int KT, bool COMBINE, bool WHOLE>
 __global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<R, KT>()) verify_lanes_kernel(const VArgs k)
 {
     constexpr int G = 4, NR = G * R, CL = kLanesThreads;   // four lanes share a quad
@@ -753,7 +755,10 @@ __global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<R, KT>()) verify
     // a row with weight 0 or coefficient 0 (a non-finite row) is left out of the sums, not multiplied
     bool any_skip = false;
     for (int r = 0; r < n; ++r) any_skip |= (sh_w[r] == 0.0f) || (COMBINE && sh_c[r] == 0.0f);
-    const bool rows_whole = (n == NR);                 // no row of any lane is missing
+    // Whole tiles run without a test per row: a lane that is short of rows reads the partition's last row in
+    // their place (finite there, since no row is left out), and what it adds up for them meets a coefficient and a
+    // weight of 0 in the column sums and lands in sums that nobody reads.
+    const int rmax = n - 1 - rb;
 
     auto four_sum = [&](float4& s) {                   // sum over the lanes of the group, every lane gets it
 #pragma unroll
@@ -772,8 +777,9 @@ __global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<R, KT>()) verify
         float4 x[R];
 #pragma unroll
         for (int r = 0; r < R; ++r)
-            x[r] = (!GUARD || rb + r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
-                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[r] = !GUARD ? __ldcs(reinterpret_cast<const float4*>(gp + (long long)(WHOLE ? r : min(r, rmax)) * stride + col))
+                 : (rb + r < n) ? __ldcs(reinterpret_cast<const float4*>(gp + (size_t)r * stride + col))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
         if (scaled) {
 #pragma unroll
             for (int r = 0; r < R; ++r) x[r] = scale_row(x[r], sh_f[rb + r]);
@@ -858,7 +864,7 @@ __global__ void __launch_bounds__(kLanesThreads, lanes_min_ctas<R, KT>()) verify
         }
     };
     for (long long qb = q0 + tid / G; qb < q1; qb += CL / G) {
-        if (rows_whole && !any_skip && qb * 4 + 3 < len) tile(std::false_type{}, qb);
+        if (!any_skip && qb * 4 + 3 < len) tile(std::false_type{}, qb);
         else tile(std::true_type{}, qb);
     }
 
@@ -1102,12 +1108,12 @@ const void* rows_fn(int R, int KT, bool combine)
     return (R == 4) ? rows_fn_r<4>(KT, combine) : (R == 8) ? rows_fn_r<8>(KT, combine) : rows_fn_r<16>(KT, combine);
 }
 
-template <int R>
+template <int R, bool WHOLE>
 const void* lanes_fn_r(int KT, bool combine)
 {
     switch (KT) {
-        case 1: return combine ? (const void*)verify_lanes_kernel<R, 1, true> : (const void*)verify_lanes_kernel<R, 1, false>;
-        case 2: return combine ? (const void*)verify_lanes_kernel<R, 2, true> : (const void*)verify_lanes_kernel<R, 2, false>;
+        case 1: return combine ? (const void*)verify_lanes_kernel<R, 1, true, WHOLE> : (const void*)verify_lanes_kernel<R, 1, false, WHOLE>;
+        case 2: return combine ? (const void*)verify_lanes_kernel<R, 2, true, WHOLE> : (const void*)verify_lanes_kernel<R, 2, false, WHOLE>;
         default: return nullptr;
     }
 }
@@ -1117,7 +1123,8 @@ inline int lanes_rows(int n) { return n <= 48 ? 12 : 16; }
 const void* lanes_fn(int n, int KT, bool combine)
 {
     const int R = lanes_rows(n);
-    return R == 12 ? lanes_fn_r<12>(KT, combine) : lanes_fn_r<16>(KT, combine);
+    if (n == 4 * R) return R == 12 ? lanes_fn_r<12, true>(KT, combine) : lanes_fn_r<16, true>(KT, combine);
+    return R == 12 ? lanes_fn_r<12, false>(KT, combine) : lanes_fn_r<16, false>(KT, combine);
 }
 
 int lanes_ctas_per_sm(int n, int KT, bool combine)
